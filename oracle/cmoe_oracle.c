@@ -1,0 +1,230 @@
+/*
+ * CPU oracle for the clustered-MoE layer forward.  TEST INFRASTRUCTURE ONLY:
+ * see cmoe_oracle.h for what it computes, its precision, and its pins.
+ * Nothing here is blocked, fused or reordered beyond the definitions cited.
+ */
+#include "cmoe_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* IEEE binary16 -> binary32, exact: 1 sign, 5 exponent (bias 15), 10 mantissa bits. */
+float cmoe_ref_half_to_float(uint16_t h) {
+  uint32_t sign = (uint32_t)(h & 0x8000u) << 16;
+  uint32_t expo = (h >> 10) & 0x1Fu;
+  uint32_t mant = h & 0x3FFu;
+  float v;
+  if (expo == 0) {                      /* zero / subnormal: mant * 2^-24 */
+    v = (float)mant * 5.9604644775390625e-8f;
+    return sign ? -v : v;
+  }
+  uint32_t bits;
+  if (expo == 31) bits = sign | 0x7F800000u | (mant << 13);          /* inf / nan */
+  else            bits = sign | ((expo + 112u) << 23) | (mant << 13); /* rebias 15 -> 127 */
+  memcpy(&v, &bits, sizeof v);
+  return v;
+}
+
+/* INT4 storage format of the residual factors (Sec. 3.4 "Precision and Memory
+ * Management"): two's-complement 4-bit code, even flat index in the low nibble,
+ * times the fp16 scale shared by its group of 32 consecutive flat elements. */
+float cmoe_ref_dequant(const uint8_t* q, const uint16_t* s, int64_t idx) {
+  uint8_t byte = q[idx / 2];
+  int code = (idx % 2 == 0) ? (byte & 0xF) : (byte >> 4);
+  if (code >= 8) code -= 16;
+  return (float)code * cmoe_ref_half_to_float(s[idx / 32]);
+}
+
+static int desc_ok(const cmoe_ref_desc* D) {
+  if (!D || D->d <= 0 || D->d_ff <= 0 || D->E <= 0 || D->G <= 0 || D->r < 0) return 0;
+  if (D->E % D->G) return 0;
+  if (D->k < 1 || D->k > D->E / D->G) return 0;
+  return 1;
+}
+
+int cmoe_ref_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+/* Two-stage hierarchical routing (Sec. 3.3, Eq. 9 and Eq. 10). */
+int cmoe_ref_route(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
+                   int32_t* cluster_id, int32_t* expert_slot, float* gates,
+                   float* z_out, float* l_out) {
+  if (!desc_ok(D)) return -1;
+  const int d = D->d, G = D->G, K = D->E / D->G, k = D->k;
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    float* z = (float*)malloc(sizeof(float) * (size_t)G);
+    float* l = (float*)malloc(sizeof(float) * (size_t)K);
+    char* taken = (char*)calloc((size_t)K, 1);
+    /* stage 1: z_g = u_g . x ; the softmax of Eq. 9 is monotone, top-1 = argmax */
+    for (int g = 0; g < G; ++g) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j)
+        acc += (double)cmoe_ref_half_to_float(x[(size_t)t * d + j]) * (double)D->C[(size_t)j * G + g];
+      if (D->b_c) acc += (double)D->b_c[g];
+      z[g] = (float)acc;
+    }
+    int gs = 0;
+    for (int g = 1; g < G; ++g) if (z[g] > z[gs]) gs = g;      /* lowest index wins ties */
+    cluster_id[t] = gs;
+    /* stage 2: l_i = v_i . x over the K experts of the chosen cluster */
+    for (int i = 0; i < K; ++i) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j)
+        acc += (double)cmoe_ref_half_to_float(x[(size_t)t * d + j]) *
+               (double)D->R[((size_t)gs * d + j) * K + i];
+      if (D->b_e) acc += (double)D->b_e[(size_t)gs * K + i];
+      l[i] = (float)acc;
+    }
+    /* top-k by repeated argmax: descending logit, lowest index first on ties */
+    int sel[64];
+    for (int s = 0; s < k; ++s) {
+      int best = -1;
+      for (int i = 0; i < K; ++i)
+        if (!taken[i] && (best < 0 || l[i] > l[best])) best = i;
+      taken[best] = 1;
+      sel[s] = best;
+      expert_slot[(size_t)t * k + s] = gs * K + best;
+    }
+    /* gates: softmax of Eq. 10 restricted to, and renormalised over, the kept experts */
+    double lmax = (double)l[sel[0]], denom = 0.0;
+    for (int s = 0; s < k; ++s) denom += exp((double)l[sel[s]] - lmax);
+    for (int s = 0; s < k; ++s)
+      gates[(size_t)t * k + s] = (float)(exp((double)l[sel[s]] - lmax) / denom);
+    if (z_out) memcpy(z_out + (size_t)t * G, z, sizeof(float) * (size_t)G);
+    if (l_out) memcpy(l_out + (size_t)t * K, l, sizeof(float) * (size_t)K);
+    free(z); free(l); free(taken);
+  }
+  return 0;
+}
+
+/* Eq. 7: W_e = W_base^g + U_e V_e, formed explicitly.
+ * which = 1: W1_e[j][f] = B1_g[j][f] + sum_p U1_e[j][p] V1_e[p][f],  U1 stored [E][r][d],    V1 stored [E][d_ff][r]
+ * which = 2: W2_e[f][c] = B2_g[f][c] + sum_p U2_e[f][p] V2_e[p][c],  U2 stored [E][r][d_ff], V2 stored [E][d][r] */
+int cmoe_ref_form_weight(const cmoe_ref_desc* D, int32_t e, int32_t which, float* W) {
+  if (!desc_ok(D) || e < 0 || e >= D->E || (which != 1 && which != 2)) return -1;
+  const int K = D->E / D->G, g = e / K, r = D->r;
+  const int64_t din = (which == 1) ? D->d : D->d_ff;
+  const int64_t dout = (which == 1) ? D->d_ff : D->d;
+  const uint16_t* B = ((which == 1) ? D->B1 : D->B2) + (size_t)g * din * dout;
+  const uint8_t* Uq = (which == 1) ? D->U1q : D->U2q;
+  const uint16_t* Us = (which == 1) ? D->U1s : D->U2s;
+  const uint8_t* Vq = (which == 1) ? D->V1q : D->V2q;
+  const uint16_t* Vs = (which == 1) ? D->V1s : D->V2s;
+  /* deq(U_e) as [din][r] and deq(V_e) as [r][dout] */
+  float* Ud = (float*)malloc(sizeof(float) * (size_t)(din * r + 1));
+  float* Vd = (float*)malloc(sizeof(float) * (size_t)(dout * r + 1));
+  for (int64_t a = 0; a < din; ++a)
+    for (int p = 0; p < r; ++p)       /* U_e[a][p] lives at flat index (e*r + p)*din + a */
+      Ud[a * r + p] = cmoe_ref_dequant(Uq, Us, ((int64_t)e * r + p) * din + a);
+  for (int p = 0; p < r; ++p)
+    for (int64_t b = 0; b < dout; ++b) /* V_e[p][b] lives at flat index (e*dout + b)*r + p */
+      Vd[p * dout + b] = cmoe_ref_dequant(Vq, Vs, ((int64_t)e * dout + b) * r + p);
+#pragma omp parallel
+  {
+    double* acc = (double*)malloc(sizeof(double) * (size_t)dout);
+#pragma omp for schedule(static)
+    for (int64_t a = 0; a < din; ++a) {
+      for (int64_t b = 0; b < dout; ++b) acc[b] = (double)cmoe_ref_half_to_float(B[a * dout + b]);
+      for (int p = 0; p < r; ++p) {
+        double u = (double)Ud[a * r + p];
+        for (int64_t b = 0; b < dout; ++b) acc[b] += u * (double)Vd[p * dout + b];
+      }
+      for (int64_t b = 0; b < dout; ++b) W[a * dout + b] = (float)acc[b];
+    }
+    free(acc);
+  }
+  free(Ud); free(Vd);
+  return 0;
+}
+
+static float gelu_erf(float u) {
+  return (float)(0.5 * (double)u * (1.0 + erf((double)u / sqrt(2.0))));
+}
+
+/* y_t = sum_{e in top-k} p_e * GELU(x_t W1_e) W2_e  for the listed tokens. */
+int cmoe_ref_forward(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
+                     const int32_t* token_idx, int32_t n_idx, float* y) {
+  if (!desc_ok(D)) return -1;
+  const int d = D->d, d_ff = D->d_ff, k = D->k, E = D->E;
+  if (n_idx <= 0) return 0;
+  /* routes of the requested tokens */
+  uint16_t* xs = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)n_idx * d);
+  for (int n = 0; n < n_idx; ++n) {
+    int t = token_idx ? token_idx[n] : n;
+    if (t < 0 || t >= T) { free(xs); return -1; }
+    memcpy(xs + (size_t)n * d, x + (size_t)t * d, sizeof(uint16_t) * (size_t)d);
+  }
+  int32_t* cid = (int32_t*)malloc(sizeof(int32_t) * (size_t)n_idx);
+  int32_t* slot = (int32_t*)malloc(sizeof(int32_t) * (size_t)n_idx * k);
+  float* gate = (float*)malloc(sizeof(float) * (size_t)n_idx * k);
+  cmoe_ref_route(D, xs, n_idx, cid, slot, gate, NULL, NULL);
+
+  /* per (token, kept expert) output of that expert's FFN */
+  float* f_out = (float*)calloc((size_t)n_idx * k * d, sizeof(float));
+  float* W1 = (float*)malloc(sizeof(float) * (size_t)d * d_ff);
+  float* W2 = (float*)malloc(sizeof(float) * (size_t)d_ff * d);
+  for (int e = 0; e < E; ++e) {
+    int used = 0;
+    for (int64_t i = 0; i < (int64_t)n_idx * k; ++i) if (slot[i] == e) { used = 1; break; }
+    if (!used) continue;                       /* experts without tokens are never formed */
+    cmoe_ref_form_weight(D, e, 1, W1);
+    cmoe_ref_form_weight(D, e, 2, W2);
+#pragma omp parallel
+    {
+      double* acc = (double*)malloc(sizeof(double) * (size_t)(d_ff > d ? d_ff : d));
+      float* a = (float*)malloc(sizeof(float) * (size_t)d_ff);
+#pragma omp for schedule(dynamic, 1)
+      for (int64_t i = 0; i < (int64_t)n_idx * k; ++i) {
+        if (slot[i] != e) continue;
+        const uint16_t* xt = xs + (size_t)(i / k) * d;
+        /* h = x W1_e */
+        for (int f = 0; f < d_ff; ++f) acc[f] = 0.0;
+        for (int j = 0; j < d; ++j) {
+          double xj = (double)cmoe_ref_half_to_float(xt[j]);
+          const float* w = W1 + (size_t)j * d_ff;
+          for (int f = 0; f < d_ff; ++f) acc[f] += xj * (double)w[f];
+        }
+        for (int f = 0; f < d_ff; ++f) a[f] = gelu_erf((float)acc[f]);
+        /* out = a W2_e */
+        for (int c = 0; c < d; ++c) acc[c] = 0.0;
+        for (int f = 0; f < d_ff; ++f) {
+          double af = (double)a[f];
+          const float* w = W2 + (size_t)f * d;
+          for (int c = 0; c < d; ++c) acc[c] += af * (double)w[c];
+        }
+        float* o = f_out + (size_t)i * d;
+        for (int c = 0; c < d; ++c) o[c] = (float)acc[c];
+      }
+      free(acc); free(a);
+    }
+  }
+  /* gated combine, in slot order */
+  for (int n = 0; n < n_idx; ++n)
+    for (int c = 0; c < d; ++c) {
+      double acc = 0.0;
+      for (int s = 0; s < k; ++s)
+        acc += (double)gate[(size_t)n * k + s] * (double)f_out[((size_t)n * k + s) * d + c];
+      y[(size_t)n * d + c] = (float)acc;
+    }
+  free(xs); free(cid); free(slot); free(gate); free(f_out); free(W1); free(W2);
+  return 0;
+}
+
+/* Storage of the compressed layer vs the E dense experts it stands for (Eq. 8,
+ * applied to both FFN matrices): per cluster one base of d*d_ff per matrix, per
+ * expert r*(d + d_ff) factor elements per matrix. */
+void cmoe_ref_param_count(const cmoe_ref_desc* D, int64_t* stored, int64_t* dense) {
+  int64_t W = 2 * (int64_t)D->d * D->d_ff;
+  *dense = (int64_t)D->E * W;
+  *stored = (int64_t)D->G * W + (int64_t)D->E * 2 * D->r * ((int64_t)D->d + D->d_ff);
+}
