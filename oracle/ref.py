@@ -24,10 +24,10 @@ class _Desc(C.Structure):
 _lib = None
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        L = C.CDLL(_build.build())
+def load(path: str):
+    """Open an oracle shared object and declare its prototypes."""
+    if True:
+        L = C.CDLL(path)
         L.cmoe_ref_half_to_float.restype = C.c_float
         L.cmoe_ref_half_to_float.argtypes = [C.c_uint16]
         L.cmoe_ref_dequant.restype = C.c_float
@@ -41,7 +41,13 @@ def lib():
         L.cmoe_ref_param_count.restype = None
         L.cmoe_ref_param_count.argtypes = [C.POINTER(_Desc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.cmoe_ref_num_threads.restype = C.c_int
-        _lib = L
+    return L
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = load(_build.build())
     return _lib
 
 
