@@ -1,0 +1,130 @@
+/*
+ * cmoe - forward pass of a clustered Mixture-of-Experts layer on one NVIDIA B200 (sm_100a).
+ *
+ * The layer (row-vector convention, y = x W):
+ *   routing   two-stage hierarchical routing (Sec. 3.3): each token picks its top-1 cluster
+ *             g* = argmax_g u_g.x (Eq. 9), then the top-k of the K = E/G experts inside that
+ *             cluster by l_i = v_i.x with a softmax over them (Eq. 10); the gates are that softmax
+ *             renormalised over the k kept experts.
+ *   experts   every expert weight is a shared base plus a low-rank residual (Eq. 6, Eq. 7):
+ *             W1_e = B1_g + U1_e V1_e (d x d_ff),  W2_e = B2_g + U2_e V2_e (d_ff x d), bases in FP16,
+ *             factors in symmetric INT4 with one FP16 scale per 32 elements (Sec. 3.4).  The library
+ *             never forms W_e: it uses  x W_e = x B_g + (x U_e) V_e  so that the base product is
+ *             computed once per token and shared by the token's k experts (text after Eq. 7).
+ *   combine   y = sum_{e in top-k} p_e GELU(x W1_e) W2_e, GELU(u) = u/2 (1 + erf(u / sqrt 2)).
+ *
+ * Conventions
+ *   - Every pointer below is a DEVICE pointer on the current CUDA device unless it says "host".
+ *   - All arrays are dense, row-major, last index fastest.  fp16 values are IEEE binary16 bits.
+ *   - Expert slot e = g*K + i is expert i of cluster g.
+ *   - The library allocates no device memory: the caller passes a workspace arena.  The query
+ *     cmoe_workspace_bytes() says how large it must be for a descriptor.
+ *   - Every function returns CMOE_OK (0) or a negative cmoe_error; nothing throws or aborts.
+ *     Argument errors are found on the host before anything is launched.
+ *   - cmoe_route / cmoe_forward are asynchronous on the given stream, issue only kernel launches and
+ *     cudaMemsetAsync on it, never synchronise, and touch only the arena and the given outputs.
+ *     They are not re-entrant on one handle (the arena holds the call's scratch).
+ */
+#ifndef CMOE_H
+#define CMOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  CMOE_OK = 0,
+  CMOE_ERR_INVALID_ARG = -1,         /* NULL pointer, negative size, misaligned pointer              */
+  CMOE_ERR_UNSUPPORTED_SHAPE = -2,   /* descriptor outside the supported envelope (see cmoe_desc)    */
+  CMOE_ERR_WORKSPACE_TOO_SMALL = -3, /* workspace_bytes < cmoe_workspace_bytes(desc)                 */
+  CMOE_ERR_T_EXCEEDS_MAX = -4,       /* T > desc.T_max                                               */
+  CMOE_ERR_CUDA = -5,                /* a CUDA runtime/driver call failed; see cmoe_last_cuda_error  */
+  CMOE_ERR_TIMEOUT = -6              /* a bounded device-side wait expired (reported by cmoe_status) */
+} cmoe_error;
+
+typedef struct cmoe_layer cmoe_layer; /* opaque, host object owned by the library */
+
+/*
+ * Layer descriptor (Sec. 3.2-3.4).  Supported envelope: E % G == 0, K = E/G <= 32, G <= 64,
+ * 1 <= k <= min(K, 8), d % 32 == 0, d_ff % 32 == 0, r in {0, 4, 8, 16, 32}, quant_group == 32,
+ * T_max >= 1.  With r == 0 the factor pointers are ignored (plain shared-base experts).
+ * All weight pointers must be 16-byte aligned.
+ */
+typedef struct {
+  int32_t d, d_ff, E, G, r, k;
+  int32_t quant_group;          /* must be 32                                                      */
+  int32_t T_max;                /* largest T any later call may pass                               */
+  const float* C;               /* [d][G]       fp32  cluster prototypes; column g is u_g (Eq. 9)  */
+  const float* R;               /* [G][d][K]    fp32  in-cluster router; columns are v_i (Eq. 10)  */
+  const float* b_c;             /* [G] or NULL        optional bias added to the cluster logits    */
+  const float* b_e;             /* [G][K] or NULL     optional bias added to the expert logits     */
+  const uint16_t* B1;           /* [G][d][d_ff] fp16  shared base of the up-projection (Eq. 6)     */
+  const uint16_t* B2;           /* [G][d_ff][d] fp16  shared base of the down-projection           */
+  /* Residual factors (Eq. 7), packed INT4: two codes per byte, even flat index in the low nibble,
+   * two's complement in [-8, 7]; the reduction index is the fastest one:
+   *   U1q [E][r][d]   (U1_e is d x r)      V1q [E][d_ff][r] (V1_e is r x d_ff)
+   *   U2q [E][r][d_ff](U2_e is d_ff x r)   V2q [E][d][r]    (V2_e is r x d)                        */
+  const uint8_t *U1q, *V1q, *U2q, *V2q;
+  /* one fp16 scale per 32 consecutive elements of the flattened factor (value = code * scale)     */
+  const uint16_t *U1s, *V1s, *U2s, *V2s;
+  const int32_t* expert_global_id; /* [E] or NULL (identity): label written to expert_ids          */
+  void* workspace;              /* caller-owned device arena, 256-byte aligned                     */
+  size_t workspace_bytes;
+} cmoe_desc;
+
+/* Pure host query: bytes of workspace cmoe_create needs for this descriptor (pointer fields are
+ * not read).  Returns CMOE_ERR_UNSUPPORTED_SHAPE / CMOE_ERR_INVALID_ARG for a bad descriptor. */
+int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes);
+
+/* Validates the descriptor, copies and re-lays-out all weights into the arena (bases transposed to
+ * reduction-index-fastest), and returns a handle.  Synchronous: it runs its kernels on the legacy
+ * default stream and waits for them; work queued by the caller on other non-blocking streams that
+ * produces the weights must have finished.  After it returns the source weight buffers may be
+ * freed; the arena must outlive the handle and must not be written by the caller. */
+int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
+
+/* Two-stage routing only (Sec. 3.3, Eq. 9-10) for x = fp16 [T][d]:
+ *   cluster_id [T]     chosen cluster g*
+ *   expert_ids [T][k]  labels of the kept experts, by descending logit (lowest index first on ties)
+ *   gates      [T][k]  fp32, softmax over the kept logits (sums to 1 per token)
+ * 0 <= T <= T_max; T == 0 is a successful no-op.  x must be 16-byte aligned. */
+int cmoe_route(cmoe_layer* layer, const void* x, int32_t T,
+               int32_t* cluster_id, int32_t* expert_ids, float* gates, void* cuda_stream);
+
+/* Whole layer: y = fp16 [T][d] in the original token order, for x = fp16 [T][d].  Routing uses the
+ * same kernel as cmoe_route, so the two can never disagree.  x and y must be 16-byte aligned and
+ * must not overlap.  The rank-r partial sums of the down-projection are accumulated with floating
+ * point atomics, so y is reproducible only up to fp32 summation order. */
+int cmoe_forward(cmoe_layer* layer, const void* x, int32_t T, void* y, void* cuda_stream);
+
+/* Waits for the stream and returns the device status word of the handle: CMOE_OK, or
+ * CMOE_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the output of that call is then
+ * undefined; the handle stays usable and the word is cleared). */
+int cmoe_status(cmoe_layer* layer, void* cuda_stream);
+
+/* Per-handle facts for tests and benchmarks (host struct, filled by cmoe_get_info). */
+typedef struct {
+  int32_t path;              /* 0 generic CUDA-core path, 1 tcgen05 grouped-GEMM path, 2 weight-streaming path */
+  int32_t launches_route;    /* kernels + memsets one cmoe_route call enqueues                     */
+  int32_t launches_forward;  /* kernels + memsets one cmoe_forward call enqueues                   */
+  int32_t row_align;         /* permuted-row alignment of a cluster segment                        */
+  int32_t T_pad_max;         /* rows of the permuted activations buffers                           */
+  int32_t reserved[3];
+} cmoe_info;
+int cmoe_get_info(const cmoe_layer* layer, cmoe_info* out);
+
+/* cudaError_t (as int) of the last failed CUDA call on this handle, 0 if none. */
+int cmoe_last_cuda_error(const cmoe_layer* layer);
+
+/* Frees the host object.  The arena is the caller's. */
+int cmoe_destroy(cmoe_layer* layer);
+
+const char* cmoe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CMOE_H */

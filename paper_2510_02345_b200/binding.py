@@ -1,0 +1,197 @@
+"""Thin ctypes binding over libcmoe.so: argument marshalling only.
+
+The functions carry the names of the C boundary (include/cmoe.h).  PyTorch is
+used for device memory and streams; every step of the layer runs in the
+library's CUDA kernels.  There is no CPU fallback: if the shared library is
+missing or no CUDA device is present, loading or calling fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(PKG, "libcmoe.so")
+
+CMOE_OK = 0
+ERRORS = {
+    -1: "CMOE_ERR_INVALID_ARG", -2: "CMOE_ERR_UNSUPPORTED_SHAPE", -3: "CMOE_ERR_WORKSPACE_TOO_SMALL",
+    -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
+}
+EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_status",
+           "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror"]
+
+
+class CmoeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {ERRORS.get(code, code)} ({strerror(code)})")
+
+
+class cmoe_desc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("d", "d_ff", "E", "G", "r", "k", "quant_group", "T_max")] + [
+        (n, C.c_void_p) for n in ("C", "R", "b_c", "b_e", "B1", "B2", "U1q", "V1q", "U2q", "V2q",
+                                  "U1s", "V1s", "U2s", "V2s", "expert_global_id", "workspace")
+    ] + [("workspace_bytes", C.c_size_t)]
+
+
+class cmoe_info(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max")] + [
+        ("reserved", C.c_int32 * 3)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libcmoe.so (built in-tree by paper_2510_02345_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2510_02345_b200.build` "
+                "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.cmoe_workspace_bytes.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_size_t)]
+        L.cmoe_create.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_void_p)]
+        L.cmoe_route.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.cmoe_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.cmoe_status.argtypes = [C.c_void_p, C.c_void_p]
+        L.cmoe_get_info.argtypes = [C.c_void_p, C.POINTER(cmoe_info)]
+        L.cmoe_last_cuda_error.argtypes = [C.c_void_p]
+        L.cmoe_destroy.argtypes = [C.c_void_p]
+        L.cmoe_strerror.argtypes = [C.c_int]
+        L.cmoe_strerror.restype = C.c_char_p
+        for name in EXPORTS:
+            if name != "cmoe_strerror":
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().cmoe_strerror(code).decode()
+
+
+def _check(rc: int, where: str):
+    if rc != CMOE_OK:
+        raise CmoeError(rc, where)
+
+
+# ---- the C calls, one Python function each ------------------------------------------------------
+def cmoe_workspace_bytes(desc: cmoe_desc) -> int:
+    out = C.c_size_t(0)
+    _check(lib().cmoe_workspace_bytes(C.byref(desc), C.byref(out)), "cmoe_workspace_bytes")
+    return out.value
+
+
+def cmoe_create(desc: cmoe_desc) -> C.c_void_p:
+    handle = C.c_void_p()
+    _check(lib().cmoe_create(C.byref(desc), C.byref(handle)), "cmoe_create")
+    return handle
+
+
+def cmoe_route(handle, x_ptr: int, T: int, cluster_id_ptr: int, expert_ids_ptr: int, gates_ptr: int, stream: int):
+    _check(lib().cmoe_route(handle, x_ptr, T, cluster_id_ptr, expert_ids_ptr, gates_ptr, stream), "cmoe_route")
+
+
+def cmoe_forward(handle, x_ptr: int, T: int, y_ptr: int, stream: int):
+    _check(lib().cmoe_forward(handle, x_ptr, T, y_ptr, stream), "cmoe_forward")
+
+
+def cmoe_status(handle, stream: int) -> int:
+    return lib().cmoe_status(handle, stream)
+
+
+def cmoe_get_info(handle) -> cmoe_info:
+    info = cmoe_info()
+    _check(lib().cmoe_get_info(handle, C.byref(info)), "cmoe_get_info")
+    return info
+
+
+def cmoe_destroy(handle):
+    _check(lib().cmoe_destroy(handle), "cmoe_destroy")
+
+
+# ---- convenience owner of the device buffers ---------------------------------------------------
+class ClusteredMoELayer:
+    """Uploads a layer (numpy arrays in the boundary layouts) and owns the arena.
+
+    route(x) / forward(x) take CUDA fp16 tensors [T][d] and launch on torch's current stream.
+    """
+
+    _NP_FIELDS = (("C", np.float32), ("R", np.float32), ("b_c", np.float32), ("b_e", np.float32),
+                  ("B1", np.float16), ("B2", np.float16),
+                  ("U1q", np.uint8), ("V1q", np.uint8), ("U2q", np.uint8), ("V2q", np.uint8),
+                  ("U1s", np.float16), ("V1s", np.float16), ("U2s", np.float16), ("V2s", np.float16),
+                  ("expert_global_id", np.int32))
+
+    def __init__(self, layer: dict, T_max: int | None = None, device: str = "cuda:0", keep_source: bool = False):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required (there is no CPU path)")
+        s = layer["shape"]
+        self.shape = s
+        self.device = torch.device(device)
+        self.T_max = int(T_max if T_max is not None else layer.get("T", s.T))
+        torch.cuda.set_device(self.device)
+        src = {}
+        for name, dt in self._NP_FIELDS:
+            a = layer.get(name)
+            if a is None or a.size == 0:
+                src[name] = None
+            else:
+                src[name] = torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(self.device)
+        desc = cmoe_desc()
+        desc.d, desc.d_ff, desc.E, desc.G, desc.r, desc.k = s.d, s.d_ff, s.E, s.G, s.r, s.k
+        desc.quant_group, desc.T_max = 32, self.T_max
+        for name, _ in self._NP_FIELDS:
+            setattr(desc, name, None if src[name] is None else src[name].data_ptr())
+        nbytes = cmoe_workspace_bytes(desc)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        desc.workspace, desc.workspace_bytes = base, nbytes
+        self.workspace_bytes = nbytes
+        torch.cuda.synchronize(self.device)
+        self.handle = cmoe_create(desc)
+        self.info = cmoe_get_info(self.handle)
+        self._src = src if keep_source else None   # the library holds its own copies in the arena
+
+    def _stream(self) -> int:
+        import torch
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def route(self, x):
+        import torch
+        T = x.shape[0]
+        k = self.shape.k
+        assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.shape[1] == self.shape.d
+        cid = torch.empty(T, dtype=torch.int32, device=x.device)
+        eid = torch.empty((T, k), dtype=torch.int32, device=x.device)
+        gates = torch.empty((T, k), dtype=torch.float32, device=x.device)
+        cmoe_route(self.handle, x.data_ptr(), T, cid.data_ptr(), eid.data_ptr(), gates.data_ptr(), self._stream())
+        return cid, eid, gates
+
+    def forward(self, x, out=None):
+        import torch
+        T = x.shape[0]
+        assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.shape[1] == self.shape.d
+        y = out if out is not None else torch.empty_like(x)
+        cmoe_forward(self.handle, x.data_ptr(), T, y.data_ptr(), self._stream())
+        return y
+
+    def status(self) -> int:
+        return cmoe_status(self.handle, self._stream())
+
+    def close(self):
+        if getattr(self, "handle", None):
+            cmoe_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

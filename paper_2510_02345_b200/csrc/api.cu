@@ -1,0 +1,286 @@
+// The C boundary of libcmoe (include/cmoe.h): descriptor validation, the arena plan, weight
+// re-layout at create time and the launch sequences of cmoe_route / cmoe_forward.
+#include <new>
+
+#include "cmoe_internal.h"
+
+using namespace cmoe;
+
+namespace {
+
+struct Arena {
+  size_t used = 0;
+  char* base = nullptr;
+  template <typename T>
+  T* take(size_t count) {
+    size_t off = (used + 255) / 256 * 256;
+    used = off + count * sizeof(T);
+    return base ? reinterpret_cast<T*>(base + off) : nullptr;
+  }
+};
+
+long long binom_ll(int n, int m) {
+  if (m > n) return 0;
+  long long r = 1;
+  for (int i = 1; i <= m; ++i) {
+    r = r * (n - m + i) / i;
+    if (r > (1ll << 40)) return r;
+  }
+  return r;
+}
+
+int validate_dims(const cmoe_desc* desc, Dims* D) {
+  if (!desc) return CMOE_ERR_INVALID_ARG;
+  if (desc->d <= 0 || desc->d_ff <= 0 || desc->E <= 0 || desc->G <= 0 || desc->k <= 0 ||
+      desc->r < 0 || desc->T_max <= 0)
+    return CMOE_ERR_INVALID_ARG;
+  if (desc->E % desc->G) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  const int K = desc->E / desc->G;
+  if (desc->G > kMaxG || K > kMaxK || desc->k > K || desc->k > kMaxKsel) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  if (desc->d % 32 || desc->d_ff % 32) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  if (!(desc->r == 0 || desc->r == 4 || desc->r == 8 || desc->r == 16 || desc->r == 32))
+    return CMOE_ERR_UNSUPPORTED_SHAPE;
+  if (desc->quant_group != 32) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  if (desc->T_max > (1 << 22)) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  D->d = desc->d; D->d_ff = desc->d_ff; D->E = desc->E; D->G = desc->G; D->K = K;
+  D->r = desc->r; D->k = desc->k; D->T_max = desc->T_max;
+  const long long combos = binom_ll(K, desc->k);
+  if (combos <= 64) { D->nsub = (int)combos; D->sub_is_combo = 1; }
+  else              { D->nsub = K;           D->sub_is_combo = 0; }
+  D->nkey = D->G * D->nsub;
+  if (D->nkey > kMaxKeys) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  D->row_align = 128;
+  D->T_pad_max = t_pad_bound(*D, D->T_max);
+  return CMOE_OK;
+}
+
+// Lays the arena out; with a null base it only measures.
+void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
+  const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r, k = D.k;
+  const size_t T = D.T_max, P = D.T_pad_max;
+  const size_t nblk = (T + kPermBlock - 1) / kPermBlock;
+  Weights w{};
+  Scratch s{};
+  w.Ct = A.take<float>(G * d);
+  w.Rt = A.take<float>(E * d);
+  w.bc = A.take<float>(G);
+  w.be = A.take<float>(E);
+  w.label = A.take<int>(E);
+  w.B1t = A.take<__half>(G * d * f);
+  w.B2t = A.take<__half>(G * d * f);
+  w.U1q = A.take<uint8_t>(E * r * d / 2 + 16);
+  w.V1q = A.take<uint8_t>(E * f * r / 2 + 16);
+  w.U2q = A.take<uint8_t>(E * r * f / 2 + 16);
+  w.V2q = A.take<uint8_t>(E * d * r / 2 + 16);
+  w.U1s = A.take<__half>(E * r * d / 32 + 8);
+  w.V1s = A.take<__half>(E * f * r / 32 + 8);
+  w.U2s = A.take<__half>(E * r * f / 32 + 8);
+  w.V2s = A.take<__half>(E * d * r / 32 + 8);
+  s.cluster_id = A.take<int>(T);
+  s.slot = A.take<int>(T * k);
+  s.gates = A.take<float>(T * k);
+  s.keys = A.take<int>(T);
+  s.block_counts = A.take<int>(nblk * D.nkey);
+  s.block_base = A.take<int>(nblk * D.nkey);
+  s.key_cnt = A.take<int>(D.nkey);
+  s.key_off = A.take<int>(D.nkey);
+  s.seg_off = A.take<int>(G + 1);
+  s.seg_cnt = A.take<int>(G);
+  s.n_rows = A.take<int>(1);
+  s.tile_cluster = A.take<int>(P / D.row_align);
+  s.row_token = A.take<int>(P);
+  s.row_slot = A.take<int>(P * k);
+  s.row_gate = A.take<float>(P * k);
+  s.x_perm = A.take<__half>(P * d);
+  s.t = A.take<float>(P * k * r + 4);
+  s.abar = A.take<__half>(P * f);
+  s.s = A.take<float>(P * k * r + 4);
+  s.status = A.take<int>(1);
+  if (W) *W = w;
+  if (S) *S = s;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+#define CMOE_CUDA(layer, expr)                                   \
+  do {                                                           \
+    cudaError_t _e = (expr);                                     \
+    if (_e != cudaSuccess) {                                     \
+      (layer)->last_cuda_error = (int)_e;                        \
+      return CMOE_ERR_CUDA;                                      \
+    }                                                            \
+  } while (0)
+
+int check_call(cmoe_layer* L, const void* x, int32_t T) {
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  if (T < 0) return CMOE_ERR_INVALID_ARG;
+  if (T > L->dims.T_max) return CMOE_ERR_T_EXCEEDS_MAX;
+  if (T > 0 && (!x || !aligned16(x))) return CMOE_ERR_INVALID_ARG;
+  return CMOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) {
+  if (!out_bytes) return CMOE_ERR_INVALID_ARG;
+  Dims D{};
+  int rc = validate_dims(desc, &D);
+  if (rc) return rc;
+  Arena A;
+  plan(D, A, nullptr, nullptr);
+  *out_bytes = (A.used + 255) / 256 * 256;
+  return CMOE_OK;
+}
+
+int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
+  if (!out_layer) return CMOE_ERR_INVALID_ARG;
+  *out_layer = nullptr;
+  Dims D{};
+  int rc = validate_dims(desc, &D);
+  if (rc) return rc;
+  if (!desc->C || !desc->R || !desc->B1 || !desc->B2 || !desc->workspace) return CMOE_ERR_INVALID_ARG;
+  if (D.r > 0 && (!desc->U1q || !desc->V1q || !desc->U2q || !desc->V2q || !desc->U1s ||
+                  !desc->V1s || !desc->U2s || !desc->V2s))
+    return CMOE_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(desc->workspace) & 255) != 0) return CMOE_ERR_INVALID_ARG;
+  const void* ptrs[] = {desc->C, desc->R, desc->B1, desc->B2};
+  for (const void* p : ptrs)
+    if (!aligned16(p)) return CMOE_ERR_INVALID_ARG;
+  size_t need = 0;
+  cmoe_workspace_bytes(desc, &need);
+  if (desc->workspace_bytes < need) return CMOE_ERR_WORKSPACE_TOO_SMALL;
+
+  cmoe_layer* L = new (std::nothrow) cmoe_layer();
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  L->dims = D;
+  L->path = kPathGeneric;
+  L->last_cuda_error = 0;
+  L->host_status = nullptr;
+  Arena A;
+  A.base = static_cast<char*>(desc->workspace);
+  plan(D, A, &L->w, &L->sc);
+
+  cudaStream_t st = 0;
+  const Weights& W = L->w;
+  const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r;
+  auto fail = [&](cudaError_t) {
+    delete L;
+    return CMOE_ERR_CUDA;
+  };
+  cudaError_t e;
+  // router: C [d][G] -> Ct [G][d];  R [G][d][K] -> Rt [G][K][d]
+  if ((e = launch_transpose_f32(desc->C, const_cast<float*>(W.Ct), 1, D.d, D.G, st))) return fail(e);
+  if ((e = launch_transpose_f32(desc->R, const_cast<float*>(W.Rt), D.G, D.d, D.K, st))) return fail(e);
+  if (desc->b_c) e = cudaMemcpyAsync(const_cast<float*>(W.bc), desc->b_c, G * 4, cudaMemcpyDeviceToDevice, st);
+  else           e = cudaMemsetAsync(const_cast<float*>(W.bc), 0, G * 4, st);
+  if (e) return fail(e);
+  if (desc->b_e) e = cudaMemcpyAsync(const_cast<float*>(W.be), desc->b_e, E * 4, cudaMemcpyDeviceToDevice, st);
+  else           e = cudaMemsetAsync(const_cast<float*>(W.be), 0, E * 4, st);
+  if (e) return fail(e);
+  if (desc->expert_global_id) {
+    e = cudaMemcpyAsync(const_cast<int*>(W.label), desc->expert_global_id, E * 4, cudaMemcpyDeviceToDevice, st);
+  } else {
+    int* ids = new (std::nothrow) int[E];
+    if (!ids) { delete L; return CMOE_ERR_INVALID_ARG; }
+    for (size_t i = 0; i < E; ++i) ids[i] = (int)i;
+    e = cudaMemcpy(const_cast<int*>(W.label), ids, E * 4, cudaMemcpyHostToDevice);
+    delete[] ids;
+  }
+  if (e) return fail(e);
+  // bases: B1 [G][d][d_ff] -> B1t [G][d_ff][d];  B2 [G][d_ff][d] -> B2t [G][d][d_ff]
+  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B1), const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st))) return fail(e);
+  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B2), const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st))) return fail(e);
+  if (r > 0) {
+    struct { const void* src; const void* dst; size_t bytes; } cp[] = {
+        {desc->U1q, W.U1q, E * r * d / 2}, {desc->V1q, W.V1q, E * f * r / 2},
+        {desc->U2q, W.U2q, E * r * f / 2}, {desc->V2q, W.V2q, E * d * r / 2},
+        {desc->U1s, W.U1s, E * r * d / 32 * 2}, {desc->V1s, W.V1s, E * f * r / 32 * 2},
+        {desc->U2s, W.U2s, E * r * f / 32 * 2}, {desc->V2s, W.V2s, E * d * r / 32 * 2}};
+    for (auto& c : cp)
+      if ((e = cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, c.bytes, cudaMemcpyDeviceToDevice, st))) return fail(e);
+  }
+  if ((e = cudaMemsetAsync(L->sc.status, 0, sizeof(int), st))) return fail(e);
+  if ((e = cudaStreamSynchronize(st))) return fail(e);
+  *out_layer = L;
+  return CMOE_OK;
+}
+
+int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int32_t* expert_ids,
+               float* gates, void* cuda_stream) {
+  int rc = check_call(L, x, T);
+  if (rc) return rc;
+  if (T == 0) return CMOE_OK;
+  if (!cluster_id || !expert_ids || !gates) return CMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CMOE_CUDA(L, launch_router(L->dims, L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
+                             gates, nullptr, st));
+  return CMOE_OK;
+}
+
+int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream) {
+  int rc = check_call(L, x, T);
+  if (rc) return rc;
+  if (T == 0) return CMOE_OK;
+  if (!y || !aligned16(y)) return CMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Dims& D = L->dims;
+  const Scratch& S = L->sc;
+  const __half* xh = static_cast<const __half*>(x);
+  CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  CMOE_CUDA(L, launch_permute(D, S, xh, T, st));
+  if (D.r > 0)
+    CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
+  CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st));
+  return CMOE_OK;
+}
+
+int cmoe_status(cmoe_layer* L, void* cuda_stream) {
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int word = 0;
+  CMOE_CUDA(L, cudaMemcpyAsync(&word, L->sc.status, sizeof(int), cudaMemcpyDeviceToHost, st));
+  CMOE_CUDA(L, cudaStreamSynchronize(st));
+  if (word != 0) {
+    CMOE_CUDA(L, cudaMemsetAsync(L->sc.status, 0, sizeof(int), st));
+    CMOE_CUDA(L, cudaStreamSynchronize(st));
+    return CMOE_ERR_TIMEOUT;
+  }
+  return CMOE_OK;
+}
+
+int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
+  if (!L || !out) return CMOE_ERR_INVALID_ARG;
+  *out = cmoe_info{};
+  out->path = L->path;
+  out->launches_route = 1;
+  out->launches_forward = 1 + kPermuteLaunches + (L->dims.r > 0 ? 1 : 0) +
+                          (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1);
+  out->row_align = L->dims.row_align;
+  out->T_pad_max = L->dims.T_pad_max;
+  return CMOE_OK;
+}
+
+int cmoe_last_cuda_error(const cmoe_layer* L) { return L ? L->last_cuda_error : 0; }
+
+int cmoe_destroy(cmoe_layer* L) {
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  delete L;
+  return CMOE_OK;
+}
+
+const char* cmoe_strerror(int code) {
+  switch (code) {
+    case CMOE_OK: return "ok";
+    case CMOE_ERR_INVALID_ARG: return "invalid argument";
+    case CMOE_ERR_UNSUPPORTED_SHAPE: return "descriptor outside the supported envelope";
+    case CMOE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CMOE_ERR_T_EXCEEDS_MAX: return "T exceeds T_max";
+    case CMOE_ERR_CUDA: return "CUDA call failed";
+    case CMOE_ERR_TIMEOUT: return "bounded device wait expired";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,106 @@
+// Internal declarations shared by the translation units of libcmoe: the handle, the arena plan,
+// the per-call scratch views and the kernel launchers.  Nothing here is part of the C boundary.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "cmoe.h"
+
+namespace cmoe {
+
+constexpr int kMaxG = 64;          // clusters
+constexpr int kMaxK = 32;          // experts per cluster (one lane each in the router's top-k)
+constexpr int kMaxKsel = 8;        // k
+constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
+constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels
+
+enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
+
+struct Dims {
+  int d, d_ff, E, G, K, r, k;
+  int nsub;        // permutation sub-keys per cluster (expert combinations, or lowest expert)
+  int nkey;        // G * nsub
+  int T_max;
+  int T_pad_max;   // rows of the permuted buffers
+  int row_align;   // a cluster's rows start at a multiple of this
+  int sub_is_combo;
+};
+
+// Weights as re-laid-out in the arena by cmoe_create.
+struct Weights {
+  const float* Ct;   // [G][d]     cluster prototypes, one row per cluster
+  const float* Rt;   // [E][d]     expert router vectors, one row per expert slot
+  const float* bc;   // [G]        (zeros when the caller passed NULL)
+  const float* be;   // [E]
+  const int* label;  // [E]        expert label written to expert_ids
+  const __half* B1t; // [G][d_ff][d]   base of the up-projection, reduction index fastest
+  const __half* B2t; // [G][d][d_ff]   base of the down-projection, reduction index fastest
+  const uint8_t *U1q, *V1q, *U2q, *V2q;  // packed INT4 in the boundary layouts
+  const __half *U1s, *V1s, *U2s, *V2s;   // fp16 scale per 32 flat elements
+};
+
+// Per-call scratch in the arena.
+struct Scratch {
+  // token order
+  int* cluster_id;    // [T]
+  int* slot;          // [T][k]  local expert index inside the cluster, routing order
+  float* gates;       // [T][k]
+  int* keys;          // [T]     permutation key = cluster * nsub + sub
+  // permutation tables
+  int* block_counts;  // [nblk][nkey]
+  int* block_base;    // [nblk][nkey]  rows of this key owned by earlier blocks
+  int* key_cnt;       // [nkey]
+  int* key_off;       // [nkey]  first permuted row of the key
+  int* seg_off;       // [G+1]   first permuted row of each cluster (multiple of row_align)
+  int* seg_cnt;       // [G]     tokens of each cluster
+  int* n_rows;        // [1]     seg_off[G]
+  int* tile_cluster;  // [T_pad_max / row_align]
+  // permuted-row order
+  int* row_token;     // [T_pad]     source token, -1 for padding rows
+  int* row_slot;      // [T_pad][k]  expert slot ids (g*K+i), ascending
+  float* row_gate;    // [T_pad][k]  gates in the same order (0 for padding rows)
+  __half* x_perm;     // [T_pad][d]
+  float* t;           // [T_pad][k][r]   x U1_e
+  __half* abar;       // [T_pad][d_ff]   sum_j p_j GELU(h_j)
+  float* s;           // [T_pad][k][r]   GELU(h_j) U2_e, accumulated with atomics
+  int* status;        // [1]
+};
+
+}  // namespace cmoe
+
+struct cmoe_layer {
+  cmoe::Dims dims;
+  cmoe::Weights w;
+  cmoe::Scratch sc;
+  int path;
+  int last_cuda_error;
+  int* host_status;   // pinned? plain host word used by cmoe_status
+};
+
+namespace cmoe {
+
+inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+inline int t_pad_bound(const Dims& D, int T) { return round_up(T, D.row_align) + D.G * D.row_align; }
+
+// ---- launchers (each returns the cudaError_t of its launches) ----------------------------------
+// router.cu
+cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int T,
+                          int* cluster_id, int* expert_ids, float* gates, int* slot_local,
+                          cudaStream_t st);
+// permute.cu : histogram, scan, scatter (+ row gather), padding rows
+cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st);
+constexpr int kPermuteLaunches = 4;
+// generic_path.cu : CUDA-core path for any supported shape
+cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,
+                               cudaStream_t st);
+constexpr int kGenericFfnLaunches = 3;
+// repack.cu : create-time layout changes
+cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
+                                  cudaStream_t st);
+cudaError_t launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols,
+                                 cudaStream_t st);
+
+}  // namespace cmoe

@@ -1,0 +1,210 @@
+// Token permutation: a stable counting sort of the tokens by (cluster, expert combination), with
+// every cluster's segment of permuted rows starting at a multiple of row_align so that GEMM tiles
+// never straddle two clusters.  The paper only implies this step ("tokens are assigned to a
+// cluster, then to experts inside it", Sec. 3.3); the mechanism is this library's.
+//
+//   hist     per-block histogram of the keys (block = 256 consecutive tokens)
+//   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table
+//   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
+//            writes the row tables and moves the token's activations with 16-byte vectors
+//   pad      fills the padding rows of each segment (zero activations, zero gates)
+//
+// The result is deterministic: rows of one key keep the token order.
+#include "cmoe_internal.h"
+#include "device_utils.cuh"
+
+namespace cmoe {
+
+namespace {
+
+__device__ __forceinline__ int binom(int n, int m) {
+  if (m > n) return 0;
+  long long r = 1;
+  for (int i = 1; i <= m; ++i) r = r * (n - m + i) / i;
+  return (int)r;
+}
+
+// Sort the token's k local expert indices ascending (gates follow) and return the sub-key.
+__device__ __forceinline__ int canonical_slots(const int* __restrict__ slot, const float* __restrict__ gate,
+                                               int k, int sub_is_combo, int* cs, float* cg) {
+#pragma unroll
+  for (int j = 0; j < kMaxKsel; ++j)
+    if (j < k) { cs[j] = slot[j]; cg[j] = gate[j]; }
+#pragma unroll
+  for (int a = 1; a < kMaxKsel; ++a)
+    if (a < k) {
+#pragma unroll
+      for (int b = kMaxKsel - 1; b > 0; --b)
+        if (b <= a && cs[b] < cs[b - 1]) {
+          int ti = cs[b]; cs[b] = cs[b - 1]; cs[b - 1] = ti;
+          float tg = cg[b]; cg[b] = cg[b - 1]; cg[b - 1] = tg;
+        }
+    }
+  if (!sub_is_combo) return cs[0];
+  int rank = 0;                    // combinatorial number system: sum_i C(c_i, i+1)
+#pragma unroll
+  for (int j = 0; j < kMaxKsel; ++j)
+    if (j < k) rank += binom(cs[j], j + 1);
+  return rank;
+}
+
+__global__ void __launch_bounds__(kPermBlock)
+hist_kernel(int T, int k, int nsub, int nkey, int sub_is_combo,
+            const int* __restrict__ cluster_id, const int* __restrict__ slot,
+            const float* __restrict__ gates, int* __restrict__ keys, int* __restrict__ block_counts) {
+  extern __shared__ int sh_cnt[];
+  for (int i = threadIdx.x; i < nkey; i += blockDim.x) sh_cnt[i] = 0;
+  __syncthreads();
+  int t = blockIdx.x * kPermBlock + threadIdx.x;
+  if (t < T) {
+    int cs[kMaxKsel];
+    float cg[kMaxKsel];
+    int sub = canonical_slots(slot + (size_t)t * k, gates + (size_t)t * k, k, sub_is_combo, cs, cg);
+    int key = cluster_id[t] * nsub + sub;
+    keys[t] = key;
+    atomicAdd(&sh_cnt[key], 1);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < nkey; i += blockDim.x)
+    block_counts[(size_t)blockIdx.x * nkey + i] = sh_cnt[i];
+}
+
+__global__ void __launch_bounds__(1024)
+scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
+            const int* __restrict__ block_counts, int* __restrict__ block_base,
+            int* __restrict__ key_cnt, int* __restrict__ key_off, int* __restrict__ seg_off,
+            int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster) {
+  __shared__ int sh_seg[kMaxG + 1];
+  for (int key = threadIdx.x; key < nkey; key += blockDim.x) {
+    int run = 0;
+    for (int b = 0; b < nblk; ++b) {
+      int c = block_counts[(size_t)b * nkey + key];
+      block_base[(size_t)b * nkey + key] = run;
+      run += c;
+    }
+    key_cnt[key] = run;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int off = 0;
+    for (int g = 0; g < G; ++g) {
+      sh_seg[g] = off;
+      seg_off[g] = off;
+      int cnt = 0;
+      for (int s = 0; s < nsub; ++s) {
+        key_off[g * nsub + s] = off + cnt;
+        cnt += key_cnt[g * nsub + s];
+      }
+      seg_cnt[g] = cnt;
+      off += (cnt + row_align - 1) / row_align * row_align;
+    }
+    sh_seg[G] = off;
+    seg_off[G] = off;
+    *n_rows = off;
+  }
+  __syncthreads();
+  const int ntile = sh_seg[G] / row_align;
+  for (int tile = threadIdx.x; tile < max_tiles; tile += blockDim.x) {
+    int g = -1;
+    if (tile < ntile) {
+      int row = tile * row_align;
+      g = 0;
+      while (g + 1 < G && sh_seg[g + 1] <= row) ++g;
+    }
+    tile_cluster[tile] = g;
+  }
+}
+
+__global__ void __launch_bounds__(kPermBlock)
+scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
+               const __half* __restrict__ x, const int* __restrict__ cluster_id,
+               const int* __restrict__ slot, const float* __restrict__ gates,
+               const int* __restrict__ keys, const int* __restrict__ block_base,
+               const int* __restrict__ key_off,
+               int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
+               __half* __restrict__ x_perm) {
+  extern __shared__ int sh_next[];   // next free row of each key for this block
+  for (int i = threadIdx.x; i < nkey; i += blockDim.x)
+    sh_next[i] = key_off[i] + block_base[(size_t)blockIdx.x * nkey + i];
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int t = blockIdx.x * kPermBlock + threadIdx.x;
+  const bool live = t < T;
+  const int key = live ? keys[t] : -1 - lane;     // dead lanes get unique keys: groups of one
+  const unsigned peers = __match_any_sync(0xffffffffu, key);
+  const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+  const bool leader = rank_in_warp == 0;
+  int row = -1;
+  // warps take their rows in warp order, so rows of a key stay in token order
+  for (int w = 0; w < kPermBlock / 32; ++w) {
+    if (warp == w && live) {
+      row = sh_next[key] + rank_in_warp;
+    }
+    __syncthreads();
+    if (warp == w && live && leader) sh_next[key] += __popc(peers);
+    __syncthreads();
+  }
+  if (live) {
+    int cs[kMaxKsel];
+    float cg[kMaxKsel];
+    canonical_slots(slot + (size_t)t * k, gates + (size_t)t * k, k, sub_is_combo, cs, cg);
+    const int g = cluster_id[t];
+    row_token[row] = t;
+#pragma unroll
+    for (int j = 0; j < kMaxKsel; ++j)
+      if (j < k) {
+        row_slot[(size_t)row * k + j] = g * K + cs[j];
+        row_gate[(size_t)row * k + j] = cg[j];
+      }
+  }
+  // row move: the warp copies its 32 tokens' rows one after the other, 16 bytes per lane
+  const int vec_per_row = d / 8;
+  for (int i = 0; i < 32; ++i) {
+    int src_t = __shfl_sync(0xffffffffu, t, i);
+    int dst_r = __shfl_sync(0xffffffffu, row, i);
+    if (dst_r < 0) continue;
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)src_t * d);
+    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)dst_r * d);
+    for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+  }
+}
+
+__global__ void __launch_bounds__(256)
+pad_kernel(int d, int K, int k, const int* __restrict__ seg_off, const int* __restrict__ seg_cnt,
+           int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
+           __half* __restrict__ x_perm) {
+  const int g = blockIdx.x;
+  const int first = seg_off[g] + seg_cnt[g], last = seg_off[g + 1];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int vec_per_row = d / 8;
+  for (int row = first + warp; row < last; row += nwarp) {
+    if (lane == 0) row_token[row] = -1;
+    if (lane < k) {
+      row_slot[(size_t)row * k + lane] = g * K + lane;   // any valid experts of the cluster
+      row_gate[(size_t)row * k + lane] = 0.f;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
+    for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st) {
+  const int nblk = (T + kPermBlock - 1) / kPermBlock;
+  const size_t sh = sizeof(int) * (size_t)D.nkey;
+  hist_kernel<<<nblk, kPermBlock, sh, st>>>(T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
+                                            S.slot, S.gates, S.keys, S.block_counts);
+  scan_kernel<<<1, 1024, 0, st>>>(nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
+                                  S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
+                                  S.seg_cnt, S.n_rows, S.tile_cluster);
+  scatter_kernel<<<nblk, kPermBlock, sh, st>>>(T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
+                                               S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
+                                               S.key_off, S.row_token, S.row_slot, S.row_gate,
+                                               S.x_perm);
+  pad_kernel<<<D.G, 256, 0, st>>>(D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
+                                  S.row_gate, S.x_perm);
+  return cudaGetLastError();
+}
+
+}  // namespace cmoe
