@@ -1,0 +1,387 @@
+#!/usr/bin/env python
+"""Benchmark of the clustered-MoE layer forward (cmoe_forward through the C ABI).
+
+A step is one pass of the whole hot path (router, permutation, expert FFNs with the fused
+residuals, gated combine, un-permute) over one batch of synthetic tokens.  Default workload: the
+GPT-2-medium-shaped layer (T=16384, d=1024, d_ff=4096, E=32, G=8, r=16, top-2), the compute-bound
+headline configuration; `--all` adds one short line per other workload under "workloads".
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all] [--impl reference]
+
+Prints ONE JSON line on rank 0.  With N > 1 (torchrun) every rank runs an independent replica of
+the same layer on its own GPU and token batch ("replicas only": the path has no exchange step).
+`--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2510_02345_b200 import inputs  # noqa: E402
+
+METRIC = "clustered_moe_layer_fwd_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_FP16_TFLOPS = 2250.0   # dense, vendor figure
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ------------------------------------------------------------------ algorithmic work of the method
+def algorithmic_work(s, T, active_clusters, active_experts):
+    """Flops and bytes the factored method must do (base once per token, G+K router logits)."""
+    d, f, r, k, G, K, E = s.d, s.d_ff, s.r, s.k, s.G, s.K, s.E
+    flops = 4 * T * d * f + 4 * k * T * r * (d + f) + 2 * T * d * (G + K)
+    nbytes = 2 * (2 * d * f) * active_clusters + (2 * r * (d + f)) * (0.5 + 2 / 32) * active_experts \
+        + 4 * d * (G + E) + 2 * T * d * 2
+    return float(flops), float(nbytes)
+
+
+def stage_work(s, T, stage, active_clusters, active_experts):
+    """(flops, bytes) of one stage's own algorithmic share (used for the dominant kernel)."""
+    d, f, r, k = s.d, s.d_ff, s.r, s.k
+    if stage == "up":      # x B1 + t V1 + a U2 ; reads x, B1, V1, U2 ; its output abar is an intermediate
+        return (2 * T * f * (d + 2 * k * r),
+                2 * d * f * active_clusters + 2 * r * f * 0.5625 * active_experts + 2 * T * d)
+    if stage == "down":    # abar B2 + s V2 ; reads B2, V2 ; writes y
+        return (2 * T * d * (f + k * r),
+                2 * d * f * active_clusters + r * d * 0.5625 * active_experts + 2 * T * d)
+    return (0.0, 0.0)
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thr = None
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 7:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thr = threading.Thread(target=self._run, daemon=True)
+        self._thr.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thr.join(timeout=10)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm = [float(p[0]) for p in self.samples]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(p[3 + i].lower().startswith("active") for p in self.samples)]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(self.samples[0][1]),
+                "power_w_max": max(float(p[2]) for p in self.samples), "reasons": reasons,
+                "samples": len(self.samples)}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ the CUDA arm
+def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks, dev_index, sync_ranks=True):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer, cmoe_profile_enable, cmoe_profile_read
+    s = inputs.CONFIGS[name]
+    L = inputs.make_layer(s, seed=0)
+    x_np = L["x"] if seed_offset == 0 else inputs.make_tokens(s, s.T, seed=seed_offset)
+    dev = torch.device(f"cuda:{dev_index}")
+    torch.cuda.set_device(dev)
+    m = ClusteredMoELayer(L, device=str(dev))
+    T = x_np.shape[0]
+    x = torch.from_numpy(x_np).to(dev)
+    y = torch.empty_like(x)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+    stream = torch.cuda.current_stream(dev)
+
+    cid, eid, _ = m.route(x)
+    torch.cuda.synchronize(dev)
+    active_clusters = int(torch.unique(cid).numel())
+    active_experts = int(torch.unique(eid).numel())
+    loads = torch.bincount(eid.flatten().long(), minlength=s.E).float()
+    i_load = float(loads.std(unbiased=False) / loads.mean())
+
+    for _ in range(max(3, warmup)):
+        flush.zero_()
+        m.forward(x, out=y)
+    torch.cuda.synchronize(dev)
+
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    sampler = ClockSampler(dev_index) if want_clocks else None
+    if sampler:
+        sampler.__enter__()
+        time.sleep(0.25)
+    if sync_ranks:
+        barrier()
+    torch.cuda.synchronize(dev)
+    t0 = time.perf_counter()
+    for i in range(steps):
+        flush.zero_()                      # L2 flush, outside the per-step events
+        starts[i].record(stream)
+        m.forward(x, out=y)
+        ends[i].record(stream)
+    torch.cuda.synchronize(dev)
+    if sync_ranks:
+        barrier()
+    wall = time.perf_counter() - t0
+    if sampler:
+        time.sleep(0.1)
+        sampler.__exit__()
+    assert m.status() == 0
+    per_step = [starts[i].elapsed_time(ends[i]) for i in range(steps)]
+    dev_ms = sum(per_step)
+
+    # stage times: a second pass of the same steps with the library's stage events on
+    cmoe_profile_enable(m.handle, True)
+    stage_ms = {}
+    for _ in range(steps):
+        flush.zero_()
+        m.forward(x, out=y)
+        for k_, v in cmoe_profile_read(m.handle).items():
+            stage_ms[k_] = stage_ms.get(k_, 0.0) + v / steps
+    cmoe_profile_enable(m.handle, False)
+
+    e2e = None
+    if want_e2e:
+        xh = torch.from_numpy(x_np).pin_memory()
+        yh = torch.empty((T, s.d), dtype=torch.float16).pin_memory()
+        xd = torch.empty_like(x)
+        for _ in range(2):
+            xd.copy_(xh, non_blocking=True); m.forward(xd, out=y); yh.copy_(y, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(3, min(steps, 20))
+        tot = 0.0
+        for _ in range(n_e2e):
+            flush.zero_()
+            e0.record(stream)
+            xd.copy_(xh, non_blocking=True)          # host -> device, pinned
+            m.forward(xd, out=y)
+            yh.copy_(y, non_blocking=True)           # device -> host
+            e1.record(stream)
+            e1.synchronize()
+            tot += e0.elapsed_time(e1)
+        e2e = {"ms_per_step": tot / n_e2e, "h2d_bytes_per_step": int(xh.numel() * 2),
+               "d2h_bytes_per_step": int(yh.numel() * 2), "steps": n_e2e}
+
+    res = dict(name=name, shape=s, T=T, dev_ms=dev_ms, steps=steps, wall_s=wall, per_step=per_step,
+               stage_ms=stage_ms, active_clusters=active_clusters, active_experts=active_experts,
+               i_load=i_load, info=m.info, e2e=e2e, clocks=sampler.summary() if sampler else None)
+    m.close()
+    del m, x, y, flush
+    torch.cuda.empty_cache()
+    return res
+
+
+_dist = None
+
+
+def barrier():
+    if _dist is not None:
+        _dist.barrier()
+
+
+def roofline_for(res, peaks, peaks_kind):
+    s, T = res["shape"], res["T"]
+    stage = max(("up", "down"), key=lambda n: res["stage_ms"].get(n, 0.0))
+    ms = res["stage_ms"][stage]
+    flops, nbytes = stage_work(s, T, stage, res["active_clusters"], res["active_experts"])
+    intensity = flops / max(nbytes, 1.0)
+    if intensity > 300:           # ridge of the B200 is ~250 flop/B
+        peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        ach = flops / (ms * 1e-3) / 1e12
+        return {"bound": "tensor", "kernel": stage, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                "frac": ach / peak, "traffic": None, "peak_kind": f"{peaks_kind} cuBLAS bf16 sustained (fp16 has the same rate)",
+                "kernel_ms": ms, "flops_per_launch": flops}
+    peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    ach = nbytes / (ms * 1e-3) / 1e9
+    return {"bound": "hbm", "kernel": stage, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+            "traffic": None, "peak_kind": f"{peaks_kind} copy bandwidth", "kernel_ms": ms,
+            "bytes_per_launch": nbytes}
+
+
+def whole_layer_fractions(res, n_gpus):
+    s, T = res["shape"], res["T"]
+    flops, nbytes = algorithmic_work(s, T, res["active_clusters"], res["active_experts"])
+    sec = res["dev_ms"] / res["steps"] * 1e-3
+    return {"algorithmic_tflops": flops / sec / 1e12, "algorithmic_gbs": nbytes / sec / 1e9,
+            "frac_of_nominal_fp16_2250T": flops / sec / 1e12 / NOMINAL_FP16_TFLOPS,
+            "frac_of_nominal_hbm_8TBs": nbytes / sec / 1e9 / NOMINAL_HBM_GBS}
+
+
+# ------------------------------------------------------------------ the CPU oracle arm
+def oracle_rate(name, target_s=15.0, max_tokens=None):
+    """tokens/s of the CPU oracle on a bounded sample (first n tokens) of the workload."""
+    from oracle import ref
+    s = inputs.CONFIGS[name]
+    L = inputs.make_layer(s, seed=0)
+    o = ref.Layer(L)
+    T = L["x"].shape[0]
+    probe = min(T, 64)
+    t0 = time.perf_counter(); o.forward(L["x"][:probe]); dt = time.perf_counter() - t0
+    n = int(min(T, max(probe, probe * target_s / max(dt, 1e-3))))
+    if max_tokens:
+        n = min(n, max_tokens)
+    n = max(1, n)
+    t0 = time.perf_counter(); o.forward(L["x"][:n]); dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": UNIT, "cores": ref.num_threads(), "kind": "oracle",
+            "sample": f"first {n} of {T} tokens of '{name}', one call, {dt:.1f} s, expert weights formed explicitly inside the timed call"}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from oracle import ref
+    name = args.workload
+    s = inputs.CONFIGS[name]
+    L = inputs.make_layer(s, seed=0)
+    o = ref.Layer(L)
+    T = L["x"].shape[0]
+    # size the per-step sample so that the whole run stays within a few minutes
+    probe = min(T, 64)
+    t0 = time.perf_counter(); o.forward(L["x"][:probe]); dt = time.perf_counter() - t0
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n = int(max(1, min(T, probe * budget / max(dt, 1e-3))))
+    for _ in range(args.warmup):
+        o.forward(L["x"][:n])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        o.forward(L["x"][:n])
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": name, "T": T, "d": s.d, "d_ff": s.d_ff, "E": s.E, "G": s.G, "r": s.r, "k": s.k,
+                       "sample_tokens_per_step": n},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": ref.num_threads(), "kind": "oracle",
+                             "sample": f"first {n} of {T} tokens per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ main
+def main():
+    global _dist
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="gpt2m", choices=list(inputs.CONFIGS))
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--all", action="store_true", help="also time the other four workloads (short runs)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+        _dist = dist
+
+    steps, warmup = args.steps, max(3, args.warmup)
+    res = time_workload(args.workload, steps, warmup, rank, seed_offset=rank, want_e2e=True,
+                        want_clocks=True, dev_index=local_rank)
+    dev_ms = res["dev_ms"]
+    e2e_ms = res["e2e"]["ms_per_step"]
+    if world > 1:
+        t = torch.tensor([dev_ms, e2e_ms], device=f"cuda:{local_rank}", dtype=torch.float64)
+        _dist.all_reduce(t, op=_dist.ReduceOp.MAX)     # timing only: max over ranks
+        dev_ms, e2e_ms = float(t[0]), float(t[1])
+    s, T = res["shape"], res["T"]
+    ms_per_step = dev_ms / steps
+    value = world * T / (ms_per_step * 1e-3)
+
+    if rank == 0:
+        peaks, kind = load_peaks()
+        roof = roofline_for(res, peaks, kind)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f16", "data": "synthetic",
+            "config": {"workload": args.workload, "T_per_gpu": T, "d": s.d, "d_ff": s.d_ff, "E": s.E, "G": s.G,
+                       "r": s.r, "k": s.k, "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": "flushed between steps by a 256 MB write outside the per-step CUDA events",
+                       "timing": "sum of per-step CUDA-event intervals on the launch stream",
+                       "path": int(res["info"].path),
+                       "active_clusters": res["active_clusters"], "active_experts": res["active_experts"],
+                       "expert_load_cov": res["i_load"]},
+            "clocks": res["clocks"],
+            "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": res["e2e"]["h2d_bytes_per_step"],
+                    "d2h_bytes_per_step": res["e2e"]["d2h_bytes_per_step"], "ms_per_step": e2e_ms},
+            "gpu_launches": int(res["info"].launches_forward) * steps,
+            "roofline": roof,
+            "layer": whole_layer_fractions(res, world),
+            "stage_ms": res["stage_ms"],
+            "wall_ms_per_step_incl_flush": res["wall_s"] / steps * 1e3,
+        }
+        if args.all:
+            others = {}
+            for name in inputs.CONFIG_ORDER:
+                if name == args.workload:
+                    continue
+                r2 = time_workload(name, max(5, steps // 3), 3, rank, 0, False, False, local_rank, sync_ranks=False)
+                ms2 = r2["dev_ms"] / r2["steps"]
+                others[name] = {"tokens_per_s": r2["T"] / (ms2 * 1e-3), "ms_per_step": ms2,
+                                "roofline": roofline_for(r2, peaks, kind), "layer": whole_layer_fractions(r2, 1),
+                                "stage_ms": r2["stage_ms"], "path": int(r2["info"].path),
+                                "active_clusters": r2["active_clusters"], "active_experts": r2["active_experts"]}
+            line["workloads"] = others
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = oracle_rate(args.workload)
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        _dist.barrier()
+        _dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

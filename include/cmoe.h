@@ -108,13 +108,25 @@ int cmoe_status(cmoe_layer* layer, void* cuda_stream);
 /* Per-handle facts for tests and benchmarks (host struct, filled by cmoe_get_info). */
 typedef struct {
   int32_t path;              /* 0 generic CUDA-core path, 1 tcgen05 grouped-GEMM path, 2 weight-streaming path */
-  int32_t launches_route;    /* kernels + memsets one cmoe_route call enqueues                     */
-  int32_t launches_forward;  /* kernels + memsets one cmoe_forward call enqueues                   */
+  int32_t launches_route;    /* kernel launches one cmoe_route call enqueues                       */
+  int32_t launches_forward;  /* kernel launches one cmoe_forward call enqueues (memsets excluded)  */
   int32_t row_align;         /* permuted-row alignment of a cluster segment                        */
   int32_t T_pad_max;         /* rows of the permuted activations buffers                           */
-  int32_t reserved[3];
+  int32_t memsets_forward;   /* cudaMemsetAsync calls one cmoe_forward enqueues                    */
+  int32_t n_stages;          /* stages cmoe_profile_read reports for this handle                   */
+  int32_t reserved[1];
 } cmoe_info;
 int cmoe_get_info(const cmoe_layer* layer, cmoe_info* out);
+
+/* Stage timing for benchmarks.  While enabled, cmoe_forward records a CUDA event on the stream
+ * before each of its stages and after the last one (no synchronisation).  cmoe_profile_read waits
+ * for the last recorded forward and writes the milliseconds of each stage of that call to
+ * stage_ms[0..n_stages-1] (n_stages <= CMOE_MAX_STAGES); cmoe_stage_name names a stage, or returns
+ * NULL past the last one.  Enabling creates the events; it allocates no device memory. */
+#define CMOE_MAX_STAGES 8
+int cmoe_profile_enable(cmoe_layer* layer, int on);
+int cmoe_profile_read(cmoe_layer* layer, float* stage_ms, int32_t* n_stages);
+const char* cmoe_stage_name(const cmoe_layer* layer, int32_t stage);
 
 /* cudaError_t (as int) of the last failed CUDA call on this handle, 0 if none. */
 int cmoe_last_cuda_error(const cmoe_layer* layer);

@@ -21,7 +21,9 @@ ERRORS = {
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
 EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_status",
-           "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror"]
+           "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
+           "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name"]
+CMOE_MAX_STAGES = 8
 
 
 class CmoeError(RuntimeError):
@@ -38,8 +40,8 @@ class cmoe_desc(C.Structure):
 
 
 class cmoe_info(C.Structure):
-    _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max")] + [
-        ("reserved", C.c_int32 * 3)]
+    _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max",
+                                         "memsets_forward", "n_stages")] + [("reserved", C.c_int32 * 1)]
 
 
 _lib = None
@@ -64,8 +66,12 @@ def lib():
         L.cmoe_destroy.argtypes = [C.c_void_p]
         L.cmoe_strerror.argtypes = [C.c_int]
         L.cmoe_strerror.restype = C.c_char_p
+        L.cmoe_profile_enable.argtypes = [C.c_void_p, C.c_int]
+        L.cmoe_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
+        L.cmoe_stage_name.argtypes = [C.c_void_p, C.c_int32]
+        L.cmoe_stage_name.restype = C.c_char_p
         for name in EXPORTS:
-            if name != "cmoe_strerror":
+            if name not in ("cmoe_strerror", "cmoe_stage_name"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -109,6 +115,18 @@ def cmoe_get_info(handle) -> cmoe_info:
     info = cmoe_info()
     _check(lib().cmoe_get_info(handle, C.byref(info)), "cmoe_get_info")
     return info
+
+
+def cmoe_profile_enable(handle, on: bool):
+    _check(lib().cmoe_profile_enable(handle, 1 if on else 0), "cmoe_profile_enable")
+
+
+def cmoe_profile_read(handle) -> dict:
+    """{stage name: milliseconds} of the last profiled cmoe_forward on this handle."""
+    ms = (C.c_float * CMOE_MAX_STAGES)()
+    n = C.c_int32(0)
+    _check(lib().cmoe_profile_read(handle, ms, C.byref(n)), "cmoe_profile_read")
+    return {lib().cmoe_stage_name(handle, i).decode(): float(ms[i]) for i in range(n.value)}
 
 
 def cmoe_destroy(handle):

@@ -157,7 +157,15 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   L->dims = D;
   L->path = kPathGeneric;
   L->last_cuda_error = 0;
-  L->host_status = nullptr;
+  L->profiling = 0;
+  L->events_created = 0;
+  L->events_recorded = 0;
+  L->n_stages = 5;
+  L->stage_names[0] = "router";
+  L->stage_names[1] = "permute";
+  L->stage_names[2] = "residual_t";
+  L->stage_names[3] = "up";
+  L->stage_names[4] = "down";
   Arena A;
   A.base = static_cast<char*>(desc->workspace);
   plan(D, A, &L->w, &L->sc);
@@ -228,11 +236,24 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   const Dims& D = L->dims;
   const Scratch& S = L->sc;
   const __half* xh = static_cast<const __half*>(x);
+  int stage = 0;
+#define CMOE_MARK()                                                        \
+  do {                                                                     \
+    if (L->profiling) CMOE_CUDA(L, cudaEventRecord(L->events[stage], st)); \
+    ++stage;                                                               \
+  } while (0)
+  CMOE_MARK();
   CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  CMOE_MARK();
   CMOE_CUDA(L, launch_permute(D, S, xh, T, st));
   if (D.r > 0)
     CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
-  CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st));
+  CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st,
+                                  L->profiling ? L->events + stage : nullptr));
+  stage += 3;
+  CMOE_MARK();   // end of the last stage
+#undef CMOE_MARK
+  if (L->profiling) L->events_recorded = 1;
   return CMOE_OK;
 }
 
@@ -255,17 +276,47 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   *out = cmoe_info{};
   out->path = L->path;
   out->launches_route = 1;
-  out->launches_forward = 1 + kPermuteLaunches + (L->dims.r > 0 ? 1 : 0) +
+  out->launches_forward = 1 + kPermuteLaunches +
                           (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1);
+  out->memsets_forward = L->dims.r > 0 ? 1 : 0;
+  out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;
   out->T_pad_max = L->dims.T_pad_max;
   return CMOE_OK;
+}
+
+int cmoe_profile_enable(cmoe_layer* L, int on) {
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  if (on && !L->events_created) {
+    for (int i = 0; i <= CMOE_MAX_STAGES; ++i) CMOE_CUDA(L, cudaEventCreate(&L->events[i]));
+    L->events_created = 1;
+  }
+  L->profiling = on ? 1 : 0;
+  L->events_recorded = 0;
+  return CMOE_OK;
+}
+
+int cmoe_profile_read(cmoe_layer* L, float* stage_ms, int32_t* n_stages) {
+  if (!L || !stage_ms || !n_stages) return CMOE_ERR_INVALID_ARG;
+  if (!L->events_created || !L->events_recorded) return CMOE_ERR_INVALID_ARG;
+  CMOE_CUDA(L, cudaEventSynchronize(L->events[L->n_stages]));
+  for (int i = 0; i < L->n_stages; ++i)
+    CMOE_CUDA(L, cudaEventElapsedTime(&stage_ms[i], L->events[i], L->events[i + 1]));
+  *n_stages = L->n_stages;
+  return CMOE_OK;
+}
+
+const char* cmoe_stage_name(const cmoe_layer* L, int32_t stage) {
+  if (!L || stage < 0 || stage >= L->n_stages) return nullptr;
+  return L->stage_names[stage];
 }
 
 int cmoe_last_cuda_error(const cmoe_layer* L) { return L ? L->last_cuda_error : 0; }
 
 int cmoe_destroy(cmoe_layer* L) {
   if (!L) return CMOE_ERR_INVALID_ARG;
+  if (L->events_created)
+    for (int i = 0; i <= CMOE_MAX_STAGES; ++i) cudaEventDestroy(L->events[i]);
   delete L;
   return CMOE_OK;
 }

@@ -77,7 +77,13 @@ struct cmoe_layer {
   cmoe::Scratch sc;
   int path;
   int last_cuda_error;
-  int* host_status;   // pinned? plain host word used by cmoe_status
+  // optional stage timing (cmoe_profile_*)
+  int profiling;
+  int n_stages;
+  const char* stage_names[CMOE_MAX_STAGES];
+  cudaEvent_t events[CMOE_MAX_STAGES + 1];
+  int events_created;
+  int events_recorded;
 };
 
 namespace cmoe {
@@ -94,8 +100,9 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st);
 constexpr int kPermuteLaunches = 4;
 // generic_path.cu : CUDA-core path for any supported shape
+// `marks` (or null): three events recorded before the residual-t, up and down stages
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,
-                               cudaStream_t st);
+                               cudaStream_t st, cudaEvent_t* marks);
 constexpr int kGenericFfnLaunches = 3;
 // repack.cu : create-time layout changes
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
