@@ -131,6 +131,34 @@ const char* cmoe_stage_name(const cmoe_layer* layer, int32_t stage);
 /* cudaError_t (as int) of the last failed CUDA call on this handle, 0 if none. */
 int cmoe_last_cuda_error(const cmoe_layer* layer);
 
+/* Routing for callers that cannot allocate device memory at all.  (The paper has no counterpart
+ * of this call; it exists for integration reasons only.)
+ *
+ * cmoe_route needs a handle, and a handle needs an arena that somebody allocated.  Code that runs
+ * where allocation is off the table - a plugin inside a host application whose GPU memory pool is
+ * frozen after start-up, a dispatcher that must place tokens before any layer has been created -
+ * can call this instead.  It takes the router exactly as cmoe_desc describes it (C [d][G],
+ * R [G][d][K], optional b_c [G] and b_e [G][K], all device pointers) plus x = fp16 [T][d], and
+ * writes the same three outputs as cmoe_route, with identity expert labels.  Its only scratch is a
+ * fixed array of CMOE_ROUTE_STATIC_BYTES inside the library image, which every GPU that loads the
+ * library holds until the process exits; it calls no cudaMalloc/cudaFree and no allocating library
+ * routine.
+ *
+ *   - Limit: 4*(G+E)*d bytes of router plus a few KB must fit in the array; a larger router is
+ *     rejected with CMOE_ERR_WORKSPACE_TOO_SMALL before anything is launched.  The shape rules of
+ *     cmoe_desc for d, E, G, k apply (CMOE_ERR_UNSUPPORTED_SHAPE otherwise).
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the array.  Each call rewrites everything it reads, so calls in
+ *     stream order are independent of each other, but two calls whose GPU work overlaps (issued
+ *     on different streams without ordering) race and give undefined routes.
+ *   - Asynchronous on the given stream like cmoe_route; T == 0 is a successful no-op. */
+#define CMOE_ROUTE_STATIC_BYTES (2u << 20)
+int cmoe_route_static(int32_t d, int32_t E, int32_t G, int32_t k,
+                      const float* C, const float* R, const float* b_c, const float* b_e,
+                      const void* x, int32_t T,
+                      int32_t* cluster_id, int32_t* expert_ids, float* gates, void* cuda_stream);
+
 /* Frees the host object.  The arena is the caller's. */
 int cmoe_destroy(cmoe_layer* layer);
 

@@ -22,7 +22,7 @@ ERRORS = {
 }
 EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
-           "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name"]
+           "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
 CMOE_MAX_STAGES = 8
 
 
@@ -70,6 +70,7 @@ def lib():
         L.cmoe_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_float), C.POINTER(C.c_int32)]
         L.cmoe_stage_name.argtypes = [C.c_void_p, C.c_int32]
         L.cmoe_stage_name.restype = C.c_char_p
+        L.cmoe_route_static.argtypes = [C.c_int32] * 4 + [C.c_void_p] * 5 + [C.c_int32] + [C.c_void_p] * 4
         for name in EXPORTS:
             if name not in ("cmoe_strerror", "cmoe_stage_name"):
                 getattr(L, name).restype = C.c_int
@@ -127,6 +128,14 @@ def cmoe_profile_read(handle) -> dict:
     n = C.c_int32(0)
     _check(lib().cmoe_profile_read(handle, ms, C.byref(n)), "cmoe_profile_read")
     return {lib().cmoe_stage_name(handle, i).decode(): float(ms[i]) for i in range(n.value)}
+
+
+def cmoe_route_static(d: int, E: int, G: int, k: int, C_ptr, R_ptr, b_c_ptr, b_e_ptr, x_ptr, T: int,
+                      cluster_id_ptr, expert_ids_ptr, gates_ptr, stream: int):
+    """Handle-free routing for callers that cannot allocate: the library's fixed device array is
+    the only scratch (see include/cmoe.h).  Raises CmoeError on a non-zero return code."""
+    _check(lib().cmoe_route_static(d, E, G, k, C_ptr, R_ptr, b_c_ptr, b_e_ptr, x_ptr, T,
+                                   cluster_id_ptr, expert_ids_ptr, gates_ptr, stream), "cmoe_route_static")
 
 
 def cmoe_destroy(handle):
