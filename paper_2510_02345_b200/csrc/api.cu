@@ -1,5 +1,6 @@
 // The C boundary of libcmoe (include/cmoe.h): descriptor validation, the arena plan, weight
 // re-layout at create time and the launch sequences of cmoe_route / cmoe_forward.
+#include <cstdlib>
 #include <new>
 
 #include "cmoe_internal.h"
@@ -211,6 +212,14 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   }
   if ((e = cudaMemsetAsync(L->sc.status, 0, sizeof(int), st))) return fail(e);
   if ((e = cudaStreamSynchronize(st))) return fail(e);
+  // path choice: tensor-core grouped GEMMs when the shape allows and there are enough tokens to
+  // fill 128-row tiles; CMOE_FORCE_PATH=0 keeps the generic path (for A/B checks)
+  const char* force = std::getenv("CMOE_FORCE_PATH");
+  const int forced = force ? std::atoi(force) : -1;
+  if (tc_supported(D) && D.T_max > 128 && forced != kPathGeneric) {
+    if ((e = tc_init(L))) return fail(e);
+    L->path = kPathTensor;
+  }
   *out_layer = L;
   return CMOE_OK;
 }
@@ -248,8 +257,11 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   CMOE_CUDA(L, launch_permute(D, S, xh, T, st));
   if (D.r > 0)
     CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
-  CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st,
-                                  L->profiling ? L->events + stage : nullptr));
+  if (L->path == kPathTensor)
+    CMOE_CUDA(L, launch_tc_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
+  else
+    CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st,
+                                    L->profiling ? L->events + stage : nullptr));
   stage += 3;
   CMOE_MARK();   // end of the last stage
 #undef CMOE_MARK

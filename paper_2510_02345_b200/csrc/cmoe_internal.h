@@ -84,6 +84,8 @@ struct cmoe_layer {
   cudaEvent_t events[CMOE_MAX_STAGES + 1];
   int events_created;
   int events_recorded;
+  // tensor-core path: tensor maps and launch shapes (opaque here, see tc_path.cu)
+  alignas(128) unsigned char tc_state[1024];
 };
 
 namespace cmoe {
@@ -104,6 +106,12 @@ constexpr int kPermuteLaunches = 4;
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,
                                cudaStream_t st, cudaEvent_t* marks);
 constexpr int kGenericFfnLaunches = 3;
+// t = x_perm U1_e for every permuted row and kept expert (no-op when r == 0)
+cudaError_t launch_residual_t(const Dims& D, const Weights& W, const Scratch& S, int T, cudaStream_t st);
+// tc_path.cu : tcgen05/TMEM/TMA grouped GEMMs with the fused epilogues
+bool tc_supported(const Dims& D);
+cudaError_t tc_init(cmoe_layer* L);
+cudaError_t launch_tc_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // repack.cu : create-time layout changes
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
                                   cudaStream_t st);

@@ -185,16 +185,22 @@ ffn_tile_kernel(int Kd, int N, int K, int k, int r, int row_align,
 
 }  // namespace
 
+cudaError_t launch_residual_t(const Dims& D, const Weights& W, const Scratch& S, int T, cudaStream_t st) {
+  if (D.r <= 0) return cudaSuccess;
+  const int rows_bound = t_pad_bound(D, T);
+  int blocks = (rows_bound * D.k + 7) / 8;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  residual_t_kernel<<<blocks, 256, 0, st>>>(D.d, D.k, D.r, S.n_rows, S.x_perm, S.row_slot, W.U1q,
+                                            W.U1s, S.t);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,
                                cudaStream_t st, cudaEvent_t* marks) {
   const int rows_bound = t_pad_bound(D, T);
   if (marks) cudaEventRecord(marks[0], st);
-  if (D.r > 0) {
-    int blocks = (rows_bound * D.k + 7) / 8;
-    if (blocks > 148 * 16) blocks = 148 * 16;
-    residual_t_kernel<<<blocks, 256, 0, st>>>(D.d, D.k, D.r, S.n_rows, S.x_perm, S.row_slot, W.U1q,
-                                              W.U1s, S.t);
-  }
+  cudaError_t e0 = launch_residual_t(D, W, S, T, st);
+  if (e0 != cudaSuccess) return e0;
   if (marks) cudaEventRecord(marks[1], st);
   dim3 gu((D.d_ff + BN - 1) / BN, rows_bound / BM);
   ffn_tile_kernel<true><<<gu, 256, 0, st>>>(D.d, D.d_ff, D.K, D.k, D.r, D.row_align, S.n_rows,

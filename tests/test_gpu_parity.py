@@ -160,3 +160,34 @@ def test_permutation_equivariance_on_gpu():
     torch.cuda.synchronize()
     # rows move with their tokens (summation order of the rank-r partials may differ slightly)
     assert torch.allclose(yp, y[perm], atol=2e-3, rtol=1e-3)
+
+
+# ---- shapes that take the tensor-core path (d, d_ff multiples of 128, T_max > 128) ----------------
+@pytest.mark.parametrize("T", [129, 200, 640, 1111])
+def test_tensor_path_ragged(T):
+    s = inputs.small_shape(T=T, d=128, d_ff=256, E=8, G=2, r=16, k=2)
+    L = inputs.make_layer(s, 12)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1
+
+
+@pytest.mark.parametrize("kw", [
+    dict(d=128, d_ff=384, E=8, G=2, r=0, k=2),
+    dict(d=256, d_ff=128, E=6, G=3, r=8, k=1),
+    dict(d=384, d_ff=256, E=16, G=2, r=32, k=2),     # K = 8, down tile 128 wide
+    dict(d=256, d_ff=512, E=4, G=4, r=4, k=1),       # one expert per cluster
+    dict(d=512, d_ff=256, E=12, G=3, r=16, k=2),     # down tile 256 wide
+], ids=["r0", "r8k1", "K8r32", "K1r4", "bn256"])
+def test_tensor_path_variants(kw):
+    s = inputs.small_shape(T=700, **kw)
+    L = inputs.make_layer(s, 13)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1
+
+
+def test_tensor_path_empty_cluster():
+    s = inputs.small_shape(T=400, d=128, d_ff=256, E=12, G=3, r=16, k=2)
+    L = inputs.make_layer(s, 14)
+    L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1 and not np.any(got["cid"] == 1)
