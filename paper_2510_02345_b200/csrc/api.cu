@@ -52,6 +52,7 @@ int validate_dims(const cmoe_desc* desc, Dims* D) {
   if (D->nkey > kMaxKeys) return CMOE_ERR_UNSUPPORTED_SHAPE;
   D->row_align = 128;
   D->T_pad_max = t_pad_bound(*D, D->T_max);
+  D->tc2 = (tc2_supported(*D) && D->T_max > 128) ? 1 : 0;
   return CMOE_OK;
 }
 
@@ -97,6 +98,16 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   s.abar = A.take<__half>(P * f);
   s.s = A.take<float>(P * k * r + 4);
   s.status = A.take<int>(1);
+  if (D.tc2 && r > 0) {
+    s.U1f = A.take<__half>(G * 64 * d);
+    s.V1f = A.take<__half>(G * f * 64);
+    s.U2f = A.take<__half>(G * 64 * f);
+    s.V2f = A.take<__half>(G * d * 64);
+    s.A0 = A.take<__half>(P * 64);
+    s.Ad = A.take<__half>(P * 64);
+    s.As = A.take<__half>(P * 64);
+    s.tile_mask = A.take<int>(P / D.row_align * 2);
+  }
   if (W) *W = w;
   if (S) *S = s;
 }
@@ -216,9 +227,17 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   // fill 128-row tiles; CMOE_FORCE_PATH=0 keeps the generic path (for A/B checks)
   const char* force = std::getenv("CMOE_FORCE_PATH");
   const int forced = force ? std::atoi(force) : -1;
-  if (tc_supported(D) && D.T_max > 128 && forced != kPathGeneric) {
+  const char* variant = std::getenv("CMOE_TC_VARIANT");     // 1 keeps the CUDA-core residual epilogues
+  const int forced_variant = variant ? std::atoi(variant) : 0;
+  L->tc_variant = 0;
+  if (D.tc2 && forced != kPathGeneric && forced_variant != 1) {
+    if ((e = tc2_init(L))) return fail(e);
+    L->path = kPathTensor;
+    L->tc_variant = 2;
+  } else if (tc_supported(D) && D.T_max > 128 && forced != kPathGeneric) {
     if ((e = tc_init(L))) return fail(e);
     L->path = kPathTensor;
+    L->tc_variant = 1;
   }
   *out_layer = L;
   return CMOE_OK;
@@ -257,7 +276,9 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   CMOE_CUDA(L, launch_permute(D, S, xh, T, st));
   if (D.r > 0)
     CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
-  if (L->path == kPathTensor)
+  if (L->path == kPathTensor && L->tc_variant == 2)
+    CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
+  else if (L->path == kPathTensor)
     CMOE_CUDA(L, launch_tc_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else
     CMOE_CUDA(L, launch_generic_ffn(D, L->w, S, T, static_cast<__half*>(y), st,
@@ -289,7 +310,9 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->path = L->path;
   out->launches_route = 1;
   out->launches_forward = 1 + kPermuteLaunches +
-                          (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1);
+                          (L->path == kPathTensor && L->tc_variant == 2
+                               ? tc2_launch_count(L->dims)
+                               : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
   out->memsets_forward = L->dims.r > 0 ? 1 : 0;
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;

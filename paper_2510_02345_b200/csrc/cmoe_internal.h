@@ -27,6 +27,7 @@ struct Dims {
   int T_pad_max;   // rows of the permuted buffers
   int row_align;   // a cluster's rows start at a multiple of this
   int sub_is_combo;
+  int tc2;         // the shape takes the tensor-core path with tensor-core residuals (tc2_path.cu)
 };
 
 // Weights as re-laid-out in the arena by cmoe_create.
@@ -67,6 +68,10 @@ struct Scratch {
   __half* abar;       // [T_pad][d_ff]   sum_j p_j GELU(h_j)
   float* s;           // [T_pad][k][r]   GELU(h_j) U2_e, accumulated with atomics
   int* status;        // [1]
+  // tensor-core path with tensor-core residuals only (see tc2_path.cu)
+  __half *U1f, *V1f, *U2f, *V2f;   // INT4 factors decoded to fp16 operand matrices, per call
+  __half *A0, *Ad, *As;            // [T_pad][64] expanded-rank-index operands
+  int* tile_mask;                  // [T_pad / 128][2]
 };
 
 }  // namespace cmoe
@@ -76,6 +81,7 @@ struct cmoe_layer {
   cmoe::Weights w;
   cmoe::Scratch sc;
   int path;
+  int tc_variant;   // 1: tc_path.cu, 2: tc2_path.cu (when path == kPathTensor)
   int last_cuda_error;
   // optional stage timing (cmoe_profile_*)
   int profiling;
@@ -85,7 +91,7 @@ struct cmoe_layer {
   int events_created;
   int events_recorded;
   // tensor-core path: tensor maps and launch shapes (opaque here, see tc_path.cu)
-  alignas(128) unsigned char tc_state[1024];
+  alignas(128) unsigned char tc_state[2048];
 };
 
 namespace cmoe {
@@ -112,6 +118,11 @@ cudaError_t launch_residual_t(const Dims& D, const Weights& W, const Scratch& S,
 bool tc_supported(const Dims& D);
 cudaError_t tc_init(cmoe_layer* L);
 cudaError_t launch_tc_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
+// tc2_path.cu : the same with the rank-r residual products on the tensor cores as well
+bool tc2_supported(const Dims& D);
+cudaError_t tc2_init(cmoe_layer* L);
+int tc2_launch_count(const Dims& D);
+cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // repack.cu : create-time layout changes
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
                                   cudaStream_t st);

@@ -1,0 +1,1024 @@
+// Tensor-core path of the expert FFNs with the rank-r residuals on the tensor cores as well
+// (sm_100a: tcgen05 MMAs with TMEM accumulators, operands staged in shared memory by TMA).
+//
+// The factored form of the text after Eq. 7, x W_e = x B_g + (x U_e) V_e, is kept, but every
+// rank-r product is phrased as a GEMM over an "expanded rank index" c = i*r + p (i = expert of the
+// cluster, p = rank), KE = 64 wide, so that one tile may mix rows routed to different experts:
+//
+//   stage   INT4 factors of the layer -> fp16 operand matrices in scratch (decoded in registers)
+//             U1f [G][KE][d]   V1f [G][d_ff][KE]   U2f [G][KE][d_ff]   V2f [G][d][KE]
+//   t       Tall = x_perm U1f_g^T (128 x KE per tile); row-wise selection writes
+//             A0 [row][c] = t of the row's first kept expert inside that expert's block, else 0
+//             Ad [row][c] = +t of the second kept expert in its block, -t of the first in its block
+//   up      P = x_perm B1_g^T + A0 V1f^T  (= h of the first expert),  Q = Ad V1f^T  (h_2 - h_1);
+//           epilogue: a_j = GELU(h_j), abar = sum_j p_j a_j (fp16 to HBM), a_j (fp16) to shared
+//           memory as the A operand of  S_j += a_j U2f^T  (accumulated in TMEM over the N tiles of
+//           a row tile, then the row's own block is added to s with fp32 atomics)
+//   expand  As [row][c] = p_j s_j inside the block of expert e_j (fp16)
+//   down    y = abar B2_g^T + As V2f^T, stored un-permuted
+//
+// The base product is computed once per token and shared by its k experts; the extra tensor work
+// is the KE-deep steps (skipped per tile for experts no row of the tile uses) and the S products.
+// Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
+// all roles leave their loops, TMEM is freed and the kernel returns.
+#include "cmoe_internal.h"
+#include "device_utils.cuh"
+#include "tc_ptx.cuh"
+
+namespace cmoe {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int BM = 128;          // rows per tile (UMMA M)
+constexpr int BK = 64;           // halves per K chunk: one 128-byte swizzle row
+constexpr int KE = 64;           // width of the expanded rank index
+constexpr int BN_UP = 128;
+constexpr uint32_t kTmemCols = 512;
+constexpr size_t kSmemLimit = 232448;   // 227 KB
+constexpr int kMaxStages = 8;
+
+// ------------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------------
+
+// all lanes wait; the warp agrees on the outcome so that it never diverges around .sync.aligned code
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __all_sync(0xffffffffu, ok);
+}
+
+// GELU(u) ~ u/2 (1 + tanh(u (c1 + c2 u^2))) with c1, c2 fitted to the erf form (max abs deviation
+// 2.7e-4 over the reals) and the hardware tanh (relative error 2^-11): below the fp16 rounding of
+// the stored activation.
+__device__ __forceinline__ float gelu_fast(float u) {
+  const float u2 = u * u;
+  const float w = fmaf(u2, 0.03470089f, 0.80015708f);
+  float th;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(u * w));
+  const float hu = 0.5f * u;
+  return fmaf(hu, th, hu);
+}
+
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+  __half2 h = __floats2half2_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&h);
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// stage: INT4 factors -> fp16 operand matrices (one thread per 32-bit word = 8 codes)
+// ------------------------------------------------------------------------------------------------
+struct FactorStage {
+  const uint8_t* q[4];     // U1, V1, U2, V2
+  const __half* s[4];
+  __half* dst[4];
+  long long words[4];      // 32-bit words of each packed factor
+  int dim[4];              // non-rank extent: d, d_ff, d_ff, d
+  int K, r;
+};
+
+__global__ void __launch_bounds__(256)
+stage_factors_kernel(const FactorStage fs) {
+  const int which = blockIdx.y;
+  const long long wd = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (wd >= fs.words[which]) return;
+  const int dim = fs.dim[which], K = fs.K, r = fs.r;
+  const uint32_t word = reinterpret_cast<const uint32_t*>(fs.q[which])[wd];
+  const long long flat0 = wd * 8;
+  const float sc = __half2float(fs.s[which][flat0 >> 5]);
+  __align__(16) __half v[8];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) v[n] = __float2half_rn((float)sext4((int)(word >> (4 * n))) * sc);
+  __half* dst = fs.dst[which];
+  if ((which & 1) == 0) {
+    // U [E][r][dim]: row (e, p) of length dim -> row g*KE + i*r + p
+    const long long row = flat0 / dim;
+    const int c = (int)(flat0 - row * dim);
+    const long long g = row / (K * r);
+    const int n = (int)(row - g * (K * r));
+    *reinterpret_cast<uint4*>(dst + ((g * KE + n) * dim + c)) = *reinterpret_cast<const uint4*>(v);
+  } else if (r >= 8) {
+    // V [E][dim][r]: (e, n, p0..p0+7) -> [g][n][i*r + p0 ..]
+    const long long en = flat0 / r;
+    const int p0 = (int)(flat0 - en * r);
+    const long long e = en / dim;
+    const int n = (int)(en - e * dim);
+    const long long g = e / K;
+    const int i = (int)(e - g * K);
+    *reinterpret_cast<uint4*>(dst + ((g * dim + n) * KE + i * r + p0)) = *reinterpret_cast<const uint4*>(v);
+  } else {
+    // r == 4: the word holds two output columns of four ranks each
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const long long en = (flat0 + 4 * h) / 4;
+      const long long e = en / dim;
+      const int n = (int)(en - e * dim);
+      const long long g = e / K;
+      const int i = (int)(e - g * K);
+      *reinterpret_cast<uint2*>(dst + ((g * dim + n) * KE + i * 4)) = reinterpret_cast<const uint2*>(v)[h];
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// t: Tall = x_perm U1f_g^T, one 128-row tile per CTA, then the row-wise selection into A0 / Ad
+// ------------------------------------------------------------------------------------------------
+struct TParams {
+  const int* n_rows;
+  const int* tile_cluster;
+  const int* row_slot;
+  const int* row_token;
+  __half* A0;          // [rows][KE]
+  __half* Ad;          // [rows][KE]  (k == 2 only)
+  int* tile_mask;      // [tiles][2]  16-wide steps of the expanded index used by slot 0 / slot 1
+  int* status;
+  int KC, K, r;
+};
+
+constexpr int T_THREADS = 192;
+constexpr int T_STAGES = 6;
+constexpr uint32_t T_STAGE_BYTES = BM * BK * 2 + KE * BK * 2;   // 24 KB
+
+template <int KSEL>
+__global__ void __launch_bounds__(T_THREADS, 1)
+tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU1,
+             const TParams p) {
+  const int mt = blockIdx.x;
+  if (mt >= *p.n_rows / BM) return;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)T_STAGES * T_STAGE_BYTES);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages), tfull = smem_u32(bars + 2 * kMaxStages);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* sh_mask = reinterpret_cast<int*>(tmem_holder + 2);     // [2]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < T_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(tfull, 1);
+    *abort_flag = 0;
+    sh_mask[0] = 0; sh_mask[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_holder)), "r"(64u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  const int g = p.tile_cluster[mt];
+  const int KC = p.KC;
+  bool failed = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      for (int kc = 0; kc < KC; ++kc) {
+        const uint32_t s = kc % T_STAGES, ph = (kc / T_STAGES) & 1u;
+        if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+        const uint32_t a_dst = base + s * T_STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
+        mbar_expect_tx(full0 + 8 * s, T_STAGE_BYTES);
+        tma_load_2d(a_dst, &tmX, full0 + 8 * s, kc * BK, mt * BM);
+        tma_load_2d(b_dst, &tmU1, full0 + 8 * s, kc * BK, g * KE);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = idesc_f16(BM, KE);
+      for (int kc = 0; kc < KC; ++kc) {
+        const uint32_t s = kc % T_STAGES, ph = (kc / T_STAGES) & 1u;
+        if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t a_src = base + s * T_STAGE_BYTES, b_src = a_src + BM * BK * 2;
+        const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+#pragma unroll
+        for (int ks = 0; ks < BK / 16; ++ks)
+          umma_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (kc | ks) != 0 ? 1u : 0u);
+        umma_commit(empty0 + 8 * s);
+      }
+      if (!failed) umma_commit(tfull);
+    }
+  } else {
+    const int q = warp & 3;
+    const int row = mt * BM + q * 32 + lane;
+    const int r = p.r;
+    const int lo0 = (p.row_slot[(size_t)row * KSEL] - g * p.K) * r;
+    const int lo1 = KSEL == 2 ? (p.row_slot[(size_t)row * KSEL + 1] - g * p.K) * r : -1;
+    const bool real = p.row_token[row] >= 0;
+    if (warp_wait(tfull, 0, abort_flag)) {
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t v[32];
+        tmem_ld32_nowait(taddr + half * 32, v);
+        tmem_ld_wait();
+        uint32_t o0[16], od[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          float a[2], dl[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const int cc = half * 32 + c + u;
+            const float t = __uint_as_float(v[c + u]);
+            const bool in0 = cc >= lo0 && cc < lo0 + r;
+            const bool in1 = KSEL == 2 && cc >= lo1 && cc < lo1 + r;
+            a[u] = in0 ? t : 0.f;
+            dl[u] = in1 ? t : (in0 ? -t : 0.f);
+          }
+          o0[c >> 1] = pack_half2(a[0], a[1]);
+          od[c >> 1] = pack_half2(dl[0], dl[1]);
+        }
+        uint4* d0 = reinterpret_cast<uint4*>(p.A0 + (size_t)row * KE + half * 32);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) d0[i] = make_uint4(o0[4 * i], o0[4 * i + 1], o0[4 * i + 2], o0[4 * i + 3]);
+        if (KSEL == 2) {
+          uint4* dd = reinterpret_cast<uint4*>(p.Ad + (size_t)row * KE + half * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dd[i] = make_uint4(od[4 * i], od[4 * i + 1], od[4 * i + 2], od[4 * i + 3]);
+        }
+      }
+      // 16-wide steps of the expanded index that rows of this tile use
+      int m0 = 0, m1 = 0;
+      if (real) {
+        for (int c = lo0; c < lo0 + r; c += (r < 16 ? r : 16)) m0 |= 1 << (c >> 4);
+        if (KSEL == 2)
+          for (int c = lo1; c < lo1 + r; c += (r < 16 ? r : 16)) m1 |= 1 << (c >> 4);
+      }
+      m0 = __reduce_or_sync(0xffffffffu, (unsigned)m0);
+      m1 = __reduce_or_sync(0xffffffffu, (unsigned)m1);
+      if (lane == 0) { atomicOr(&sh_mask[0], m0); atomicOr(&sh_mask[1], m1); }
+    } else {
+      failed = true;
+    }
+    tc_fence_before();
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
+  }
+  __syncthreads();
+  if (threadIdx.x == 64) { p.tile_mask[2 * mt] = sh_mask[0]; p.tile_mask[2 * mt + 1] = sh_mask[1]; }
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) { }    // let copies already issued land
+    __syncthreads();
+  }
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(64u) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// up
+// ------------------------------------------------------------------------------------------------
+struct Up2Params {
+  const int* n_rows;
+  const int* tile_cluster;
+  const int* tile_mask;
+  const int* row_slot;
+  const float* row_gate;
+  const int* row_token;
+  float* s_out;        // [rows][k][r] fp32, zeroed by the caller
+  __half* abar;        // [rows][N]
+  int* status;
+  int KC, NT, N, K, k, r, log2r;
+};
+
+constexpr int UP_THREADS = 352;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 S products
+constexpr uint32_t UP_STAGE_BYTES = BM * BK * 2 + BN_UP * BK * 2;   // 32 KB
+constexpr uint32_t A_CHUNK_BYTES = BM * BK * 2;                     // 16 KB: 128 rows x 64 activations
+constexpr uint32_t U2_TILE_BYTES = KE * BN_UP * 2;                  // 16 KB: two 64x64 chunks
+
+template <bool HAS_R, int KSEL>
+struct UpCfg {
+  static constexpr int STAGES = HAS_R ? 4 : 6;
+  static constexpr int NA = HAS_R ? 2 * KSEL : 1;          // activation chunks per tile = ring size
+  static constexpr int NEXT = HAS_R ? KSEL : 0;            // expanded-index chunks after the main loop
+  static constexpr uint32_t RING = STAGES * UP_STAGE_BYTES;
+  static constexpr uint32_t ARING = HAS_R ? NA * A_CHUNK_BYTES : 0;
+  static constexpr uint32_t U2 = HAS_R ? 2 * U2_TILE_BYTES : 0;
+  static constexpr uint32_t BAR_OFF = RING + ARING + U2;
+  static constexpr size_t SMEM = 1024 + BAR_OFF + 48 * 8;
+};
+
+template <bool HAS_R, int KSEL>
+__global__ void __launch_bounds__(UP_THREADS, 1)
+tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmB1,
+              const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmAd,
+              const __grid_constant__ CUtensorMap tmV1, const __grid_constant__ CUtensorMap tmU2,
+              const Up2Params p) {
+  using Cfg = UpCfg<HAS_R, KSEL>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  const uint32_t aring = base + Cfg::RING;
+  const uint32_t u2base = aring + Cfg::ARING;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Cfg::BAR_OFF);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
+  const uint32_t tfull0 = smem_u32(bars + 16), tempty0 = smem_u32(bars + 18), qempty = smem_u32(bars + 20);
+  const uint32_t afull0 = smem_u32(bars + 21), aempty0 = smem_u32(bars + 25);
+  const uint32_t u2full0 = smem_u32(bars + 29), u2empty0 = smem_u32(bars + 31);
+  const uint32_t sfull = smem_u32(bars + 33), sempty = smem_u32(bars + 34);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 36);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 8); }
+    mbar_init(qempty, 8);
+    for (int a = 0; a < 4; ++a) { mbar_init(afull0 + 8 * a, 4); mbar_init(aempty0 + 8 * a, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(u2full0 + 8 * a, 1); mbar_init(u2empty0 + 8 * a, 1); }
+    mbar_init(sfull, 1);
+    mbar_init(sempty, 4 * KSEL);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+  // TMEM columns: P (two buffers) 0..255, Q 256..383, S_0 384..447, S_1 448..511
+  const uint32_t tmem_q = tmem_base + 256, tmem_s = tmem_base + 384;
+
+  const int NT = p.NT, KC = p.KC;
+  const long long total = (long long)(*p.n_rows / BM) * NT;
+  const int w0 = (int)(total * blockIdx.x / gridDim.x);
+  const int w1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+  bool failed = false;
+
+  if (warp == 0) {
+    // ---------------- TMA producer: KC chunks of (x_perm, B1) then the expanded-index chunks
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int w = w0; w < w1 && !failed; ++w) {
+        const int mt = w / NT, nt = w - mt * NT;
+        const int g = p.tile_cluster[mt];
+        const int brow = g * p.N + nt * BN_UP;
+        for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
+          mbar_expect_tx(full0 + 8 * s, UP_STAGE_BYTES);
+          if (c < KC) {
+            tma_load_2d(a_dst, &tmX, full0 + 8 * s, c * BK, mt * BM);
+            tma_load_2d(b_dst, &tmB1, full0 + 8 * s, c * BK, brow);
+          } else {
+            tma_load_2d(a_dst, c == KC ? &tmA0 : &tmAd, full0 + 8 * s, 0, mt * BM);
+            tma_load_2d(b_dst, &tmV1, full0 + 8 * s, 0, brow);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer of P and Q
+    if (lane == 0) {
+      constexpr uint32_t IDESC = idesc_f16(BM, BN_UP);
+      uint32_t it = 0, tile_i = 0;
+      for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
+        const int mt = w / NT;
+        const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN_UP;
+        for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+          if (c == KC + 1) {
+            // Q has one buffer: the epilogue of the previous tile must have drained it
+            if (!mbar_wait(qempty, (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+            tc_fence_after();
+          }
+          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a_src = base + s * UP_STAGE_BYTES, b_src = a_src + BM * BK * 2;
+          const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+          if (c < KC) {
+#pragma unroll
+            for (int ks = 0; ks < BK / 16; ++ks)
+              umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
+          } else if (c == KC) {
+            const int m = p.tile_mask[2 * mt];
+#pragma unroll
+            for (int ks = 0; ks < KE / 16; ++ks)
+              if ((m >> ks) & 1) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+          } else {
+            int m = p.tile_mask[2 * mt] | p.tile_mask[2 * mt + 1];
+            if (m == 0) m = 1;           // Q must be written at least once (A is zero there)
+            uint32_t accum = 0;
+#pragma unroll
+            for (int ks = 0; ks < KE / 16; ++ks)
+              if ((m >> ks) & 1) { umma_f16(tmem_q, adesc + 2 * ks, bdesc + 2 * ks, IDESC, accum); accum = 1; }
+          }
+          umma_commit(empty0 + 8 * s);
+        }
+        if (failed) break;
+        umma_commit(tfull0 + 8 * acc);
+      }
+    }
+  } else if (warp == 10) {
+    // ---------------- S products: S_j += a_j U2f^T as the epilogue hands activation chunks over
+    if (HAS_R && lane == 0 && w0 < w1) {
+      constexpr uint32_t IDESC_S = idesc_f16(BM, KE);
+      auto load_u2 = [&](int w, uint32_t ti) -> bool {
+        const int mt = w / NT, nt = w - mt * NT;
+        const int g = p.tile_cluster[mt];
+        const uint32_t ub = ti & 1u, uph = (ti >> 1) & 1u;
+        if (!mbar_wait(u2empty0 + 8 * ub, uph ^ 1u, abort_flag)) return false;
+        const uint32_t dst = u2base + ub * U2_TILE_BYTES;
+        mbar_expect_tx(u2full0 + 8 * ub, U2_TILE_BYTES);
+        tma_load_2d(dst, &tmU2, u2full0 + 8 * ub, nt * BN_UP, g * KE);
+        tma_load_2d(dst + KE * BK * 2, &tmU2, u2full0 + 8 * ub, nt * BN_UP + BK, g * KE);
+        return true;
+      };
+      uint32_t tile_i = 0, flushes = 0;
+      bool fresh = true;                    // the next product of each slot overwrites S
+      uint32_t written = 0;                 // bit j: S_j has been written since the last flush
+      if (!load_u2(w0, 0)) failed = true;
+      for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
+        const int mt = w / NT;
+        if (w + 1 < w1 && !load_u2(w + 1, tile_i + 1)) { failed = true; break; }
+        const uint32_t ub = tile_i & 1u, uph = (tile_i >> 1) & 1u;
+        if (!mbar_wait(u2full0 + 8 * ub, uph, abort_flag)) { failed = true; break; }
+        if (fresh && flushes > 0) {
+          // the epilogue must have read the previous row tile's S before it is overwritten
+          if (!mbar_wait(sempty, (flushes - 1) & 1u, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+        }
+        if (fresh) { written = 0; fresh = false; }
+        for (int c = 0; c < 2 * KSEL; ++c) {
+          const uint32_t n = tile_i * (2 * KSEL) + c;
+          const uint32_t slot = n % Cfg::NA, aph = (n / Cfg::NA) & 1u;
+          if (!mbar_wait(afull0 + 8 * slot, aph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const int hf = c / KSEL, j = c - hf * KSEL;
+          const uint64_t adesc = umma_desc(aring + slot * A_CHUNK_BYTES);
+          const uint64_t bdesc = umma_desc(u2base + ub * U2_TILE_BYTES + hf * (KE * BK * 2));
+#pragma unroll
+          for (int ks = 0; ks < BK / 16; ++ks) {
+            umma_f16(tmem_s + j * KE, adesc + 2 * ks, bdesc + 2 * ks, IDESC_S, (written >> j) & 1u);
+            written |= 1u << j;
+          }
+          umma_commit(aempty0 + 8 * slot);
+        }
+        if (failed) break;
+        umma_commit(u2empty0 + 8 * ub);
+        const bool last_of_run = (w + 1 == w1) || ((w + 1) / NT != mt);
+        if (last_of_run) { umma_commit(sfull); fresh = true; ++flushes; }
+      }
+    }
+  } else {
+    // ---------------- epilogue warps: quadrant q of the TMEM lanes, column half hf of the tile
+    const int q = warp & 3;
+    const int hf = (warp - 2) >> 2;
+    const int rowc = q * 32 + lane;                        // row inside the tile
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    uint32_t tile_i = 0, flushes = 0;
+    for (int w = w0; w < w1; ++w, ++tile_i) {
+      const int mt = w / NT, nt = w - mt * NT;
+      const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
+      const int row = mt * BM + rowc;
+      const float g0 = p.row_gate[(size_t)row * p.k];
+      const float g1 = p.k == 2 ? p.row_gate[(size_t)row * p.k + 1] : 0.f;
+      if (!warp_wait(tfull0 + 8 * acc, aph, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int grp = 0; grp < 2; ++grp) {
+        const int col0 = hf * 64 + grp * 32;
+        uint32_t vp[32], vq[32];
+        tmem_ld32_nowait(taddr + acc * BN_UP + col0, vp);
+        if (HAS_R && KSEL == 2) tmem_ld32_nowait(taddr + 256 + col0, vq);
+        tmem_ld_wait();
+        if (HAS_R && grp == 0) {
+          // the S products that read this warp's chunk slots one tile ago must have finished
+          bool ok = true;
+#pragma unroll
+          for (int j = 0; j < KSEL; ++j) {
+            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+            ok = ok && mbar_wait(aempty0 + 8 * (n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
+          }
+          if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+        }
+        uint32_t ob[16], oa0[16], oa1[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          float ab[2], a0[2], a1[2];
+#pragma unroll
+          for (int u = 0; u < 2; ++u) {
+            const float h0 = __uint_as_float(vp[c + u]);
+            a0[u] = gelu_fast(h0);
+            if (HAS_R && KSEL == 2) {
+              a1[u] = gelu_fast(h0 + __uint_as_float(vq[c + u]));
+              ab[u] = fmaf(g1, a1[u], g0 * a0[u]);
+            } else {
+              a1[u] = 0.f;
+              ab[u] = (g0 + g1) * a0[u];
+            }
+          }
+          ob[c >> 1] = pack_half2(ab[0], ab[1]);
+          if (HAS_R) {
+            oa0[c >> 1] = pack_half2(a0[0], a0[1]);
+            if (KSEL == 2) oa1[c >> 1] = pack_half2(a1[0], a1[1]);
+          }
+        }
+        uint4* dst = reinterpret_cast<uint4*>(p.abar + (size_t)row * p.N + nt * BN_UP + col0);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
+        if (HAS_R) {
+          // a_j into its chunk as a K-major 128-byte-swizzled A operand: 16-byte unit u of row
+          // rowc sits at rowc*128 + ((u ^ (rowc & 7)) << 4)
+#pragma unroll
+          for (int j = 0; j < KSEL; ++j) {
+            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+            const uint32_t cb = aring + (n % Cfg::NA) * A_CHUNK_BYTES + rowc * 128;
+            const uint32_t* src = j == 0 ? oa0 : oa1;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t unit = (uint32_t)(grp * 4 + i);
+              st_shared_v4(cb + ((unit ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2],
+                           src[4 * i + 3]);
+            }
+          }
+        }
+      }
+      if (failed) break;
+      if (HAS_R) {
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+#pragma unroll
+          for (int j = 0; j < KSEL; ++j) {
+            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+            mbar_arrive(afull0 + 8 * (n % Cfg::NA));
+          }
+        }
+      }
+      // accumulators drained: hand P (and Q) back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(tempty0 + 8 * acc); mbar_arrive(qempty); }
+      const bool last_of_run = (w + 1 == w1) || ((w + 1) / NT != mt);
+      if (HAS_R && last_of_run) {
+        if (hf < KSEL) {
+          // S_hf is complete for this row tile: add the row's own expert block to s
+          if (!warp_wait(sfull, flushes & 1u, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const int g = p.tile_cluster[mt];
+          const int e = p.row_slot[(size_t)row * KSEL + hf] - g * p.K;
+          const bool real = p.row_token[row] >= 0;
+          float* srow = p.s_out + ((size_t)row * KSEL + hf) * p.r;
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            uint32_t v[32];
+            tmem_ld32_nowait(taddr + 384 + hf * KE + half * 32, v);
+            tmem_ld_wait();
+            if (real) {
+#pragma unroll
+              for (int c = 0; c < 32; ++c) {
+                const int cc = half * 32 + c;
+                if ((cc >> p.log2r) == e) atomicAdd(srow + (cc & (p.r - 1)), __uint_as_float(v[c]));
+              }
+            }
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sempty);
+        }
+        ++flushes;
+      }
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) { }    // let copies already issued land
+    __syncthreads();
+  }
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// expand: As[row][c] = sum_j [c in block of e_j] p_j s_j[c mod r]   (fp16)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_cluster,
+                const int* __restrict__ row_slot, const float* __restrict__ row_gate,
+                const float* __restrict__ s, __half* __restrict__ As, int K, int k, int r, int log2r) {
+  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+  const int row = idx >> 3, c0 = (idx & 7) * 8;
+  if (row >= *n_rows) return;
+  const int g = tile_cluster[row / BM];
+  __align__(16) __half out[8];
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const int c = c0 + n, i = c >> log2r, pr = c & (r - 1);
+    float v = 0.f;
+    for (int j = 0; j < k; ++j)
+      if (row_slot[(size_t)row * k + j] - g * K == i) v = fmaf(row_gate[(size_t)row * k + j], s[((size_t)row * k + j) * r + pr], v);
+    out[n] = __float2half_rn(v);
+  }
+  *reinterpret_cast<uint4*>(As + (size_t)row * KE + c0) = *reinterpret_cast<const uint4*>(out);
+}
+
+// ------------------------------------------------------------------------------------------------
+// down
+// ------------------------------------------------------------------------------------------------
+struct Down2Params {
+  const int* n_rows;
+  const int* tile_cluster;
+  const int* tile_mask;
+  const int* row_token;
+  __half* y;           // [T][N], original token order
+  int* status;
+  int KC, NT, N;
+};
+
+constexpr int DN_THREADS = 192;
+
+template <int BN, bool HAS_R>
+struct DownCfg {
+  static constexpr uint32_t STAGE_BYTES = BM * BK * 2 + BN * BK * 2;
+  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 32 * 8;
+};
+
+template <int BN, bool HAS_R>
+__global__ void __launch_bounds__(DN_THREADS, 1)
+tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB2,
+                const __grid_constant__ CUtensorMap tmAs, const __grid_constant__ CUtensorMap tmV2,
+                const Down2Params p) {
+  using Cfg = DownCfg<BN, HAS_R>;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr uint32_t STAGE_BYTES = Cfg::STAGE_BYTES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)STAGES * STAGE_BYTES);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
+  const uint32_t tfull0 = smem_u32(bars + 16), tempty0 = smem_u32(bars + 18);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 20);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int NT = p.NT, KC = p.KC;
+  const int total = (*p.n_rows / BM) * NT;
+  constexpr int NEXT = HAS_R ? 1 : 0;
+  bool failed = false;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int w = blockIdx.x; w < total && !failed; w += gridDim.x) {
+        const int mt = w / NT, nt = w - mt * NT;
+        const int g = p.tile_cluster[mt];
+        const int brow = g * p.N + nt * BN;
+        for (int c = 0; c < KC + NEXT; ++c, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
+          mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+          if (c < KC) {
+            tma_load_2d(a_dst, &tmA, full0 + 8 * s, c * BK, mt * BM);
+            tma_load_2d(b_dst, &tmB2, full0 + 8 * s, c * BK, brow);
+          } else {
+            tma_load_2d(a_dst, &tmAs, full0 + 8 * s, 0, mt * BM);
+            tma_load_2d(b_dst, &tmV2, full0 + 8 * s, 0, brow);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t IDESC = idesc_f16(BM, BN);
+      uint32_t it = 0, tile_i = 0;
+      for (int w = blockIdx.x; w < total && !failed; w += gridDim.x, ++tile_i) {
+        const int mt = w / NT;
+        const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int c = 0; c < KC + NEXT; ++c, ++it) {
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + BM * BK * 2;
+          const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+          if (c < KC) {
+#pragma unroll
+            for (int ks = 0; ks < BK / 16; ++ks)
+              umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
+          } else {
+            const int m = p.tile_mask[2 * mt] | p.tile_mask[2 * mt + 1];
+#pragma unroll
+            for (int ks = 0; ks < KE / 16; ++ks)
+              if ((m >> ks) & 1) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+          }
+          umma_commit(empty0 + 8 * s);
+        }
+        if (failed) break;
+        umma_commit(tfull0 + 8 * acc);
+      }
+    }
+  } else {
+    const int q = warp & 3;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    uint32_t tile_i = 0;
+    for (int w = blockIdx.x; w < total; w += gridDim.x, ++tile_i) {
+      const int mt = w / NT, nt = w - mt * NT;
+      const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
+      const int tok = p.row_token[mt * BM + q * 32 + lane];
+      if (!warp_wait(tfull0 + 8 * acc, aph, abort_flag)) { failed = true; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t v[32];
+        tmem_ld32_nowait(taddr + acc * BN + c0, v);
+        tmem_ld_wait();
+        if (tok >= 0) {
+          uint32_t o[16];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) o[c >> 1] = pack_half2(__uint_as_float(v[c]), __uint_as_float(v[c + 1]));
+          uint4* dst = reinterpret_cast<uint4*>(p.y + (size_t)tok * p.N + nt * BN + c0);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    const unsigned long long t0 = global_ns();
+    while (global_ns() - t0 < 200000ull) { }
+    __syncthreads();
+  }
+  tc_fence_after();
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// fp16 matrix [rows][cols] row-major; box = box_rows x 64 halves, 128-byte swizzle
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct Tc2State {
+  CUtensorMap mX, mB1, mA0, mAd, mV1, mU2;     // up
+  CUtensorMap mU1;                             // t
+  CUtensorMap mAbar, mB2, mAs, mV2;            // down
+  int bn_down;
+  int sm_count;
+  int log2r;
+};
+static_assert(sizeof(Tc2State) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
+
+template <typename Kern>
+cudaError_t set_smem(Kern kern, size_t bytes) {
+  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+template <bool HAS_R, int KSEL>
+cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStream_t st) {
+  auto kern = tc2_up_kernel<HAS_R, KSEL>;
+  constexpr size_t sm = UpCfg<HAS_R, KSEL>::SMEM;
+  static_assert(sm <= kSmemLimit, "up kernel shared memory");
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = set_smem(kern, sm);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  kern<<<grid, UP_THREADS, sm, st>>>(ts.mX, ts.mB1, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
+  return cudaGetLastError();
+}
+
+template <int BN, bool HAS_R>
+cudaError_t launch_down(const Tc2State& ts, const Down2Params& p, int grid, cudaStream_t st) {
+  auto kern = tc2_down_kernel<BN, HAS_R>;
+  constexpr size_t sm = DownCfg<BN, HAS_R>::SMEM;
+  static_assert(sm <= kSmemLimit, "down kernel shared memory");
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = set_smem(kern, sm);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  kern<<<grid, DN_THREADS, sm, st>>>(ts.mAbar, ts.mB2, ts.mAs, ts.mV2, p);
+  return cudaGetLastError();
+}
+
+template <int KSEL>
+cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_t st) {
+  auto kern = tc2_t_kernel<KSEL>;
+  constexpr size_t sm = 1024 + (size_t)T_STAGES * T_STAGE_BYTES + 32 * 8;
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = set_smem(kern, sm);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  kern<<<grid, T_THREADS, sm, st>>>(ts.mX, ts.mU1, p);
+  return cudaGetLastError();
+}
+
+int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
+
+}  // namespace
+
+bool tc2_supported(const Dims& D) {
+  if (D.d % 128 || D.d_ff % 128) return false;
+  if (D.k != 1 && D.k != 2) return false;
+  if (!(D.r == 0 || D.r == 4 || D.r == 8 || D.r == 16 || D.r == 32)) return false;
+  if (D.K * D.r > KE) return false;
+  if (D.row_align != BM) return false;
+  return true;
+}
+
+cudaError_t tc2_init(cmoe_layer* L) {
+  const Dims& D = L->dims;
+  const Scratch& S = L->sc;
+  Tc2State* ts = reinterpret_cast<Tc2State*>(L->tc_state);
+  ts->bn_down = (D.d % 256 == 0) ? 256 : 128;
+  ts->log2r = D.r > 0 ? ilog2(D.r) : 0;
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
+  bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
+            make_map(&ts->mB1, L->w.B1t, G * D.d_ff, D.d, BN_UP) &&
+            make_map(&ts->mAbar, S.abar, P, D.d_ff, BM) &&
+            make_map(&ts->mB2, L->w.B2t, G * D.d, D.d_ff, ts->bn_down);
+  if (ok && D.r > 0) {
+    ok = make_map(&ts->mA0, S.A0, P, KE, BM) && make_map(&ts->mAd, S.Ad, P, KE, BM) &&
+         make_map(&ts->mAs, S.As, P, KE, BM) &&
+         make_map(&ts->mV1, S.V1f, G * D.d_ff, KE, BN_UP) &&
+         make_map(&ts->mV2, S.V2f, G * D.d, KE, ts->bn_down) &&
+         make_map(&ts->mU1, S.U1f, G * KE, D.d, KE) &&
+         make_map(&ts->mU2, S.U2f, G * KE, D.d_ff, KE);
+    // the padding rows / columns of the staged factors (K*r < 64) stay zero for the handle's life
+    const size_t f16 = sizeof(__half);
+    if (ok) {
+      if ((e = cudaMemset(S.U1f, 0, G * KE * D.d * f16)) != cudaSuccess) return e;
+      if ((e = cudaMemset(S.V1f, 0, G * D.d_ff * KE * f16)) != cudaSuccess) return e;
+      if ((e = cudaMemset(S.U2f, 0, G * KE * D.d_ff * f16)) != cudaSuccess) return e;
+      if ((e = cudaMemset(S.V2f, 0, G * D.d * KE * f16)) != cudaSuccess) return e;
+    }
+  } else if (ok) {
+    // unused maps still have to be valid kernel arguments
+    ts->mA0 = ts->mX; ts->mAd = ts->mX; ts->mV1 = ts->mB1; ts->mU2 = ts->mB1; ts->mU1 = ts->mB1;
+    ts->mAs = ts->mAbar; ts->mV2 = ts->mB2;
+  }
+  return ok ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int tc2_launch_count(const Dims& D) { return D.r > 0 ? 5 : 2; }
+
+cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
+  const Dims& D = L->dims;
+  const Weights& W = L->w;
+  const Scratch& S = L->sc;
+  const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
+  const int rows_bound = t_pad_bound(D, T);
+  const int mt_bound = rows_bound / BM;
+  cudaError_t e;
+  if (marks) cudaEventRecord(marks[0], st);
+  if (D.r > 0) {
+    FactorStage fs{};
+    const uint8_t* q[4] = {W.U1q, W.V1q, W.U2q, W.V2q};
+    const __half* sc[4] = {W.U1s, W.V1s, W.U2s, W.V2s};
+    __half* dst[4] = {S.U1f, S.V1f, S.U2f, S.V2f};
+    const int dim[4] = {D.d, D.d_ff, D.d_ff, D.d};
+    long long maxw = 0;
+    for (int i = 0; i < 4; ++i) {
+      fs.q[i] = q[i]; fs.s[i] = sc[i]; fs.dst[i] = dst[i]; fs.dim[i] = dim[i];
+      fs.words[i] = (long long)D.E * D.r * dim[i] / 8;
+      if (fs.words[i] > maxw) maxw = fs.words[i];
+    }
+    fs.K = D.K; fs.r = D.r;
+    dim3 grid((unsigned)((maxw + 255) / 256), 4);
+    stage_factors_kernel<<<grid, 256, 0, st>>>(fs);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    TParams tp{};
+    tp.n_rows = S.n_rows; tp.tile_cluster = S.tile_cluster; tp.row_slot = S.row_slot; tp.row_token = S.row_token;
+    tp.A0 = S.A0; tp.Ad = S.Ad; tp.tile_mask = S.tile_mask; tp.status = S.status;
+    tp.KC = D.d / BK; tp.K = D.K; tp.r = D.r;
+    e = D.k == 2 ? launch_t<2>(ts, tp, mt_bound, st) : launch_t<1>(ts, tp, mt_bound, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (marks) cudaEventRecord(marks[1], st);
+  Up2Params up{};
+  up.n_rows = S.n_rows; up.tile_cluster = S.tile_cluster; up.tile_mask = S.tile_mask; up.row_slot = S.row_slot;
+  up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
+  up.KC = D.d / BK; up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
+  {
+    const long long total = (long long)mt_bound * up.NT;
+    const int grid = (int)(total < ts.sm_count ? total : ts.sm_count);
+    if (D.r == 0)      e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates
+    else if (D.k == 2) e = launch_up<true, 2>(ts, up, grid, st);
+    else               e = launch_up<true, 1>(ts, up, grid, st);
+    if (e != cudaSuccess) return e;
+  }
+  if (marks) cudaEventRecord(marks[2], st);
+  if (D.r > 0) {
+    const int threads = rows_bound * 8;
+    s_expand_kernel<<<(threads + 255) / 256, 256, 0, st>>>(S.n_rows, S.tile_cluster, S.row_slot, S.row_gate, S.s,
+                                                           S.As, D.K, D.k, D.r, ts.log2r);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  Down2Params dn{};
+  dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask; dn.row_token = S.row_token;
+  dn.y = y; dn.status = S.status; dn.KC = D.d_ff / BK; dn.NT = D.d / ts.bn_down; dn.N = D.d;
+  {
+    const long long total = (long long)mt_bound * dn.NT;
+    const int grid = (int)(total < ts.sm_count ? total : ts.sm_count);
+    if (ts.bn_down == 256) e = D.r > 0 ? launch_down<256, true>(ts, dn, grid, st) : launch_down<256, false>(ts, dn, grid, st);
+    else                   e = D.r > 0 ? launch_down<128, true>(ts, dn, grid, st) : launch_down<128, false>(ts, dn, grid, st);
+  }
+  return e;
+}
+
+}  // namespace cmoe
