@@ -295,6 +295,7 @@ struct Up2Params {
   __half* abar;        // [rows][N]
   int* status;
   int KC, NT, N, K, k, r, log2r;
+  int unit;            // N tiles per work unit (divides NT)
 };
 
 constexpr int UP_THREADS = 352;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 S products
@@ -364,9 +365,18 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
   const uint32_t tmem_q = tmem_base + 256, tmem_s = tmem_base + 384;
 
   const int NT = p.NT, KC = p.KC;
-  const long long total = (long long)(*p.n_rows / BM) * NT;
-  const int w0 = (int)(total * blockIdx.x / gridDim.x);
-  const int w1 = (int)(total * (blockIdx.x + 1) / gridDim.x);
+  // Work units of `unit` consecutive N tiles of one row tile, dealt round-robin to the CTAs: at any
+  // time the CTAs work on neighbouring row tiles, i.e. inside one or two clusters, whose base then
+  // stays in L2.  Local tile i of this CTA is tile i % unit of its (i / unit)-th unit.
+  const int unit = p.unit, upm = NT / unit;
+  const int n_units = (*p.n_rows / BM) * upm;
+  const int w0 = 0;
+  const int w1 = blockIdx.x < n_units ? ((n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * unit : 0;
+  auto tile_of = [&](int i, int& mt, int& nt) {
+    const int uu = i / unit, u = blockIdx.x + uu * gridDim.x;
+    mt = u / upm;
+    nt = (u - mt * upm) * unit + (i - uu * unit);
+  };
   bool failed = false;
 
   if (warp == 0) {
@@ -374,7 +384,8 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     if (lane == 0) {
       uint32_t it = 0;
       for (int w = w0; w < w1 && !failed; ++w) {
-        const int mt = w / NT, nt = w - mt * NT;
+        int mt, nt;
+        tile_of(w, mt, nt);
         const int g = p.tile_cluster[mt];
         const int brow = g * p.N + nt * BN_UP;
         for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
@@ -398,7 +409,8 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       constexpr uint32_t IDESC = idesc_f16(BM, BN_UP);
       uint32_t it = 0, tile_i = 0;
       for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
-        const int mt = w / NT;
+        int mt, nt_unused;
+        tile_of(w, mt, nt_unused);
         const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
         if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
@@ -442,7 +454,8 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     if (HAS_R && lane == 0 && w0 < w1) {
       constexpr uint32_t IDESC_S = idesc_f16(BM, KE);
       auto load_u2 = [&](int w, uint32_t ti) -> bool {
-        const int mt = w / NT, nt = w - mt * NT;
+        int mt, nt;
+        tile_of(w, mt, nt);
         const int g = p.tile_cluster[mt];
         const uint32_t ub = ti & 1u, uph = (ti >> 1) & 1u;
         if (!mbar_wait(u2empty0 + 8 * ub, uph ^ 1u, abort_flag)) return false;
@@ -457,7 +470,6 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       uint32_t written = 0;                 // bit j: S_j has been written since the last flush
       if (!load_u2(w0, 0)) failed = true;
       for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
-        const int mt = w / NT;
         if (w + 1 < w1 && !load_u2(w + 1, tile_i + 1)) { failed = true; break; }
         const uint32_t ub = tile_i & 1u, uph = (tile_i >> 1) & 1u;
         if (!mbar_wait(u2full0 + 8 * ub, uph, abort_flag)) { failed = true; break; }
@@ -484,7 +496,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
         }
         if (failed) break;
         umma_commit(u2empty0 + 8 * ub);
-        const bool last_of_run = (w + 1 == w1) || ((w + 1) / NT != mt);
+        const bool last_of_run = (w + 1) % unit == 0;
         if (last_of_run) { umma_commit(sfull); fresh = true; ++flushes; }
       }
     }
@@ -496,7 +508,8 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     uint32_t tile_i = 0, flushes = 0;
     for (int w = w0; w < w1; ++w, ++tile_i) {
-      const int mt = w / NT, nt = w - mt * NT;
+      int mt, nt;
+      tile_of(w, mt, nt);
       const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
       const int row = mt * BM + rowc;
       const float g0 = p.row_gate[(size_t)row * p.k];
@@ -578,7 +591,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       tc_fence_before();
       __syncwarp();
       if (lane == 0) { mbar_arrive(tempty0 + 8 * acc); mbar_arrive(qempty); }
-      const bool last_of_run = (w + 1 == w1) || ((w + 1) / NT != mt);
+      const bool last_of_run = (w + 1) % unit == 0;
       if (HAS_R && last_of_run) {
         if (hf < KSEL) {
           // S_hf is complete for this row tile: add the row's own expert block to s
@@ -903,6 +916,15 @@ cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_
   return cudaGetLastError();
 }
 
+// N tiles per work unit of the up kernel: the largest divisor of NT up to 4 (S is flushed once per
+// unit) that still leaves every SM a unit
+int pick_unit(int NT, int mt_bound, int sms) {
+  int unit = 1;
+  for (int u = 2; u <= 4; ++u)
+    if (NT % u == 0 && (long long)mt_bound * (NT / u) >= 2LL * sms) unit = u;
+  return unit;
+}
+
 int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 
 }  // namespace
@@ -995,7 +1017,8 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
   up.KC = D.d / BK; up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
   {
-    const long long total = (long long)mt_bound * up.NT;
+    up.unit = pick_unit(up.NT, mt_bound, ts.sm_count);
+    const long long total = (long long)mt_bound * (up.NT / up.unit);
     const int grid = (int)(total < ts.sm_count ? total : ts.sm_count);
     if (D.r == 0)      e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates
     else if (D.k == 2) e = launch_up<true, 2>(ts, up, grid, st);
