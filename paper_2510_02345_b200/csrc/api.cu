@@ -50,9 +50,9 @@ int validate_dims(const cmoe_desc* desc, Dims* D) {
   else              { D->nsub = K;           D->sub_is_combo = 0; }
   D->nkey = D->G * D->nsub;
   if (D->nkey > kMaxKeys) return CMOE_ERR_UNSUPPORTED_SHAPE;
-  D->row_align = 128;
-  D->T_pad_max = t_pad_bound(*D, D->T_max);
   D->tc2 = (tc2_supported(*D) && D->T_max > 128) ? 1 : 0;
+  D->row_align = D->tc2 ? 256 : 128;     // CTA pairs work on 256-row tiles of one cluster
+  D->T_pad_max = t_pad_bound(*D, D->T_max);
   return CMOE_OK;
 }
 
@@ -106,7 +106,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
     s.A0 = A.take<__half>(P * 64);
     s.Ad = A.take<__half>(P * 64);
     s.As = A.take<__half>(P * 64);
-    s.tile_mask = A.take<int>(P / D.row_align * 2);
+    s.tile_mask = A.take<int>(P / 128 * 2);
   }
   if (W) *W = w;
   if (S) *S = s;
@@ -227,10 +227,8 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   // fill 128-row tiles; CMOE_FORCE_PATH=0 keeps the generic path (for A/B checks)
   const char* force = std::getenv("CMOE_FORCE_PATH");
   const int forced = force ? std::atoi(force) : -1;
-  const char* variant = std::getenv("CMOE_TC_VARIANT");     // 1 keeps the CUDA-core residual epilogues
-  const int forced_variant = variant ? std::atoi(variant) : 0;
   L->tc_variant = 0;
-  if (D.tc2 && forced != kPathGeneric && forced_variant != 1) {
+  if (D.tc2 && forced != kPathGeneric) {
     if ((e = tc2_init(L))) return fail(e);
     L->path = kPathTensor;
     L->tc_variant = 2;

@@ -17,6 +17,12 @@
 //   expand  As [row][c] = p_j s_j inside the block of expert e_j (fp16)
 //   down    y = abar B2_g^T + As V2f^T, stored un-permuted
 //
+// The up and down kernels run as CTA pairs (thread-block clusters of two, tcgen05 cta_group::2) on
+// 256-row tiles: each CTA loads its 128 rows of A and half of the B tile, the leader CTA issues the
+// MMAs, each CTA's 128 accumulator rows land in its own TMEM and are drained by its own epilogue
+// warps.  This halves the B traffic from L2 per CTA, which is what bounds 128-wide tiles.  A
+// cluster's rows therefore start at multiples of 256.
+//
 // The base product is computed once per token and shared by its k experts; the extra tensor work
 // is the KE-deep steps (skipped per tile for experts no row of the tile uses) and the S products.
 // Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
@@ -178,7 +184,7 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
-  const int g = p.tile_cluster[mt];
+  const int g = p.tile_cluster[mt >> 1];      // the cluster table has one entry per 256 rows
   const int KC = p.KC;
   bool failed = false;
 
@@ -282,12 +288,12 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
 }
 
 // ------------------------------------------------------------------------------------------------
-// up
+// up: CTA pairs (cta_group::2) on 256 x 128 tiles; each CTA owns 128 rows
 // ------------------------------------------------------------------------------------------------
 struct Up2Params {
   const int* n_rows;
-  const int* tile_cluster;
-  const int* tile_mask;
+  const int* tile_cluster;   // per 256-row tile
+  const int* tile_mask;      // per 128-row tile, two words
   const int* row_slot;
   const float* row_gate;
   const int* row_token;
@@ -299,13 +305,20 @@ struct Up2Params {
 };
 
 constexpr int UP_THREADS = 352;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 S products
-constexpr uint32_t UP_STAGE_BYTES = BM * BK * 2 + BN_UP * BK * 2;   // 32 KB
+constexpr uint32_t UP_A_BYTES = BM * BK * 2;                        // 16 KB: this CTA's 128 rows
+constexpr uint32_t UP_B_BYTES = (BN_UP / 2) * BK * 2;               //  8 KB: this CTA's half of the B tile
+constexpr uint32_t UP_STAGE_BYTES = UP_A_BYTES + UP_B_BYTES;        // 24 KB
 constexpr uint32_t A_CHUNK_BYTES = BM * BK * 2;                     // 16 KB: 128 rows x 64 activations
-constexpr uint32_t U2_TILE_BYTES = KE * BN_UP * 2;                  // 16 KB: two 64x64 chunks
+constexpr uint32_t U2_CHUNK_BYTES = (KE / 2) * BK * 2;              //  4 KB: this CTA's 32 rows of a 64 x 64 chunk
+constexpr uint32_t U2_TILE_BYTES = 2 * U2_CHUNK_BYTES;
+
+// barrier slots (64-bit words after the buffers)
+enum : int { B_FULL = 0, B_EMPTY = 8, B_TFULL = 16, B_TEMPTY = 18, B_QEMPTY = 20, B_AFULL = 21, B_AEMPTY = 25,
+             B_U2FULL = 29, B_U2EMPTY = 31, B_SFULL = 33, B_SEMPTY = 34, B_COUNT = 36 };
 
 template <bool HAS_R, int KSEL>
 struct UpCfg {
-  static constexpr int STAGES = HAS_R ? 4 : 6;
+  static constexpr int STAGES = HAS_R ? 6 : 8;
   static constexpr int NA = HAS_R ? 2 * KSEL : 1;          // activation chunks per tile = ring size
   static constexpr int NEXT = HAS_R ? KSEL : 0;            // expanded-index chunks after the main loop
   static constexpr uint32_t RING = STAGES * UP_STAGE_BYTES;
@@ -330,191 +343,203 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
   const uint32_t aring = base + Cfg::RING;
   const uint32_t u2base = aring + Cfg::ARING;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Cfg::BAR_OFF);
-  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
-  const uint32_t tfull0 = smem_u32(bars + 16), tempty0 = smem_u32(bars + 18), qempty = smem_u32(bars + 20);
-  const uint32_t afull0 = smem_u32(bars + 21), aempty0 = smem_u32(bars + 25);
-  const uint32_t u2full0 = smem_u32(bars + 29), u2empty0 = smem_u32(bars + 31);
-  const uint32_t sfull = smem_u32(bars + 33), sempty = smem_u32(bars + 34);
-  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 36);
+  const uint32_t bar0 = smem_u32(bars);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + B_COUNT);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  // the same barrier words in the leader's and in the peer's shared memory (shared::cluster addresses)
+  const uint32_t cbar[2] = {mapa(bar0, 0), mapa(bar0, 1)};
+  const uint32_t lbar = cbar[0];
+  auto local = [&](int slot) { return bar0 + 8u * slot; };
+  auto lead = [&](int slot) { return lbar + 8u * slot; };
+  auto commit_both = [&](int slot) { umma2_commit(cbar[0] + 8u * slot); umma2_commit(cbar[1] + 8u * slot); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 8); }
-    mbar_init(qempty, 8);
-    for (int a = 0; a < 4; ++a) { mbar_init(afull0 + 8 * a, 4); mbar_init(aempty0 + 8 * a, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(u2full0 + 8 * a, 1); mbar_init(u2empty0 + 8 * a, 1); }
-    mbar_init(sfull, 1);
-    mbar_init(sempty, 4 * KSEL);
+    for (int s = 0; s < STAGES; ++s) { mbar_init(local(B_FULL + s), 1); mbar_init(local(B_EMPTY + s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 16); }
+    mbar_init(local(B_QEMPTY), 16);
+    for (int a = 0; a < 4; ++a) { mbar_init(local(B_AFULL + a), 8); mbar_init(local(B_AEMPTY + a), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(local(B_U2FULL + a), 1); mbar_init(local(B_U2EMPTY + a), 1); }
+    mbar_init(local(B_SFULL), 1);
+    mbar_init(local(B_SEMPTY), 8 * KSEL);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
     __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();          // both CTAs' barriers are initialised before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
   // TMEM columns: P (two buffers) 0..255, Q 256..383, S_0 384..447, S_1 448..511
   const uint32_t tmem_q = tmem_base + 256, tmem_s = tmem_base + 384;
 
   const int NT = p.NT, KC = p.KC;
-  // Work units of `unit` consecutive N tiles of one row tile, dealt round-robin to the CTAs: at any
-  // time the CTAs work on neighbouring row tiles, i.e. inside one or two clusters, whose base then
-  // stays in L2.  Local tile i of this CTA is tile i % unit of its (i / unit)-th unit.
+  // Work units of `unit` consecutive N tiles of one 256-row tile, dealt round-robin to the CTA pairs:
+  // at any time the pairs work on neighbouring row tiles, i.e. inside one or two clusters, whose base
+  // then stays in L2.  Local tile i of this pair is tile i % unit of its (i / unit)-th unit.
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
   const int unit = p.unit, upm = NT / unit;
-  const int n_units = (*p.n_rows / BM) * upm;
-  const int w0 = 0;
-  const int w1 = blockIdx.x < n_units ? ((n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1) * unit : 0;
-  auto tile_of = [&](int i, int& mt, int& nt) {
-    const int uu = i / unit, u = blockIdx.x + uu * gridDim.x;
-    mt = u / upm;
-    nt = (u - mt * upm) * unit + (i - uu * unit);
+  const int n_units = (*p.n_rows / (2 * BM)) * upm;
+  const int w1 = pair < n_units ? ((n_units - 1 - pair) / npairs + 1) * unit : 0;
+  auto tile_of = [&](int i, int& pt, int& nt) {
+    const int uu = i / unit, u = pair + uu * npairs;
+    pt = u / upm;
+    nt = (u - pt * upm) * unit + (i - uu * unit);
   };
   bool failed = false;
 
   if (warp == 0) {
-    // ---------------- TMA producer: KC chunks of (x_perm, B1) then the expanded-index chunks
+    // ---------------- TMA producer (both CTAs): this CTA's rows of A and its half of B; the bytes
+    // of both CTAs are counted on the leader's barrier
     if (lane == 0) {
       uint32_t it = 0;
-      for (int w = w0; w < w1 && !failed; ++w) {
-        int mt, nt;
-        tile_of(w, mt, nt);
-        const int g = p.tile_cluster[mt];
-        const int brow = g * p.N + nt * BN_UP;
+      for (int w = 0; w < w1 && !failed; ++w) {
+        int pt, nt;
+        tile_of(w, pt, nt);
+        const int g = p.tile_cluster[pt];
+        const int arow = (2 * pt + (int)rank) * BM;
+        const int brow = g * p.N + nt * BN_UP + (int)rank * (BN_UP / 2);
         for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
-          const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
-          mbar_expect_tx(full0 + 8 * s, UP_STAGE_BYTES);
+          if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + UP_A_BYTES;
+          if (leader) mbar_expect_tx(local(B_FULL + s), 2 * UP_STAGE_BYTES);
           if (c < KC) {
-            tma_load_2d(a_dst, &tmX, full0 + 8 * s, c * BK, mt * BM);
-            tma_load_2d(b_dst, &tmB1, full0 + 8 * s, c * BK, brow);
+            tma2_load_2d(a_dst, &tmX, lead(B_FULL + s), c * BK, arow);
+            tma2_load_2d(b_dst, &tmB1, lead(B_FULL + s), c * BK, brow);
           } else {
-            tma_load_2d(a_dst, c == KC ? &tmA0 : &tmAd, full0 + 8 * s, 0, mt * BM);
-            tma_load_2d(b_dst, &tmV1, full0 + 8 * s, 0, brow);
+            tma2_load_2d(a_dst, c == KC ? &tmA0 : &tmAd, lead(B_FULL + s), 0, arow);
+            tma2_load_2d(b_dst, &tmV1, lead(B_FULL + s), 0, brow);
           }
         }
       }
     }
   } else if (warp == 1) {
-    // ---------------- MMA issuer of P and Q
-    if (lane == 0) {
-      constexpr uint32_t IDESC = idesc_f16(BM, BN_UP);
+    // ---------------- MMA issuer of P and Q (leader CTA only)
+    if (lane == 0 && leader) {
+      constexpr uint32_t IDESC = idesc_f16(2 * BM, BN_UP);
       uint32_t it = 0, tile_i = 0;
-      for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
-        int mt, nt_unused;
-        tile_of(w, mt, nt_unused);
+      for (int w = 0; w < w1 && !failed; ++w, ++tile_i) {
+        int pt, nt_unused;
+        tile_of(w, pt, nt_unused);
         const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
-        if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+        if (!mbar_wait_cluster(local(B_TEMPTY + acc), aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN_UP;
+        const int m0 = HAS_R ? (p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 2]) : 0;
+        const int m1 = HAS_R ? (p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 3]) : 0;
         for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (c == KC + 1) {
-            // Q has one buffer: the epilogue of the previous tile must have drained it
-            if (!mbar_wait(qempty, (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+            // Q has one buffer: both epilogues of the previous tile must have drained it
+            if (!mbar_wait_cluster(local(B_QEMPTY), (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
             tc_fence_after();
           }
-          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+          if (!mbar_wait_cluster(local(B_FULL + s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
-          const uint32_t a_src = base + s * UP_STAGE_BYTES, b_src = a_src + BM * BK * 2;
+          const uint32_t a_src = base + s * UP_STAGE_BYTES, b_src = a_src + UP_A_BYTES;
           const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
           if (c < KC) {
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks)
-              umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
+              umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
           } else if (c == KC) {
-            const int m = p.tile_mask[2 * mt];
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m >> ks) & 1) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+              if ((m0 >> ks) & 1) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
           } else {
-            int m = p.tile_mask[2 * mt] | p.tile_mask[2 * mt + 1];
+            int m = m0 | m1;
             if (m == 0) m = 1;           // Q must be written at least once (A is zero there)
             uint32_t accum = 0;
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m >> ks) & 1) { umma_f16(tmem_q, adesc + 2 * ks, bdesc + 2 * ks, IDESC, accum); accum = 1; }
+              if ((m >> ks) & 1) { umma2_f16(tmem_q, adesc + 2 * ks, bdesc + 2 * ks, IDESC, accum); accum = 1; }
           }
-          umma_commit(empty0 + 8 * s);
+          commit_both(B_EMPTY + s);
         }
         if (failed) break;
-        umma_commit(tfull0 + 8 * acc);
+        commit_both(B_TFULL + acc);
       }
     }
   } else if (warp == 10) {
-    // ---------------- S products: S_j += a_j U2f^T as the epilogue hands activation chunks over
-    if (HAS_R && lane == 0 && w0 < w1) {
-      constexpr uint32_t IDESC_S = idesc_f16(BM, KE);
+    // ---------------- S products: S_j += a_j U2f^T as the epilogues hand activation chunks over.
+    // Both CTAs load their 32 rows of each U2f chunk; the leader issues the MMAs.
+    if (HAS_R && lane == 0 && w1 > 0) {
+      constexpr uint32_t IDESC_S = idesc_f16(2 * BM, KE);
       auto load_u2 = [&](int w, uint32_t ti) -> bool {
-        int mt, nt;
-        tile_of(w, mt, nt);
-        const int g = p.tile_cluster[mt];
+        int pt, nt;
+        tile_of(w, pt, nt);
+        const int g = p.tile_cluster[pt];
         const uint32_t ub = ti & 1u, uph = (ti >> 1) & 1u;
-        if (!mbar_wait(u2empty0 + 8 * ub, uph ^ 1u, abort_flag)) return false;
+        if (!mbar_wait_cluster(local(B_U2EMPTY + ub), uph ^ 1u, abort_flag)) return false;
         const uint32_t dst = u2base + ub * U2_TILE_BYTES;
-        mbar_expect_tx(u2full0 + 8 * ub, U2_TILE_BYTES);
-        tma_load_2d(dst, &tmU2, u2full0 + 8 * ub, nt * BN_UP, g * KE);
-        tma_load_2d(dst + KE * BK * 2, &tmU2, u2full0 + 8 * ub, nt * BN_UP + BK, g * KE);
+        if (leader) mbar_expect_tx(local(B_U2FULL + ub), 2 * U2_TILE_BYTES);
+        tma2_load_2d(dst, &tmU2, lead(B_U2FULL + ub), nt * BN_UP, g * KE + (int)rank * (KE / 2));
+        tma2_load_2d(dst + U2_CHUNK_BYTES, &tmU2, lead(B_U2FULL + ub), nt * BN_UP + BK, g * KE + (int)rank * (KE / 2));
         return true;
       };
       uint32_t tile_i = 0, flushes = 0;
       bool fresh = true;                    // the next product of each slot overwrites S
       uint32_t written = 0;                 // bit j: S_j has been written since the last flush
-      if (!load_u2(w0, 0)) failed = true;
-      for (int w = w0; w < w1 && !failed; ++w, ++tile_i) {
+      if (!load_u2(0, 0)) failed = true;
+      for (int w = 0; w < w1 && !failed; ++w, ++tile_i) {
         if (w + 1 < w1 && !load_u2(w + 1, tile_i + 1)) { failed = true; break; }
+        if (!leader) continue;
         const uint32_t ub = tile_i & 1u, uph = (tile_i >> 1) & 1u;
-        if (!mbar_wait(u2full0 + 8 * ub, uph, abort_flag)) { failed = true; break; }
+        if (!mbar_wait_cluster(local(B_U2FULL + ub), uph, abort_flag)) { failed = true; break; }
         if (fresh && flushes > 0) {
-          // the epilogue must have read the previous row tile's S before it is overwritten
-          if (!mbar_wait(sempty, (flushes - 1) & 1u, abort_flag)) { failed = true; break; }
+          // both epilogues must have read the previous unit's S before it is overwritten
+          if (!mbar_wait_cluster(local(B_SEMPTY), (flushes - 1) & 1u, abort_flag)) { failed = true; break; }
           tc_fence_after();
         }
         if (fresh) { written = 0; fresh = false; }
         for (int c = 0; c < 2 * KSEL; ++c) {
           const uint32_t n = tile_i * (2 * KSEL) + c;
           const uint32_t slot = n % Cfg::NA, aph = (n / Cfg::NA) & 1u;
-          if (!mbar_wait(afull0 + 8 * slot, aph, abort_flag)) { failed = true; break; }
+          if (!mbar_wait_cluster(local(B_AFULL + slot), aph, abort_flag)) { failed = true; break; }
           tc_fence_after();
           const int hf = c / KSEL, j = c - hf * KSEL;
           const uint64_t adesc = umma_desc(aring + slot * A_CHUNK_BYTES);
-          const uint64_t bdesc = umma_desc(u2base + ub * U2_TILE_BYTES + hf * (KE * BK * 2));
+          const uint64_t bdesc = umma_desc(u2base + ub * U2_TILE_BYTES + hf * U2_CHUNK_BYTES);
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks) {
-            umma_f16(tmem_s + j * KE, adesc + 2 * ks, bdesc + 2 * ks, IDESC_S, (written >> j) & 1u);
+            umma2_f16(tmem_s + j * KE, adesc + 2 * ks, bdesc + 2 * ks, IDESC_S, (written >> j) & 1u);
             written |= 1u << j;
           }
-          umma_commit(aempty0 + 8 * slot);
+          commit_both(B_AEMPTY + slot);
         }
         if (failed) break;
-        umma_commit(u2empty0 + 8 * ub);
-        const bool last_of_run = (w + 1) % unit == 0;
-        if (last_of_run) { umma_commit(sfull); fresh = true; ++flushes; }
+        commit_both(B_U2EMPTY + ub);
+        if ((w + 1) % unit == 0) { commit_both(B_SFULL); fresh = true; ++flushes; }
       }
     }
   } else {
-    // ---------------- epilogue warps: quadrant q of the TMEM lanes, column half hf of the tile
+    // ---------------- epilogue warps (both CTAs): quadrant q of this CTA's TMEM lanes, column half hf
     const int q = warp & 3;
     const int hf = (warp - 2) >> 2;
-    const int rowc = q * 32 + lane;                        // row inside the tile
+    const int rowc = q * 32 + lane;                        // row inside this CTA's 128 rows
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     uint32_t tile_i = 0, flushes = 0;
-    for (int w = w0; w < w1; ++w, ++tile_i) {
-      int mt, nt;
-      tile_of(w, mt, nt);
+    for (int w = 0; w < w1; ++w, ++tile_i) {
+      int pt, nt;
+      tile_of(w, pt, nt);
       const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
-      const int row = mt * BM + rowc;
+      const int row = (2 * pt + (int)rank) * BM + rowc;
       const float g0 = p.row_gate[(size_t)row * p.k];
       const float g1 = p.k == 2 ? p.row_gate[(size_t)row * p.k + 1] : 0.f;
-      if (!warp_wait(tfull0 + 8 * acc, aph, abort_flag)) { failed = true; break; }
+      {
+        const bool ok = mbar_wait_cluster(local(B_TFULL + acc), aph, abort_flag);
+        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+      }
       tc_fence_after();
 #pragma unroll 1
       for (int grp = 0; grp < 2; ++grp) {
@@ -529,7 +554,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < KSEL; ++j) {
             const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
-            ok = ok && mbar_wait(aempty0 + 8 * (n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
+            ok = ok && mbar_wait_cluster(local(B_AEMPTY + n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
           }
           if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
         }
@@ -568,8 +593,8 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
             const uint32_t* src = j == 0 ? oa0 : oa1;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              const uint32_t unit = (uint32_t)(grp * 4 + i);
-              st_shared_v4(cb + ((unit ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2],
+              const uint32_t un = (uint32_t)(grp * 4 + i);
+              st_shared_v4(cb + ((un ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2],
                            src[4 * i + 3]);
             }
           }
@@ -583,21 +608,21 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 #pragma unroll
           for (int j = 0; j < KSEL; ++j) {
             const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
-            mbar_arrive(afull0 + 8 * (n % Cfg::NA));
+            mbar_arrive_cluster(lead(B_AFULL + n % Cfg::NA));
           }
         }
       }
-      // accumulators drained: hand P (and Q) back to the MMA warp
+      // accumulators drained: hand P (and Q) back to the leader's MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(tempty0 + 8 * acc); mbar_arrive(qempty); }
-      const bool last_of_run = (w + 1) % unit == 0;
-      if (HAS_R && last_of_run) {
+      if (lane == 0) { mbar_arrive_cluster(lead(B_TEMPTY + acc)); mbar_arrive_cluster(lead(B_QEMPTY)); }
+      if (HAS_R && (w + 1) % unit == 0) {
         if (hf < KSEL) {
-          // S_hf is complete for this row tile: add the row's own expert block to s
-          if (!warp_wait(sfull, flushes & 1u, abort_flag)) { failed = true; break; }
+          // S_hf is complete for this unit: add the row's own expert block to s
+          const bool ok = mbar_wait_cluster(local(B_SFULL), flushes & 1u, abort_flag);
+          if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
           tc_fence_after();
-          const int g = p.tile_cluster[mt];
+          const int g = p.tile_cluster[pt];
           const int e = p.row_slot[(size_t)row * KSEL + hf] - g * p.K;
           const bool real = p.row_token[row] >= 0;
           float* srow = p.s_out + ((size_t)row * KSEL + hf) * p.r;
@@ -616,7 +641,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(sempty);
+          if (lane == 0) mbar_arrive_cluster(lead(B_SEMPTY));
         }
         ++flushes;
       }
@@ -625,17 +650,19 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 
   if (failed) {
     *abort_flag = 1;
+    st_cluster_u32(mapa(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u), 1u);   // the peer gives up too
     atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
   }
   __syncthreads();
   if (*abort_flag) {
     const unsigned long long t0 = global_ns();
     while (global_ns() - t0 < 200000ull) { }    // let copies already issued land
-    __syncthreads();
   }
+  tc_fence_before();
+  cluster_sync_all();      // neither CTA leaves while the other may still use its shared memory or barriers
   tc_fence_after();
   if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -648,7 +675,7 @@ s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_clu
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   const int row = idx >> 3, c0 = (idx & 7) * 8;
   if (row >= *n_rows) return;
-  const int g = tile_cluster[row / BM];
+  const int g = tile_cluster[row / (2 * BM)];
   __align__(16) __half out[8];
 #pragma unroll
   for (int n = 0; n < 8; ++n) {
@@ -662,24 +689,26 @@ s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_clu
 }
 
 // ------------------------------------------------------------------------------------------------
-// down
+// down: CTA pairs on 256 x BN tiles
 // ------------------------------------------------------------------------------------------------
 struct Down2Params {
   const int* n_rows;
-  const int* tile_cluster;
-  const int* tile_mask;
+  const int* tile_cluster;   // per 256-row tile
+  const int* tile_mask;      // per 128-row tile, two words
   const int* row_token;
   __half* y;           // [T][N], original token order
   int* status;
   int KC, NT, N;
 };
 
-constexpr int DN_THREADS = 192;
+constexpr int DN_THREADS = 192;   // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
 
 template <int BN, bool HAS_R>
 struct DownCfg {
-  static constexpr uint32_t STAGE_BYTES = BM * BK * 2 + BN * BK * 2;
-  static constexpr int STAGES = BN == 256 ? 4 : 6;
+  static constexpr uint32_t A_BYTES = BM * BK * 2;
+  static constexpr uint32_t B_BYTES = (BN / 2) * BK * 2;       // this CTA's half of the B tile
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = BN == 256 ? 6 : 8;
   static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 32 * 8;
 };
 
@@ -696,97 +725,108 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)STAGES * STAGE_BYTES);
-  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
-  const uint32_t tfull0 = smem_u32(bars + 16), tempty0 = smem_u32(bars + 18);
+  const uint32_t bar0 = smem_u32(bars);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = rank == 0;
+  const uint32_t cbar[2] = {mapa(bar0, 0), mapa(bar0, 1)};
+  auto local = [&](int slot) { return bar0 + 8u * slot; };
+  auto lead = [&](int slot) { return cbar[0] + 8u * slot; };
+  auto commit_both = [&](int slot) { umma2_commit(cbar[0] + 8u * slot); umma2_commit(cbar[1] + 8u * slot); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, 4); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(local(B_FULL + s), 1); mbar_init(local(B_EMPTY + s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 8); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
     __syncwarp();
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
+  cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
   const int NT = p.NT, KC = p.KC;
-  const int total = (*p.n_rows / BM) * NT;
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int total = (*p.n_rows / (2 * BM)) * NT;
   constexpr int NEXT = HAS_R ? 1 : 0;
   bool failed = false;
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t it = 0;
-      for (int w = blockIdx.x; w < total && !failed; w += gridDim.x) {
-        const int mt = w / NT, nt = w - mt * NT;
-        const int g = p.tile_cluster[mt];
-        const int brow = g * p.N + nt * BN;
+      for (int w = pair; w < total && !failed; w += npairs) {
+        const int pt = w / NT, nt = w - pt * NT;
+        const int g = p.tile_cluster[pt];
+        const int arow = (2 * pt + (int)rank) * BM;
+        const int brow = g * p.N + nt * BN + (int)rank * (BN / 2);
         for (int c = 0; c < KC + NEXT; ++c, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
-          const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
-          mbar_expect_tx(full0 + 8 * s, STAGE_BYTES);
+          if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
+          if (leader) mbar_expect_tx(local(B_FULL + s), 2 * STAGE_BYTES);
           if (c < KC) {
-            tma_load_2d(a_dst, &tmA, full0 + 8 * s, c * BK, mt * BM);
-            tma_load_2d(b_dst, &tmB2, full0 + 8 * s, c * BK, brow);
+            tma2_load_2d(a_dst, &tmA, lead(B_FULL + s), c * BK, arow);
+            tma2_load_2d(b_dst, &tmB2, lead(B_FULL + s), c * BK, brow);
           } else {
-            tma_load_2d(a_dst, &tmAs, full0 + 8 * s, 0, mt * BM);
-            tma_load_2d(b_dst, &tmV2, full0 + 8 * s, 0, brow);
+            tma2_load_2d(a_dst, &tmAs, lead(B_FULL + s), 0, arow);
+            tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, brow);
           }
         }
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t IDESC = idesc_f16(BM, BN);
+    if (lane == 0 && leader) {
+      constexpr uint32_t IDESC = idesc_f16(2 * BM, BN);
       uint32_t it = 0, tile_i = 0;
-      for (int w = blockIdx.x; w < total && !failed; w += gridDim.x, ++tile_i) {
-        const int mt = w / NT;
+      for (int w = pair; w < total && !failed; w += npairs, ++tile_i) {
+        const int pt = w / NT;
         const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
-        if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+        if (!mbar_wait_cluster(local(B_TEMPTY + acc), aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
         for (int c = 0; c < KC + NEXT; ++c, ++it) {
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+          if (!mbar_wait_cluster(local(B_FULL + s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
-          const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + BM * BK * 2;
+          const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + Cfg::A_BYTES;
           const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
           if (c < KC) {
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks)
-              umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
+              umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
           } else {
-            const int m = p.tile_mask[2 * mt] | p.tile_mask[2 * mt + 1];
+            const int m = p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 2] | p.tile_mask[4 * pt + 3];
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m >> ks) & 1) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+              if ((m >> ks) & 1) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
           }
-          umma_commit(empty0 + 8 * s);
+          commit_both(B_EMPTY + s);
         }
         if (failed) break;
-        umma_commit(tfull0 + 8 * acc);
+        commit_both(B_TFULL + acc);
       }
     }
   } else {
     const int q = warp & 3;
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     uint32_t tile_i = 0;
-    for (int w = blockIdx.x; w < total; w += gridDim.x, ++tile_i) {
-      const int mt = w / NT, nt = w - mt * NT;
+    for (int w = pair; w < total; w += npairs, ++tile_i) {
+      const int pt = w / NT, nt = w - pt * NT;
       const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
-      const int tok = p.row_token[mt * BM + q * 32 + lane];
-      if (!warp_wait(tfull0 + 8 * acc, aph, abort_flag)) { failed = true; break; }
+      const int tok = p.row_token[(2 * pt + (int)rank) * BM + q * 32 + lane];
+      {
+        const bool ok = mbar_wait_cluster(local(B_TFULL + acc), aph, abort_flag);
+        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+      }
       tc_fence_after();
 #pragma unroll 1
       for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -804,23 +844,25 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+      if (lane == 0) mbar_arrive_cluster(lead(B_TEMPTY + acc));
     }
   }
 
   if (failed) {
     *abort_flag = 1;
+    st_cluster_u32(mapa(smem_u32(const_cast<int*>(abort_flag)), rank ^ 1u), 1u);
     atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
   }
   __syncthreads();
   if (*abort_flag) {
     const unsigned long long t0 = global_ns();
     while (global_ns() - t0 < 200000ull) { }
-    __syncthreads();
   }
+  tc_fence_before();
+  cluster_sync_all();
   tc_fence_after();
   if (warp == 0)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -872,6 +914,24 @@ cudaError_t set_smem(Kern kern, size_t bytes) {
   return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
+// launch as thread-block clusters of two CTAs (grid = 2 x pairs)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3((unsigned)threads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 template <bool HAS_R, int KSEL>
 cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStream_t st) {
   auto kern = tc2_up_kernel<HAS_R, KSEL>;
@@ -883,8 +943,7 @@ cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStre
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<grid, UP_THREADS, sm, st>>>(ts.mX, ts.mB1, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
-  return cudaGetLastError();
+  return launch_pairs(kern, grid, UP_THREADS, sm, st, ts.mX, ts.mB1, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
 }
 
 template <int BN, bool HAS_R>
@@ -898,8 +957,7 @@ cudaError_t launch_down(const Tc2State& ts, const Down2Params& p, int grid, cuda
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<grid, DN_THREADS, sm, st>>>(ts.mAbar, ts.mB2, ts.mAs, ts.mV2, p);
-  return cudaGetLastError();
+  return launch_pairs(kern, grid, DN_THREADS, sm, st, ts.mAbar, ts.mB2, ts.mAs, ts.mV2, p);
 }
 
 template <int KSEL>
@@ -918,10 +976,10 @@ cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_
 
 // N tiles per work unit of the up kernel: the largest divisor of NT up to 4 (S is flushed once per
 // unit) that still leaves every SM a unit
-int pick_unit(int NT, int mt_bound, int sms) {
+int pick_unit(int NT, int pt_bound, int pairs) {
   int unit = 1;
   for (int u = 2; u <= 4; ++u)
-    if (NT % u == 0 && (long long)mt_bound * (NT / u) >= 2LL * sms) unit = u;
+    if (NT % u == 0 && (long long)pt_bound * (NT / u) >= 2LL * pairs) unit = u;
   return unit;
 }
 
@@ -934,8 +992,7 @@ bool tc2_supported(const Dims& D) {
   if (D.k != 1 && D.k != 2) return false;
   if (!(D.r == 0 || D.r == 4 || D.r == 8 || D.r == 16 || D.r == 32)) return false;
   if (D.K * D.r > KE) return false;
-  if (D.row_align != BM) return false;
-  return true;
+  return true;      // (cmoe_create then aligns the clusters' row segments to 256)
 }
 
 cudaError_t tc2_init(cmoe_layer* L) {
@@ -951,16 +1008,16 @@ cudaError_t tc2_init(cmoe_layer* L) {
   if (e != cudaSuccess) return e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
-            make_map(&ts->mB1, L->w.B1t, G * D.d_ff, D.d, BN_UP) &&
+            make_map(&ts->mB1, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
             make_map(&ts->mAbar, S.abar, P, D.d_ff, BM) &&
-            make_map(&ts->mB2, L->w.B2t, G * D.d, D.d_ff, ts->bn_down);
+            make_map(&ts->mB2, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
   if (ok && D.r > 0) {
     ok = make_map(&ts->mA0, S.A0, P, KE, BM) && make_map(&ts->mAd, S.Ad, P, KE, BM) &&
          make_map(&ts->mAs, S.As, P, KE, BM) &&
-         make_map(&ts->mV1, S.V1f, G * D.d_ff, KE, BN_UP) &&
-         make_map(&ts->mV2, S.V2f, G * D.d, KE, ts->bn_down) &&
+         make_map(&ts->mV1, S.V1f, G * D.d_ff, KE, BN_UP / 2) &&
+         make_map(&ts->mV2, S.V2f, G * D.d, KE, ts->bn_down / 2) &&
          make_map(&ts->mU1, S.U1f, G * KE, D.d, KE) &&
-         make_map(&ts->mU2, S.U2f, G * KE, D.d_ff, KE);
+         make_map(&ts->mU2, S.U2f, G * KE, D.d_ff, KE / 2);
     // the padding rows / columns of the staged factors (K*r < 64) stay zero for the handle's life
     const size_t f16 = sizeof(__half);
     if (ok) {
@@ -985,7 +1042,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   const Scratch& S = L->sc;
   const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
   const int rows_bound = t_pad_bound(D, T);
-  const int mt_bound = rows_bound / BM;
+  const int mt_bound = rows_bound / BM, pt_bound = rows_bound / (2 * BM);
   cudaError_t e;
   if (marks) cudaEventRecord(marks[0], st);
   if (D.r > 0) {
@@ -1017,9 +1074,10 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
   up.KC = D.d / BK; up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
   {
-    up.unit = pick_unit(up.NT, mt_bound, ts.sm_count);
-    const long long total = (long long)mt_bound * (up.NT / up.unit);
-    const int grid = (int)(total < ts.sm_count ? total : ts.sm_count);
+    const int pairs = ts.sm_count / 2;
+    up.unit = pick_unit(up.NT, pt_bound, pairs);
+    const long long total = (long long)pt_bound * (up.NT / up.unit);
+    const int grid = 2 * (int)(total < pairs ? total : pairs);
     if (D.r == 0)      e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates
     else if (D.k == 2) e = launch_up<true, 2>(ts, up, grid, st);
     else               e = launch_up<true, 1>(ts, up, grid, st);
@@ -1036,8 +1094,9 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask; dn.row_token = S.row_token;
   dn.y = y; dn.status = S.status; dn.KC = D.d_ff / BK; dn.NT = D.d / ts.bn_down; dn.N = D.d;
   {
-    const long long total = (long long)mt_bound * dn.NT;
-    const int grid = (int)(total < ts.sm_count ? total : ts.sm_count);
+    const int pairs = ts.sm_count / 2;
+    const long long total = (long long)pt_bound * dn.NT;
+    const int grid = 2 * (int)(total < pairs ? total : pairs);
     if (ts.bn_down == 256) e = D.r > 0 ? launch_down<256, true>(ts, dn, grid, st) : launch_down<256, false>(ts, dn, grid, st);
     else                   e = D.r > 0 ? launch_down<128, true>(ts, dn, grid, st) : launch_down<128, false>(ts, dn, grid, st);
   }

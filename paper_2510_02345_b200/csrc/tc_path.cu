@@ -27,7 +27,7 @@ constexpr int BK = 64;          // halves per K chunk: one 128-byte swizzle row
 constexpr int kThreads = 192;
 constexpr int kMaxStages = 8;
 constexpr uint32_t kTmemCols = 512;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr long long kWaitLimitCycles = 4000000000ll;          // about 2 s of SM clocks
 constexpr size_t kSmemLimit = 232448;                        // 227 KB
 
 struct TcParams {
@@ -75,12 +75,12 @@ __device__ __forceinline__ unsigned long long global_ns() {
 // Bounded wait: false if the time limit ran out or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
+  const long long t0 = clock64();      // the SM's own counter: reading the global timer costs about a microsecond
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 255u) == 0) {
+    if ((++spins & 63u) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) return false;
+      if (clock64() - t0 > kWaitLimitCycles) return false;
     }
   }
   return true;
