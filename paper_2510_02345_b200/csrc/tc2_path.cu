@@ -55,18 +55,6 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
   return __all_sync(0xffffffffu, ok);
 }
 
-// GELU(u) ~ u/2 (1 + tanh(u (c1 + c2 u^2))) with c1, c2 fitted to the erf form (max abs deviation
-// 2.7e-4 over the reals) and the hardware tanh (relative error 2^-11): below the fp16 rounding of
-// the stored activation.
-__device__ __forceinline__ float gelu_fast(float u) {
-  const float u2 = u * u;
-  const float w = fmaf(u2, 0.03470089f, 0.80015708f);
-  float th;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(th) : "f"(u * w));
-  const float hu = 0.5f * u;
-  return fmaf(hu, th, hu);
-}
-
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
   __half2 h = __floats2half2_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
@@ -304,10 +292,19 @@ struct Up2Params {
   int unit;            // N tiles per work unit (divides NT)
 };
 
-constexpr int UP_THREADS = 352;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue, warp 10 S products
-constexpr uint32_t UP_A_BYTES = BM * BK * 2;                        // 16 KB: this CTA's 128 rows
-constexpr uint32_t UP_B_BYTES = (BN_UP / 2) * BK * 2;               //  8 KB: this CTA's half of the B tile
-constexpr uint32_t UP_STAGE_BYTES = UP_A_BYTES + UP_B_BYTES;        // 24 KB
+// Warp roles: 0 and 3 TMA (alternating stages), 1 MMA, 2 S products, 4..19 epilogue.
+// One thread can issue a TMA tile load only every few hundred cycles, and everything a single
+// thread does between two MMAs delays the next one, so a stage carries two 64-wide K atoms (eight
+// MMAs per barrier round trip) and two threads feed the ring.  The epilogue is sixteen warps (four
+// per scheduler) working in packed fp16, because with fewer it, not the tensor pipe, sets the pace.
+constexpr int UP_THREADS = 640;
+constexpr int UP_EPI_WARP0 = 4, UP_EPI_WARPS = 16;
+constexpr int KA = 2;                                               // K atoms of 64 halves per stage
+constexpr uint32_t UP_A_ATOM = BM * BK * 2;                         // 16 KB: this CTA's 128 rows, one atom
+constexpr uint32_t UP_B_ATOM = (BN_UP / 2) * BK * 2;                //  8 KB: this CTA's half of the B tile
+constexpr uint32_t UP_A_BYTES = KA * UP_A_ATOM;
+constexpr uint32_t UP_B_BYTES = KA * UP_B_ATOM;
+constexpr uint32_t UP_STAGE_BYTES = UP_A_BYTES + UP_B_BYTES;        // 48 KB
 constexpr uint32_t A_CHUNK_BYTES = BM * BK * 2;                     // 16 KB: 128 rows x 64 activations
 constexpr uint32_t U2_CHUNK_BYTES = (KE / 2) * BK * 2;              //  4 KB: this CTA's 32 rows of a 64 x 64 chunk
 constexpr uint32_t U2_TILE_BYTES = 2 * U2_CHUNK_BYTES;
@@ -318,9 +315,9 @@ enum : int { B_FULL = 0, B_EMPTY = 8, B_TFULL = 16, B_TEMPTY = 18, B_QEMPTY = 20
 
 template <bool HAS_R, int KSEL>
 struct UpCfg {
-  static constexpr int STAGES = HAS_R ? 6 : 8;
+  static constexpr int STAGES = HAS_R ? 3 : 4;
   static constexpr int NA = HAS_R ? 2 * KSEL : 1;          // activation chunks per tile = ring size
-  static constexpr int NEXT = HAS_R ? KSEL : 0;            // expanded-index chunks after the main loop
+  static constexpr int NEXT = HAS_R ? 1 : 0;               // one expanded-index stage after the main loop (atom j feeds P / Q)
   static constexpr uint32_t RING = STAGES * UP_STAGE_BYTES;
   static constexpr uint32_t ARING = HAS_R ? NA * A_CHUNK_BYTES : 0;
   static constexpr uint32_t U2 = HAS_R ? 2 * U2_TILE_BYTES : 0;
@@ -328,9 +325,24 @@ struct UpCfg {
   static constexpr size_t SMEM = 1024 + BAR_OFF + 48 * 8;
 };
 
+// GELU(u) ~ u/2 (1 + tanh(u (c1 + c2 u^2))) on two fp16 values at once, with c1, c2 fitted to the erf
+// form (max abs deviation 2.7e-4 over the reals) and the hardware tanh; the error is of the size of the
+// fp16 rounding of the stored activation.
+__device__ __forceinline__ __half2 gelu_fast2(__half2 u) {
+  const __half2 u2 = __hmul2(u, u);
+  const __half2 w = __hfma2(u2, __float2half2_rn(0.03470089f), __float2half2_rn(0.80015708f));
+  const __half2 z = __hmul2(u, w);
+  uint32_t zi = *reinterpret_cast<const uint32_t*>(&z), ti;
+  asm("tanh.approx.f16x2 %0, %1;" : "=r"(ti) : "r"(zi));
+  const __half2 th = *reinterpret_cast<const __half2*>(&ti);
+  const __half2 hu = __hmul2(u, __float2half2_rn(0.5f));
+  return __hfma2(hu, th, hu);
+}
+__device__ __forceinline__ uint32_t h2u(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
 template <bool HAS_R, int KSEL>
 __global__ void __launch_bounds__(UP_THREADS, 1)
-tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmB1,
+tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ CUtensorMap tmB13,
               const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmAd,
               const __grid_constant__ CUtensorMap tmV1, const __grid_constant__ CUtensorMap tmU2,
               const Up2Params p) {
@@ -359,12 +371,12 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(local(B_FULL + s), 1); mbar_init(local(B_EMPTY + s), 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 16); }
-    mbar_init(local(B_QEMPTY), 16);
-    for (int a = 0; a < 4; ++a) { mbar_init(local(B_AFULL + a), 8); mbar_init(local(B_AEMPTY + a), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 2 * UP_EPI_WARPS); }
+    mbar_init(local(B_QEMPTY), 2 * UP_EPI_WARPS);
+    for (int a = 0; a < 4; ++a) { mbar_init(local(B_AFULL + a), UP_EPI_WARPS); mbar_init(local(B_AEMPTY + a), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(local(B_U2FULL + a), 1); mbar_init(local(B_U2EMPTY + a), 1); }
     mbar_init(local(B_SFULL), 1);
-    mbar_init(local(B_SEMPTY), 8 * KSEL);
+    mbar_init(local(B_SEMPTY), UP_EPI_WARPS * KSEL);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -397,28 +409,34 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
   };
   bool failed = false;
 
-  if (warp == 0) {
-    // ---------------- TMA producer (both CTAs): this CTA's rows of A and its half of B; the bytes
-    // of both CTAs are counted on the leader's barrier
+  if (warp == 0 || warp == 3) {
+    // ---------------- TMA producers (both CTAs, two threads taking alternate stages): this CTA's rows
+    // of A and its half of B; the bytes of both CTAs are counted on the leader's barrier
     if (lane == 0) {
-      uint32_t it = 0;
-      for (int w = 0; w < w1 && !failed; ++w) {
+      const int spt = KC + Cfg::NEXT;                   // stages per tile
+      const uint32_t n_it = (uint32_t)w1 * spt;
+      for (uint32_t it = warp == 0 ? 0u : 1u; it < n_it && !failed; it += 2) {
+        const int w = it / spt, c = it - w * spt;
         int pt, nt;
         tile_of(w, pt, nt);
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
         const int brow = g * p.N + nt * BN_UP + (int)rank * (BN_UP / 2);
-        for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
-          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
-          const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + UP_A_BYTES;
+        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+        if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
+        const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + UP_A_BYTES;
+        if (c < KC) {
           if (leader) mbar_expect_tx(local(B_FULL + s), 2 * UP_STAGE_BYTES);
-          if (c < KC) {
-            tma2_load_2d(a_dst, &tmX, lead(B_FULL + s), c * BK, arow);
-            tma2_load_2d(b_dst, &tmB1, lead(B_FULL + s), c * BK, brow);
-          } else {
-            tma2_load_2d(a_dst, c == KC ? &tmA0 : &tmAd, lead(B_FULL + s), 0, arow);
-            tma2_load_2d(b_dst, &tmV1, lead(B_FULL + s), 0, brow);
+          tma2_load_3d(a_dst, &tmX3, lead(B_FULL + s), 0, arow, c * KA);
+          tma2_load_3d(b_dst, &tmB13, lead(B_FULL + s), 0, brow, c * KA);
+        } else {
+          // expanded-index stage: atom 0 = (A0, V1f) for P, atom 1 = (Ad, V1f) for Q
+          if (leader) mbar_expect_tx(local(B_FULL + s), 2 * KSEL * (UP_A_ATOM + UP_B_ATOM));
+          tma2_load_2d(a_dst, &tmA0, lead(B_FULL + s), 0, arow);
+          tma2_load_2d(b_dst, &tmV1, lead(B_FULL + s), 0, brow);
+          if (KSEL == 2) {
+            tma2_load_2d(a_dst + UP_A_ATOM, &tmAd, lead(B_FULL + s), 0, arow);
+            tma2_load_2d(b_dst + UP_B_ATOM, &tmV1, lead(B_FULL + s), 0, brow);
           }
         }
       }
@@ -427,50 +445,56 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
     // ---------------- MMA issuer of P and Q (leader CTA only)
     if (lane == 0 && leader) {
       constexpr uint32_t IDESC = idesc_f16(2 * BM, BN_UP);
-      uint32_t it = 0, tile_i = 0;
+      uint32_t s = 0, ph = 0, tile_i = 0;
       for (int w = 0; w < w1 && !failed; ++w, ++tile_i) {
         int pt, nt_unused;
         tile_of(w, pt, nt_unused);
         const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
+        const int m0 = HAS_R ? (p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 2]) : 0;
+        const int m1 = HAS_R ? (p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 3]) : 0;
         if (!mbar_wait_cluster(local(B_TEMPTY + acc), aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN_UP;
-        const int m0 = HAS_R ? (p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 2]) : 0;
-        const int m1 = HAS_R ? (p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 3]) : 0;
-        for (int c = 0; c < KC + Cfg::NEXT; ++c, ++it) {
-          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (c == KC + 1) {
-            // Q has one buffer: both epilogues of the previous tile must have drained it
-            if (!mbar_wait_cluster(local(B_QEMPTY), (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
-            tc_fence_after();
-          }
+        for (int c = 0; c < KC + Cfg::NEXT; ++c) {
           if (!mbar_wait_cluster(local(B_FULL + s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a_src = base + s * UP_STAGE_BYTES, b_src = a_src + UP_A_BYTES;
           const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
           if (c < KC) {
+            // the second atom's tiles follow the first's: descriptor addresses are in 16-byte units
+            umma2_f16(d_tmem, adesc, bdesc, IDESC, c != 0 ? 1u : 0u);
+#pragma unroll
+            for (int ks = 1; ks < BK / 16; ++ks) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
 #pragma unroll
             for (int ks = 0; ks < BK / 16; ++ks)
-              umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
-          } else if (c == KC) {
+              umma2_f16(d_tmem, adesc + (UP_A_ATOM >> 4) + 2 * ks, bdesc + (UP_B_ATOM >> 4) + 2 * ks, IDESC, 1u);
+          } else {
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
               if ((m0 >> ks) & 1) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
-          } else {
-            int m = m0 | m1;
-            if (m == 0) m = 1;           // Q must be written at least once (A is zero there)
-            uint32_t accum = 0;
+            if (KSEL == 2) {
+              // Q has one buffer: both epilogues of the previous tile must have drained it
+              if (!mbar_wait_cluster(local(B_QEMPTY), (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+              tc_fence_after();
+              int m = m0 | m1;
+              if (m == 0) m = 1;           // Q must be written at least once (A is zero there)
+              uint32_t accum = 0;
 #pragma unroll
-            for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m >> ks) & 1) { umma2_f16(tmem_q, adesc + 2 * ks, bdesc + 2 * ks, IDESC, accum); accum = 1; }
+              for (int ks = 0; ks < KE / 16; ++ks)
+                if ((m >> ks) & 1) {
+                  umma2_f16(tmem_q, adesc + (UP_A_ATOM >> 4) + 2 * ks, bdesc + (UP_B_ATOM >> 4) + 2 * ks, IDESC, accum);
+                  accum = 1;
+                }
+            }
           }
           commit_both(B_EMPTY + s);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (failed) break;
         commit_both(B_TFULL + acc);
       }
     }
-  } else if (warp == 10) {
+  } else if (warp == 2) {
     // ---------------- S products: S_j += a_j U2f^T as the epilogues hand activation chunks over.
     // Both CTAs load their 32 rows of each U2f chunk; the leader issues the MMAs.
     if (HAS_R && lane == 0 && w1 > 0) {
@@ -523,9 +547,12 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       }
     }
   } else {
-    // ---------------- epilogue warps (both CTAs): quadrant q of this CTA's TMEM lanes, column half hf
-    const int q = warp & 3;
-    const int hf = (warp - 2) >> 2;
+    // ---------------- epilogue warps (both CTAs): quadrant q of this CTA's TMEM lanes, 32 of the
+    // tile's 128 columns (quarter cq); packed fp16 arithmetic after h_2 = P + Q in fp32
+    const int ew = warp - UP_EPI_WARP0;
+    const int q = warp & 3;                                // the TMEM lanes a warp may read: 32 (warp % 4) ..
+    const int cq = ew >> 2;
+    const int hf = cq >> 1;                                // which 64-column activation chunk
     const int rowc = q * 32 + lane;                        // row inside this CTA's 128 rows
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     uint32_t tile_i = 0, flushes = 0;
@@ -534,21 +561,23 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       tile_of(w, pt, nt);
       const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
       const int row = (2 * pt + (int)rank) * BM + rowc;
-      const float g0 = p.row_gate[(size_t)row * p.k];
-      const float g1 = p.k == 2 ? p.row_gate[(size_t)row * p.k + 1] : 0.f;
+      const float g0f = p.row_gate[(size_t)row * p.k];
+      const float g1f = p.k == 2 ? p.row_gate[(size_t)row * p.k + 1] : 0.f;
+      const __half2 g0 = __float2half2_rn((HAS_R && KSEL == 2) ? g0f : g0f + g1f), g1 = __float2half2_rn(g1f);
       {
         const bool ok = mbar_wait_cluster(local(B_TFULL + acc), aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       }
       tc_fence_after();
-#pragma unroll 1
-      for (int grp = 0; grp < 2; ++grp) {
-        const int col0 = hf * 64 + grp * 32;
-        uint32_t vp[32], vq[32];
-        tmem_ld32_nowait(taddr + acc * BN_UP + col0, vp);
-        if (HAS_R && KSEL == 2) tmem_ld32_nowait(taddr + 256 + col0, vq);
+      uint32_t ob[2][8];                                   // abar, stored after the hand-overs below
+#pragma unroll
+      for (int sub = 0; sub < 2; ++sub) {
+        const int col0 = cq * 32 + sub * 16;
+        uint32_t vp[16], vq[16];
+        tmem_ld16_nowait(taddr + acc * BN_UP + col0, vp);
+        if (HAS_R && KSEL == 2) tmem_ld16_nowait(taddr + 256 + col0, vq);
         tmem_ld_wait();
-        if (HAS_R && grp == 0) {
+        if (HAS_R && sub == 0) {
           // the S products that read this warp's chunk slots one tile ago must have finished
           bool ok = true;
 #pragma unroll
@@ -558,42 +587,33 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
           }
           if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
         }
-        uint32_t ob[16], oa0[16], oa1[16];
+        uint32_t oa0[8], oa1[8];
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float ab[2], a0[2], a1[2];
-#pragma unroll
-          for (int u = 0; u < 2; ++u) {
-            const float h0 = __uint_as_float(vp[c + u]);
-            a0[u] = gelu_fast(h0);
-            if (HAS_R && KSEL == 2) {
-              a1[u] = gelu_fast(h0 + __uint_as_float(vq[c + u]));
-              ab[u] = fmaf(g1, a1[u], g0 * a0[u]);
-            } else {
-              a1[u] = 0.f;
-              ab[u] = (g0 + g1) * a0[u];
-            }
+        for (int c = 0; c < 16; c += 2) {
+          const float p0 = __uint_as_float(vp[c]), p1 = __uint_as_float(vp[c + 1]);
+          const __half2 a0 = gelu_fast2(__floats2half2_rn(p0, p1));
+          __half2 ab;
+          if (HAS_R && KSEL == 2) {
+            const __half2 a1 = gelu_fast2(__floats2half2_rn(p0 + __uint_as_float(vq[c]), p1 + __uint_as_float(vq[c + 1])));
+            ab = __hfma2(g1, a1, __hmul2(g0, a0));
+            oa1[c >> 1] = h2u(a1);
+          } else {
+            ab = __hmul2(g0, a0);
           }
-          ob[c >> 1] = pack_half2(ab[0], ab[1]);
-          if (HAS_R) {
-            oa0[c >> 1] = pack_half2(a0[0], a0[1]);
-            if (KSEL == 2) oa1[c >> 1] = pack_half2(a1[0], a1[1]);
-          }
+          ob[sub][c >> 1] = h2u(ab);
+          oa0[c >> 1] = h2u(a0);
         }
-        uint4* dst = reinterpret_cast<uint4*>(p.abar + (size_t)row * p.N + nt * BN_UP + col0);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) dst[i] = make_uint4(ob[4 * i], ob[4 * i + 1], ob[4 * i + 2], ob[4 * i + 3]);
         if (HAS_R) {
           // a_j into its chunk as a K-major 128-byte-swizzled A operand: 16-byte unit u of row
-          // rowc sits at rowc*128 + ((u ^ (rowc & 7)) << 4)
+          // rowc sits at rowc*128 + ((u ^ (rowc & 7)) << 4); this warp owns units 4 (cq & 1) + 2 sub + {0, 1}
 #pragma unroll
           for (int j = 0; j < KSEL; ++j) {
             const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
             const uint32_t cb = aring + (n % Cfg::NA) * A_CHUNK_BYTES + rowc * 128;
             const uint32_t* src = j == 0 ? oa0 : oa1;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t un = (uint32_t)(grp * 4 + i);
+            for (int i = 0; i < 2; ++i) {
+              const uint32_t un = (uint32_t)((cq & 1) * 4 + sub * 2 + i);
               st_shared_v4(cb + ((un ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2],
                            src[4 * i + 3]);
             }
@@ -616,9 +636,20 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
       tc_fence_before();
       __syncwarp();
       if (lane == 0) { mbar_arrive_cluster(lead(B_TEMPTY + acc)); mbar_arrive_cluster(lead(B_QEMPTY)); }
+      // abar goes out last: a release at cluster scope waits for the thread's earlier global stores,
+      // and by the next tile's hand-overs these have long landed
+      {
+        uint4* dst = reinterpret_cast<uint4*>(p.abar + (size_t)row * p.N + nt * BN_UP + cq * 32);
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          dst[2 * sub] = make_uint4(ob[sub][0], ob[sub][1], ob[sub][2], ob[sub][3]);
+          dst[2 * sub + 1] = make_uint4(ob[sub][4], ob[sub][5], ob[sub][6], ob[sub][7]);
+        }
+      }
       if (HAS_R && (w + 1) % unit == 0) {
         if (hf < KSEL) {
-          // S_hf is complete for this unit: add the row's own expert block to s
+          // S_hf is complete for this unit.  The warp walks over the expert blocks of the expanded
+          // index (this warp: every other block); lanes whose row uses the block add it to s.
           const bool ok = mbar_wait_cluster(local(B_SFULL), flushes & 1u, abort_flag);
           if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
           tc_fence_after();
@@ -626,17 +657,41 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ C
           const int e = p.row_slot[(size_t)row * KSEL + hf] - g * p.K;
           const bool real = p.row_token[row] >= 0;
           float* srow = p.s_out + ((size_t)row * KSEL + hf) * p.r;
-#pragma unroll 1
-          for (int half = 0; half < 2; ++half) {
-            uint32_t v[32];
-            tmem_ld32_nowait(taddr + 384 + hf * KE + half * 32, v);
-            tmem_ld_wait();
-            if (real) {
+          const int r = p.r;
+          for (int i = cq & 1; i < p.K; i += 2) {
+            const uint32_t ta = taddr + 384 + hf * KE + i * r;
+            const bool mine = real && e == i;
+            if (r == 16) {
+              uint32_t v[16];
+              tmem_ld16_nowait(ta, v);
+              tmem_ld_wait();
+              if (mine) {
 #pragma unroll
-              for (int c = 0; c < 32; ++c) {
-                const int cc = half * 32 + c;
-                if ((cc >> p.log2r) == e) atomicAdd(srow + (cc & (p.r - 1)), __uint_as_float(v[c]));
+                for (int c = 0; c < 16; c += 4)
+                  red_add_v4(srow + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
               }
+            } else if (r == 32) {
+              uint32_t v[32];
+              tmem_ld32_nowait(ta, v);
+              tmem_ld_wait();
+              if (mine) {
+#pragma unroll
+                for (int c = 0; c < 32; c += 4)
+                  red_add_v4(srow + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+              }
+            } else if (r == 8) {
+              uint32_t v[8];
+              tmem_ld8_nowait(ta, v);
+              tmem_ld_wait();
+              if (mine) {
+                red_add_v4(srow, __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+                red_add_v4(srow + 4, __uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
+              }
+            } else {
+              uint32_t v[4];
+              tmem_ld4_nowait(ta, v);
+              tmem_ld_wait();
+              if (mine) red_add_v4(srow, __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
             }
           }
           tc_fence_before();
@@ -701,20 +756,22 @@ struct Down2Params {
   int KC, NT, N;
 };
 
-constexpr int DN_THREADS = 192;   // warp 0 TMA, warp 1 MMA, warps 2..5 epilogue
+constexpr int DN_THREADS = 224;   // warps 0 and 6 TMA (alternating stages), warp 1 MMA, warps 2..5 epilogue
 
 template <int BN, bool HAS_R>
 struct DownCfg {
-  static constexpr uint32_t A_BYTES = BM * BK * 2;
-  static constexpr uint32_t B_BYTES = (BN / 2) * BK * 2;       // this CTA's half of the B tile
-  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = BN == 256 ? 6 : 8;
+  static constexpr uint32_t A_ATOM = BM * BK * 2;
+  static constexpr uint32_t B_ATOM = (BN / 2) * BK * 2;        // this CTA's half of the B tile, one K atom
+  static constexpr uint32_t A_BYTES = KA * A_ATOM;
+  static constexpr uint32_t B_BYTES = KA * B_ATOM;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;   // 64 KB (BN = 256) / 48 KB
+  static constexpr int STAGES = BN == 256 ? 3 : 4;
   static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 32 * 8;
 };
 
 template <int BN, bool HAS_R>
 __global__ void __launch_bounds__(DN_THREADS, 1)
-tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB2,
+tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant__ CUtensorMap tmB23,
                 const __grid_constant__ CUtensorMap tmAs, const __grid_constant__ CUtensorMap tmV2,
                 const Down2Params p) {
   using Cfg = DownCfg<BN, HAS_R>;
@@ -760,26 +817,30 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   constexpr int NEXT = HAS_R ? 1 : 0;
   bool failed = false;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 6) {
+    // two producer threads take alternate stages
     if (lane == 0) {
-      uint32_t it = 0;
-      for (int w = pair; w < total && !failed; w += npairs) {
+      const int spt = KC + NEXT;
+      const int my_tiles = pair < total ? (total - 1 - pair) / npairs + 1 : 0;
+      const uint32_t n_it = (uint32_t)my_tiles * spt;
+      for (uint32_t it = warp == 0 ? 0u : 1u; it < n_it && !failed; it += 2) {
+        const int ti = it / spt, c = it - ti * spt;
+        const int w = pair + ti * npairs;
         const int pt = w / NT, nt = w - pt * NT;
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
         const int brow = g * p.N + nt * BN + (int)rank * (BN / 2);
-        for (int c = 0; c < KC + NEXT; ++c, ++it) {
-          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-          if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
-          const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
+        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+        if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
+        const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
+        if (c < KC) {
           if (leader) mbar_expect_tx(local(B_FULL + s), 2 * STAGE_BYTES);
-          if (c < KC) {
-            tma2_load_2d(a_dst, &tmA, lead(B_FULL + s), c * BK, arow);
-            tma2_load_2d(b_dst, &tmB2, lead(B_FULL + s), c * BK, brow);
-          } else {
-            tma2_load_2d(a_dst, &tmAs, lead(B_FULL + s), 0, arow);
-            tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, brow);
-          }
+          tma2_load_3d(a_dst, &tmA3, lead(B_FULL + s), 0, arow, c * KA);
+          tma2_load_3d(b_dst, &tmB23, lead(B_FULL + s), 0, brow, c * KA);
+        } else {
+          if (leader) mbar_expect_tx(local(B_FULL + s), 2 * (Cfg::A_ATOM + Cfg::B_ATOM));
+          tma2_load_2d(a_dst, &tmAs, lead(B_FULL + s), 0, arow);
+          tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, brow);
         }
       }
     }
@@ -798,12 +859,16 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           if (!mbar_wait_cluster(local(B_FULL + s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
           const uint32_t a_src = base + s * STAGE_BYTES, b_src = a_src + Cfg::A_BYTES;
-          const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
           if (c < KC) {
 #pragma unroll
-            for (int ks = 0; ks < BK / 16; ++ks)
-              umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | ks) != 0 ? 1u : 0u);
+            for (int a = 0; a < KA; ++a) {
+              const uint64_t adesc = umma_desc(a_src + a * Cfg::A_ATOM), bdesc = umma_desc(b_src + a * Cfg::B_ATOM);
+#pragma unroll
+              for (int ks = 0; ks < BK / 16; ++ks)
+                umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (c | a | ks) != 0 ? 1u : 0u);
+            }
           } else {
+            const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
             const int m = p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 2] | p.tile_mask[4 * pt + 3];
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
@@ -899,10 +964,24 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen as [cols / 64][rows][64]: a box of 64 x box_rows x KA lands in shared memory as KA
+// consecutive 128-byte-swizzled [box_rows][64] tiles, one per K atom.
+bool make_map3(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t gdim[3] = {(cuuint64_t)BK, rows, cols / BK};
+  cuuint64_t gstride[2] = {cols * 2, (cuuint64_t)BK * 2};
+  cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, (cuuint32_t)KA};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, const_cast<void*>(ptr), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Tc2State {
-  CUtensorMap mX, mB1, mA0, mAd, mV1, mU2;     // up
+  CUtensorMap mX, mX3, mB13, mA0, mAd, mV1, mU2;   // up (mX: 2-D, for the t kernel)
   CUtensorMap mU1;                             // t
-  CUtensorMap mAbar, mB2, mAs, mV2;            // down
+  CUtensorMap mAbar3, mB23, mAs, mV2;          // down
   int bn_down;
   int sm_count;
   int log2r;
@@ -943,7 +1022,7 @@ cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStre
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pairs(kern, grid, UP_THREADS, sm, st, ts.mX, ts.mB1, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
+  return launch_pairs(kern, grid, UP_THREADS, sm, st, ts.mX3, ts.mB13, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
 }
 
 template <int BN, bool HAS_R>
@@ -957,7 +1036,7 @@ cudaError_t launch_down(const Tc2State& ts, const Down2Params& p, int grid, cuda
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pairs(kern, grid, DN_THREADS, sm, st, ts.mAbar, ts.mB2, ts.mAs, ts.mV2, p);
+  return launch_pairs(kern, grid, DN_THREADS, sm, st, ts.mAbar3, ts.mB23, ts.mAs, ts.mV2, p);
 }
 
 template <int KSEL>
@@ -1008,9 +1087,10 @@ cudaError_t tc2_init(cmoe_layer* L) {
   if (e != cudaSuccess) return e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
-            make_map(&ts->mB1, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
-            make_map(&ts->mAbar, S.abar, P, D.d_ff, BM) &&
-            make_map(&ts->mB2, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
+            make_map3(&ts->mX3, S.x_perm, P, D.d, BM) &&
+            make_map3(&ts->mB13, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
+            make_map3(&ts->mAbar3, S.abar, P, D.d_ff, BM) &&
+            make_map3(&ts->mB23, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
   if (ok && D.r > 0) {
     ok = make_map(&ts->mA0, S.A0, P, KE, BM) && make_map(&ts->mAd, S.Ad, P, KE, BM) &&
          make_map(&ts->mAs, S.As, P, KE, BM) &&
@@ -1028,8 +1108,8 @@ cudaError_t tc2_init(cmoe_layer* L) {
     }
   } else if (ok) {
     // unused maps still have to be valid kernel arguments
-    ts->mA0 = ts->mX; ts->mAd = ts->mX; ts->mV1 = ts->mB1; ts->mU2 = ts->mB1; ts->mU1 = ts->mB1;
-    ts->mAs = ts->mAbar; ts->mV2 = ts->mB2;
+    ts->mA0 = ts->mX; ts->mAd = ts->mX; ts->mV1 = ts->mX; ts->mU2 = ts->mX; ts->mU1 = ts->mX;
+    ts->mAs = ts->mX; ts->mV2 = ts->mX;
   }
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
@@ -1072,7 +1152,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   Up2Params up{};
   up.n_rows = S.n_rows; up.tile_cluster = S.tile_cluster; up.tile_mask = S.tile_mask; up.row_slot = S.row_slot;
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
-  up.KC = D.d / BK; up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
+  up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
   {
     const int pairs = ts.sm_count / 2;
     up.unit = pick_unit(up.NT, pt_bound, pairs);
@@ -1092,7 +1172,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   }
   Down2Params dn{};
   dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask; dn.row_token = S.row_token;
-  dn.y = y; dn.status = S.status; dn.KC = D.d_ff / BK; dn.NT = D.d / ts.bn_down; dn.N = D.d;
+  dn.y = y; dn.status = S.status; dn.KC = D.d_ff / (BK * KA); dn.NT = D.d / ts.bn_down; dn.N = D.d;
   {
     const int pairs = ts.sm_count / 2;
     const long long total = (long long)pt_bound * dn.NT;
