@@ -1,7 +1,18 @@
 // Fused two-stage router (Sec. 3.3): cluster logits z = x C and top-1 cluster (Eq. 9), expert
 // logits l = x R_g* over the K experts of that cluster, top-k and renormalised softmax gates
-// (Eq. 10).  One warp per token; all dot products are fp32 FMAs in a fixed order, so the result
-// does not depend on the launch shape.
+// (Eq. 10).  All dot products are fp32 FMAs in a fixed order per kernel, so a token's route does not
+// depend on where in the batch it sits; which kernel runs depends only on the batch size.
+//
+//   router_tile_kernel   many tokens: a block takes 64 tokens, a warp eight of them at a time, so
+//                        that a router row fetched by a lane is used for eight tokens.  Stage 1
+//                        reads the cluster prototypes from shared memory; for stage 2 the block
+//                        orders its tokens by cluster, so that the eight tokens of a warp mostly
+//                        share one cluster's expert rows.
+//   router_token_kernel  few tokens (decode): one block per token, the warps split d.
+//
+// In both, lane l of a warp owns the columns 256 s + 8 l .. + 7 of the 256-column segments it
+// visits, a lane's partial sum runs over its columns in ascending order, and partial sums are
+// combined by an xor butterfly (and, in the second kernel, by adding the warps' sums in warp order).
 #include "cmoe_internal.h"
 #include "device_utils.cuh"
 
@@ -9,92 +20,252 @@ namespace cmoe {
 
 namespace {
 
-// dot of the token row with one fp32 router row, lanes striding 8-element chunks
-__device__ __forceinline__ float row_dot(const __half* __restrict__ xr, const float* __restrict__ wr,
-                                         int d, int lane) {
-  float acc = 0.f;
-  for (int c = lane * 8; c < d; c += 256) {
-    uint4 xv = *reinterpret_cast<const uint4*>(xr + c);
-    float4 w0 = *reinterpret_cast<const float4*>(wr + c);
-    float4 w1 = *reinterpret_cast<const float4*>(wr + c + 4);
-    const __half2* xh = reinterpret_cast<const __half2*>(&xv);
-    float2 a = __half22float2(xh[0]), b = __half22float2(xh[1]);
-    float2 c2 = __half22float2(xh[2]), e = __half22float2(xh[3]);
-    acc = fmaf(a.x, w0.x, acc);  acc = fmaf(a.y, w0.y, acc);
-    acc = fmaf(b.x, w0.z, acc);  acc = fmaf(b.y, w0.w, acc);
-    acc = fmaf(c2.x, w1.x, acc); acc = fmaf(c2.y, w1.y, acc);
-    acc = fmaf(e.x, w1.z, acc);  acc = fmaf(e.y, w1.w, acc);
-  }
-  return warp_sum(acc);
+constexpr int kTokPerWarp = 8;
+constexpr int kTileWarps = 8;
+constexpr int kTileTokens = kTokPerWarp * kTileWarps;     // 64
+constexpr int kGroup = 8;                                  // router rows accumulated at once
+
+__device__ __forceinline__ void fma8(float& acc, const uint4& xv, const float4& w0, const float4& w1) {
+  const __half2* xh = reinterpret_cast<const __half2*>(&xv);
+  const float2 a = __half22float2(xh[0]), b = __half22float2(xh[1]);
+  const float2 c = __half22float2(xh[2]), e = __half22float2(xh[3]);
+  acc = fmaf(a.x, w0.x, acc); acc = fmaf(a.y, w0.y, acc);
+  acc = fmaf(b.x, w0.z, acc); acc = fmaf(b.y, w0.w, acc);
+  acc = fmaf(c.x, w1.x, acc); acc = fmaf(c.y, w1.y, acc);
+  acc = fmaf(e.x, w1.z, acc); acc = fmaf(e.y, w1.w, acc);
 }
 
-__global__ void __launch_bounds__(256)
-router_kernel(const __half* __restrict__ x, int T, int d, int G, int K, int k,
-              const float* __restrict__ Ct, const float* __restrict__ Rt,
-              const float* __restrict__ bc, const float* __restrict__ be,
-              const int* __restrict__ label,
-              int* __restrict__ cluster_id, int* __restrict__ expert_ids,
-              float* __restrict__ gates, int* __restrict__ slot_local) {
-  const int lane = threadIdx.x & 31;
-  const int warps_per_block = blockDim.x >> 5;
-  for (int t = blockIdx.x * warps_per_block + (threadIdx.x >> 5); t < T;
-       t += gridDim.x * warps_per_block) {
-    const __half* xr = x + (size_t)t * d;
-    // stage 1: top-1 cluster = argmax of the logits (softmax of Eq. 9 is monotone)
-    int gs = 0;
-    float zbest = 0.f;
-    for (int g = 0; g < G; ++g) {
-      float z = row_dot(xr, Ct + (size_t)g * d, d, lane) + bc[g];
-      if (g == 0 || z > zbest) { zbest = z; gs = g; }   // strict >: lowest index wins ties
-    }
-    // stage 2: lane i keeps the logit of expert i of the chosen cluster
-    float myl = -INFINITY;
+// Top-k of K logits (ties: lowest index), gates = softmax over the kept logits (Eq. 10
+// renormalised over the kept experts); one thread per token, logits read from `lg`.
+__device__ __forceinline__ void select_and_store(const float* lg, int K, int k, int g, int t,
+                                                 const int* __restrict__ label, int* __restrict__ expert_ids,
+                                                 float* __restrict__ gates, int* __restrict__ slot_local) {
+  unsigned taken = 0;
+  float selv[kMaxKsel];
+  int seli[kMaxKsel];
+  for (int s = 0; s < k; ++s) {
+    float best = -INFINITY;
+    int bi = 0;
+    bool have = false;
     for (int i = 0; i < K; ++i) {
-      float l = row_dot(xr, Rt + (size_t)(gs * K + i) * d, d, lane) + be[gs * K + i];
-      if (lane == i) myl = l;
+      if ((taken >> i) & 1u) continue;
+      const float v = lg[i];
+      if (!have || v > best) { best = v; bi = i; have = true; }   // strict >: lowest index wins ties
     }
-    // top-k by k rounds of warp arg-max (ties: lowest index)
-    float selv[kMaxKsel];
-    int seli[kMaxKsel];
-    bool taken = (lane >= K);
+    taken |= 1u << bi;
+    selv[s] = best;
+    seli[s] = bi;
+  }
+  const float lmax = selv[0];
+  float ev[kMaxKsel];
+  float sum = 0.f;
+  for (int s = 0; s < k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
+  for (int s = 0; s < k; ++s) {
+    if (gates) gates[(size_t)t * k + s] = ev[s] / sum;
+    if (expert_ids) expert_ids[(size_t)t * k + s] = label[g * K + seli[s]];
+    if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
+  }
+}
+
+struct RouterArgs {
+  const __half* x;
+  int T, d, G, K, k;
+  const float *Ct, *Rt, *bc, *be;
+  const int* label;
+  int* cluster_id;
+  int* expert_ids;
+  float* gates;
+  int* slot_local;
+  int dc;          // columns of the cluster prototypes staged in shared memory at a time
+};
+
+__global__ void __launch_bounds__(kTileWarps * 32)
+router_tile_kernel(const RouterArgs a) {
+  extern __shared__ float sm_f[];
+  float* Cs = sm_f;                                        // [up to 8 clusters][dc]
+  float* lg = Cs + (size_t)kGroup * a.dc;                  // [64][K] expert logits
+  __shared__ int s_cid[kTileTokens];
+  __shared__ int s_order[kTileTokens];
+  __shared__ float s_zbest[kTileTokens];
+
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tok0 = blockIdx.x * kTileTokens;
+  const int d = a.d, G = a.G, K = a.K;
+
+  // ---- stage 1: cluster logits of the warp's eight tokens, clusters in groups of eight
+  const int wt0 = tok0 + warp * kTokPerWarp;
+  for (int g0 = 0; g0 < G; g0 += kGroup) {
+    const int ng = min(kGroup, G - g0);
+    float acc[kTokPerWarp][kGroup];
 #pragma unroll
-    for (int s = 0; s < kMaxKsel; ++s) {
-      if (s < k) {
-        float v = taken ? -INFINITY : myl;
-        int idx = taken ? 64 : lane;
+    for (int t = 0; t < kTokPerWarp; ++t)
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          float ov = __shfl_xor_sync(0xffffffffu, v, o);
-          int oi = __shfl_xor_sync(0xffffffffu, idx, o);
-          if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+      for (int j = 0; j < kGroup; ++j) acc[t][j] = 0.f;
+    for (int c0 = 0; c0 < d; c0 += a.dc) {
+      const int cw = min(a.dc, d - c0);
+      __syncthreads();                                     // the previous chunk is no longer read
+      for (int i = threadIdx.x * 4; i < ng * cw; i += blockDim.x * 4) {
+        const int j = i / cw, c = i - j * cw;
+        *reinterpret_cast<float4*>(Cs + (size_t)j * a.dc + c) =
+            *reinterpret_cast<const float4*>(a.Ct + (size_t)(g0 + j) * d + c0 + c);
+      }
+      __syncthreads();
+      for (int c = lane * 8; c < cw; c += 256) {
+        uint4 xv[kTokPerWarp];
+#pragma unroll
+        for (int t = 0; t < kTokPerWarp; ++t) {
+          const int tok = min(wt0 + t, a.T - 1);
+          xv[t] = *reinterpret_cast<const uint4*>(a.x + (size_t)tok * d + c0 + c);
         }
-        selv[s] = v;
-        seli[s] = idx;
-        if (lane == idx) taken = true;
+#pragma unroll
+        for (int j = 0; j < kGroup; ++j) {
+          if (j < ng) {
+            const float4 w0 = *reinterpret_cast<const float4*>(Cs + (size_t)j * a.dc + c);
+            const float4 w1 = *reinterpret_cast<const float4*>(Cs + (size_t)j * a.dc + c + 4);
+#pragma unroll
+            for (int t = 0; t < kTokPerWarp; ++t) fma8(acc[t][j], xv[t], w0, w1);
+          }
+        }
       }
     }
-    if (lane == 0) cluster_id[t] = gs;
-    // gates: softmax over the kept logits (= Eq. 10 renormalised over the kept experts)
-    {
-      const float lmax = selv[0];
-      float ev[kMaxKsel];
-      float sum = 0.f;
+    // combine the lanes' partial sums; lane t keeps the running arg-max of token t
 #pragma unroll
-      for (int s = 0; s < kMaxKsel; ++s)
-        if (s < k) {
-          ev[s] = expf(selv[s] - lmax);
-          sum += ev[s];
+    for (int t = 0; t < kTokPerWarp; ++t) {
+#pragma unroll
+      for (int j = 0; j < kGroup; ++j) {
+        const float z = warp_sum(acc[t][j]);
+        if (j < ng && lane == t) {
+          const float zb = z + a.bc[g0 + j];
+          const int slot = warp * kTokPerWarp + t;
+          if ((g0 + j) == 0 || zb > s_zbest[slot]) { s_zbest[slot] = zb; s_cid[slot] = g0 + j; }   // strict >: lowest index wins ties
+        }
+      }
+    }
+    __syncwarp();
+  }
+  __syncthreads();
+
+  // ---- order the block's tokens by cluster (stable), so that a warp's eight tokens share rows
+  if (threadIdx.x < kTileTokens) {
+    const int me = threadIdx.x, c = s_cid[me];
+    int rank = 0;
+    for (int u = 0; u < kTileTokens; ++u) {
+      const int cu = s_cid[u];
+      rank += (cu < c || (cu == c && u < me)) ? 1 : 0;
+    }
+    s_order[rank] = me;
+    if (tok0 + me < a.T) a.cluster_id[tok0 + me] = c;
+  }
+  __syncthreads();
+
+  // ---- stage 2: expert logits; the warp takes eight tokens of the ordered list, run by run
+  int slot_of[kTokPerWarp], cl_of[kTokPerWarp];
+#pragma unroll
+  for (int t = 0; t < kTokPerWarp; ++t) {
+    slot_of[t] = s_order[warp * kTokPerWarp + t];
+    cl_of[t] = s_cid[slot_of[t]];
+  }
+  int j0 = 0;
+  while (j0 < kTokPerWarp) {
+    int g = 0;
+#pragma unroll
+    for (int t = 0; t < kTokPerWarp; ++t)
+      if (t == j0) g = cl_of[t];
+    unsigned active = 0;                                   // tokens of this run
+    int j1 = j0;
+#pragma unroll
+    for (int t = 0; t < kTokPerWarp; ++t)
+      if (t >= j0 && cl_of[t] == g) { active |= 1u << t; j1 = t + 1; }
+    for (int i0 = 0; i0 < K; i0 += 4) {
+      const int ni = min(4, K - i0);
+      float acc[kTokPerWarp][4];
+#pragma unroll
+      for (int t = 0; t < kTokPerWarp; ++t)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[t][i] = 0.f;
+      for (int c = lane * 8; c < d; c += 256) {
+        uint4 xv[kTokPerWarp];
+#pragma unroll
+        for (int t = 0; t < kTokPerWarp; ++t) {
+          xv[t] = make_uint4(0, 0, 0, 0);
+          if ((active >> t) & 1u) {
+            const int tok = min(tok0 + slot_of[t], a.T - 1);
+            xv[t] = *reinterpret_cast<const uint4*>(a.x + (size_t)tok * d + c);
+          }
         }
 #pragma unroll
-      for (int s = 0; s < kMaxKsel; ++s)
-        if (s < k && lane == 0) {
-          int slot = gs * K + seli[s];
-          if (gates) gates[(size_t)t * k + s] = ev[s] / sum;
-          if (expert_ids) expert_ids[(size_t)t * k + s] = label[slot];
-          if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
+        for (int i = 0; i < 4; ++i) {
+          if (i < ni) {
+            const float* wr = a.Rt + (size_t)(g * K + i0 + i) * d + c;
+            const float4 w0 = __ldg(reinterpret_cast<const float4*>(wr));
+            const float4 w1 = __ldg(reinterpret_cast<const float4*>(wr + 4));
+#pragma unroll
+            for (int t = 0; t < kTokPerWarp; ++t) fma8(acc[t][i], xv[t], w0, w1);
+          }
         }
+      }
+#pragma unroll
+      for (int t = 0; t < kTokPerWarp; ++t) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float l = warp_sum(acc[t][i]);
+          if (i < ni && ((active >> t) & 1u) && lane == t)
+            lg[(size_t)slot_of[t] * K + i0 + i] = l + a.be[g * K + i0 + i];
+        }
+      }
+    }
+    j0 = j1;
+  }
+  __syncthreads();
+
+  // ---- top-k and gates: one thread per token
+  if (threadIdx.x < kTileTokens && tok0 + threadIdx.x < a.T)
+    select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
+                     a.expert_ids, a.gates, a.slot_local);
+}
+
+// One block per token; warp w covers the 256-column segments w, w + nwarp, ...
+__global__ void __launch_bounds__(256)
+router_token_kernel(const RouterArgs a) {
+  __shared__ float part[8][kMaxG];      // also reused for the expert logits (kMaxK <= kMaxG)
+  __shared__ float lg[kMaxG];
+  __shared__ int s_g;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  const int t = blockIdx.x, d = a.d;
+  const __half* xr = a.x + (size_t)t * d;
+  for (int pass = 0; pass < 2; ++pass) {
+    const int n = pass == 0 ? a.G : a.K;
+    const float* W = pass == 0 ? a.Ct : a.Rt + (size_t)s_g * a.K * d;
+    for (int j = 0; j < n; ++j) {
+      float acc = 0.f;
+      for (int c = warp * 256 + lane * 8; c < d; c += nwarp * 256) {
+        const uint4 xv = *reinterpret_cast<const uint4*>(xr + c);
+        const float* wr = W + (size_t)j * d + c;
+        fma8(acc, xv, __ldg(reinterpret_cast<const float4*>(wr)), __ldg(reinterpret_cast<const float4*>(wr + 4)));
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) part[warp][j] = acc;
+    }
+    __syncthreads();
+    if (threadIdx.x < n) {
+      float v = 0.f;
+      for (int w = 0; w < nwarp; ++w) v += part[w][threadIdx.x];
+      lg[threadIdx.x] = v + (pass == 0 ? a.bc[threadIdx.x] : a.be[s_g * a.K + threadIdx.x]);
+    }
+    __syncthreads();
+    if (pass == 0) {
+      if (threadIdx.x == 0) {
+        int gs = 0;
+        float zb = lg[0];
+        for (int g = 1; g < a.G; ++g)
+          if (lg[g] > zb) { zb = lg[g]; gs = g; }          // strict >: lowest index wins ties
+        s_g = gs;
+        a.cluster_id[t] = gs;
+      }
+      __syncthreads();
     }
   }
+  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local);
 }
 
 }  // namespace
@@ -103,11 +274,28 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
                           cudaStream_t st) {
   if (T <= 0) return cudaSuccess;
-  const int warps = 8;
-  int blocks = (T + warps - 1) / warps;
-  if (blocks > 148 * 8) blocks = 148 * 8;
-  router_kernel<<<blocks, warps * 32, 0, st>>>(x, T, D.d, D.G, D.K, D.k, W.Ct, W.Rt, W.bc, W.be,
-                                               W.label, cluster_id, expert_ids, gates, slot_local);
+  RouterArgs a{};
+  a.x = x; a.T = T; a.d = D.d; a.G = D.G; a.K = D.K; a.k = D.k;
+  a.Ct = W.Ct; a.Rt = W.Rt; a.bc = W.bc; a.be = W.be; a.label = W.label;
+  a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;
+  if (T < 1024) {
+    // few tokens: the per-token kernel puts every token on its own SM
+    router_token_kernel<<<T, 256, 0, st>>>(a);
+    return cudaGetLastError();
+  }
+  // chunk of the prototypes staged at a time: at most 32 KB for a group of eight clusters
+  const int rows = D.G < kGroup ? D.G : kGroup;
+  int dc = 32768 / (4 * rows) / 256 * 256;
+  if (dc > D.d) dc = D.d;
+  a.dc = dc;
+  const size_t sh = sizeof(float) * ((size_t)kGroup * dc + (size_t)kTileTokens * D.K);
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(router_tile_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  router_tile_kernel<<<(T + kTileTokens - 1) / kTileTokens, kTileWarps * 32, sh, st>>>(a);
   return cudaGetLastError();
 }
 

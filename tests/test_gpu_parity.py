@@ -162,6 +162,28 @@ def test_permutation_equivariance_on_gpu():
     assert torch.allclose(yp, y[perm], atol=2e-3, rtol=1e-3)
 
 
+# ---- batches large enough for the tiled router kernel (T >= 1024), on odd router shapes ---------------
+@pytest.mark.parametrize("kw", [
+    dict(T=1100, d=96, d_ff=64, E=36, G=12, r=0, k=2),      # more than eight clusters, K = 3
+    dict(T=1500, d=160, d_ff=64, E=10, G=2, r=0, k=3),      # K = 5: a ragged group of expert rows
+    dict(T=1027, d=1056, d_ff=32, E=8, G=8, r=0, k=1),      # d not a multiple of 256, one expert per cluster
+    dict(T=2048, d=2304, d_ff=32, E=64, G=2, r=0, k=8),     # prototypes staged in several chunks, K = 32
+], ids=["G12", "K5", "d1056", "d2304_K32"])
+def test_router_tile_kernel_shapes(kw):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(**kw)
+    L = inputs.make_layer(s, 17)
+    rng = np.random.default_rng(1)
+    L["b_c"] = (rng.standard_normal(s.G) * 0.2).astype(np.float32)
+    L["b_e"] = (rng.standard_normal((s.G, s.K)) * 0.2).astype(np.float32)
+    m = ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    cid, eid, gates = m.route(x)
+    torch.cuda.synchronize()
+    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+
+
 # ---- shapes that take the tensor-core path (d, d_ff multiples of 128, T_max > 128) ----------------
 @pytest.mark.parametrize("T", [129, 200, 640, 1111])
 def test_tensor_path_ragged(T):
