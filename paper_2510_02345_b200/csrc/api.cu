@@ -51,7 +51,9 @@ int validate_dims(const cmoe_desc* desc, Dims* D) {
   D->nkey = D->G * D->nsub;
   if (D->nkey > kMaxKeys) return CMOE_ERR_UNSUPPORTED_SHAPE;
   D->tc2 = (tc2_supported(*D) && D->T_max > 128) ? 1 : 0;
-  D->row_align = D->tc2 ? 256 : 128;     // CTA pairs work on 256-row tiles of one cluster
+  D->stream = (!D->tc2 && stream_supported(*D)) ? 1 : 0;
+  // CTA pairs work on 256-row tiles of one cluster; the streaming path on 16-row token blocks
+  D->row_align = D->tc2 ? 256 : (D->stream ? 16 : 128);
   D->T_pad_max = t_pad_bound(*D, D->T_max);
   return CMOE_OK;
 }
@@ -107,6 +109,10 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
     s.Ad = A.take<__half>(P * 64);
     s.As = A.take<__half>(P * 64);
     s.tile_mask = A.take<int>(P / 128 * 2);
+  }
+  if (D.stream) {
+    if (r > 0) s.a_slot = A.take<__half>(P * k * f);
+    s.y32 = A.take<float>(P * d);
   }
   if (W) *W = w;
   if (S) *S = s;
@@ -232,6 +238,9 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
     if ((e = tc2_init(L))) return fail(e);
     L->path = kPathTensor;
     L->tc_variant = 2;
+  } else if (D.stream && forced != kPathGeneric) {
+    if ((e = stream_init(L))) return fail(e);
+    L->path = kPathStream;
   } else if (tc_supported(D) && D.T_max > 128 && forced != kPathGeneric) {
     if ((e = tc_init(L))) return fail(e);
     L->path = kPathTensor;
@@ -276,6 +285,8 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
+  else if (L->path == kPathStream)
+    CMOE_CUDA(L, launch_stream_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else if (L->path == kPathTensor)
     CMOE_CUDA(L, launch_tc_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else
@@ -310,8 +321,8 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->launches_forward = 1 + kPermuteLaunches +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L->dims)
-                               : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
-  out->memsets_forward = L->dims.r > 0 ? 1 : 0;
+                               : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
+  out->memsets_forward = (L->dims.r > 0 ? 1 : 0) + (L->path == kPathStream ? 1 : 0);
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;
   out->T_pad_max = L->dims.T_pad_max;

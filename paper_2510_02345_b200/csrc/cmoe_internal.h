@@ -28,6 +28,7 @@ struct Dims {
   int row_align;   // a cluster's rows start at a multiple of this
   int sub_is_combo;
   int tc2;         // the shape takes the tensor-core path with tensor-core residuals (tc2_path.cu)
+  int stream;      // the shape takes the weight-streaming path (stream_path.cu)
 };
 
 // Weights as re-laid-out in the arena by cmoe_create.
@@ -72,6 +73,9 @@ struct Scratch {
   __half *U1f, *V1f, *U2f, *V2f;   // INT4 factors decoded to fp16 operand matrices, per call
   __half *A0, *Ad, *As;            // [T_pad][64] expanded-rank-index operands
   int* tile_mask;                  // [T_pad / 128][2]
+  // weight-streaming path only (see stream_path.cu)
+  __half* a_slot;                  // [T_pad][k][d_ff]  GELU(h_j) of every kept expert
+  float* y32;                      // [T_pad][d]        fp32 sum of the K ranges of the down-projection
 };
 
 }  // namespace cmoe
@@ -123,6 +127,11 @@ bool tc2_supported(const Dims& D);
 cudaError_t tc2_init(cmoe_layer* L);
 int tc2_launch_count(const Dims& D);
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
+// stream_path.cu : small batches, bound by streaming the bases from HBM
+bool stream_supported(const Dims& D);
+cudaError_t stream_init(cmoe_layer* L);
+int stream_launch_count(const Dims& D);
+cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // repack.cu : create-time layout changes
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
                                   cudaStream_t st);

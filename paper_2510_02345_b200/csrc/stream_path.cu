@@ -1,0 +1,474 @@
+// Weight-streaming path of the expert FFNs for small batches (decode): with a handful of tokens per
+// cluster the layer is bound by reading the FP16 bases once from HBM, so the kernels are laid out
+// around the weight stream (sm_100a: TMA into shared memory, tcgen05 MMAs with TMEM accumulators).
+//
+// The roles of the two GEMM operands are swapped with respect to the large-batch path: the WEIGHTS
+// are the 128-row A operand (a tile of output features, streamed once), the cluster's few tokens
+// are the narrow B operand (N = 16..64, re-read from L2), and the accumulator holds
+// D[feature][token].  Tensor-core rows cost nothing here; bytes do.
+//
+//   t      t_j = x U1_e for every (row, kept expert)                 (CUDA cores, tiny)
+//   up     D = B1t_g[f-tile] x_g^T; epilogue per feature f (one thread each): h_j = D + t_j V1_e[f],
+//          a_j = GELU(h_j) (erf form) -> fp16, abar = sum_j p_j a_j -> fp16; the INT4 codes of
+//          V1_e[f, :] are read and decoded in registers right here
+//   s      s_j = a_j U2_e                                            (CUDA cores, tiny)
+//   down   D = B2t_g[c-tile, K range] abar_g^T, split along K over several CTAs, added to a fp32
+//          copy of y with atomics
+//   final  y = fp16(y32 + sum_j p_j s_j V2_e), stored un-permuted
+//
+// A cluster's rows are aligned to 16 (the MMA's N granularity) and cut into segments of at most 64
+// rows; a work unit is (segment, tile of features[, K range]), dealt round-robin to the CTAs.
+// Every device wait is bounded (status word CMOE_ERR_TIMEOUT on expiry).
+#include "cmoe_internal.h"
+#include "device_utils.cuh"
+#include "tc_ptx.cuh"
+
+namespace cmoe {
+
+namespace {
+
+using namespace ptx;
+
+constexpr int SBK = 64;            // halves per K atom: one 128-byte swizzle row
+constexpr int SKA = 2;             // K atoms per stage
+constexpr int SNB = 64;            // most token rows per segment (MMA N)
+constexpr int SMAXSEG = 160;       // segments: at most G + T_pad / 64
+constexpr int S_THREADS = 256;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..7 epilogue
+constexpr uint32_t S_B_ATOM = SNB * SBK * 2;             // 8 KB
+constexpr uint32_t S_TMEM_COLS = 128;                    // two accumulators of up to 64 columns
+
+struct StreamParams {
+  const int* seg_off;        // [G+1] first permuted row of each cluster (multiples of 16)
+  const int* row_slot;       // [rows][k]
+  const float* row_gate;     // [rows][k]
+  const int* row_token;      // [rows]
+  // up
+  const float* t;            // [rows][k][r]
+  const uint8_t* V1q;        // packed INT4 in the boundary layout
+  const __half* V1s;
+  __half* a_slot;            // [rows][k][d_ff]  GELU(h_j) of every kept expert
+  __half* abar;              // [rows][d_ff]
+  // down
+  float* y32;                // [rows][d], zeroed by the caller
+  int* status;
+  int G, K, k, r;
+  int Kd;                    // reduction length (d for up, d_ff for down)
+  int M;                     // output features (d_ff for up, d for down)
+  int ksplit;                // down: K ranges per tile
+};
+
+template <int MROWS>
+struct SCfg {
+  static constexpr uint32_t A_ATOM = MROWS * SBK * 2;
+  static constexpr uint32_t A_BYTES = SKA * A_ATOM;
+  static constexpr uint32_t B_BYTES = SKA * S_B_ATOM;
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = MROWS == 64 ? 6 : 4;                 // 32 KB x 6 / 48 KB x 4
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 64 * 8 + SMAXSEG * 12 + 64;
+};
+
+// UP: MROWS = 64 feature rows per tile (the MMA still spans 128 rows; the upper half of the
+// accumulator is never read).  DOWN: 128 rows.
+template <bool UP>
+__global__ void __launch_bounds__(S_THREADS, 1)
+stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmTok,
+              const StreamParams p) {
+  constexpr int MROWS = UP ? 64 : 128;
+  using Cfg = SCfg<MROWS>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* sm = smem_raw + (base - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)STAGES * Cfg::STAGE_BYTES);
+  const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8);
+  const uint32_t tfull0 = smem_u32(bars + 16), tempty0 = smem_u32(bars + 18);
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 20);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  int* n_seg_p = reinterpret_cast<int*>(tmem_holder + 2);
+  int* seg_row0 = reinterpret_cast<int*>(bars + 64);       // [SMAXSEG]
+  int* seg_rows = seg_row0 + SMAXSEG;
+  int* seg_g = seg_rows + SMAXSEG;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kEpiWarps = MROWS / 32;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, kEpiWarps); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // segments of at most SNB rows
+    int n = 0;
+    for (int g = 0; g < p.G; ++g) {
+      const int r0 = p.seg_off[g], r1 = p.seg_off[g + 1];
+      for (int r = r0; r < r1 && n < SMAXSEG; r += SNB) {
+        seg_row0[n] = r; seg_rows[n] = min(SNB, r1 - r); seg_g[n] = g; ++n;
+      }
+    }
+    *n_seg_p = n;
+  }
+  if (warp == 2) {
+    __syncwarp();
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_holder)), "r"(S_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  // work units: u = (seg * n_mt + mt) * ksplit + ks
+  const int n_mt = p.M / MROWS;
+  const int ksplit = UP ? 1 : p.ksplit;
+  const int KCH = p.Kd / (SBK * SKA);                    // stages in the whole reduction
+  const int n_units = *n_seg_p * n_mt * ksplit;
+  const int my_units = (int)blockIdx.x < n_units ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  auto unit_of = [&](int i, int& seg, int& mt, int& c_begin, int& c_end) {
+    const int u = blockIdx.x + i * gridDim.x;
+    const int ks = u % ksplit, sm_ = u / ksplit;
+    mt = sm_ % n_mt;
+    seg = sm_ / n_mt;
+    c_begin = (int)((long long)KCH * ks / ksplit);
+    c_end = (int)((long long)KCH * (ks + 1) / ksplit);
+  };
+  bool failed = false;
+
+  if (warp == 0 || warp == 3) {
+    // ---------------- TMA producers: two threads take alternate stages of the flattened stage sequence
+    if (lane == 0) {
+      uint32_t it = 0;                                     // stage counter over all units
+      const uint32_t mine = warp == 0 ? 0u : 1u;
+      for (int i = 0; i < my_units && !failed; ++i) {
+        int seg, mt, c0, c1;
+        unit_of(i, seg, mt, c0, c1);
+        const int g = seg_g[seg], row0 = seg_row0[seg], nb = seg_rows[seg] / 16;
+        const int wrow = g * p.M + mt * MROWS;
+        for (int c = c0; c < c1; ++c, ++it) {
+          if ((it & 1u) != mine) continue;
+          const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+          if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * Cfg::STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
+          mbar_expect_tx(full0 + 8 * s, Cfg::A_BYTES + (uint32_t)nb * SKA * 16 * SBK * 2);
+          tma_load_3d(a_dst, &tmW, full0 + 8 * s, 0, wrow, c * SKA);
+          // the tokens: 16 rows per box; atom a of block b lands at atom a, rows 16 b .. of the B tile
+          for (int b = 0; b < nb; ++b)
+            for (int a = 0; a < SKA; ++a)
+              tma_load_2d(b_dst + a * S_B_ATOM + b * (16 * SBK * 2), &tmTok, full0 + 8 * s, (c * SKA + a) * SBK, row0 + 16 * b);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      uint32_t s = 0, ph = 0;
+      for (int i = 0; i < my_units && !failed; ++i) {
+        int seg, mt, c0, c1;
+        unit_of(i, seg, mt, c0, c1);
+        const uint32_t idesc = idesc_f16(128, seg_rows[seg]);
+        const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
+        if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * SNB;
+        for (int c = c0; c < c1; ++c) {
+          if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint32_t a_src = base + s * Cfg::STAGE_BYTES, b_src = a_src + Cfg::A_BYTES;
+          const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+          umma_f16(d_tmem, adesc, bdesc, idesc, c != c0 ? 1u : 0u);
+#pragma unroll
+          for (int ks = 1; ks < SBK / 16; ++ks) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
+#pragma unroll
+          for (int ks = 0; ks < SBK / 16; ++ks)
+            umma_f16(d_tmem, adesc + (Cfg::A_ATOM >> 4) + 2 * ks, bdesc + (S_B_ATOM >> 4) + 2 * ks, idesc, 1u);
+          umma_commit(empty0 + 8 * s);
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (failed) break;
+        umma_commit(tfull0 + 8 * acc);
+      }
+    }
+  } else if (warp >= 4 && warp < 4 + kEpiWarps) {
+    // ---------------- epilogue warps: one thread per output feature of the tile
+    const int q = warp & 3;
+    const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
+    const int r = p.r, k = p.k, M = p.M;
+    for (int i = 0; i < my_units; ++i) {
+      int seg, mt, c0, c1;
+      unit_of(i, seg, mt, c0, c1);
+      const int row0 = seg_row0[seg], nrows = seg_rows[seg];
+      const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
+      const int f = mt * MROWS + q * 32 + lane;            // output feature (up) / output column (down)
+      {
+        const bool ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag);
+        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+      }
+      tc_fence_after();
+      for (int tb = 0; tb < nrows; tb += 16) {
+        uint32_t v[16];
+        tmem_ld16_nowait(taddr + acc * SNB + tb, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; ++c) {
+          const int row = row0 + tb + c;
+          const bool real = p.row_token[row] >= 0;         // the same for every thread
+          const float dv = __uint_as_float(v[c]);
+          if (UP) {
+            float ab = 0.f;
+            if (real) {
+              for (int j = 0; j < k; ++j) {
+                const int e = p.row_slot[(size_t)row * k + j];
+                float h = dv;
+                if (r > 0) {
+                  // h += t_j . V1_e[f, :]: r codes of one scale group, decoded in registers
+                  const float* tp = p.t + ((size_t)row * k + j) * r;
+                  const long long flat = ((long long)e * M + f) * r;
+                  const float sc = __half2float(p.V1s[flat >> 5]);
+                  float dot = 0.f;
+                  if (r >= 8) {
+                    const uint32_t* wq = reinterpret_cast<const uint32_t*>(p.V1q + (flat >> 1));
+                    for (int w8 = 0; w8 < r / 8; ++w8) {
+                      const uint32_t word = wq[w8];
+#pragma unroll
+                      for (int n = 0; n < 8; ++n) dot = fmaf(tp[w8 * 8 + n], (float)sext4((int)(word >> (4 * n))), dot);
+                    }
+                  } else {
+                    const uint32_t word = *reinterpret_cast<const uint16_t*>(p.V1q + (flat >> 1));
+#pragma unroll
+                    for (int n = 0; n < 4; ++n) dot = fmaf(tp[n], (float)sext4((int)(word >> (4 * n))), dot);
+                  }
+                  h = fmaf(sc, dot, h);
+                }
+                const float a = gelu_erf(h);
+                ab = fmaf(p.row_gate[(size_t)row * k + j], a, ab);
+                if (r > 0) p.a_slot[((size_t)row * k + j) * M + f] = __float2half_rn(a);
+              }
+            }
+            p.abar[(size_t)row * M + f] = __float2half_rn(ab);
+          } else {
+            if (real) atomicAdd(p.y32 + (size_t)row * M + f, dv);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty0 + 8 * acc);
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
+  }
+  __syncthreads();
+  if (*abort_flag) {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 400000ll) { }       // let copies already issued land
+    __syncthreads();
+  }
+  tc_fence_after();
+  if (warp == 2)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(S_TMEM_COLS) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// rank-r projections of one vector per (row, kept expert):  out[item][p] = sum_c in[item][c] U_e[p][c]
+// with U packed INT4 [E][r][len].  t = x U1 (in = the row's activations) and s = a_j U2 (in = the
+// activation of that row and slot).  One block per item, a warp per rank index, lanes over the
+// 32-element scale groups.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
+               const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
+               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+  const int item = blockIdx.x;
+  const int row = item / k;
+  if (row >= seg_off[G] || row_token[row] < 0) {
+    if (row < seg_off[G]) for (int pr = threadIdx.x; pr < r; pr += blockDim.x) out[(size_t)item * r + pr] = 0.f;
+    return;
+  }
+  const int e = row_slot[item];
+  const __half* xin = in + (size_t)(in_per_slot ? item : row) * len;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  for (int pr = warp; pr < r; pr += nwarp) {
+    const long long base = ((long long)e * r + pr) * len;
+    float acc = 0.f;
+    for (int grp = lane; grp * 32 < len; grp += 32) {
+      const uint4 pk = *reinterpret_cast<const uint4*>(Uq + ((base + grp * 32) >> 1));
+      const float sc = __half2float(Us[(base >> 5) + grp]);
+      const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
+      float part = 0.f;
+#pragma unroll
+      for (int qd = 0; qd < 4; ++qd) {
+        const uint4 xv = *reinterpret_cast<const uint4*>(xin + grp * 32 + qd * 8);
+        const __half* xh = reinterpret_cast<const __half*>(&xv);
+#pragma unroll
+        for (int n = 0; n < 8; ++n) part = fmaf(__half2float(xh[n]), (float)sext4((int)(w[qd] >> (4 * n))), part);
+      }
+      acc = fmaf(part, sc, acc);
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) out[(size_t)item * r + pr] = acc;
+  }
+}
+
+// y[tok] = fp16(y32[row] + sum_j p_j s_j V2_e), one thread per (row, output column)
+__global__ void __launch_bounds__(256)
+stream_final_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r,
+                    const float* __restrict__ y32, const float* __restrict__ s, const int* __restrict__ row_slot,
+                    const float* __restrict__ row_gate, const int* __restrict__ row_token,
+                    const uint8_t* __restrict__ V2q, const __half* __restrict__ V2s, __half* __restrict__ y) {
+  const int row = blockIdx.y;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= seg_off[G] || c >= d) return;
+  const int tok = row_token[row];
+  if (tok < 0) return;
+  float v = y32[(size_t)row * d + c];
+  for (int j = 0; j < k && r > 0; ++j) {
+    const int e = row_slot[(size_t)row * k + j];
+    const float* sj = s + ((size_t)row * k + j) * r;
+    const long long flat = ((long long)e * d + c) * r;
+    float u = 0.f;
+    for (int pr = 0; pr < r; ++pr) u = fmaf(sj[pr], deq4(V2q, V2s, flat + pr), u);
+    v = fmaf(row_gate[(size_t)row * k + j], u, v);
+  }
+  y[(size_t)tok * d + c] = __float2half_rn(v);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// fp16 matrix [rows][cols]; katoms == 0: 2-D box of box_rows x 64 halves; otherwise the matrix is seen
+// as [cols / 64][rows][64] and the box takes katoms K atoms (consecutive swizzled tiles in shared memory)
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t katoms) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t gdim[3] = {katoms ? (cuuint64_t)SBK : cols, rows, cols / SBK};
+  cuuint64_t gstride[2] = {cols * 2, (cuuint64_t)SBK * 2};
+  cuuint32_t box[3] = {(cuuint32_t)SBK, box_rows, katoms};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, katoms ? 3 : 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct StreamState {
+  CUtensorMap mW1, mX, mW2, mAbar;
+  int sm_count;
+  int ksplit;
+};
+static_assert(sizeof(StreamState) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
+
+template <bool UP>
+cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mTok, const StreamParams& p, int grid, cudaStream_t st) {
+  auto kern = stream_kernel<UP>;
+  constexpr size_t sm = SCfg<UP ? 64 : 128>::SMEM;
+  static_assert(sm <= 232448, "stream kernel shared memory");
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  kern<<<grid, S_THREADS, sm, st>>>(mW, mTok, p);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+bool stream_supported(const Dims& D) {
+  return D.d % 128 == 0 && D.d_ff % 128 == 0 && D.T_max <= 128;
+}
+
+cudaError_t stream_init(cmoe_layer* L) {
+  const Dims& D = L->dims;
+  const Scratch& S = L->sc;
+  StreamState* ts = reinterpret_cast<StreamState*>(L->tc_state);
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (e != cudaSuccess) return e;
+  const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
+  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 64, SKA) && make_map(&ts->mX, S.x_perm, P, D.d, 16, 0) &&
+                  make_map(&ts->mW2, L->w.B2t, G * D.d, D.d_ff, 128, SKA) && make_map(&ts->mAbar, S.abar, P, D.d_ff, 16, 0);
+  // K ranges per down tile: fill the SMs evenly, keep at least four stages per range
+  const int kch = D.d_ff / (SBK * SKA);
+  const long long tiles = (long long)D.G * (D.d / 128);
+  int best = 1;
+  double best_eff = 0.0;
+  for (int ks = 1; ks <= 16 && kch / ks >= 4; ++ks) {
+    const long long units = tiles * ks, waves = (units + ts->sm_count - 1) / ts->sm_count;
+    const double eff = (double)units / (double)(waves * ts->sm_count);
+    if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
+  }
+  ts->ksplit = best;
+  return ok ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int stream_launch_count(const Dims& D) { return D.r > 0 ? 5 : 3; }
+
+cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
+  const Dims& D = L->dims;
+  const Weights& W = L->w;
+  const Scratch& S = L->sc;
+  const StreamState& ts = *reinterpret_cast<const StreamState*>(L->tc_state);
+  const int rows_bound = t_pad_bound(D, T);
+  cudaError_t e;
+  if (marks) cudaEventRecord(marks[0], st);
+  if ((e = cudaMemsetAsync(S.y32, 0, sizeof(float) * (size_t)rows_bound * D.d, st)) != cudaSuccess) return e;
+  if (D.r > 0) {
+    lowrank_kernel<<<rows_bound * D.k, 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
+                                                      W.U1q, W.U1s, S.t);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  if (marks) cudaEventRecord(marks[1], st);
+  StreamParams p{};
+  p.seg_off = S.seg_off; p.row_slot = S.row_slot; p.row_gate = S.row_gate; p.row_token = S.row_token;
+  p.t = S.t; p.V1q = W.V1q; p.V1s = W.V1s; p.a_slot = S.a_slot; p.abar = S.abar; p.y32 = S.y32; p.status = S.status;
+  p.G = D.G; p.K = D.K; p.k = D.k; p.r = D.r;
+  const int seg_bound = D.G + rows_bound / SNB;
+  {
+    p.Kd = D.d; p.M = D.d_ff; p.ksplit = 1;
+    const long long units = (long long)seg_bound * (D.d_ff / 64);
+    const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
+    if ((e = launch_stream<true>(ts.mW1, ts.mX, p, grid, st)) != cudaSuccess) return e;
+  }
+  if (marks) cudaEventRecord(marks[2], st);
+  if (D.r > 0) {
+    lowrank_kernel<<<rows_bound * D.k, 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
+                                                      W.U2q, W.U2s, S.s);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  }
+  {
+    p.Kd = D.d_ff; p.M = D.d; p.ksplit = ts.ksplit;
+    const long long units = (long long)seg_bound * (D.d / 128) * ts.ksplit;
+    const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
+    if ((e = launch_stream<false>(ts.mW2, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
+  }
+  dim3 fgrid((D.d + 255) / 256, rows_bound);
+  stream_final_kernel<<<fgrid, 256, 0, st>>>(S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
+                                             S.row_token, W.V2q, W.V2s, y);
+  return cudaGetLastError();
+}
+
+}  // namespace cmoe

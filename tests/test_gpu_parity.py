@@ -213,3 +213,40 @@ def test_tensor_path_empty_cluster():
     L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)
     got = full_check(L, L["x"])
     assert got["module"].info.path == 1 and not np.any(got["cid"] == 1)
+
+
+# ---- shapes that take the weight-streaming path (T_max <= 128, d and d_ff multiples of 128) ---------
+@pytest.mark.parametrize("kw", [
+    dict(T=1, d=128, d_ff=128, E=8, G=2, r=4, k=2),
+    dict(T=5, d=256, d_ff=384, E=8, G=2, r=16, k=2),
+    dict(T=64, d=128, d_ff=256, E=16, G=2, r=32, k=3),      # K = 8, odd k, largest rank
+    dict(T=100, d=256, d_ff=128, E=4, G=1, r=8, k=2),       # one cluster: two token segments (64 + 36)
+    dict(T=128, d=384, d_ff=640, E=6, G=3, r=0, k=2),       # no residual, ragged K split
+    dict(T=77, d=128, d_ff=256, E=5, G=5, r=4, k=1),        # one expert per cluster
+], ids=["T1", "T5", "K8k3r32", "G1_two_segments", "r0", "K1"])
+def test_stream_path_variants(kw):
+    s = inputs.small_shape(**kw)
+    L = inputs.make_layer(s, 21)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 2
+
+
+def test_stream_path_empty_cluster_and_reuse():
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=90, d=128, d_ff=256, E=12, G=3, r=16, k=2)
+    L = inputs.make_layer(s, 22)
+    L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 2 and not np.any(got["cid"] == 1)
+    m = ClusteredMoELayer(L, T_max=128)
+    o = ref.Layer(L)
+    for T in (128, 3, 40):                                  # the same handle, different batch sizes
+        x_np = inputs.make_tokens(s, T, seed=T)
+        x = torch.from_numpy(x_np).cuda()
+        cid, eid, gates = m.route(x)
+        y = m.forward(x)
+        torch.cuda.synchronize()
+        decided, _ = check_routes(s, o.route(x_np), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+        check_y(y.float().cpu().numpy(), o.forward(x_np), decided)
+    assert m.status() == 0
