@@ -6,8 +6,10 @@
 //   hist     per-block histogram of the keys (block = 256 consecutive tokens)
 //   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
-//            writes the row tables and moves the token's activations with 16-byte vectors
-//   pad      fills the padding rows of each segment (zero activations, zero gates)
+//            writes the row tables
+//   pad      fills the table entries of the padding rows of each segment (no token, zero gates)
+//   move     copies every token's activations to its row with 16-byte vectors (a block per row;
+//            padding rows get zeros)
 //
 // The result is deterministic: rows of one key keep the token order.
 #include "cmoe_internal.h"
@@ -157,15 +159,22 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
         row_gate[(size_t)row * k + j] = cg[j];
       }
   }
-  // row move: the warp copies its 32 tokens' rows one after the other, 16 bytes per lane
+}
+
+// x_perm[row] = x[row_token[row]], zeros for padding rows; a block per row, 16 bytes per thread
+__global__ void __launch_bounds__(128)
+move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ row_token,
+                 const __half* __restrict__ x, __half* __restrict__ x_perm) {
   const int vec_per_row = d / 8;
-  for (int i = 0; i < 32; ++i) {
-    int src_t = __shfl_sync(0xffffffffu, t, i);
-    int dst_r = __shfl_sync(0xffffffffu, row, i);
-    if (dst_r < 0) continue;
-    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)src_t * d);
-    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)dst_r * d);
-    for (int v = lane; v < vec_per_row; v += 32) dst[v] = src[v];
+  for (int row = blockIdx.x; row < *n_rows; row += gridDim.x) {
+    const int tok = row_token[row];
+    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
+    if (tok >= 0) {
+      const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)tok * d);
+      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = src[v];
+    } else {
+      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+    }
   }
 }
 
@@ -176,15 +185,12 @@ pad_kernel(int d, int K, int k, const int* __restrict__ seg_off, const int* __re
   const int g = blockIdx.x;
   const int first = seg_off[g] + seg_cnt[g], last = seg_off[g + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  const int vec_per_row = d / 8;
   for (int row = first + warp; row < last; row += nwarp) {
     if (lane == 0) row_token[row] = -1;
     if (lane < k) {
       row_slot[(size_t)row * k + lane] = g * K + lane;   // any valid experts of the cluster
       row_gate[(size_t)row * k + lane] = 0.f;
     }
-    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
-    for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0, 0, 0, 0);
   }
 }
 
@@ -204,6 +210,8 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                                                S.x_perm);
   pad_kernel<<<D.G, 256, 0, st>>>(D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
                                   S.row_gate, S.x_perm);
+  const int rows_bound = t_pad_bound(D, T);
+  move_rows_kernel<<<rows_bound < 148 * 32 ? rows_bound : 148 * 32, 128, 0, st>>>(D.d, S.n_rows, S.row_token, x, S.x_perm);
   return cudaGetLastError();
 }
 

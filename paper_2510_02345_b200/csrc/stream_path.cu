@@ -63,17 +63,19 @@ struct SCfg {
   static constexpr uint32_t A_BYTES = SKA * A_ATOM;
   static constexpr uint32_t B_BYTES = SKA * S_B_ATOM;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
-  static constexpr int STAGES = MROWS == 64 ? 6 : 4;                 // 32 KB x 6 / 48 KB x 4
+  static constexpr int STAGES = 4;                                   // 48 KB each
   static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 64 * 8 + SMAXSEG * 12 + 64;
 };
 
-// UP: MROWS = 64 feature rows per tile (the MMA still spans 128 rows; the upper half of the
-// accumulator is never read).  DOWN: 128 rows.
+// Tiles have 128 feature rows.  In the up kernel the tiles of the last, incomplete round of the
+// round-robin are cut into halves of 64 rows (loaded with tmWh; the MMA still spans 128 rows and the
+// upper half of the accumulator is not read), so that the tail occupies twice as many SMs for half
+// as long.  The down kernel gets its granularity from the K ranges.
 template <bool UP>
 __global__ void __launch_bounds__(S_THREADS, 1)
-stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmTok,
-              const StreamParams p) {
-  constexpr int MROWS = UP ? 64 : 128;
+stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWh,
+              const __grid_constant__ CUtensorMap tmTok, const StreamParams p) {
+  constexpr int MROWS = 128;
   using Cfg = SCfg<MROWS>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -123,10 +125,19 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
   const int n_mt = p.M / MROWS;
   const int ksplit = UP ? 1 : p.ksplit;
   const int KCH = p.Kd / (SBK * SKA);                    // stages in the whole reduction
-  const int n_units = *n_seg_p * n_mt * ksplit;
+  const int n_tiles = *n_seg_p * n_mt * ksplit;
+  int n_whole = n_tiles;                                 // units [0, n_whole) are whole tiles, the rest halves
+  if (UP) {
+    const int tail = n_tiles % (int)gridDim.x;
+    if (tail > 0 && 2 * tail <= (int)gridDim.x) n_whole = n_tiles - tail;
+  }
+  const int n_units = n_whole + 2 * (n_tiles - n_whole);
   const int my_units = (int)blockIdx.x < n_units ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  auto unit_of = [&](int i, int& seg, int& mt, int& c_begin, int& c_end) {
-    const int u = blockIdx.x + i * gridDim.x;
+  // half: -1 for a whole tile, else which 64 rows of the tile
+  auto unit_of = [&](int i, int& seg, int& mt, int& half, int& c_begin, int& c_end) {
+    int u = blockIdx.x + i * gridDim.x;
+    half = -1;
+    if (u >= n_whole) { half = (u - n_whole) & 1; u = n_whole + ((u - n_whole) >> 1); }
     const int ks = u % ksplit, sm_ = u / ksplit;
     mt = sm_ % n_mt;
     seg = sm_ / n_mt;
@@ -141,17 +152,18 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
       uint32_t it = 0;                                     // stage counter over all units
       const uint32_t mine = warp == 0 ? 0u : 1u;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, c0, c1;
-        unit_of(i, seg, mt, c0, c1);
+        int seg, mt, half, c0, c1;
+        unit_of(i, seg, mt, half, c0, c1);
         const int g = seg_g[seg], row0 = seg_row0[seg], nb = seg_rows[seg] / 16;
-        const int wrow = g * p.M + mt * MROWS;
+        const int wrow = g * p.M + mt * MROWS + (half > 0 ? 64 : 0);
+        const uint32_t a_bytes = half < 0 ? Cfg::A_BYTES : Cfg::A_BYTES / 2;
         for (int c = c0; c < c1; ++c, ++it) {
           if ((it & 1u) != mine) continue;
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
           const uint32_t a_dst = base + s * Cfg::STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
-          mbar_expect_tx(full0 + 8 * s, Cfg::A_BYTES + (uint32_t)nb * SKA * 16 * SBK * 2);
-          tma_load_3d(a_dst, &tmW, full0 + 8 * s, 0, wrow, c * SKA);
+          mbar_expect_tx(full0 + 8 * s, a_bytes + (uint32_t)nb * SKA * 16 * SBK * 2);
+          tma_load_3d(a_dst, half < 0 ? &tmW : &tmWh, full0 + 8 * s, 0, wrow, c * SKA);
           // the tokens: 16 rows per box; atom a of block b lands at atom a, rows 16 b .. of the B tile
           for (int b = 0; b < nb; ++b)
             for (int a = 0; a < SKA; ++a)
@@ -164,9 +176,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, c0, c1;
-        unit_of(i, seg, mt, c0, c1);
+        int seg, mt, half, c0, c1;
+        unit_of(i, seg, mt, half, c0, c1);
         const uint32_t idesc = idesc_f16(128, seg_rows[seg]);
+        const uint32_t a_atom16 = (half < 0 ? Cfg::A_ATOM : Cfg::A_ATOM / 2) >> 4;   // second K atom, in 16-byte units
         const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
         if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
@@ -181,7 +194,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
           for (int ks = 1; ks < SBK / 16; ++ks) umma_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
 #pragma unroll
           for (int ks = 0; ks < SBK / 16; ++ks)
-            umma_f16(d_tmem, adesc + (Cfg::A_ATOM >> 4) + 2 * ks, bdesc + (S_B_ATOM >> 4) + 2 * ks, idesc, 1u);
+            umma_f16(d_tmem, adesc + a_atom16 + 2 * ks, bdesc + (S_B_ATOM >> 4) + 2 * ks, idesc, 1u);
           umma_commit(empty0 + 8 * s);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -195,11 +208,11 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int r = p.r, k = p.k, M = p.M;
     for (int i = 0; i < my_units; ++i) {
-      int seg, mt, c0, c1;
-      unit_of(i, seg, mt, c0, c1);
-      const int row0 = seg_row0[seg], nrows = seg_rows[seg];
+      int seg, mt, half, c0, c1;
+      unit_of(i, seg, mt, half, c0, c1);
+      const int row0 = seg_row0[seg], nrows = half >= 0 && q >= 2 ? 0 : seg_rows[seg];   // half tiles: two warps have no rows
       const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
-      const int f = mt * MROWS + q * 32 + lane;            // output feature (up) / output column (down)
+      const int f = mt * MROWS + (half > 0 ? 64 : 0) + q * 32 + lane;   // output feature (up) / output column (down)
       {
         const bool ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -275,8 +288,8 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
 // ------------------------------------------------------------------------------------------------
 // rank-r projections of one vector per (row, kept expert):  out[item][p] = sum_c in[item][c] U_e[p][c]
 // with U packed INT4 [E][r][len].  t = x U1 (in = the row's activations) and s = a_j U2 (in = the
-// activation of that row and slot).  One block per item, a warp per rank index, lanes over the
-// 32-element scale groups.
+// activation of that row and slot).  A block per (item, eight rank indices), a warp per rank index,
+// lanes over the 32-element scale groups.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
@@ -285,13 +298,13 @@ lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, in
   const int item = blockIdx.x;
   const int row = item / k;
   if (row >= seg_off[G] || row_token[row] < 0) {
-    if (row < seg_off[G]) for (int pr = threadIdx.x; pr < r; pr += blockDim.x) out[(size_t)item * r + pr] = 0.f;
+    if (row < seg_off[G] && blockIdx.y == 0) for (int pr = threadIdx.x; pr < r; pr += blockDim.x) out[(size_t)item * r + pr] = 0.f;
     return;
   }
   const int e = row_slot[item];
   const __half* xin = in + (size_t)(in_per_slot ? item : row) * len;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  for (int pr = warp; pr < r; pr += nwarp) {
+  for (int pr = blockIdx.y * nwarp + warp; pr < r; pr += gridDim.y * nwarp) {
     const long long base = ((long long)e * r + pr) * len;
     float acc = 0.f;
     for (int grp = lane; grp * 32 < len; grp += 32) {
@@ -328,10 +341,21 @@ stream_final_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r,
   for (int j = 0; j < k && r > 0; ++j) {
     const int e = row_slot[(size_t)row * k + j];
     const float* sj = s + ((size_t)row * k + j) * r;
-    const long long flat = ((long long)e * d + c) * r;
+    const long long flat = ((long long)e * d + c) * r;      // the r codes of (e, c) share one scale group
     float u = 0.f;
-    for (int pr = 0; pr < r; ++pr) u = fmaf(sj[pr], deq4(V2q, V2s, flat + pr), u);
-    v = fmaf(row_gate[(size_t)row * k + j], u, v);
+    if (r >= 8) {
+      const uint32_t* wq = reinterpret_cast<const uint32_t*>(V2q + (flat >> 1));
+      for (int w8 = 0; w8 < r / 8; ++w8) {
+        const uint32_t word = wq[w8];
+#pragma unroll
+        for (int n = 0; n < 8; ++n) u = fmaf(sj[w8 * 8 + n], (float)sext4((int)(word >> (4 * n))), u);
+      }
+    } else {
+      const uint32_t word = *reinterpret_cast<const uint16_t*>(V2q + (flat >> 1));
+#pragma unroll
+      for (int n = 0; n < 4; ++n) u = fmaf(sj[n], (float)sext4((int)(word >> (4 * n))), u);
+    }
+    v = fmaf(row_gate[(size_t)row * k + j] * __half2float(V2s[flat >> 5]), u, v);
   }
   y[(size_t)tok * d + c] = __float2half_rn(v);
 }
@@ -372,16 +396,17 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
 }
 
 struct StreamState {
-  CUtensorMap mW1, mX, mW2, mAbar;
+  CUtensorMap mW1, mW1h, mX, mW2, mAbar;
   int sm_count;
   int ksplit;
 };
 static_assert(sizeof(StreamState) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
 
 template <bool UP>
-cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mTok, const StreamParams& p, int grid, cudaStream_t st) {
+cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mWh, const CUtensorMap& mTok, const StreamParams& p, int grid,
+                          cudaStream_t st) {
   auto kern = stream_kernel<UP>;
-  constexpr size_t sm = SCfg<UP ? 64 : 128>::SMEM;
+  constexpr size_t sm = SCfg<128>::SMEM;
   static_assert(sm <= 232448, "stream kernel shared memory");
   static bool attr_set = false;
   if (!attr_set) {
@@ -389,7 +414,7 @@ cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mTok, const 
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<grid, S_THREADS, sm, st>>>(mW, mTok, p);
+  kern<<<grid, S_THREADS, sm, st>>>(mW, mWh, mTok, p);
   return cudaGetLastError();
 }
 
@@ -409,7 +434,8 @@ cudaError_t stream_init(cmoe_layer* L) {
   e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
-  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 64, SKA) && make_map(&ts->mX, S.x_perm, P, D.d, 16, 0) &&
+  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 128, SKA) && make_map(&ts->mW1h, L->w.B1t, G * D.d_ff, D.d, 64, SKA) &&
+                  make_map(&ts->mX, S.x_perm, P, D.d, 16, 0) &&
                   make_map(&ts->mW2, L->w.B2t, G * D.d, D.d_ff, 128, SKA) && make_map(&ts->mAbar, S.abar, P, D.d_ff, 16, 0);
   // K ranges per down tile: fill the SMs evenly, keep at least four stages per range
   const int kch = D.d_ff / (SBK * SKA);
@@ -437,7 +463,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   if (marks) cudaEventRecord(marks[0], st);
   if ((e = cudaMemsetAsync(S.y32, 0, sizeof(float) * (size_t)rows_bound * D.d, st)) != cudaSuccess) return e;
   if (D.r > 0) {
-    lowrank_kernel<<<rows_bound * D.k, 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
+    lowrank_kernel<<<dim3(rows_bound * D.k, (D.r + 7) / 8), 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
                                                       W.U1q, W.U1s, S.t);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -449,13 +475,13 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   const int seg_bound = D.G + rows_bound / SNB;
   {
     p.Kd = D.d; p.M = D.d_ff; p.ksplit = 1;
-    const long long units = (long long)seg_bound * (D.d_ff / 64);
+    const long long units = (long long)seg_bound * (D.d_ff / 128);
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<true>(ts.mW1, ts.mX, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<true>(ts.mW1, ts.mW1h, ts.mX, p, grid, st)) != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
-    lowrank_kernel<<<rows_bound * D.k, 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
+    lowrank_kernel<<<dim3(rows_bound * D.k, (D.r + 7) / 8), 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
                                                       W.U2q, W.U2s, S.s);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -463,7 +489,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     p.Kd = D.d_ff; p.M = D.d; p.ksplit = ts.ksplit;
     const long long units = (long long)seg_bound * (D.d / 128) * ts.ksplit;
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<false>(ts.mW2, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<false>(ts.mW2, ts.mW2, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
   }
   dim3 fgrid((D.d + 255) / 256, rows_bound);
   stream_final_kernel<<<fgrid, 256, 0, st>>>(S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
