@@ -110,7 +110,8 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
                           cudaStream_t st);
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st);
-constexpr int kPermuteLaunches = 5;
+constexpr int kPermuteLaunches = 5;        // 2 for batches of at most 256 tokens (permute_launches)
+inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
 // generic_path.cu : CUDA-core path for any supported shape
 // `marks` (or null): three events recorded before the residual-t, up and down stages
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,

@@ -194,9 +194,101 @@ pad_kernel(int d, int K, int k, const int* __restrict__ seg_off, const int* __re
   }
 }
 
+// The whole permutation of a small batch (T <= 256) in one block: keys, counts, offsets, the stable
+// rank of every token inside its key (by counting the earlier tokens with the same key), the row
+// tables and the padding rows.  Gives exactly the tables the four kernels above give.
+constexpr int kSmallT = 256;
+
+__global__ void __launch_bounds__(kSmallT)
+permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_combo, int row_align, int max_tiles,
+                     const int* __restrict__ cluster_id, const int* __restrict__ slot, const float* __restrict__ gates,
+                     int* __restrict__ seg_off, int* __restrict__ seg_cnt, int* __restrict__ n_rows,
+                     int* __restrict__ tile_cluster, int* __restrict__ row_token, int* __restrict__ row_slot,
+                     float* __restrict__ row_gate) {
+  extern __shared__ int sh[];
+  int* cnt = sh;                   // [nkey] tokens per key, then first row of the key
+  int* keys = cnt + nkey;          // [kSmallT]
+  __shared__ int s_seg[kMaxG + 1];
+  __shared__ int s_cnt[kMaxG];
+  const int t = threadIdx.x;
+  for (int i = t; i < nkey; i += blockDim.x) cnt[i] = 0;
+  __syncthreads();
+  int cs[kMaxKsel];
+  float cg[kMaxKsel];
+  int key = -1, g = 0;
+  if (t < T) {
+    const int sub = canonical_slots(slot + (size_t)t * k, gates + (size_t)t * k, k, sub_is_combo, cs, cg);
+    g = cluster_id[t];
+    key = g * nsub + sub;
+    atomicAdd(&cnt[key], 1);
+  }
+  keys[t] = key;
+  __syncthreads();
+  if (t == 0) {
+    int off = 0;
+    for (int c = 0; c < G; ++c) {
+      s_seg[c] = off;
+      seg_off[c] = off;
+      int n = 0;
+      for (int sb = 0; sb < nsub; ++sb) {
+        const int here = cnt[c * nsub + sb];
+        cnt[c * nsub + sb] = off + n;          // first row of the key
+        n += here;
+      }
+      seg_cnt[c] = n;
+      s_cnt[c] = n;
+      off += (n + row_align - 1) / row_align * row_align;
+    }
+    s_seg[G] = off;
+    seg_off[G] = off;
+    *n_rows = off;
+  }
+  __syncthreads();
+  if (t < T) {
+    int rank = 0;
+    for (int u = 0; u < t; ++u) rank += keys[u] == key ? 1 : 0;
+    const int row = cnt[key] + rank;
+    row_token[row] = t;
+    for (int j = 0; j < k; ++j) {
+      row_slot[(size_t)row * k + j] = g * K + cs[j];
+      row_gate[(size_t)row * k + j] = cg[j];
+    }
+  }
+  // padding rows of every cluster, and the cluster of every tile
+  for (int row = t; row < s_seg[G]; row += blockDim.x) {
+    int c = 0;
+    while (c + 1 < G && s_seg[c + 1] <= row) ++c;
+    if (row - s_seg[c] >= s_cnt[c]) {                  // past the cluster's tokens
+      row_token[row] = -1;
+      for (int j = 0; j < k; ++j) {
+        row_slot[(size_t)row * k + j] = c * K + j;     // any valid experts of the cluster
+        row_gate[(size_t)row * k + j] = 0.f;
+      }
+    }
+  }
+  const int ntile = s_seg[G] / row_align;
+  for (int tile = t; tile < max_tiles; tile += blockDim.x) {
+    int c = -1;
+    if (tile < ntile) {
+      const int row = tile * row_align;
+      c = 0;
+      while (c + 1 < G && s_seg[c + 1] <= row) ++c;
+    }
+    tile_cluster[tile] = c;
+  }
+}
+
 }  // namespace
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st) {
+  const int rows_bound = t_pad_bound(D, T);
+  if (T <= kSmallT) {
+    permute_small_kernel<<<1, kSmallT, sizeof(int) * ((size_t)D.nkey + kSmallT), st>>>(
+        T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
+        S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate);
+    move_rows_kernel<<<rows_bound, 128, 0, st>>>(D.d, S.n_rows, S.row_token, x, S.x_perm);
+    return cudaGetLastError();
+  }
   const int nblk = (T + kPermBlock - 1) / kPermBlock;
   const size_t sh = sizeof(int) * (size_t)D.nkey;
   hist_kernel<<<nblk, kPermBlock, sh, st>>>(T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
@@ -210,7 +302,6 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                                                S.x_perm);
   pad_kernel<<<D.G, 256, 0, st>>>(D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
                                   S.row_gate, S.x_perm);
-  const int rows_bound = t_pad_bound(D, T);
   move_rows_kernel<<<rows_bound < 148 * 32 ? rows_bound : 148 * 32, 128, 0, st>>>(D.d, S.n_rows, S.row_token, x, S.x_perm);
   return cudaGetLastError();
 }

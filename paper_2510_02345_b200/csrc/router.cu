@@ -8,11 +8,11 @@
 //                        reads the cluster prototypes from shared memory; for stage 2 the block
 //                        orders its tokens by cluster, so that the eight tokens of a warp mostly
 //                        share one cluster's expert rows.
-//   router_token_kernel  few tokens (decode): one block per token, the warps split d.
+//   router_token_kernel  few tokens (decode): one block per token, a warp per router row.
 //
 // In both, lane l of a warp owns the columns 256 s + 8 l .. + 7 of the 256-column segments it
 // visits, a lane's partial sum runs over its columns in ascending order, and partial sums are
-// combined by an xor butterfly (and, in the second kernel, by adding the warps' sums in warp order).
+// combined by the same xor butterfly, so both kernels give a token the same logits.
 #include "cmoe_internal.h"
 #include "device_utils.cuh"
 
@@ -224,11 +224,11 @@ router_tile_kernel(const RouterArgs a) {
                      a.expert_ids, a.gates, a.slot_local);
 }
 
-// One block per token; warp w covers the 256-column segments w, w + nwarp, ...
+// One block per token; warp w computes the rows w, w + nwarp, ... of the router matrix, each over all of d
+// (so a dot product is summed in the same order as in the tiled kernel).
 __global__ void __launch_bounds__(256)
 router_token_kernel(const RouterArgs a) {
-  __shared__ float part[8][kMaxG];      // also reused for the expert logits (kMaxK <= kMaxG)
-  __shared__ float lg[kMaxG];
+  __shared__ float lg[kMaxG];           // cluster logits, then the expert logits (kMaxK <= kMaxG)
   __shared__ int s_g;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int t = blockIdx.x, d = a.d;
@@ -236,21 +236,16 @@ router_token_kernel(const RouterArgs a) {
   for (int pass = 0; pass < 2; ++pass) {
     const int n = pass == 0 ? a.G : a.K;
     const float* W = pass == 0 ? a.Ct : a.Rt + (size_t)s_g * a.K * d;
-    for (int j = 0; j < n; ++j) {
+    const float* bias = pass == 0 ? a.bc : a.be + s_g * a.K;
+    for (int j = warp; j < n; j += nwarp) {
+      const float* wr = W + (size_t)j * d;
       float acc = 0.f;
-      for (int c = warp * 256 + lane * 8; c < d; c += nwarp * 256) {
-        const uint4 xv = *reinterpret_cast<const uint4*>(xr + c);
-        const float* wr = W + (size_t)j * d + c;
-        fma8(acc, xv, __ldg(reinterpret_cast<const float4*>(wr)), __ldg(reinterpret_cast<const float4*>(wr + 4)));
-      }
+#pragma unroll 4
+      for (int c = lane * 8; c < d; c += 256)
+        fma8(acc, *reinterpret_cast<const uint4*>(xr + c), __ldg(reinterpret_cast<const float4*>(wr + c)),
+             __ldg(reinterpret_cast<const float4*>(wr + c + 4)));
       acc = warp_sum(acc);
-      if (lane == 0) part[warp][j] = acc;
-    }
-    __syncthreads();
-    if (threadIdx.x < n) {
-      float v = 0.f;
-      for (int w = 0; w < nwarp; ++w) v += part[w][threadIdx.x];
-      lg[threadIdx.x] = v + (pass == 0 ? a.bc[threadIdx.x] : a.be[s_g * a.K + threadIdx.x]);
+      if (lane == 0) lg[j] = acc + bias[j];
     }
     __syncthreads();
     if (pass == 0) {

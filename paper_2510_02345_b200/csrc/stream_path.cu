@@ -33,7 +33,7 @@ constexpr int SBK = 64;            // halves per K atom: one 128-byte swizzle ro
 constexpr int SKA = 2;             // K atoms per stage
 constexpr int SNB = 64;            // most token rows per segment (MMA N)
 constexpr int SMAXSEG = 160;       // segments: at most G + T_pad / 64
-constexpr int S_THREADS = 256;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..7 epilogue
+constexpr int S_THREADS = 384;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..11 epilogue
 constexpr uint32_t S_B_ATOM = SNB * SBK * 2;             // 8 KB
 constexpr uint32_t S_TMEM_COLS = 128;                    // two accumulators of up to 64 columns
 
@@ -93,7 +93,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
   int* seg_g = seg_rows + SMAXSEG;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int kEpiWarps = MROWS / 32;
+  constexpr int kEpiWarps = 8;       // two warps per TMEM lane quadrant: even and odd token columns
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -202,9 +202,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         umma_commit(tfull0 + 8 * acc);
       }
     }
-  } else if (warp >= 4 && warp < 4 + kEpiWarps) {
+  } else if (warp >= 4) {
     // ---------------- epilogue warps: one thread per output feature of the tile
     const int q = warp & 3;
+    const int parity = (warp - 4) >> 2;                  // which token columns of the accumulator this warp takes
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int r = p.r, k = p.k, M = p.M;
     for (int i = 0; i < my_units; ++i) {
@@ -223,10 +224,11 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         tmem_ld16_nowait(taddr + acc * SNB + tb, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int c = 0; c < 16; ++c) {
+        for (int c2 = 0; c2 < 8; ++c2) {
+          const int c = 2 * c2 + parity;
           const int row = row0 + tb + c;
           const bool real = p.row_token[row] >= 0;         // the same for every thread
-          const float dv = __uint_as_float(v[c]);
+          const float dv = __uint_as_float(parity ? v[2 * c2 + 1] : v[2 * c2]);
           if (UP) {
             float ab = 0.f;
             if (real) {
@@ -235,23 +237,33 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                 float h = dv;
                 if (r > 0) {
                   // h += t_j . V1_e[f, :]: r codes of one scale group, decoded in registers
-                  const float* tp = p.t + ((size_t)row * k + j) * r;
+                  const float4* tp = reinterpret_cast<const float4*>(p.t + ((size_t)row * k + j) * r);
                   const long long flat = ((long long)e * M + f) * r;
                   const float sc = __half2float(p.V1s[flat >> 5]);
-                  float dot = 0.f;
+                  float dot0 = 0.f, dot1 = 0.f;
                   if (r >= 8) {
                     const uint32_t* wq = reinterpret_cast<const uint32_t*>(p.V1q + (flat >> 1));
                     for (int w8 = 0; w8 < r / 8; ++w8) {
                       const uint32_t word = wq[w8];
-#pragma unroll
-                      for (int n = 0; n < 8; ++n) dot = fmaf(tp[w8 * 8 + n], (float)sext4((int)(word >> (4 * n))), dot);
+                      const float4 ta = tp[2 * w8], tb4 = tp[2 * w8 + 1];
+                      dot0 = fmaf(ta.x, (float)sext4((int)word), dot0);
+                      dot1 = fmaf(ta.y, (float)sext4((int)(word >> 4)), dot1);
+                      dot0 = fmaf(ta.z, (float)sext4((int)(word >> 8)), dot0);
+                      dot1 = fmaf(ta.w, (float)sext4((int)(word >> 12)), dot1);
+                      dot0 = fmaf(tb4.x, (float)sext4((int)(word >> 16)), dot0);
+                      dot1 = fmaf(tb4.y, (float)sext4((int)(word >> 20)), dot1);
+                      dot0 = fmaf(tb4.z, (float)sext4((int)(word >> 24)), dot0);
+                      dot1 = fmaf(tb4.w, (float)sext4((int)(word >> 28)), dot1);
                     }
                   } else {
                     const uint32_t word = *reinterpret_cast<const uint16_t*>(p.V1q + (flat >> 1));
-#pragma unroll
-                    for (int n = 0; n < 4; ++n) dot = fmaf(tp[n], (float)sext4((int)(word >> (4 * n))), dot);
+                    const float4 ta = tp[0];
+                    dot0 = fmaf(ta.x, (float)sext4((int)word), dot0);
+                    dot1 = fmaf(ta.y, (float)sext4((int)(word >> 4)), dot1);
+                    dot0 = fmaf(ta.z, (float)sext4((int)(word >> 8)), dot0);
+                    dot1 = fmaf(ta.w, (float)sext4((int)(word >> 12)), dot1);
                   }
-                  h = fmaf(sc, dot, h);
+                  h = fmaf(sc, dot0 + dot1, h);
                 }
                 const float a = gelu_erf(h);
                 ab = fmaf(p.row_gate[(size_t)row * k + j], a, ab);
@@ -307,6 +319,7 @@ lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, in
   for (int pr = blockIdx.y * nwarp + warp; pr < r; pr += gridDim.y * nwarp) {
     const long long base = ((long long)e * r + pr) * len;
     float acc = 0.f;
+#pragma unroll 4
     for (int grp = lane; grp * 32 < len; grp += 32) {
       const uint4 pk = *reinterpret_cast<const uint4*>(Uq + ((base + grp * 32) >> 1));
       const float sc = __half2float(Us[(base >> 5) + grp]);

@@ -184,6 +184,21 @@ def test_router_tile_kernel_shapes(kw):
     check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
 
 
+def test_route_does_not_depend_on_the_batch():
+    """A token's route is the same whether it arrives in a large batch (tiled router kernel) or in a small
+    one (per-token kernel): both sum every dot product in the same order."""
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    L = layer_for("bert")
+    m = ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    big = [t.clone() for t in m.route(x)]
+    small = m.route(x[1000:1300].contiguous())
+    torch.cuda.synchronize()
+    for b, s_ in zip(big, small):
+        assert torch.equal(b[1000:1300], s_)
+
+
 # ---- shapes that take the tensor-core path (d, d_ff multiples of 128, T_max > 128) ----------------
 @pytest.mark.parametrize("T", [129, 200, 640, 1111])
 def test_tensor_path_ragged(T):
