@@ -280,9 +280,13 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   CMOE_MARK();
   CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   CMOE_MARK();
-  CMOE_CUDA(L, launch_permute(D, S, xh, T, st));
-  if (D.r > 0)
-    CMOE_CUDA(L, cudaMemsetAsync(S.s, 0, sizeof(float) * (size_t)t_pad_bound(D, T) * D.k * D.r, st));
+  {
+    // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s
+    const size_t rows = (size_t)t_pad_bound(D, T);
+    void* zp = L->path == kPathStream ? static_cast<void*>(S.y32) : static_cast<void*>(S.s);
+    const size_t zb = L->path == kPathStream ? sizeof(float) * rows * D.d : sizeof(float) * rows * D.k * D.r;
+    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb));
+  }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else if (L->path == kPathStream)
@@ -322,7 +326,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L->dims)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
-  out->memsets_forward = (L->dims.r > 0 ? 1 : 0) + (L->path == kPathStream ? 1 : 0);
+  out->memsets_forward = 0;
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;
   out->T_pad_max = L->dims.T_pad_max;

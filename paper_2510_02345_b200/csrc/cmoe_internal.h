@@ -109,7 +109,9 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
                           cudaStream_t st);
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
-cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st);
+// also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
+cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
+                           size_t zero_bytes);
 constexpr int kPermuteLaunches = 5;        // 2 for batches of at most 256 tokens (permute_launches)
 inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
 // generic_path.cu : CUDA-core path for any supported shape

@@ -8,6 +8,7 @@
 //   y     = abar B2_g + sum_j p_j s_j V2_e     down kernel (linear in a_j, so the base product
 //                                              runs once on the gate-weighted sum)
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 
 namespace cmoe {
@@ -22,6 +23,7 @@ residual_t_kernel(int d, int k, int r, const int* __restrict__ n_rows,
                   const __half* __restrict__ x_perm, const int* __restrict__ row_slot,
                   const uint8_t* __restrict__ U1q, const __half* __restrict__ U1s,
                   float* __restrict__ t) {
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
   const int total = *n_rows * k;
@@ -67,7 +69,8 @@ ffn_tile_kernel(int Kd, int N, int K, int k, int r, int row_align,
                 const uint8_t* __restrict__ U2q, const __half* __restrict__ U2s, // UP only
                 const float* __restrict__ coef,      // t (UP) / s (DOWN), [rows][k][r]
                 float* __restrict__ s_out,           // UP only
-                __half* __restrict__ out) {          // abar [rows][N] (UP) / y [T][N] (DOWN)
+                __half* __restrict__ out) {
+  pdl_wait();          // abar [rows][N] (UP) / y [T][N] (DOWN)
   const int row0 = blockIdx.y * BM;
   if (row0 >= *n_rows) return;
   const int g = tile_cluster[row0 / row_align];
@@ -190,7 +193,8 @@ cudaError_t launch_residual_t(const Dims& D, const Weights& W, const Scratch& S,
   const int rows_bound = t_pad_bound(D, T);
   int blocks = (rows_bound * D.k + 7) / 8;
   if (blocks > 148 * 16) blocks = 148 * 16;
-  residual_t_kernel<<<blocks, 256, 0, st>>>(D.d, D.k, D.r, S.n_rows, S.x_perm, S.row_slot, W.U1q,
+  launch_chained(residual_t_kernel, dim3(blocks), dim3(256), 0, st, 1,
+      D.d, D.k, D.r, S.n_rows, S.x_perm, S.row_slot, W.U1q,
                                             W.U1s, S.t);
   return cudaGetLastError();
 }
@@ -203,12 +207,14 @@ cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S
   if (e0 != cudaSuccess) return e0;
   if (marks) cudaEventRecord(marks[1], st);
   dim3 gu((D.d_ff + BN - 1) / BN, rows_bound / BM);
-  ffn_tile_kernel<true><<<gu, 256, 0, st>>>(D.d, D.d_ff, D.K, D.k, D.r, D.row_align, S.n_rows,
+  launch_chained(ffn_tile_kernel<true>, dim3(gu), dim3(256), 0, st, 1,
+      D.d, D.d_ff, D.K, D.k, D.r, D.row_align, S.n_rows,
                                             S.tile_cluster, S.x_perm, W.B1t, S.row_slot, S.row_gate,
                                             S.row_token, W.V1q, W.V1s, W.U2q, W.U2s, S.t, S.s, S.abar);
   if (marks) cudaEventRecord(marks[2], st);
   dim3 gd((D.d + BN - 1) / BN, rows_bound / BM);
-  ffn_tile_kernel<false><<<gd, 256, 0, st>>>(D.d_ff, D.d, D.K, D.k, D.r, D.row_align, S.n_rows,
+  launch_chained(ffn_tile_kernel<false>, dim3(gd), dim3(256), 0, st, 1,
+      D.d_ff, D.d, D.K, D.k, D.r, D.row_align, S.n_rows,
                                              S.tile_cluster, S.abar, W.B2t, S.row_slot, S.row_gate,
                                              S.row_token, W.V2q, W.V2s, nullptr, nullptr, S.s, nullptr,
                                              y);

@@ -9,10 +9,11 @@
 //            writes the row tables
 //   pad      fills the table entries of the padding rows of each segment (no token, zero gates)
 //   move     copies every token's activations to its row with 16-byte vectors (a block per row;
-//            padding rows get zeros)
+//            padding rows get zeros) and clears the buffer the later stages accumulate into
 //
 // The result is deterministic: rows of one key keep the token order.
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 
 namespace cmoe {
@@ -54,6 +55,7 @@ __global__ void __launch_bounds__(kPermBlock)
 hist_kernel(int T, int k, int nsub, int nkey, int sub_is_combo,
             const int* __restrict__ cluster_id, const int* __restrict__ slot,
             const float* __restrict__ gates, int* __restrict__ keys, int* __restrict__ block_counts) {
+  pdl_wait();
   extern __shared__ int sh_cnt[];
   for (int i = threadIdx.x; i < nkey; i += blockDim.x) sh_cnt[i] = 0;
   __syncthreads();
@@ -76,6 +78,7 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             const int* __restrict__ block_counts, int* __restrict__ block_base,
             int* __restrict__ key_cnt, int* __restrict__ key_off, int* __restrict__ seg_off,
             int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster) {
+  pdl_wait();
   __shared__ int sh_seg[kMaxG + 1];
   for (int key = threadIdx.x; key < nkey; key += blockDim.x) {
     int run = 0;
@@ -125,6 +128,7 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
                const int* __restrict__ key_off,
                int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
                __half* __restrict__ x_perm) {
+  pdl_wait();
   extern __shared__ int sh_next[];   // next free row of each key for this block
   for (int i = threadIdx.x; i < nkey; i += blockDim.x)
     sh_next[i] = key_off[i] + block_base[(size_t)blockIdx.x * nkey + i];
@@ -164,7 +168,8 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
 // x_perm[row] = x[row_token[row]], zeros for padding rows; a block per row, 16 bytes per thread
 __global__ void __launch_bounds__(128)
 move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ row_token,
-                 const __half* __restrict__ x, __half* __restrict__ x_perm) {
+                 const __half* __restrict__ x, __half* __restrict__ x_perm, uint4* __restrict__ zero_ptr, size_t zero_n) {
+  pdl_wait();
   const int vec_per_row = d / 8;
   for (int row = blockIdx.x; row < *n_rows; row += gridDim.x) {
     const int tok = row_token[row];
@@ -176,12 +181,16 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
       for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
     }
   }
+  // the accumulation buffer of the later stages starts at zero
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += (size_t)gridDim.x * blockDim.x)
+    zero_ptr[i] = make_uint4(0, 0, 0, 0);
 }
 
 __global__ void __launch_bounds__(256)
 pad_kernel(int d, int K, int k, const int* __restrict__ seg_off, const int* __restrict__ seg_cnt,
            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
            __half* __restrict__ x_perm) {
+  pdl_wait();
   const int g = blockIdx.x;
   const int first = seg_off[g] + seg_cnt[g], last = seg_off[g + 1];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
@@ -205,6 +214,7 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
                      int* __restrict__ seg_off, int* __restrict__ seg_cnt, int* __restrict__ n_rows,
                      int* __restrict__ tile_cluster, int* __restrict__ row_token, int* __restrict__ row_slot,
                      float* __restrict__ row_gate) {
+  pdl_wait();
   extern __shared__ int sh[];
   int* cnt = sh;                   // [nkey] tokens per key, then first row of the key
   int* keys = cnt + nkey;          // [kSmallT]
@@ -280,29 +290,38 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
 
 }  // namespace
 
-cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st) {
+cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
+                           size_t zero_bytes) {
   const int rows_bound = t_pad_bound(D, T);
   if (T <= kSmallT) {
-    permute_small_kernel<<<1, kSmallT, sizeof(int) * ((size_t)D.nkey + kSmallT), st>>>(
+    launch_chained(permute_small_kernel, dim3(1), dim3(kSmallT), sizeof(int) * ((size_t)D.nkey + kSmallT), st, 1,
+      
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
         S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate);
-    move_rows_kernel<<<rows_bound, 128, 0, st>>>(D.d, S.n_rows, S.row_token, x, S.x_perm);
+    launch_chained(move_rows_kernel, dim3(rows_bound), dim3(128), 0, st, 1,
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
     return cudaGetLastError();
   }
   const int nblk = (T + kPermBlock - 1) / kPermBlock;
   const size_t sh = sizeof(int) * (size_t)D.nkey;
-  hist_kernel<<<nblk, kPermBlock, sh, st>>>(T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
+  launch_chained(hist_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
+      T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
                                             S.slot, S.gates, S.keys, S.block_counts);
-  scan_kernel<<<1, 1024, 0, st>>>(nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
+  launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
+      nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
                                   S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
                                   S.seg_cnt, S.n_rows, S.tile_cluster);
-  scatter_kernel<<<nblk, kPermBlock, sh, st>>>(T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
+  launch_chained(scatter_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
+      T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
                                                S.x_perm);
-  pad_kernel<<<D.G, 256, 0, st>>>(D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
+  launch_chained(pad_kernel, dim3(D.G), dim3(256), 0, st, 1,
+      D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
                                   S.row_gate, S.x_perm);
-  move_rows_kernel<<<rows_bound < 148 * 32 ? rows_bound : 148 * 32, 128, 0, st>>>(D.d, S.n_rows, S.row_token, x, S.x_perm);
+  const int move_grid = rows_bound < 148 * 32 ? rows_bound : 148 * 32;
+  launch_chained(move_rows_kernel, dim3(move_grid), dim3(128), 0, st, 1,
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
   return cudaGetLastError();
 }
 

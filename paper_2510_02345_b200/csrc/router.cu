@@ -14,6 +14,7 @@
 // visits, a lane's partial sum runs over its columns in ascending order, and partial sums are
 // combined by the same xor butterfly, so both kernels give a token the same logits.
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 
 namespace cmoe {
@@ -81,6 +82,7 @@ struct RouterArgs {
 
 __global__ void __launch_bounds__(kTileWarps * 32)
 router_tile_kernel(const RouterArgs a) {
+  pdl_wait();
   extern __shared__ float sm_f[];
   float* Cs = sm_f;                                        // [up to 8 clusters][dc]
   float* lg = Cs + (size_t)kGroup * a.dc;                  // [64][K] expert logits
@@ -228,6 +230,7 @@ router_tile_kernel(const RouterArgs a) {
 // (so a dot product is summed in the same order as in the tiled kernel).
 __global__ void __launch_bounds__(256)
 router_token_kernel(const RouterArgs a) {
+  pdl_wait();
   __shared__ float lg[kMaxG];           // cluster logits, then the expert logits (kMaxK <= kMaxG)
   __shared__ int s_g;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
@@ -275,7 +278,8 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
   a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;
   if (T < 1024) {
     // few tokens: the per-token kernel puts every token on its own SM
-    router_token_kernel<<<T, 256, 0, st>>>(a);
+    launch_chained(router_token_kernel, dim3(T), dim3(256), 0, st, 1,
+      a);
     return cudaGetLastError();
   }
   // chunk of the prototypes staged at a time: at most 32 KB for a group of eight clusters
@@ -290,7 +294,8 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  router_tile_kernel<<<(T + kTileTokens - 1) / kTileTokens, kTileWarps * 32, sh, st>>>(a);
+  launch_chained(router_tile_kernel, dim3((T + kTileTokens - 1) / kTileTokens), dim3(kTileWarps * 32), sh, st, 1,
+      a);
   return cudaGetLastError();
 }
 

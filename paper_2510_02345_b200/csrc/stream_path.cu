@@ -20,6 +20,7 @@
 // rows; a work unit is (segment, tile of features[, K range]), dealt round-robin to the CTAs.
 // Every device wait is bounded (status word CMOE_ERR_TIMEOUT on expiry).
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 #include "tc_ptx.cuh"
 
@@ -75,6 +76,7 @@ template <bool UP>
 __global__ void __launch_bounds__(S_THREADS, 1)
 stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWh,
               const __grid_constant__ CUtensorMap tmTok, const StreamParams p) {
+  pdl_wait();
   constexpr int MROWS = 128;
   using Cfg = SCfg<MROWS>;
   constexpr int STAGES = Cfg::STAGES;
@@ -307,6 +309,7 @@ __global__ void __launch_bounds__(256)
 lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
                const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
                const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+  pdl_wait();
   const int item = blockIdx.x;
   const int row = item / k;
   if (row >= seg_off[G] || row_token[row] < 0) {
@@ -345,6 +348,7 @@ stream_final_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r,
                     const float* __restrict__ y32, const float* __restrict__ s, const int* __restrict__ row_slot,
                     const float* __restrict__ row_gate, const int* __restrict__ row_token,
                     const uint8_t* __restrict__ V2q, const __half* __restrict__ V2s, __half* __restrict__ y) {
+  pdl_wait();
   const int row = blockIdx.y;
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= seg_off[G] || c >= d) return;
@@ -427,7 +431,8 @@ cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mWh, const C
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<grid, S_THREADS, sm, st>>>(mW, mWh, mTok, p);
+  launch_chained(kern, dim3(grid), dim3(S_THREADS), sm, st, 1,
+      mW, mWh, mTok, p);
   return cudaGetLastError();
 }
 
@@ -474,9 +479,9 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   const int rows_bound = t_pad_bound(D, T);
   cudaError_t e;
   if (marks) cudaEventRecord(marks[0], st);
-  if ((e = cudaMemsetAsync(S.y32, 0, sizeof(float) * (size_t)rows_bound * D.d, st)) != cudaSuccess) return e;
   if (D.r > 0) {
-    lowrank_kernel<<<dim3(rows_bound * D.k, (D.r + 7) / 8), 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
+    launch_chained(lowrank_kernel, dim3(rows_bound * D.k, (D.r + 7) / 8), dim3(256), 0, st, 1,
+      S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
                                                       W.U1q, W.U1s, S.t);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -494,7 +499,8 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
-    lowrank_kernel<<<dim3(rows_bound * D.k, (D.r + 7) / 8), 256, 0, st>>>(S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
+    launch_chained(lowrank_kernel, dim3(rows_bound * D.k, (D.r + 7) / 8), dim3(256), 0, st, 1,
+      S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
                                                       W.U2q, W.U2s, S.s);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
@@ -505,7 +511,8 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     if ((e = launch_stream<false>(ts.mW2, ts.mW2, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
   }
   dim3 fgrid((D.d + 255) / 256, rows_bound);
-  stream_final_kernel<<<fgrid, 256, 0, st>>>(S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
+  launch_chained(stream_final_kernel, dim3(fgrid), dim3(256), 0, st, 1,
+      S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
                                              S.row_token, W.V2q, W.V2s, y);
   return cudaGetLastError();
 }

@@ -28,6 +28,7 @@
 // Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 #include "tc_ptx.cuh"
 
@@ -78,6 +79,7 @@ struct FactorStage {
 
 __global__ void __launch_bounds__(256)
 stage_factors_kernel(const FactorStage fs) {
+  pdl_wait();
   const int which = blockIdx.y;
   const long long wd = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (wd >= fs.words[which]) return;
@@ -142,6 +144,7 @@ template <int KSEL>
 __global__ void __launch_bounds__(T_THREADS, 1)
 tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU1,
              const TParams p) {
+  pdl_wait();
   const int mt = blockIdx.x;
   if (mt >= *p.n_rows / BM) return;
   extern __shared__ uint8_t smem_raw[];
@@ -346,6 +349,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
               const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmAd,
               const __grid_constant__ CUtensorMap tmV1, const __grid_constant__ CUtensorMap tmU2,
               const Up2Params p) {
+  pdl_wait();
   using Cfg = UpCfg<HAS_R, KSEL>;
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
@@ -727,6 +731,7 @@ __global__ void __launch_bounds__(256)
 s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_cluster,
                 const int* __restrict__ row_slot, const float* __restrict__ row_gate,
                 const float* __restrict__ s, __half* __restrict__ As, int K, int k, int r, int log2r) {
+  pdl_wait();
   const int idx = blockIdx.x * blockDim.x + threadIdx.x;
   const int row = idx >> 3, c0 = (idx & 7) * 8;
   if (row >= *n_rows) return;
@@ -774,6 +779,7 @@ __global__ void __launch_bounds__(DN_THREADS, 1)
 tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant__ CUtensorMap tmB23,
                 const __grid_constant__ CUtensorMap tmAs, const __grid_constant__ CUtensorMap tmV2,
                 const Down2Params p) {
+  pdl_wait();
   using Cfg = DownCfg<BN, HAS_R>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr uint32_t STAGE_BYTES = Cfg::STAGE_BYTES;
@@ -996,19 +1002,7 @@ cudaError_t set_smem(Kern kern, size_t bytes) {
 // launch as thread-block clusters of two CTAs (grid = 2 x pairs)
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)grid, 1, 1);
-  cfg.blockDim = dim3((unsigned)threads, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+  return launch_chained(kern, dim3((unsigned)grid), dim3((unsigned)threads), smem, st, 2, args...);
 }
 
 template <bool HAS_R, int KSEL>
@@ -1049,7 +1043,8 @@ cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<grid, T_THREADS, sm, st>>>(ts.mX, ts.mU1, p);
+  launch_chained(kern, dim3(grid), dim3(T_THREADS), sm, st, 1,
+      ts.mX, ts.mU1, p);
   return cudaGetLastError();
 }
 
@@ -1139,7 +1134,8 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
     }
     fs.K = D.K; fs.r = D.r;
     dim3 grid((unsigned)((maxw + 255) / 256), 4);
-    stage_factors_kernel<<<grid, 256, 0, st>>>(fs);
+    launch_chained(stage_factors_kernel, dim3(grid), dim3(256), 0, st, 1,
+      fs);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     TParams tp{};
     tp.n_rows = S.n_rows; tp.tile_cluster = S.tile_cluster; tp.row_slot = S.row_slot; tp.row_token = S.row_token;
@@ -1166,7 +1162,8 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
     const int threads = rows_bound * 8;
-    s_expand_kernel<<<(threads + 255) / 256, 256, 0, st>>>(S.n_rows, S.tile_cluster, S.row_slot, S.row_gate, S.s,
+    launch_chained(s_expand_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, 1,
+      S.n_rows, S.tile_cluster, S.row_slot, S.row_gate, S.s,
                                                            S.As, D.K, D.k, D.r, ts.log2r);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
