@@ -110,6 +110,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
     s.As = A.take<__half>(P * 64);
     s.tile_mask = A.take<int>(P / 128 * 2);
   }
+  if (router_tc_supported(D)) s.Wsplit = A.take<__half>((size_t)2 * router_tc_rp(D) * d);
   if (D.stream) {
     if (r > 0) s.a_slot = A.take<__half>(P * k * f);
     s.y32 = A.take<float>(P * d);
@@ -246,6 +247,11 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
     L->path = kPathTensor;
     L->tc_variant = 1;
   }
+  L->router_tc = 0;
+  if (router_tc_supported(D) && !std::getenv("CMOE_ROUTER_FP32")) {
+    if ((e = router_tc_init(L))) return fail(e);
+    L->router_tc = 1;
+  }
   *out_layer = L;
   return CMOE_OK;
 }
@@ -257,8 +263,11 @@ int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int
   if (T == 0) return CMOE_OK;
   if (!cluster_id || !expert_ids || !gates) return CMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  CMOE_CUDA(L, launch_router(L->dims, L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
-                             gates, nullptr, st));
+  if (L->router_tc && T >= 1024)
+    CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st));
+  else
+    CMOE_CUDA(L, launch_router(L->dims, L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
+                               gates, nullptr, st));
   return CMOE_OK;
 }
 
@@ -278,7 +287,10 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     ++stage;                                                               \
   } while (0)
   CMOE_MARK();
-  CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  if (L->router_tc && T >= 1024)
+    CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  else
+    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   CMOE_MARK();
   {
     // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s

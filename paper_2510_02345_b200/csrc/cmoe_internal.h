@@ -2,6 +2,7 @@
 // the per-call scratch views and the kernel launchers.  Nothing here is part of the C boundary.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
@@ -76,6 +77,8 @@ struct Scratch {
   // weight-streaming path only (see stream_path.cu)
   __half* a_slot;                  // [T_pad][k][d_ff]  GELU(h_j) of every kept expert
   float* y32;                      // [T_pad][d]        fp32 sum of the K ranges of the down-projection
+  // tensor-core router only (see router_tc.cu): the fp32 router rows split into two fp16 pieces
+  __half* Wsplit;                  // [2 * rp][d]
 };
 
 }  // namespace cmoe
@@ -86,6 +89,8 @@ struct cmoe_layer {
   cmoe::Scratch sc;
   int path;
   int tc_variant;   // 1: tc_path.cu, 2: tc2_path.cu (when path == kPathTensor)
+  int router_tc;    // batches of at least 1024 tokens are routed by router_tc.cu
+  CUtensorMap router_map_w;
   int last_cuda_error;
   // optional stage timing (cmoe_profile_*)
   int profiling;
@@ -108,6 +113,12 @@ inline int t_pad_bound(const Dims& D, int T) { return round_up(T, D.row_align) +
 cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int T,
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
                           cudaStream_t st);
+// router_tc.cu : the same routing on the tensor cores (split fp16 router matrices), for large batches
+int router_tc_rp(const Dims& D);
+bool router_tc_supported(const Dims& D);
+cudaError_t router_tc_init(cmoe_layer* L);
+cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
+                             int* slot_local, cudaStream_t st);
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,

@@ -169,9 +169,10 @@ def test_permutation_equivariance_on_gpu():
     dict(T=1027, d=1056, d_ff=32, E=8, G=8, r=0, k=1),      # d not a multiple of 256, one expert per cluster
     dict(T=2048, d=2304, d_ff=32, E=64, G=2, r=0, k=8),     # prototypes staged in several chunks, K = 32
 ], ids=["G12", "K5", "d1056", "d2304_K32"])
-def test_router_tile_kernel_shapes(kw):
+def test_router_tile_kernel_shapes(kw, monkeypatch):
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer
+    monkeypatch.setenv("CMOE_ROUTER_FP32", "1")          # the CUDA-core kernels, also for these large batches
     s = inputs.small_shape(**kw)
     L = inputs.make_layer(s, 17)
     rng = np.random.default_rng(1)
@@ -184,11 +185,36 @@ def test_router_tile_kernel_shapes(kw):
     check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
 
 
-def test_route_does_not_depend_on_the_batch():
-    """A token's route is the same whether it arrives in a large batch (tiled router kernel) or in a small
-    one (per-token kernel): both sum every dot product in the same order."""
+@pytest.mark.parametrize("kw", [
+    dict(T=1100, d=128, d_ff=64, E=36, G=12, r=0, k=2),     # 48 router rows -> 96 MMA columns
+    dict(T=1500, d=256, d_ff=64, E=10, G=2, r=0, k=3),      # K = 5
+    dict(T=1027, d=1024, d_ff=32, E=8, G=8, r=0, k=1),      # ragged last tile of 128 tokens
+], ids=["G12", "K5", "ragged"])
+def test_router_tensor_core_shapes(kw):
+    """Large batches are routed on the tensor cores from split fp16 router matrices: same routes as the
+    oracle outside the near-tie band, gates to 1e-5."""
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(**kw)
+    L = inputs.make_layer(s, 18)
+    rng = np.random.default_rng(2)
+    L["b_c"] = (rng.standard_normal(s.G) * 0.2).astype(np.float32)
+    L["b_e"] = (rng.standard_normal((s.G, s.K)) * 0.2).astype(np.float32)
+    m = ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    cid, eid, gates = m.route(x)
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+
+
+def test_route_does_not_depend_on_the_batch(monkeypatch):
+    """With the fp32 CUDA-core router kernels (CMOE_ROUTER_FP32=1 keeps large batches off the tensor-core
+    router) a token's route is bit-identical whether it arrives in a large batch (tiled kernel) or in a
+    small one (per-token kernel): both sum every dot product in the same order."""
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    monkeypatch.setenv("CMOE_ROUTER_FP32", "1")
     L = layer_for("bert")
     m = ClusteredMoELayer(L)
     x = torch.from_numpy(L["x"]).cuda()
