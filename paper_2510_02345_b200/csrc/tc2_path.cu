@@ -314,7 +314,7 @@ constexpr uint32_t U2_TILE_BYTES = 2 * U2_CHUNK_BYTES;
 
 // barrier slots (64-bit words after the buffers)
 enum : int { B_FULL = 0, B_EMPTY = 8, B_TFULL = 16, B_TEMPTY = 18, B_QEMPTY = 20, B_AFULL = 21, B_AEMPTY = 25,
-             B_U2FULL = 29, B_U2EMPTY = 31, B_SFULL = 33, B_SEMPTY = 34, B_COUNT = 36 };
+             B_U2FULL = 29, B_U2EMPTY = 31, B_SFULL = 33, B_SEMPTY = 34, B_QFULL = 35, B_COUNT = 37 };
 
 template <bool HAS_R, int KSEL>
 struct UpCfg {
@@ -377,6 +377,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
     for (int s = 0; s < STAGES; ++s) { mbar_init(local(B_FULL + s), 1); mbar_init(local(B_EMPTY + s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 2 * UP_EPI_WARPS); }
     mbar_init(local(B_QEMPTY), 2 * UP_EPI_WARPS);
+    mbar_init(local(B_QFULL), 1);
     for (int a = 0; a < 4; ++a) { mbar_init(local(B_AFULL + a), UP_EPI_WARPS); mbar_init(local(B_AEMPTY + a), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(local(B_U2FULL + a), 1); mbar_init(local(B_U2EMPTY + a), 1); }
     mbar_init(local(B_SFULL), 1);
@@ -476,8 +477,10 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
               if ((m0 >> ks) & 1) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+            commit_both(B_TFULL + acc);    // P is complete: the epilogues start on the first expert
             if (KSEL == 2) {
-              // Q has one buffer: both epilogues of the previous tile must have drained it
+              // Q has one buffer: both epilogues of the previous tile must have drained it.  They are
+              // then already busy with P of this tile, so the wait and the Q product hide behind that.
               if (!mbar_wait_cluster(local(B_QEMPTY), (tile_i & 1u) ^ 1u, abort_flag)) { failed = true; break; }
               tc_fence_after();
               int m = m0 | m1;
@@ -489,13 +492,14 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
                   umma2_f16(tmem_q, adesc + (UP_A_ATOM >> 4) + 2 * ks, bdesc + (UP_B_ATOM >> 4) + 2 * ks, IDESC, accum);
                   accum = 1;
                 }
+              commit_both(B_QFULL);
             }
           }
           commit_both(B_EMPTY + s);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (failed) break;
-        commit_both(B_TFULL + acc);
+        if (!HAS_R) commit_both(B_TFULL + acc);
       }
     }
   } else if (warp == 2) {
@@ -573,68 +577,71 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       }
       tc_fence_after();
+      // Phase A (needs P only): a_1 = GELU(h_1) of the first kept expert, its share of abar, its chunk
+      // of the S operand.  Phase B (needs Q, which the leader issues meanwhile): h_2 = P + Q, a_2.
       uint32_t ob[2][8];                                   // abar, stored after the hand-overs below
+      auto put_chunk = [&](int j, int sub, const uint32_t* src) {
+        // a_j into its chunk as a K-major 128-byte-swizzled A operand: 16-byte unit u of row rowc sits at
+        // rowc*128 + ((u ^ (rowc & 7)) << 4); this warp owns units 4 (cq & 1) + 2 sub + {0, 1}
+        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        const uint32_t cb = aring + (n % Cfg::NA) * A_CHUNK_BYTES + rowc * 128;
 #pragma unroll
-      for (int sub = 0; sub < 2; ++sub) {
-        const int col0 = cq * 32 + sub * 16;
-        uint32_t vp[16], vq[16];
-        tmem_ld16_nowait(taddr + acc * BN_UP + col0, vp);
-        if (HAS_R && KSEL == 2) tmem_ld16_nowait(taddr + 256 + col0, vq);
-        tmem_ld_wait();
-        if (HAS_R && sub == 0) {
-          // the S products that read this warp's chunk slots one tile ago must have finished
-          bool ok = true;
-#pragma unroll
-          for (int j = 0; j < KSEL; ++j) {
-            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
-            ok = ok && mbar_wait_cluster(local(B_AEMPTY + n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
-          }
-          if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+        for (int i = 0; i < 2; ++i) {
+          const uint32_t un = (uint32_t)((cq & 1) * 4 + sub * 2 + i);
+          st_shared_v4(cb + ((un ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2], src[4 * i + 3]);
         }
-        uint32_t oa0[8], oa1[8];
-#pragma unroll
-        for (int c = 0; c < 16; c += 2) {
-          const float p0 = __uint_as_float(vp[c]), p1 = __uint_as_float(vp[c + 1]);
-          const __half2 a0 = gelu_fast2(__floats2half2_rn(p0, p1));
-          __half2 ab;
-          if (HAS_R && KSEL == 2) {
-            const __half2 a1 = gelu_fast2(__floats2half2_rn(p0 + __uint_as_float(vq[c]), p1 + __uint_as_float(vq[c + 1])));
-            ab = __hfma2(g1, a1, __hmul2(g0, a0));
-            oa1[c >> 1] = h2u(a1);
-          } else {
-            ab = __hmul2(g0, a0);
-          }
-          ob[sub][c >> 1] = h2u(ab);
-          oa0[c >> 1] = h2u(a0);
-        }
-        if (HAS_R) {
-          // a_j into its chunk as a K-major 128-byte-swizzled A operand: 16-byte unit u of row
-          // rowc sits at rowc*128 + ((u ^ (rowc & 7)) << 4); this warp owns units 4 (cq & 1) + 2 sub + {0, 1}
-#pragma unroll
-          for (int j = 0; j < KSEL; ++j) {
-            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
-            const uint32_t cb = aring + (n % Cfg::NA) * A_CHUNK_BYTES + rowc * 128;
-            const uint32_t* src = j == 0 ? oa0 : oa1;
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-              const uint32_t un = (uint32_t)((cq & 1) * 4 + sub * 2 + i);
-              st_shared_v4(cb + ((un ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2],
-                           src[4 * i + 3]);
-            }
-          }
-        }
-      }
-      if (failed) break;
-      if (HAS_R) {
+      };
+      auto chunk_free = [&](int j) {       // the S product that read this slot one tile ago has finished
+        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        const bool ok = mbar_wait_cluster(local(B_AEMPTY + n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
+        return __all_sync(0xffffffffu, ok);
+      };
+      auto chunk_done = [&](int j) {
         fence_async_smem();
         __syncwarp();
-        if (lane == 0) {
+        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        if (lane == 0) mbar_arrive_cluster(lead(B_AFULL + n % Cfg::NA));
+      };
+      if (HAS_R && !chunk_free(0)) { failed = true; break; }
 #pragma unroll
-          for (int j = 0; j < KSEL; ++j) {
-            const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
-            mbar_arrive_cluster(lead(B_AFULL + n % Cfg::NA));
-          }
+      for (int sub = 0; sub < 2; ++sub) {
+        uint32_t vp[16], oa0[8];
+        tmem_ld16_nowait(taddr + acc * BN_UP + cq * 32 + sub * 16, vp);
+        tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 16; c += 2) {
+          const __half2 a0 = gelu_fast2(__floats2half2_rn(__uint_as_float(vp[c]), __uint_as_float(vp[c + 1])));
+          ob[sub][c >> 1] = h2u(__hmul2(g0, a0));
+          oa0[c >> 1] = h2u(a0);
         }
+        if (HAS_R) put_chunk(0, sub, oa0);
+      }
+      if (HAS_R) chunk_done(0);
+      if (HAS_R && KSEL == 2) {
+        {
+          const bool ok = mbar_wait_cluster(local(B_QFULL), tile_i & 1u, abort_flag);
+          if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+        }
+        tc_fence_after();
+        if (!chunk_free(1)) { failed = true; break; }
+#pragma unroll
+        for (int sub = 0; sub < 2; ++sub) {
+          const int col0 = cq * 32 + sub * 16;
+          uint32_t vp[16], vq[16], oa1[8];
+          tmem_ld16_nowait(taddr + acc * BN_UP + col0, vp);
+          tmem_ld16_nowait(taddr + 256 + col0, vq);
+          tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 16; c += 2) {
+            const __half2 a1 = gelu_fast2(__floats2half2_rn(__uint_as_float(vp[c]) + __uint_as_float(vq[c]),
+                                                            __uint_as_float(vp[c + 1]) + __uint_as_float(vq[c + 1])));
+            const uint32_t prev = ob[sub][c >> 1];
+            ob[sub][c >> 1] = h2u(__hfma2(g1, a1, *reinterpret_cast<const __half2*>(&prev)));
+            oa1[c >> 1] = h2u(a1);
+          }
+          put_chunk(1, sub, oa1);
+        }
+        chunk_done(1);
       }
       // accumulators drained: hand P (and Q) back to the leader's MMA warp
       tc_fence_before();
