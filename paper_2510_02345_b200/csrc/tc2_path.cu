@@ -650,12 +650,9 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
       // abar goes out last: a release at cluster scope waits for the thread's earlier global stores,
       // and by the next tile's hand-overs these have long landed
       {
-        uint4* dst = reinterpret_cast<uint4*>(p.abar + (size_t)row * p.N + nt * BN_UP + cq * 32);
+        __half* dst = p.abar + (size_t)row * p.N + nt * BN_UP + cq * 32;     // 64-byte aligned: two whole sectors
 #pragma unroll
-        for (int sub = 0; sub < 2; ++sub) {
-          dst[2 * sub] = make_uint4(ob[sub][0], ob[sub][1], ob[sub][2], ob[sub][3]);
-          dst[2 * sub + 1] = make_uint4(ob[sub][4], ob[sub][5], ob[sub][6], ob[sub][7]);
-        }
+        for (int sub = 0; sub < 2; ++sub) st_global_v8(dst + 16 * sub, ob[sub]);
       }
       if (HAS_R && (w + 1) % unit == 0) {
         if (hf < KSEL) {
@@ -915,9 +912,9 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
           uint32_t o[16];
 #pragma unroll
           for (int c = 0; c < 32; c += 2) o[c >> 1] = pack_half2(__uint_as_float(v[c]), __uint_as_float(v[c + 1]));
-          uint4* dst = reinterpret_cast<uint4*>(p.y + (size_t)tok * p.N + nt * BN + c0);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) dst[i] = make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+          __half* dst = p.y + (size_t)tok * p.N + nt * BN + c0;                 // 64-byte aligned: two whole sectors
+          st_global_v8(dst, o);
+          st_global_v8(dst + 16, o + 8);
         }
       }
       tc_fence_before();
