@@ -539,7 +539,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
           const uint32_t slot = n % Cfg::NA, aph = (n / Cfg::NA) & 1u;
           if (!mbar_wait_cluster(local(B_AFULL + slot), aph, abort_flag)) { failed = true; break; }
           tc_fence_after();
-          const int hf = c / KSEL, j = c - hf * KSEL;
+          const int j = c >> 1, hf = c & 1;      // first-expert chunks of both halves first: the order the epilogues hand them over
           const uint64_t adesc = umma_desc(aring + slot * A_CHUNK_BYTES);
           const uint64_t bdesc = umma_desc(u2base + ub * U2_TILE_BYTES + hf * U2_CHUNK_BYTES);
 #pragma unroll
@@ -583,7 +583,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
       auto put_chunk = [&](int j, int sub, const uint32_t* src) {
         // a_j into its chunk as a K-major 128-byte-swizzled A operand: 16-byte unit u of row rowc sits at
         // rowc*128 + ((u ^ (rowc & 7)) << 4); this warp owns units 4 (cq & 1) + 2 sub + {0, 1}
-        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        const uint32_t n = tile_i * (2 * KSEL) + j * 2 + hf;
         const uint32_t cb = aring + (n % Cfg::NA) * A_CHUNK_BYTES + rowc * 128;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -592,14 +592,14 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
         }
       };
       auto chunk_free = [&](int j) {       // the S product that read this slot one tile ago has finished
-        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        const uint32_t n = tile_i * (2 * KSEL) + j * 2 + hf;
         const bool ok = mbar_wait_cluster(local(B_AEMPTY + n % Cfg::NA), ((n / Cfg::NA) & 1u) ^ 1u, abort_flag);
         return __all_sync(0xffffffffu, ok);
       };
       auto chunk_done = [&](int j) {
         fence_async_smem();
         __syncwarp();
-        const uint32_t n = tile_i * (2 * KSEL) + hf * KSEL + j;
+        const uint32_t n = tile_i * (2 * KSEL) + j * 2 + hf;
         if (lane == 0) mbar_arrive_cluster(lead(B_AFULL + n % Cfg::NA));
       };
       if (HAS_R && !chunk_free(0)) { failed = true; break; }
