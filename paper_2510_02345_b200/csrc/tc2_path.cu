@@ -600,7 +600,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
         fence_async_smem();
         __syncwarp();
         const uint32_t n = tile_i * (2 * KSEL) + j * 2 + hf;
-        if (lane == 0) mbar_arrive_cluster(lead(B_AFULL + n % Cfg::NA));
+        if (lane == 0) mbar_arrive_cluster_relaxed(lead(B_AFULL + n % Cfg::NA));   // after fence.proxy.async
       };
       if (HAS_R && !chunk_free(0)) { failed = true; break; }
 #pragma unroll
@@ -646,7 +646,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
       // accumulators drained: hand P (and Q) back to the leader's MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive_cluster(lead(B_TEMPTY + acc)); mbar_arrive_cluster(lead(B_QEMPTY)); }
+      if (lane == 0) { mbar_arrive_cluster_relaxed(lead(B_TEMPTY + acc)); mbar_arrive_cluster_relaxed(lead(B_QEMPTY)); }
       // abar goes out last: a release at cluster scope waits for the thread's earlier global stores,
       // and by the next tile's hand-overs these have long landed
       {
@@ -704,7 +704,7 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
           }
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(lead(B_SEMPTY));
+          if (lane == 0) mbar_arrive_cluster_relaxed(lead(B_SEMPTY));
         }
         ++flushes;
       }
@@ -919,7 +919,7 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(lead(B_TEMPTY + acc));
+      if (lane == 0) mbar_arrive_cluster_relaxed(lead(B_TEMPTY + acc));
     }
   }
 
