@@ -80,14 +80,23 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster) {
   pdl_wait();
   __shared__ int sh_seg[kMaxG + 1];
-  for (int key = threadIdx.x; key < nkey; key += blockDim.x) {
+  // a warp per key, lanes over the blocks: exclusive prefix sums of the key's per-block counts
+  const int lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
+  for (int key = threadIdx.x >> 5; key < nkey; key += nwarp) {
     int run = 0;
-    for (int b = 0; b < nblk; ++b) {
-      int c = block_counts[(size_t)b * nkey + key];
-      block_base[(size_t)b * nkey + key] = run;
-      run += c;
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+      const int b = b0 + lane;
+      const int c = b < nblk ? block_counts[(size_t)b * nkey + key] : 0;
+      int incl = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (b < nblk) block_base[(size_t)b * nkey + key] = run + incl - c;
+      run += __shfl_sync(0xffffffffu, incl, 31);
     }
-    key_cnt[key] = run;
+    if (lane == 0) key_cnt[key] = run;
   }
   __syncthreads();
   if (threadIdx.x == 0) {

@@ -136,7 +136,7 @@ struct TParams {
   int KC, K, r;
 };
 
-constexpr int T_THREADS = 192;
+constexpr int T_THREADS = 224;      // warps 0 and 6 TMA (alternating stages), 1 MMA, 2..5 epilogue
 constexpr int T_STAGES = 6;
 constexpr uint32_t T_STAGE_BYTES = BM * BK * 2 + KE * BK * 2;   // 24 KB
 
@@ -179,9 +179,9 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
   const int KC = p.KC;
   bool failed = false;
 
-  if (warp == 0) {
+  if (warp == 0 || warp == 6) {
     if (lane == 0) {
-      for (int kc = 0; kc < KC; ++kc) {
+      for (int kc = warp == 0 ? 0 : 1; kc < KC; kc += 2) {
         const uint32_t s = kc % T_STAGES, ph = (kc / T_STAGES) & 1u;
         if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
         const uint32_t a_dst = base + s * T_STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
@@ -206,7 +206,7 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
       }
       if (!failed) umma_commit(tfull);
     }
-  } else {
+  } else if (warp < 6) {
     const int q = warp & 3;
     const int row = mt * BM + q * 32 + lane;
     const int r = p.r;
