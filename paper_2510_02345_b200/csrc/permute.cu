@@ -80,6 +80,7 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster) {
   pdl_wait();
   __shared__ int sh_seg[kMaxG + 1];
+  __shared__ int sh_cnt[kMaxKeys];
   // a warp per key, lanes over the blocks: exclusive prefix sums of the key's per-block counts
   const int lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   for (int key = threadIdx.x >> 5; key < nkey; key += nwarp) {
@@ -96,7 +97,7 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
       if (b < nblk) block_base[(size_t)b * nkey + key] = run + incl - c;
       run += __shfl_sync(0xffffffffu, incl, 31);
     }
-    if (lane == 0) key_cnt[key] = run;
+    if (lane == 0) { key_cnt[key] = run; sh_cnt[key] = run; }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -107,7 +108,7 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
       int cnt = 0;
       for (int s = 0; s < nsub; ++s) {
         key_off[g * nsub + s] = off + cnt;
-        cnt += key_cnt[g * nsub + s];
+        cnt += sh_cnt[g * nsub + s];
       }
       seg_cnt[g] = cnt;
       off += (cnt + row_align - 1) / row_align * row_align;
