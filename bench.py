@@ -60,6 +60,36 @@ def stage_work(s, T, stage, active_clusters, active_experts):
     return (0.0, 0.0)
 
 
+# ------------------------------------------------------------------ DRAM traffic of the dominant kernel
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under
+# profiles/ (ncu_gpt2m_tc2_up_down.md, ncu_decode_stream_kernels.md).  The figure is reported only while
+# the kernel sources still have the hash they had at the capture; otherwise "traffic" is null.
+NCU_TRAFFIC = {
+    "gpt2m": {"kernel": "tc2_up_kernel<true,2>", "bytes": 119.380224e6 + 110.086912e6,
+              "sha1": {"tc2_path.cu": "a154d2d232a34cc56ed2e340e6b9af1bc977cfb0",
+                       "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 956.056064e6 + 9.835008e6,
+               "sha1": {"stream_path.cu": "ff9ca4655bcb87c2f136a404415963dd060c98a0",
+                        "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
+}
+
+
+def ncu_traffic(workload):
+    import hashlib
+    ent = NCU_TRAFFIC.get(workload)
+    if ent is None:
+        return None
+    csrc = os.path.join(ROOT, "paper_2510_02345_b200", "csrc")
+    for name, want in ent["sha1"].items():
+        try:
+            with open(os.path.join(csrc, name), "rb") as f:
+                if hashlib.sha1(f.read()).hexdigest() != want:
+                    return None
+        except OSError:
+            return None
+    return ent["bytes"]
+
+
 # ------------------------------------------------------------------ clocks
 class ClockSampler:
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -227,12 +257,12 @@ def roofline_for(res, peaks, peaks_kind):
         peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
         ach = flops / (ms * 1e-3) / 1e12
         return {"bound": "tensor", "kernel": stage, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                "frac": ach / peak, "traffic": None, "peak_kind": f"{peaks_kind} cuBLAS bf16 sustained (fp16 has the same rate)",
+                "frac": ach / peak, "traffic": ncu_traffic(res["name"]) if stage == "up" else None, "peak_kind": f"{peaks_kind} cuBLAS bf16 sustained (fp16 has the same rate)",
                 "kernel_ms": ms, "flops_per_launch": flops}
     peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
     ach = nbytes / (ms * 1e-3) / 1e9
     return {"bound": "hbm", "kernel": stage, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-            "traffic": None, "peak_kind": f"{peaks_kind} copy bandwidth", "kernel_ms": ms,
+            "traffic": ncu_traffic(res["name"]) if stage == "up" else None, "peak_kind": f"{peaks_kind} copy bandwidth", "kernel_ms": ms,
             "bytes_per_launch": nbytes}
 
 
