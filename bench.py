@@ -247,6 +247,21 @@ def barrier():
         _dist.barrier()
 
 
+def max_over_ranks(values, dist, device="cpu"):
+    """The only collective of a multi-rank run: the MAX over ranks of the device timings (the replicas
+    exchange no data).  `dist` is torch.distributed with an initialised process group."""
+    import torch
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def replicas_value(world, tokens_per_rank, ms_per_step):
+    """Whole-job tokens/s of `world` independent replicas that each process tokens_per_rank tokens per step,
+    timed by the slowest rank."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def roofline_for(res, peaks, peaks_kind):
     s, T = res["shape"], res["T"]
     stage = max(("up", "down"), key=lambda n: res["stage_ms"].get(n, 0.0))
@@ -362,12 +377,10 @@ def main():
     dev_ms = res["dev_ms"]
     e2e_ms = res["e2e"]["ms_per_step"]
     if world > 1:
-        t = torch.tensor([dev_ms, e2e_ms], device=f"cuda:{local_rank}", dtype=torch.float64)
-        _dist.all_reduce(t, op=_dist.ReduceOp.MAX)     # timing only: max over ranks
-        dev_ms, e2e_ms = float(t[0]), float(t[1])
+        dev_ms, e2e_ms = max_over_ranks([dev_ms, e2e_ms], _dist, f"cuda:{local_rank}")
     s, T = res["shape"], res["T"]
     ms_per_step = dev_ms / steps
-    value = world * T / (ms_per_step * 1e-3)
+    value = replicas_value(world, T, ms_per_step)
 
     if rank == 0:
         peaks, kind = load_peaks()

@@ -84,6 +84,10 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes);
  * default stream and waits for them; work queued by the caller on other non-blocking streams that
  * produces the weights must have finished.  After it returns the source weight buffers may be
  * freed; the arena must outlive the handle and must not be written by the caller. */
+/* Two environment variables, read by cmoe_create, exist for A/B measurements: CMOE_FORCE_PATH=0 keeps
+ * the generic CUDA-core path for every shape; CMOE_ROUTER_FP32=1 keeps batches of 1024 tokens and more
+ * on the fp32 CUDA-core router instead of the tensor-core router (split fp16 router matrices, logit
+ * error about 1e-6). */
 int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
 
 /* Two-stage routing only (Sec. 3.3, Eq. 9-10) for x = fp16 [T][d]:
@@ -107,7 +111,8 @@ int cmoe_status(cmoe_layer* layer, void* cuda_stream);
 
 /* Per-handle facts for tests and benchmarks (host struct, filled by cmoe_get_info). */
 typedef struct {
-  int32_t path;              /* 0 generic CUDA-core path, 1 tcgen05 grouped-GEMM path, 2 weight-streaming path */
+  int32_t path;              /* 0 generic CUDA-core path, 1 tcgen05 grouped-GEMM path (T_max > 128),
+                                2 weight-streaming path (T_max <= 128); chosen by cmoe_create             */
   int32_t launches_route;    /* kernel launches one cmoe_route call enqueues                       */
   int32_t launches_forward;  /* kernel launches one cmoe_forward call enqueues (memsets excluded)  */
   int32_t row_align;         /* permuted-row alignment of a cluster segment                        */
