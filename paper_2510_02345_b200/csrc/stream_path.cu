@@ -34,7 +34,7 @@ constexpr int SBK = 64;            // halves per K atom: one 128-byte swizzle ro
 constexpr int SKA = 2;             // K atoms per stage
 constexpr int SNB = 64;            // most token rows per segment (MMA N)
 constexpr int SMAXSEG = 160;       // segments: at most G + T_pad / 64
-constexpr int S_THREADS = 384;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..11 epilogue
+constexpr int S_THREADS = 640;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..19 epilogue
 constexpr uint32_t S_B_ATOM = SNB * SBK * 2;             // 8 KB
 constexpr uint32_t S_TMEM_COLS = 128;                    // two accumulators of up to 64 columns
 
@@ -69,12 +69,14 @@ struct SCfg {
 };
 
 // Tiles have 128 feature rows.  In the up kernel the tiles of the last, incomplete round of the
-// round-robin are cut into halves of 64 rows (loaded with tmWh; the MMA still spans 128 rows and the
-// upper half of the accumulator is not read), so that the tail occupies twice as many SMs for half
-// as long.  The down kernel gets its granularity from the K ranges.
+// round-robin are cut into 2, 4, 8 or 16 slices of 64 ... 8 rows (loaded with the boxes of tmWs; the
+// MMA still spans 128 rows and the rest of the accumulator is not read), as many as still fit one
+// slice per CTA, so that the tail occupies all SMs for a fraction of a tile time.  The down kernel
+// gets its granularity from the K ranges.
+struct SliceMaps { CUtensorMap m[4]; };      // boxes of 64, 32, 16, 8 weight rows
 template <bool UP>
 __global__ void __launch_bounds__(S_THREADS, 1)
-stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmWh,
+stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ SliceMaps tmWs,
               const __grid_constant__ CUtensorMap tmTok, const StreamParams p) {
   pdl_wait();
   constexpr int MROWS = 128;
@@ -95,7 +97,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
   int* seg_g = seg_rows + SMAXSEG;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int kEpiWarps = 8;       // two warps per TMEM lane quadrant: even and odd token columns
+  constexpr int kEpiWarps = 16;      // four warps per TMEM lane quadrant: token columns c with c mod 4 = 0, 1, 2, 3
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -128,18 +130,22 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
   const int ksplit = UP ? 1 : p.ksplit;
   const int KCH = p.Kd / (SBK * SKA);                    // stages in the whole reduction
   const int n_tiles = *n_seg_p * n_mt * ksplit;
-  int n_whole = n_tiles;                                 // units [0, n_whole) are whole tiles, the rest halves
+  int n_whole = n_tiles;                                 // units [0, n_whole) are whole tiles, the rest slices
+  int lg_f = 0;                                          // log2 of the slices per tail tile
   if (UP) {
     const int tail = n_tiles % (int)gridDim.x;
-    if (tail > 0 && 2 * tail <= (int)gridDim.x) n_whole = n_tiles - tail;
+    if (tail > 0) {
+      while (lg_f < 4 && (tail << (lg_f + 1)) <= (int)gridDim.x) ++lg_f;
+      if (lg_f > 0) n_whole = n_tiles - tail;
+    }
   }
-  const int n_units = n_whole + 2 * (n_tiles - n_whole);
+  const int n_units = n_whole + ((n_tiles - n_whole) << lg_f);
   const int my_units = (int)blockIdx.x < n_units ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  // half: -1 for a whole tile, else which 64 rows of the tile
-  auto unit_of = [&](int i, int& seg, int& mt, int& half, int& c_begin, int& c_end) {
+  // slice: -1 for a whole tile, else which (128 >> lg_f) rows of the tile
+  auto unit_of = [&](int i, int& seg, int& mt, int& slice, int& c_begin, int& c_end) {
     int u = blockIdx.x + i * gridDim.x;
-    half = -1;
-    if (u >= n_whole) { half = (u - n_whole) & 1; u = n_whole + ((u - n_whole) >> 1); }
+    slice = -1;
+    if (u >= n_whole) { slice = (u - n_whole) & ((1 << lg_f) - 1); u = n_whole + ((u - n_whole) >> lg_f); }
     const int ks = u % ksplit, sm_ = u / ksplit;
     mt = sm_ % n_mt;
     seg = sm_ / n_mt;
@@ -154,18 +160,19 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
       uint32_t it = 0;                                     // stage counter over all units
       const uint32_t mine = warp == 0 ? 0u : 1u;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, half, c0, c1;
-        unit_of(i, seg, mt, half, c0, c1);
+        int seg, mt, slice, c0, c1;
+        unit_of(i, seg, mt, slice, c0, c1);
         const int g = seg_g[seg], row0 = seg_row0[seg], nb = seg_rows[seg] / 16;
-        const int wrow = g * p.M + mt * MROWS + (half > 0 ? 64 : 0);
-        const uint32_t a_bytes = half < 0 ? Cfg::A_BYTES : Cfg::A_BYTES / 2;
+        const int srows = slice < 0 ? MROWS : MROWS >> lg_f;          // weight rows this unit loads
+        const int wrow = g * p.M + mt * MROWS + (slice < 0 ? 0 : slice * srows);
+        const uint32_t a_bytes = (uint32_t)srows * SBK * 2 * SKA;
         for (int c = c0; c < c1; ++c, ++it) {
           if ((it & 1u) != mine) continue;
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
           const uint32_t a_dst = base + s * Cfg::STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
           mbar_expect_tx(full0 + 8 * s, a_bytes + (uint32_t)nb * SKA * 16 * SBK * 2);
-          tma_load_3d(a_dst, half < 0 ? &tmW : &tmWh, full0 + 8 * s, 0, wrow, c * SKA);
+          tma_load_3d(a_dst, slice < 0 ? &tmW : &tmWs.m[lg_f - 1], full0 + 8 * s, 0, wrow, c * SKA);
           // the tokens: 16 rows per box; atom a of block b lands at atom a, rows 16 b .. of the B tile
           for (int b = 0; b < nb; ++b)
             for (int a = 0; a < SKA; ++a)
@@ -178,10 +185,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, half, c0, c1;
-        unit_of(i, seg, mt, half, c0, c1);
+        int seg, mt, slice, c0, c1;
+        unit_of(i, seg, mt, slice, c0, c1);
         const uint32_t idesc = idesc_f16(128, seg_rows[seg]);
-        const uint32_t a_atom16 = (half < 0 ? Cfg::A_ATOM : Cfg::A_ATOM / 2) >> 4;   // second K atom, in 16-byte units
+        const uint32_t a_atom16 = (slice < 0 ? Cfg::A_ATOM : Cfg::A_ATOM >> lg_f) >> 4;   // second K atom, in 16-byte units
         const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
         if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
@@ -207,15 +214,17 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
   } else if (warp >= 4) {
     // ---------------- epilogue warps: one thread per output feature of the tile
     const int q = warp & 3;
-    const int parity = (warp - 4) >> 2;                  // which token columns of the accumulator this warp takes
+    const int part = (warp - 4) >> 2;                    // which token columns of the accumulator this warp takes
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int r = p.r, k = p.k, M = p.M;
     for (int i = 0; i < my_units; ++i) {
-      int seg, mt, half, c0, c1;
-      unit_of(i, seg, mt, half, c0, c1);
-      const int row0 = seg_row0[seg], nrows = half >= 0 && q >= 2 ? 0 : seg_rows[seg];   // half tiles: two warps have no rows
+      int seg, mt, slice, c0, c1;
+      unit_of(i, seg, mt, slice, c0, c1);
+      const int srows = slice < 0 ? MROWS : MROWS >> lg_f;
+      const bool mine = q * 32 + lane < srows;             // slices: only the first srows accumulator lanes are real
+      const int row0 = seg_row0[seg], nrows = q * 32 < srows ? seg_rows[seg] : 0;
       const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
-      const int f = mt * MROWS + (half > 0 ? 64 : 0) + q * 32 + lane;   // output feature (up) / output column (down)
+      const int f = mt * MROWS + (slice < 0 ? 0 : slice * srows) + q * 32 + lane;   // output feature (up) / output column (down)
       {
         const bool ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -226,11 +235,11 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
         tmem_ld16_nowait(taddr + acc * SNB + tb, v);
         tmem_ld_wait();
 #pragma unroll
-        for (int c2 = 0; c2 < 8; ++c2) {
-          const int c = 2 * c2 + parity;
+        for (int c2 = 0; c2 < 4; ++c2) {
+          const int c = 4 * c2 + part;
           const int row = row0 + tb + c;
-          const bool real = p.row_token[row] >= 0;         // the same for every thread
-          const float dv = __uint_as_float(parity ? v[2 * c2 + 1] : v[2 * c2]);
+          const bool real = mine && p.row_token[row] >= 0;
+          const float dv = __uint_as_float(part == 0 ? v[4 * c2] : part == 1 ? v[4 * c2 + 1] : part == 2 ? v[4 * c2 + 2] : v[4 * c2 + 3]);
           if (UP) {
             float ab = 0.f;
             if (real) {
@@ -272,7 +281,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ C
                 if (r > 0) p.a_slot[((size_t)row * k + j) * M + f] = __float2half_rn(a);
               }
             }
-            p.abar[(size_t)row * M + f] = __float2half_rn(ab);
+            if (mine) p.abar[(size_t)row * M + f] = __float2half_rn(ab);
           } else {
             if (real) atomicAdd(p.y32 + (size_t)row * M + f, dv);
           }
@@ -413,14 +422,15 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
 }
 
 struct StreamState {
-  CUtensorMap mW1, mW1h, mX, mW2, mAbar;
+  CUtensorMap mW1, mX, mW2, mAbar;
+  SliceMaps mW1s;
   int sm_count;
   int ksplit;
 };
 static_assert(sizeof(StreamState) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
 
 template <bool UP>
-cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mWh, const CUtensorMap& mTok, const StreamParams& p, int grid,
+cudaError_t launch_stream(const CUtensorMap& mW, const SliceMaps& mWs, const CUtensorMap& mTok, const StreamParams& p, int grid,
                           cudaStream_t st) {
   auto kern = stream_kernel<UP>;
   constexpr size_t sm = SCfg<128>::SMEM;
@@ -432,7 +442,7 @@ cudaError_t launch_stream(const CUtensorMap& mW, const CUtensorMap& mWh, const C
     attr_set = true;
   }
   launch_chained(kern, dim3(grid), dim3(S_THREADS), sm, st, 1,
-      mW, mWh, mTok, p);
+      mW, mWs, mTok, p);
   return cudaGetLastError();
 }
 
@@ -452,7 +462,9 @@ cudaError_t stream_init(cmoe_layer* L) {
   e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
-  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 128, SKA) && make_map(&ts->mW1h, L->w.B1t, G * D.d_ff, D.d, 64, SKA) &&
+  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 128, SKA) && make_map(&ts->mW1s.m[0], L->w.B1t, G * D.d_ff, D.d, 64, SKA) &&
+                  make_map(&ts->mW1s.m[1], L->w.B1t, G * D.d_ff, D.d, 32, SKA) && make_map(&ts->mW1s.m[2], L->w.B1t, G * D.d_ff, D.d, 16, SKA) &&
+                  make_map(&ts->mW1s.m[3], L->w.B1t, G * D.d_ff, D.d, 8, SKA) &&
                   make_map(&ts->mX, S.x_perm, P, D.d, 16, 0) &&
                   make_map(&ts->mW2, L->w.B2t, G * D.d, D.d_ff, 128, SKA) && make_map(&ts->mAbar, S.abar, P, D.d_ff, 16, 0);
   // K ranges per down tile: fill the SMs evenly, keep at least four stages per range
@@ -495,7 +507,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     p.Kd = D.d; p.M = D.d_ff; p.ksplit = 1;
     const long long units = (long long)seg_bound * (D.d_ff / 128);
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<true>(ts.mW1, ts.mW1h, ts.mX, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<true>(ts.mW1, ts.mW1s, ts.mX, p, grid, st)) != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
@@ -508,7 +520,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     p.Kd = D.d_ff; p.M = D.d; p.ksplit = ts.ksplit;
     const long long units = (long long)seg_bound * (D.d / 128) * ts.ksplit;
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<false>(ts.mW2, ts.mW2, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<false>(ts.mW2, ts.mW1s, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
   }
   dim3 fgrid((D.d + 255) / 256, rows_bound);
   launch_chained(stream_final_kernel, dim3(fgrid), dim3(256), 0, st, 1,
