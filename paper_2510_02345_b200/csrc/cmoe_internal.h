@@ -123,7 +123,7 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
                            size_t zero_bytes);
-constexpr int kPermuteLaunches = 5;        // 2 for batches of at most 256 tokens (permute_launches)
+constexpr int kPermuteLaunches = 4;        // 2 for batches of at most 256 tokens (permute_launches)
 inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
 // generic_path.cu : CUDA-core path for any supported shape
 // `marks` (or null): three events recorded before the residual-t, up and down stages

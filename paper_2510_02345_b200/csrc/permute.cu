@@ -4,10 +4,10 @@
 // cluster, then to experts inside it", Sec. 3.3); the mechanism is this library's.
 //
 //   hist     per-block histogram of the keys (block = 256 consecutive tokens)
-//   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table
+//   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table, and the
+//            table entries of the padding rows of each segment (no token, zero gates)
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
 //            writes the row tables
-//   pad      fills the table entries of the padding rows of each segment (no token, zero gates)
 //   move     copies every token's activations to its row with 16-byte vectors (a block per row;
 //            padding rows get zeros) and clears the buffer the later stages accumulate into
 //
@@ -77,9 +77,11 @@ __global__ void __launch_bounds__(1024)
 scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             const int* __restrict__ block_counts, int* __restrict__ block_base,
             int* __restrict__ key_cnt, int* __restrict__ key_off, int* __restrict__ seg_off,
-            int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster) {
+            int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster, int K, int k,
+            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate) {
   pdl_wait();
   __shared__ int sh_seg[kMaxG + 1];
+  __shared__ int sh_segcnt[kMaxG];
   __shared__ int sh_cnt[kMaxKeys];
   // a warp per key, lanes over the blocks: exclusive prefix sums of the key's per-block counts
   const int lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
@@ -111,6 +113,7 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
         cnt += sh_cnt[g * nsub + s];
       }
       seg_cnt[g] = cnt;
+      sh_segcnt[g] = cnt;
       off += (cnt + row_align - 1) / row_align * row_align;
     }
     sh_seg[G] = off;
@@ -118,6 +121,17 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
     *n_rows = off;
   }
   __syncthreads();
+  // table entries of the padding rows of every cluster (the scatter kernel writes the token rows only)
+  for (int g = 0; g < G; ++g) {
+    const int first = sh_seg[g] + sh_segcnt[g], last = sh_seg[g + 1];
+    for (int row = first + (int)threadIdx.x; row < last; row += blockDim.x) {
+      row_token[row] = -1;
+      for (int j = 0; j < k; ++j) {
+        row_slot[(size_t)row * k + j] = g * K + j;       // any valid experts of the cluster
+        row_gate[(size_t)row * k + j] = 0.f;
+      }
+    }
+  }
   const int ntile = sh_seg[G] / row_align;
   for (int tile = threadIdx.x; tile < max_tiles; tile += blockDim.x) {
     int g = -1;
@@ -196,22 +210,6 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
     zero_ptr[i] = make_uint4(0, 0, 0, 0);
 }
 
-__global__ void __launch_bounds__(256)
-pad_kernel(int d, int K, int k, const int* __restrict__ seg_off, const int* __restrict__ seg_cnt,
-           int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
-           __half* __restrict__ x_perm) {
-  pdl_wait();
-  const int g = blockIdx.x;
-  const int first = seg_off[g] + seg_cnt[g], last = seg_off[g + 1];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  for (int row = first + warp; row < last; row += nwarp) {
-    if (lane == 0) row_token[row] = -1;
-    if (lane < k) {
-      row_slot[(size_t)row * k + lane] = g * K + lane;   // any valid experts of the cluster
-      row_gate[(size_t)row * k + lane] = 0.f;
-    }
-  }
-}
 
 // The whole permutation of a small batch (T <= 256) in one block: keys, counts, offsets, the stable
 // rank of every token inside its key (by counting the earlier tokens with the same key), the row
@@ -320,15 +318,12 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
   launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
       nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
                                   S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
-                                  S.seg_cnt, S.n_rows, S.tile_cluster);
+                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
   launch_chained(scatter_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
       T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
                                                S.x_perm);
-  launch_chained(pad_kernel, dim3(D.G), dim3(256), 0, st, 1,
-      D.d, D.K, D.k, S.seg_off, S.seg_cnt, S.row_token, S.row_slot,
-                                  S.row_gate, S.x_perm);
   const int move_grid = rows_bound < 148 * 32 ? rows_bound : 148 * 32;
   launch_chained(move_rows_kernel, dim3(move_grid), dim3(128), 0, st, 1,
       D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
