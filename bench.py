@@ -68,8 +68,8 @@ NCU_TRAFFIC = {
     "gpt2m": {"kernel": "tc2_up_kernel<true,2>", "bytes": 119.380224e6 + 110.086912e6,
               "sha1": {"tc2_path.cu": "a154d2d232a34cc56ed2e340e6b9af1bc977cfb0",
                        "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 956.056064e6 + 9.835008e6,
-               "sha1": {"stream_path.cu": "ff9ca4655bcb87c2f136a404415963dd060c98a0",
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.955200e6 + 9.806848e6,
+               "sha1": {"stream_path.cu": "003cd0de2d54c2059eaa9e7293f25ee4a5ff228d",
                         "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
 }
 
@@ -298,9 +298,14 @@ def oracle_rate(name, target_s=15.0, max_tokens=None):
     L = inputs.make_layer(s, seed=0)
     o = ref.Layer(L)
     T = L["x"].shape[0]
-    probe = min(T, 64)
-    t0 = time.perf_counter(); o.forward(L["x"][:probe]); dt = time.perf_counter() - t0
-    n = int(min(T, max(probe, probe * target_s / max(dt, 1e-3))))
+    # every call forms the expert weights first (a fixed cost) and then works per token: two probes
+    # separate the two, and the sample is sized for about target_s seconds
+    n1, n2 = min(T, 32), min(T, 256)
+    t0 = time.perf_counter(); o.forward(L["x"][:n1]); t1 = time.perf_counter() - t0
+    t0 = time.perf_counter(); o.forward(L["x"][:n2]); t2 = time.perf_counter() - t0
+    per_tok = max((t2 - t1) / max(n2 - n1, 1), 1e-7)
+    fixed = max(t1 - per_tok * n1, 0.0)
+    n = int(min(T, max(n2, (target_s - fixed) / per_tok)))
     if max_tokens:
         n = min(n, max_tokens)
     n = max(1, n)
