@@ -84,10 +84,11 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes);
  * default stream and waits for them; work queued by the caller on other non-blocking streams that
  * produces the weights must have finished.  After it returns the source weight buffers may be
  * freed; the arena must outlive the handle and must not be written by the caller. */
-/* Two environment variables, read by cmoe_create, exist for A/B measurements: CMOE_FORCE_PATH=0 keeps
+/* Three environment variables, read by cmoe_create, exist for A/B measurements: CMOE_FORCE_PATH=0 keeps
  * the generic CUDA-core path for every shape; CMOE_ROUTER_FP32=1 keeps batches of 1024 tokens and more
  * on the fp32 CUDA-core router instead of the tensor-core router (split fp16 router matrices, logit
- * error about 1e-6). */
+ * error about 1e-6); CMOE_UP_TILE=128 keeps the up projection of large batches on 128-column tiles
+ * where d_ff would allow 256-column tiles. */
 int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
 
 /* Two-stage routing only (Sec. 3.3, Eq. 9-10) for x = fp16 [T][d]:

@@ -27,43 +27,16 @@
 // is the KE-deep steps (skipped per tile for experts no row of the tile uses) and the S products.
 // Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
-#include "cmoe_internal.h"
-#include "launch.cuh"
-#include "device_utils.cuh"
-#include "tc_ptx.cuh"
+#include "tc2_common.cuh"
 
 namespace cmoe {
 
 namespace {
 
-using namespace ptx;
+using namespace tc2c;
 
-constexpr int BM = 128;          // rows per tile (UMMA M)
-constexpr int BK = 64;           // halves per K chunk: one 128-byte swizzle row
-constexpr int KE = 64;           // width of the expanded rank index
 constexpr int BN_UP = 128;
-constexpr uint32_t kTmemCols = 512;
-constexpr size_t kSmemLimit = 232448;   // 227 KB
 constexpr int kMaxStages = 8;
-
-// ------------------------------------------------------------------------------------------------
-// small helpers
-// ------------------------------------------------------------------------------------------------
-
-// all lanes wait; the warp agrees on the outcome so that it never diverges around .sync.aligned code
-__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  const bool ok = mbar_wait(bar, parity, abort_flag);
-  return __all_sync(0xffffffffu, ok);
-}
-
-__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
-  __half2 h = __floats2half2_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&h);
-}
-
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 
 // ------------------------------------------------------------------------------------------------
 // stage: INT4 factors -> fp16 operand matrices (one thread per 32-bit word = 8 codes)
@@ -281,20 +254,6 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
 // ------------------------------------------------------------------------------------------------
 // up: CTA pairs (cta_group::2) on 256 x 128 tiles; each CTA owns 128 rows
 // ------------------------------------------------------------------------------------------------
-struct Up2Params {
-  const int* n_rows;
-  const int* tile_cluster;   // per 256-row tile
-  const int* tile_mask;      // per 128-row tile, two words
-  const int* row_slot;
-  const float* row_gate;
-  const int* row_token;
-  float* s_out;        // [rows][k][r] fp32, zeroed by the caller
-  __half* abar;        // [rows][N]
-  int* status;
-  int KC, NT, N, K, k, r, log2r;
-  int unit;            // N tiles per work unit (divides NT)
-};
-
 // Warp roles: 0 and 3 TMA (alternating stages), 1 MMA, 2 S products, 4..19 epilogue.
 // One thread can issue a TMA tile load only every few hundred cycles, and everything a single
 // thread does between two MMAs delays the next one, so a stage carries two 64-wide K atoms (eight
@@ -327,21 +286,6 @@ struct UpCfg {
   static constexpr uint32_t BAR_OFF = RING + ARING + U2;
   static constexpr size_t SMEM = 1024 + BAR_OFF + 48 * 8;
 };
-
-// GELU(u) ~ u/2 (1 + tanh(u (c1 + c2 u^2))) on two fp16 values at once, with c1, c2 fitted to the erf
-// form (max abs deviation 2.7e-4 over the reals) and the hardware tanh; the error is of the size of the
-// fp16 rounding of the stored activation.
-__device__ __forceinline__ __half2 gelu_fast2(__half2 u) {
-  const __half2 u2 = __hmul2(u, u);
-  const __half2 w = __hfma2(u2, __float2half2_rn(0.03470089f), __float2half2_rn(0.80015708f));
-  const __half2 z = __hmul2(u, w);
-  uint32_t zi = *reinterpret_cast<const uint32_t*>(&z), ti;
-  asm("tanh.approx.f16x2 %0, %1;" : "=r"(ti) : "r"(zi));
-  const __half2 th = *reinterpret_cast<const __half2*>(&ti);
-  const __half2 hu = __hmul2(u, __float2half2_rn(0.5f));
-  return __hfma2(hu, th, hu);
-}
-__device__ __forceinline__ uint32_t h2u(__half2 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
 template <bool HAS_R, int KSEL>
 __global__ void __launch_bounds__(UP_THREADS, 1)
@@ -989,25 +933,16 @@ bool make_map3(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
 }
 
 struct Tc2State {
-  CUtensorMap mX, mX3, mB13, mA0, mAd, mV1, mU2;   // up (mX: 2-D, for the t kernel)
+  CUtensorMap mX, mX3, mB13, mA0, mAd, mV1, mU2;   // up (mX: 2-D, for the t kernel and the wide up kernel)
+  CUtensorMap mB1w, mV1w;                      // wide up kernel: 128-row boxes of B1t and V1f
   CUtensorMap mU1;                             // t
   CUtensorMap mAbar3, mB23, mAs, mV2;          // down
   int bn_down;
+  int up_wide;       // d_ff is a multiple of 256: the up kernel on 256-column tiles (tc2_up_wide.cu)
   int sm_count;
   int log2r;
 };
 static_assert(sizeof(Tc2State) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
-
-template <typename Kern>
-cudaError_t set_smem(Kern kern, size_t bytes) {
-  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
-
-// launch as thread-block clusters of two CTAs (grid = 2 x pairs)
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {
-  return launch_chained(kern, dim3((unsigned)grid), dim3((unsigned)threads), smem, st, 2, args...);
-}
 
 template <bool HAS_R, int KSEL>
 cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStream_t st) {
@@ -1078,6 +1013,10 @@ cudaError_t tc2_init(cmoe_layer* L) {
   const Scratch& S = L->sc;
   Tc2State* ts = reinterpret_cast<Tc2State*>(L->tc_state);
   ts->bn_down = (D.d % 256 == 0) ? 256 : 128;
+  {
+    const char* tile = getenv("CMOE_UP_TILE");
+    ts->up_wide = (D.d_ff % BN_WIDE == 0 && !(tile && atoi(tile) == 128)) ? 1 : 0;
+  }
   ts->log2r = D.r > 0 ? ilog2(D.r) : 0;
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -1088,12 +1027,14 @@ cudaError_t tc2_init(cmoe_layer* L) {
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mX3, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mB13, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
+            make_map(&ts->mB1w, L->w.B1t, G * D.d_ff, D.d, BN_WIDE / 2) &&
             make_map3(&ts->mAbar3, S.abar, P, D.d_ff, BM) &&
             make_map3(&ts->mB23, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
   if (ok && D.r > 0) {
     ok = make_map(&ts->mA0, S.A0, P, KE, BM) && make_map(&ts->mAd, S.Ad, P, KE, BM) &&
          make_map(&ts->mAs, S.As, P, KE, BM) &&
          make_map(&ts->mV1, S.V1f, G * D.d_ff, KE, BN_UP / 2) &&
+         make_map(&ts->mV1w, S.V1f, G * D.d_ff, KE, BN_WIDE / 2) &&
          make_map(&ts->mV2, S.V2f, G * D.d, KE, ts->bn_down / 2) &&
          make_map(&ts->mU1, S.U1f, G * KE, D.d, KE) &&
          make_map(&ts->mU2, S.U2f, G * KE, D.d_ff, KE / 2);
@@ -1108,7 +1049,7 @@ cudaError_t tc2_init(cmoe_layer* L) {
   } else if (ok) {
     // unused maps still have to be valid kernel arguments
     ts->mA0 = ts->mX; ts->mAd = ts->mX; ts->mV1 = ts->mX; ts->mU2 = ts->mX; ts->mU1 = ts->mX;
-    ts->mAs = ts->mX; ts->mV2 = ts->mX;
+    ts->mAs = ts->mX; ts->mV2 = ts->mX; ts->mV1w = ts->mX;
   }
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
@@ -1155,10 +1096,15 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
   {
     const int pairs = ts.sm_count / 2;
+    if (ts.up_wide) { up.KC = D.d / BK; up.NT = D.d_ff / BN_WIDE; }
     up.unit = pick_unit(up.NT, pt_bound, pairs);
     const long long total = (long long)pt_bound * (up.NT / up.unit);
     const int grid = 2 * (int)(total < pairs ? total : pairs);
-    if (D.r == 0)      e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates
+    if (ts.up_wide) {
+      const UpWideMaps maps{&ts.mX, &ts.mB1w, &ts.mA0, &ts.mAd, &ts.mV1w, &ts.mU2};
+      e = launch_up_wide(D.r > 0, D.k, maps, up, grid, st);
+    }
+    else if (D.r == 0) e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates
     else if (D.k == 2) e = launch_up<true, 2>(ts, up, grid, st);
     else               e = launch_up<true, 1>(ts, up, grid, st);
     if (e != cudaSuccess) return e;

@@ -256,6 +256,30 @@ def test_tensor_path_empty_cluster():
     assert got["module"].info.path == 1 and not np.any(got["cid"] == 1)
 
 
+# The up kernel has two tile widths: 256 columns (one accumulator updated in place for the second
+# expert) where d_ff allows, else 128 columns (two accumulators).  CMOE_UP_TILE=128 keeps the narrow one.
+@pytest.mark.parametrize("kw", [
+    dict(d=128, d_ff=768, E=8, G=2, r=16, k=2),      # three N tiles: a unit of three
+    dict(d=256, d_ff=1024, E=8, G=2, r=16, k=2),     # several units per row tile
+    dict(d=128, d_ff=512, E=8, G=2, r=0, k=2),       # no residuals
+    dict(d=128, d_ff=512, E=8, G=2, r=8, k=1),       # one kept expert: no second pass
+    dict(d=128, d_ff=256, E=16, G=2, r=8, k=2),      # K = 8
+], ids=["nt3", "units", "r0", "k1", "K8r8"])
+@pytest.mark.parametrize("tile", ["256", "128"])
+def test_up_kernel_tile_widths(kw, tile, monkeypatch):
+    monkeypatch.setenv("CMOE_UP_TILE", tile)
+    s = inputs.small_shape(T=1500, **kw)
+    L = inputs.make_layer(s, 21)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1
+
+
+def test_bert_with_the_narrow_up_kernel(monkeypatch):
+    monkeypatch.setenv("CMOE_UP_TILE", "128")
+    L = layer_for("bert")
+    full_check(L, L["x"], sample=512)
+
+
 # ---- shapes that take the weight-streaming path (T_max <= 128, d and d_ff multiples of 128) ---------
 @pytest.mark.parametrize("kw", [
     dict(T=1, d=128, d_ff=128, E=8, G=2, r=4, k=2),
