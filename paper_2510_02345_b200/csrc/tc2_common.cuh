@@ -75,10 +75,10 @@ inline cudaError_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, s
   return launch_chained(kern, dim3((unsigned)grid), dim3((unsigned)threads), smem, st, 2, args...);
 }
 
-// The tensor maps of the wide up kernel: x_perm and B1t as 2-D boxes of 64 halves x 128 rows, A0 / Ad
-// [rows][KE] (128-row boxes), V1f (128-row boxes), U2f (32-row boxes).
+// The tensor maps of the wide up kernel: x_perm and B1t as 3-D boxes of 64 halves x 128 rows x 2 K atoms,
+// A0 / Ad [rows][KE] (128-row boxes), V1f (128-row boxes), U2f (32-row boxes).
 struct UpWideMaps {
-  const CUtensorMap *x, *b1, *a0, *ad, *v1, *u2;
+  const CUtensorMap *x3, *b13, *a0, *ad, *v1, *u2;
 };
 
 constexpr int BN_WIDE = 256;     // columns per tile of the wide up kernel

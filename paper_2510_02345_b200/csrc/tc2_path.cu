@@ -934,7 +934,7 @@ bool make_map3(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
 
 struct Tc2State {
   CUtensorMap mX, mX3, mB13, mA0, mAd, mV1, mU2;   // up (mX: 2-D, for the t kernel and the wide up kernel)
-  CUtensorMap mB1w, mV1w;                      // wide up kernel: 128-row boxes of B1t and V1f
+  CUtensorMap mB13w, mV1w;                     // wide up kernel: 128-row boxes of B1t and V1f
   CUtensorMap mU1;                             // t
   CUtensorMap mAbar3, mB23, mAs, mV2;          // down
   int bn_down;
@@ -1027,7 +1027,7 @@ cudaError_t tc2_init(cmoe_layer* L) {
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mX3, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mB13, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
-            make_map(&ts->mB1w, L->w.B1t, G * D.d_ff, D.d, BN_WIDE / 2) &&
+            make_map3(&ts->mB13w, L->w.B1t, G * D.d_ff, D.d, BN_WIDE / 2) &&
             make_map3(&ts->mAbar3, S.abar, P, D.d_ff, BM) &&
             make_map3(&ts->mB23, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
   if (ok && D.r > 0) {
@@ -1096,12 +1096,12 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
   {
     const int pairs = ts.sm_count / 2;
-    if (ts.up_wide) { up.KC = D.d / BK; up.NT = D.d_ff / BN_WIDE; }
+    if (ts.up_wide) up.NT = D.d_ff / BN_WIDE;
     up.unit = pick_unit(up.NT, pt_bound, pairs);
     const long long total = (long long)pt_bound * (up.NT / up.unit);
     const int grid = 2 * (int)(total < pairs ? total : pairs);
     if (ts.up_wide) {
-      const UpWideMaps maps{&ts.mX, &ts.mB1w, &ts.mA0, &ts.mAd, &ts.mV1w, &ts.mU2};
+      const UpWideMaps maps{&ts.mX3, &ts.mB13w, &ts.mA0, &ts.mAd, &ts.mV1w, &ts.mU2};
       e = launch_up_wide(D.r > 0, D.k, maps, up, grid, st);
     }
     else if (D.r == 0) e = launch_up<false, 1>(ts, up, grid, st);    // without residuals k only enters through the gates

@@ -1,7 +1,7 @@
 // Up projection of the CTA-pair path on 256 x 256 tiles (d_ff a multiple of 256), sm_100a.
 //
-// What bounds the 128-column up kernel is the SM's shared-memory bandwidth: an N = 128 pair MMA reads
-// its operands at 96 B/clk while TMA refills the ring and the activation chunks cross shared memory
+// What bounds the 128-column up kernel is the SM's shared memory: an N = 128 pair MMA reads its
+// operands at 96 B/clk while TMA refills the ring and the activation chunks cross shared memory
 // twice.  A 256-column tile needs a third less shared-memory traffic per output element, but h_1 and
 // h_2 - h_1 as two fp32 accumulators of 256 columns, plus the S accumulators, do not fit the 512
 // TMEM columns.  So one accumulator serves both experts of a token (text after Eq. 7: one base
@@ -11,8 +11,11 @@
 //   P += Ad V1f^T                          (= h of the second kept expert)     -> epilogues copy P out
 //
 // The epilogue warps copy P into registers (packed fp16), hand P back at once and do GELU, the gated
-// sum abar and the activation chunks for S_j += a_j U2f^T (accumulated in TMEM over a unit of N tiles)
-// while the next tile's main loop runs.  TMEM columns: P 0..255, S_0 256..319, S_1 320..383.
+// sum abar and the A operand of  S_j += a_j U2f^T  while the next tile's main loop runs.  a_j never
+// touches shared memory: the epilogues store it (fp16 pairs) into spare TMEM columns and the S
+// products read their A operand from there, which leaves shared memory to a ring of three 64 KB
+// stages (two 64-wide K atoms each, 3-D TMA boxes) and the tile's U2f columns.
+// TMEM columns: P 0..255, S_0 256..319, S_1 320..383, a_j 384..511 (four chunks of 64 activations).
 // Warp roles: 0 and 3 TMA (alternating stages), 1 MMA, 2 S products and U2f loads, 4..19 epilogue
 // (twenty warps: warps are allocated in fours, and 96 registers per thread fit 20 but not 24).
 // Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
@@ -27,32 +30,33 @@ namespace {
 constexpr int UW_THREADS = 640;
 constexpr int UW_EPI_WARP0 = 4, UW_EPI_WARPS = 16;
 constexpr int UW_PRODUCERS = 2;
-constexpr uint32_t UW_A_BYTES = BM * BK * 2;                     // 16 KB: this CTA's 128 rows, one K atom
-constexpr uint32_t UW_B_BYTES = (BN_WIDE / 2) * BK * 2;          // 16 KB: this CTA's half of the B tile
-constexpr uint32_t UW_STAGE_BYTES = UW_A_BYTES + UW_B_BYTES;     // 32 KB
-constexpr uint32_t UW_CHUNK_BYTES = BM * BK * 2;                 // 16 KB: 128 rows x 64 activations
+constexpr int UW_KA = 2;                                         // K atoms of 64 halves per stage
+constexpr uint32_t UW_A_ATOM = BM * BK * 2;                      // 16 KB: this CTA's 128 rows, one K atom
+constexpr uint32_t UW_B_ATOM = (BN_WIDE / 2) * BK * 2;           // 16 KB: this CTA's half of the B tile
+constexpr uint32_t UW_A_BYTES = UW_KA * UW_A_ATOM;
+constexpr uint32_t UW_B_BYTES = UW_KA * UW_B_ATOM;
+constexpr uint32_t UW_STAGE_BYTES = UW_A_BYTES + UW_B_BYTES;     // 64 KB
 constexpr int UW_CHUNKS = BN_WIDE / BK;                          // activation chunks per tile and expert
 constexpr uint32_t UW_U2_PIECE = (KE / 2) * BK * 2;              //  4 KB: this CTA's 32 rows of a 64 x 64 piece of U2f
 constexpr uint32_t UW_U2_BYTES = UW_CHUNKS * UW_U2_PIECE;
-constexpr int UW_NA = 3;                                         // activation chunk slots
+constexpr uint32_t UW_TMEM_S = BN_WIDE, UW_TMEM_A = BN_WIDE + 2 * KE;   // first columns of S and of the a_j operand
 
-enum : int { W_FULL = 0, W_EMPTY = 8, W_TFULL = 16, W_T2FULL = 17, W_PDRAIN = 18, W_TEMPTY = 19, W_AFULL = 20,
-             W_AEMPTY = 24, W_U2FULL = 28, W_U2EMPTY = 29, W_SFULL = 30, W_SEMPTY = 31, W_COUNT = 32 };
+enum : int { W_FULL = 0, W_EMPTY = 4, W_TFULL = 8, W_T2FULL = 9, W_PDRAIN = 10, W_TEMPTY = 11, W_AFULL = 12,
+             W_AEMPTY = 16, W_U2FULL = 20, W_U2EMPTY = 22, W_SFULL = 24, W_SEMPTY = 25, W_COUNT = 26 };
 
 template <bool HAS_R, int KSEL>
 struct WideCfg {
-  static constexpr int STAGES = HAS_R ? 5 : 7;
-  static constexpr int NEXT = HAS_R ? KSEL : 0;            // expanded-index stages after the main loop: (A0, V1f), (Ad, V1f)
+  static constexpr int STAGES = 3;
+  static constexpr int NEXT = HAS_R ? 1 : 0;               // one expanded-index stage after the main loop: A0, Ad, V1f
   static constexpr uint32_t RING = STAGES * UW_STAGE_BYTES;
-  static constexpr uint32_t ARING = HAS_R ? UW_NA * UW_CHUNK_BYTES : 0;
-  static constexpr uint32_t U2 = HAS_R ? UW_U2_BYTES : 0;
-  static constexpr uint32_t BAR_OFF = RING + ARING + U2;
-  static constexpr size_t SMEM = 1024 + BAR_OFF + 40 * 8;
+  static constexpr uint32_t U2 = HAS_R ? 2 * UW_U2_BYTES : 0;
+  static constexpr uint32_t BAR_OFF = RING + U2;
+  static constexpr size_t SMEM = 1024 + BAR_OFF + 32 * 8;
 };
 
 template <bool HAS_R, int KSEL>
 __global__ void __launch_bounds__(UW_THREADS, 1)
-tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmB1,
+tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ CUtensorMap tmB13,
                    const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmAd,
                    const __grid_constant__ CUtensorMap tmV1, const __grid_constant__ CUtensorMap tmU2,
                    const Up2Params p) {
@@ -64,8 +68,7 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
-  const uint32_t aring = base + Cfg::RING;
-  const uint32_t u2base = aring + Cfg::ARING;
+  const uint32_t u2base = base + Cfg::RING;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + Cfg::BAR_OFF);
   const uint32_t bar0 = smem_u32(bars);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + W_COUNT);
@@ -86,9 +89,8 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     mbar_init(local(W_T2FULL), 1);
     mbar_init(local(W_PDRAIN), 2 * UW_EPI_WARPS);
     mbar_init(local(W_TEMPTY), 2 * UW_EPI_WARPS);
-    for (int a = 0; a < 4; ++a) { mbar_init(local(W_AFULL + a), 2 * UW_EPI_WARPS); mbar_init(local(W_AEMPTY + a), 1); }
-    mbar_init(local(W_U2FULL), 1);
-    mbar_init(local(W_U2EMPTY), 1);
+    for (int a = 0; a < UW_CHUNKS; ++a) { mbar_init(local(W_AFULL + a), 2 * UW_EPI_WARPS); mbar_init(local(W_AEMPTY + a), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(local(W_U2FULL + a), 1); mbar_init(local(W_U2EMPTY + a), 1); }
     mbar_init(local(W_SFULL), 1);
     mbar_init(local(W_SEMPTY), UW_EPI_WARPS * KSEL);
     *abort_flag = 0;
@@ -105,7 +107,7 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   cluster_sync_all();          // both CTAs' barriers are initialised before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
-  const uint32_t tmem_s = tmem_base + BN_WIDE;
+  const uint32_t tmem_s = tmem_base + UW_TMEM_S, tmem_a = tmem_base + UW_TMEM_A;
 
   const int NT = p.NT, KC = p.KC;
   // Work units of `unit` consecutive N tiles of one 256-row tile, dealt round-robin to the CTA pairs:
@@ -126,28 +128,37 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     // ---------------- TMA producers (both CTAs, two threads taking alternate stages): this CTA's rows
     // of A and its half of B; the bytes of both CTAs are counted on the leader's barrier
     if (lane == 0) {
-      const uint32_t pid = warp == 0 ? 0u : 1u;
+      // Global stage number it = w * spt + c; this thread takes it = pid, pid + 2, ...  Tile coordinates
+      // are worked out once per tile and the ring slot advances by two: integer divisions in this loop
+      // would cost the single issuing thread more than the loads themselves.
+      const int pid = warp == 0 ? 0 : 1;
       const int spt = KC + Cfg::NEXT;                   // stages per tile
-      const uint32_t n_it = (uint32_t)w1 * spt;
-      for (uint32_t it = pid; it < n_it && !failed; it += UW_PRODUCERS) {
-        const int w = it / spt, c = it - w * spt;
+      uint32_t s = (uint32_t)pid, ph = 0;
+      int c = pid;
+      for (int w = 0; w < w1 && !failed; ++w) {
         int pt, nt;
         tile_of(w, pt, nt);
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
         const int brow = g * p.N + nt * BN_WIDE + (int)rank * (BN_WIDE / 2);
-        const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-        if (!mbar_wait_cluster(local(W_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
-        const uint32_t a_dst = base + s * UW_STAGE_BYTES, b_dst = a_dst + UW_A_BYTES;
-        if (leader) mbar_expect_tx(local(W_FULL + s), 2 * UW_STAGE_BYTES);
-        if (c < KC) {
-          tma2_load_2d(a_dst, &tmX, lead(W_FULL + s), c * BK, arow);
-          tma2_load_2d(b_dst, &tmB1, lead(W_FULL + s), c * BK, brow);
-        } else {
-          // expanded-index stages: (A0, V1f) completes h of the first expert, (Ad, V1f) turns it into the second's
-          tma2_load_2d(a_dst, c == KC ? &tmA0 : &tmAd, lead(W_FULL + s), 0, arow);
-          tma2_load_2d(b_dst, &tmV1, lead(W_FULL + s), 0, brow);
+        for (; c < spt; c += UW_PRODUCERS) {
+          if (!mbar_wait_cluster(local(W_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
+          const uint32_t a_dst = base + s * UW_STAGE_BYTES, b_dst = a_dst + UW_A_BYTES;
+          if (c < KC) {
+            if (leader) mbar_expect_tx(local(W_FULL + s), 2 * UW_STAGE_BYTES);
+            tma2_load_3d(a_dst, &tmX3, lead(W_FULL + s), 0, arow, c * UW_KA);
+            tma2_load_3d(b_dst, &tmB13, lead(W_FULL + s), 0, brow, c * UW_KA);
+          } else {
+            // expanded-index stage: A0 (completes h of the first expert), Ad (turns it into the second's), V1f
+            if (leader) mbar_expect_tx(local(W_FULL + s), 2 * (KSEL * UW_A_ATOM + UW_B_ATOM));
+            tma2_load_2d(a_dst, &tmA0, lead(W_FULL + s), 0, arow);
+            if (KSEL == 2) tma2_load_2d(a_dst + UW_A_ATOM, &tmAd, lead(W_FULL + s), 0, arow);
+            tma2_load_2d(b_dst, &tmV1, lead(W_FULL + s), 0, brow);
+          }
+          s += UW_PRODUCERS;
+          if (s >= (uint32_t)STAGES) { s -= STAGES; ph ^= 1u; }
         }
+        c -= spt;
       }
     }
   } else if (warp == 1) {
@@ -170,9 +181,13 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           tc_fence_after();
           const uint32_t a_src = base + s * UW_STAGE_BYTES, b_src = a_src + UW_A_BYTES;
           const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+          // the second atom's tiles follow the first's: descriptor addresses are in 16-byte units
           umma2_f16(tmem_base, adesc, bdesc, IDESC, c != 0 ? 1u : 0u);
 #pragma unroll
           for (int ks = 1; ks < BK / 16; ++ks) umma2_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+#pragma unroll
+          for (int ks = 0; ks < BK / 16; ++ks)
+            umma2_f16(tmem_base, adesc + (UW_A_ATOM >> 4) + 2 * ks, bdesc + (UW_B_ATOM >> 4) + 2 * ks, IDESC, 1u);
           commit_both(W_EMPTY + s);
           next_stage();
         }
@@ -180,31 +195,24 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         if (HAS_R) {
           if (!mbar_wait_cluster(local(W_FULL + s), ph, abort_flag)) { failed = true; break; }
           tc_fence_after();
-          {
-            const uint32_t a_src = base + s * UW_STAGE_BYTES, b_src = a_src + UW_A_BYTES;
-            const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
+          const uint32_t a_src = base + s * UW_STAGE_BYTES, b_src = a_src + UW_A_BYTES;
+          const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
 #pragma unroll
-            for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m0 >> ks) & 1) umma2_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
-          }
+          for (int ks = 0; ks < KE / 16; ++ks)
+            if ((m0 >> ks) & 1) umma2_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
           commit_both(W_TFULL);        // P = h of the first expert
-          commit_both(W_EMPTY + s);
-          next_stage();
           if (KSEL == 2) {
-            if (!mbar_wait_cluster(local(W_FULL + s), ph, abort_flag)) { failed = true; break; }
             // P is updated in place: both CTAs' epilogues must have copied h of the first expert out
             if (!mbar_wait_cluster(local(W_PDRAIN), tph, abort_flag)) { failed = true; break; }
             tc_fence_after();
-            const uint32_t a_src = base + s * UW_STAGE_BYTES, b_src = a_src + UW_A_BYTES;
-            const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
             const int m = m0 | m1;
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
-              if ((m >> ks) & 1) umma2_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
+              if ((m >> ks) & 1) umma2_f16(tmem_base, adesc + (UW_A_ATOM >> 4) + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
             commit_both(W_T2FULL);     // P = h of the second expert
-            commit_both(W_EMPTY + s);
-            next_stage();
           }
+          commit_both(W_EMPTY + s);
+          next_stage();
         } else {
           commit_both(W_TFULL);
         }
@@ -218,20 +226,25 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       uint32_t flushes = 0;
       bool fresh = true;                    // the next product of each slot overwrites S
       uint32_t written = 0;                 // bit j: S_j has been written since the last flush
-      for (int w = 0; w < w1 && !failed; ++w) {
-        {
-          int pt, nt;
-          tile_of(w, pt, nt);
-          const int g = p.tile_cluster[pt];
-          // one buffer: the S products of the previous tile have read it
-          if (!mbar_wait_cluster(local(W_U2EMPTY), ((uint32_t)w & 1u) ^ 1u, abort_flag)) { failed = true; break; }
-          if (leader) mbar_expect_tx(local(W_U2FULL), 2 * UW_U2_BYTES);
+      auto load_u2 = [&](int w) -> bool {
+        int pt, nt;
+        tile_of(w, pt, nt);
+        const int g = p.tile_cluster[pt];
+        const uint32_t ub = (uint32_t)w & 1u, uph = ((uint32_t)w >> 1) & 1u;
+        if (!mbar_wait_cluster(local(W_U2EMPTY + ub), uph ^ 1u, abort_flag)) return false;
+        if (leader) mbar_expect_tx(local(W_U2FULL + ub), 2 * UW_U2_BYTES);
 #pragma unroll
-          for (int m = 0; m < UW_CHUNKS; ++m)
-            tma2_load_2d(u2base + m * UW_U2_PIECE, &tmU2, lead(W_U2FULL), nt * BN_WIDE + m * BK, g * KE + (int)rank * (KE / 2));
-        }
+        for (int m = 0; m < UW_CHUNKS; ++m)
+          tma2_load_2d(u2base + ub * UW_U2_BYTES + m * UW_U2_PIECE, &tmU2, lead(W_U2FULL + ub), nt * BN_WIDE + m * BK,
+                       g * KE + (int)rank * (KE / 2));
+        return true;
+      };
+      if (!load_u2(0)) failed = true;
+      for (int w = 0; w < w1 && !failed; ++w) {
+        if (w + 1 < w1 && !load_u2(w + 1)) { failed = true; break; }
         if (!leader) continue;
-        if (!mbar_wait_cluster(local(W_U2FULL), (uint32_t)w & 1u, abort_flag)) { failed = true; break; }
+        const uint32_t ub = (uint32_t)w & 1u, uph = ((uint32_t)w >> 1) & 1u;
+        if (!mbar_wait_cluster(local(W_U2FULL + ub), uph, abort_flag)) { failed = true; break; }
         if (fresh && flushes > 0) {
           // both epilogues must have read the previous unit's S before it is overwritten
           if (!mbar_wait_cluster(local(W_SEMPTY), (flushes - 1) & 1u, abort_flag)) { failed = true; break; }
@@ -239,22 +252,21 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
         if (fresh) { written = 0; fresh = false; }
         for (int c = 0; c < UW_CHUNKS * KSEL; ++c) {
-          const uint32_t n = (uint32_t)w * (UW_CHUNKS * KSEL) + c;
-          const uint32_t slot = n % UW_NA, aph = (n / UW_NA) & 1u;
-          if (!mbar_wait_cluster(local(W_AFULL + slot), aph, abort_flag)) { failed = true; break; }
-          tc_fence_after();
           const int j = c / UW_CHUNKS, m = c % UW_CHUNKS;
-          const uint64_t adesc = umma_desc(aring + slot * UW_CHUNK_BYTES);
-          const uint64_t bdesc = umma_desc(u2base + m * UW_U2_PIECE);
+          const uint32_t use = (uint32_t)w * KSEL + j;          // how often chunk slot m has been filled before
+          if (!mbar_wait_cluster(local(W_AFULL + m), use & 1u, abort_flag)) { failed = true; break; }
+          tc_fence_after();
+          const uint64_t bdesc = umma_desc(u2base + ub * UW_U2_BYTES + m * UW_U2_PIECE);
 #pragma unroll
           for (int ks = 0; ks < BK / 16; ++ks) {
-            umma2_f16(tmem_s + j * KE, adesc + 2 * ks, bdesc + 2 * ks, IDESC_S, (written >> j) & 1u);
+            // A from tensor memory: 32 columns per chunk, 8 per 16-deep step
+            umma2_f16_ts(tmem_s + j * KE, tmem_a + m * (BK / 2) + ks * 8, bdesc + 2 * ks, IDESC_S, (written >> j) & 1u);
             written |= 1u << j;
           }
-          commit_both(W_AEMPTY + slot);
+          commit_both(W_AEMPTY + m);
         }
         if (failed) break;
-        commit_both(W_U2EMPTY);
+        commit_both(W_U2EMPTY + ub);
         if ((w + 1) % unit == 0) { commit_both(W_SFULL); fresh = true; ++flushes; }
       }
     }
@@ -311,23 +323,19 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster_relaxed(lead(W_TEMPTY));
 
-      // a_j chunk m into its slot as a K-major 128-byte-swizzled A operand: 16-byte unit u of row rowc sits
-      // at rowc*128 + ((u ^ (rowc & 7)) << 4); this warp owns units 2 cq, 2 cq + 1
+      // a_j chunk m as the A operand of the S product: this thread's 16 activations (columns 64 m + 16 cq ..)
+      // go into 8 columns of its TMEM lane as fp16 pairs
       auto hand_over = [&](int j, int m, const uint32_t* src) -> bool {
-        const uint32_t n = (uint32_t)w * (UW_CHUNKS * KSEL) + j * UW_CHUNKS + m;
-        const uint32_t slot = n % UW_NA;
-        // the S product that read this slot three chunks ago has finished
-        const bool ok = mbar_wait_cluster(local(W_AEMPTY + slot), ((n / UW_NA) & 1u) ^ 1u, abort_flag);
+        const uint32_t use = (uint32_t)w * KSEL + j;
+        // the S product that read this chunk's columns one expert ago has finished
+        const bool ok = mbar_wait_cluster(local(W_AEMPTY + m), (use & 1u) ^ 1u, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) return false;
-        const uint32_t cb = aring + slot * UW_CHUNK_BYTES + rowc * 128;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          const uint32_t un = (uint32_t)(cq * 2 + i);
-          st_shared_v4(cb + ((un ^ (uint32_t)(rowc & 7)) << 4), src[4 * i], src[4 * i + 1], src[4 * i + 2], src[4 * i + 3]);
-        }
-        fence_async_smem();
+        tc_fence_after();
+        tmem_st8(taddr + UW_TMEM_A + m * (BK / 2) + cq * 8, src);
+        tmem_st_wait();
+        tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_cluster_relaxed(lead(W_AFULL + slot));   // after fence.proxy.async
+        if (lane == 0) mbar_arrive_cluster_relaxed(lead(W_AFULL + m));
         return true;
       };
       // first expert: a_1 = GELU(h_1), its share of abar (kept in h1), its chunks of the S operand
@@ -376,7 +384,7 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           float* srow = p.s_out + ((size_t)row * KSEL + j) * p.r;
           const int r = p.r;
           for (int i = cq & 1; i < p.K; i += 2) {
-            const uint32_t ta = taddr + BN_WIDE + j * KE + i * r;
+            const uint32_t ta = taddr + UW_TMEM_S + j * KE + i * r;
             const bool mine = real && e == i;
             if (r == 16) {
               uint32_t v[16];
@@ -448,7 +456,7 @@ cudaError_t launch_w(const UpWideMaps& m, const Up2Params& p, int grid, cudaStre
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  return launch_pairs(kern, grid, UW_THREADS, sm, st, *m.x, *m.b1, *m.a0, *m.ad, *m.v1, *m.u2, p);
+  return launch_pairs(kern, grid, UW_THREADS, sm, st, *m.x3, *m.b13, *m.a0, *m.ad, *m.v1, *m.u2, p);
 }
 
 }  // namespace
