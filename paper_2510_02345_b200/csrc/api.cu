@@ -179,6 +179,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   L->profiling = 0;
   L->events_created = 0;
   L->events_recorded = 0;
+  L->side_created = 0;
   L->n_stages = 5;
   L->stage_names[0] = "router";
   L->stage_names[1] = "permute";
@@ -193,10 +194,16 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   const Weights& W = L->w;
   const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r;
   auto fail = [&](cudaError_t) {
-    delete L;
+    cmoe_destroy(L);
     return CMOE_ERR_CUDA;
   };
   cudaError_t e;
+  if ((e = cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking))) return fail(e);
+  L->side_created = 1;
+  if ((e = cudaEventCreateWithFlags(&L->side_fork, cudaEventDisableTiming))) return fail(e);
+  L->side_created = 2;
+  if ((e = cudaEventCreateWithFlags(&L->side_join, cudaEventDisableTiming))) return fail(e);
+  L->side_created = 3;
   // router: C [d][G] -> Ct [G][d];  R [G][d][K] -> Rt [G][K][d]
   if ((e = launch_transpose_f32(desc->C, const_cast<float*>(W.Ct), 1, D.d, D.G, st))) return fail(e);
   if ((e = launch_transpose_f32(desc->R, const_cast<float*>(W.Rt), D.G, D.d, D.K, st))) return fail(e);
@@ -210,7 +217,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
     e = cudaMemcpyAsync(const_cast<int*>(W.label), desc->expert_global_id, E * 4, cudaMemcpyDeviceToDevice, st);
   } else {
     int* ids = new (std::nothrow) int[E];
-    if (!ids) { delete L; return CMOE_ERR_INVALID_ARG; }
+    if (!ids) { cmoe_destroy(L); return CMOE_ERR_INVALID_ARG; }
     for (size_t i = 0; i < E; ++i) ids[i] = (int)i;
     e = cudaMemcpy(const_cast<int*>(W.label), ids, E * 4, cudaMemcpyHostToDevice);
     delete[] ids;
@@ -377,6 +384,9 @@ int cmoe_destroy(cmoe_layer* L) {
   if (!L) return CMOE_ERR_INVALID_ARG;
   if (L->events_created)
     for (int i = 0; i <= CMOE_MAX_STAGES; ++i) cudaEventDestroy(L->events[i]);
+  if (L->side_created >= 3) cudaEventDestroy(L->side_join);
+  if (L->side_created >= 2) cudaEventDestroy(L->side_fork);
+  if (L->side_created >= 1) { cudaStreamSynchronize(L->side_stream); cudaStreamDestroy(L->side_stream); }
   delete L;
   return CMOE_OK;
 }

@@ -99,6 +99,11 @@ struct cmoe_layer {
   cudaEvent_t events[CMOE_MAX_STAGES + 1];
   int events_created;
   int events_recorded;
+  // a second stream for work that does not depend on the kernel running on the caller's stream (forked and
+  // joined with the two events inside one forward); created with the handle, never allocated per call
+  cudaStream_t side_stream;
+  cudaEvent_t side_fork, side_join;
+  int side_created;
   // tensor-core path: tensor maps and launch shapes (opaque here, see tc_path.cu)
   alignas(128) unsigned char tc_state[2048];
 };

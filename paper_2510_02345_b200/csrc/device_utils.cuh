@@ -17,6 +17,16 @@ __device__ __forceinline__ float deq4(const uint8_t* __restrict__ q, const __hal
   return (float)code * __half2float(s[flat >> 5]);
 }
 
+// The eight codes of a 32-bit word of a packed INT4 factor as floats, without integer-to-float
+// conversions: (nibble ^ 8) = code + 8 is placed in the mantissa of 2^23, then 2^23 + 8 is subtracted.
+__device__ __forceinline__ void int4x8_to_float(uint32_t word, float* out) {
+#pragma unroll
+  for (int n = 0; n < 8; ++n) {
+    const uint32_t bits = ((word >> (4 * n)) & 0xFu) ^ 0x4B000008u;
+    out[n] = __uint_as_float(bits) - 8388616.0f;
+  }
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

@@ -236,6 +236,14 @@ router_token_kernel(const RouterArgs a) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int t = blockIdx.x, d = a.d;
   const __half* xr = a.x + (size_t)t * d;
+  {
+    // the second pass reads the expert rows of a cluster that is not known yet: bring all of them into
+    // L2 while the cluster logits are computed (every thread of the grid asks for one 128-byte line at a time)
+    const size_t bytes = (size_t)a.G * a.K * d * sizeof(float);
+    const size_t step = (size_t)gridDim.x * blockDim.x * 128;
+    for (size_t off = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 128; off < bytes; off += step)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(a.Rt) + off));
+  }
   for (int pass = 0; pass < 2; ++pass) {
     const int n = pass == 0 ? a.G : a.K;
     const float* W = pass == 0 ? a.Ct : a.Rt + (size_t)s_g * a.K * d;
@@ -243,7 +251,7 @@ router_token_kernel(const RouterArgs a) {
     for (int j = warp; j < n; j += nwarp) {
       const float* wr = W + (size_t)j * d;
       float acc = 0.f;
-#pragma unroll 4
+#pragma unroll 8
       for (int c = lane * 8; c < d; c += 256)
         fma8(acc, *reinterpret_cast<const uint4*>(xr + c), __ldg(reinterpret_cast<const float4*>(wr + c)),
              __ldg(reinterpret_cast<const float4*>(wr + c + 4)));

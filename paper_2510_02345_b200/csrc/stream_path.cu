@@ -255,16 +255,17 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
                   if (r >= 8) {
                     const uint32_t* wq = reinterpret_cast<const uint32_t*>(p.V1q + (flat >> 1));
                     for (int w8 = 0; w8 < r / 8; ++w8) {
-                      const uint32_t word = wq[w8];
+                      float cf[8];
+                      int4x8_to_float(wq[w8], cf);
                       const float4 ta = tp[2 * w8], tb4 = tp[2 * w8 + 1];
-                      dot0 = fmaf(ta.x, (float)sext4((int)word), dot0);
-                      dot1 = fmaf(ta.y, (float)sext4((int)(word >> 4)), dot1);
-                      dot0 = fmaf(ta.z, (float)sext4((int)(word >> 8)), dot0);
-                      dot1 = fmaf(ta.w, (float)sext4((int)(word >> 12)), dot1);
-                      dot0 = fmaf(tb4.x, (float)sext4((int)(word >> 16)), dot0);
-                      dot1 = fmaf(tb4.y, (float)sext4((int)(word >> 20)), dot1);
-                      dot0 = fmaf(tb4.z, (float)sext4((int)(word >> 24)), dot0);
-                      dot1 = fmaf(tb4.w, (float)sext4((int)(word >> 28)), dot1);
+                      dot0 = fmaf(ta.x, cf[0], dot0);
+                      dot1 = fmaf(ta.y, cf[1], dot1);
+                      dot0 = fmaf(ta.z, cf[2], dot0);
+                      dot1 = fmaf(ta.w, cf[3], dot1);
+                      dot0 = fmaf(tb4.x, cf[4], dot0);
+                      dot1 = fmaf(tb4.y, cf[5], dot1);
+                      dot0 = fmaf(tb4.z, cf[6], dot0);
+                      dot1 = fmaf(tb4.w, cf[7], dot1);
                     }
                   } else {
                     const uint32_t word = *reinterpret_cast<const uint16_t*>(p.V1q + (flat >> 1));
@@ -314,11 +315,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
 // activation of that row and slot).  A block per (item, eight rank indices), a warp per rank index,
 // lanes over the 32-element scale groups.
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
-               const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
-               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
-  pdl_wait();
+__device__ __forceinline__ void
+lowrank_body(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
+             const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
+             const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
   const int item = blockIdx.x;
   const int row = item / k;
   if (row >= seg_off[G] || row_token[row] < 0) {
@@ -328,27 +328,62 @@ lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, in
   const int e = row_slot[item];
   const __half* xin = in + (size_t)(in_per_slot ? item : row) * len;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  {
+    // all code lines of this block's first rank rows are requested at once (into L2): the loop below then
+    // meets DRAM latency once, not once per unrolled batch
+    const int lines = len >> 8;                                   // 128-byte lines of one rank row (len / 2 bytes)
+    const int pr0 = blockIdx.y * nwarp, nr = min(nwarp, r - pr0);
+    for (int i = threadIdx.x; i < nr * lines; i += blockDim.x) {
+      const int rr = i / lines, l = i - rr * lines;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(Uq + ((((long long)e * r + pr0 + rr) * len) >> 1) + (size_t)l * 128));
+    }
+  }
   for (int pr = blockIdx.y * nwarp + warp; pr < r; pr += gridDim.y * nwarp) {
     const long long base = ((long long)e * r + pr) * len;
     float acc = 0.f;
-#pragma unroll 4
+#pragma unroll 8
     for (int grp = lane; grp * 32 < len; grp += 32) {
-      const uint4 pk = *reinterpret_cast<const uint4*>(Uq + ((base + grp * 32) >> 1));
+      const uint4 pk = __ldg(reinterpret_cast<const uint4*>(Uq + ((base + grp * 32) >> 1)));
       const float sc = __half2float(Us[(base >> 5) + grp]);
       const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
       float part = 0.f;
 #pragma unroll
       for (int qd = 0; qd < 4; ++qd) {
         const uint4 xv = *reinterpret_cast<const uint4*>(xin + grp * 32 + qd * 8);
-        const __half* xh = reinterpret_cast<const __half*>(&xv);
+        const __half2* xh = reinterpret_cast<const __half2*>(&xv);
+        float cf[8];
+        int4x8_to_float(w[qd], cf);
 #pragma unroll
-        for (int n = 0; n < 8; ++n) part = fmaf(__half2float(xh[n]), (float)sext4((int)(w[qd] >> (4 * n))), part);
+        for (int n = 0; n < 4; ++n) {
+          const float2 xf = __half22float2(xh[n]);
+          part = fmaf(xf.x, cf[2 * n], part);
+          part = fmaf(xf.y, cf[2 * n + 1], part);
+        }
       }
       acc = fmaf(part, sc, acc);
     }
     acc = warp_sum(acc);
     if (lane == 0) out[(size_t)item * r + pr] = acc;
   }
+}
+
+__global__ void __launch_bounds__(256)
+lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
+               const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
+               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+  pdl_wait();
+  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out);
+}
+
+// The same for the second stream: s = a_j U2 is not needed before the last kernel of the forward, so it
+// runs beside the down kernel.  That kernel holds 640 threads x 96 registers of every SM; four warps of
+// 32 registers are what fits next to it.
+constexpr int kSideThreads = 128;
+__global__ void __launch_bounds__(kSideThreads, 16)
+lowrank_side_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
+                    const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
+                    const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out);
 }
 
 // y[tok] = fp16(y32[row] + sum_j p_j s_j V2_e), one thread per (row, output column)
@@ -372,9 +407,10 @@ stream_final_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r,
     if (r >= 8) {
       const uint32_t* wq = reinterpret_cast<const uint32_t*>(V2q + (flat >> 1));
       for (int w8 = 0; w8 < r / 8; ++w8) {
-        const uint32_t word = wq[w8];
+        float cf[8];
+        int4x8_to_float(wq[w8], cf);
 #pragma unroll
-        for (int n = 0; n < 8; ++n) u = fmaf(sj[w8 * 8 + n], (float)sext4((int)(word >> (4 * n))), u);
+        for (int n = 0; n < 8; ++n) u = fmaf(sj[w8 * 8 + n], cf[n], u);
       }
     } else {
       const uint32_t word = *reinterpret_cast<const uint16_t*>(V2q + (flat >> 1));
@@ -511,10 +547,14 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
-    launch_chained(lowrank_kernel, dim3(rows_bound * D.k, (D.r + 7) / 8), dim3(256), 0, st, 1,
-      S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token,
-                                                      W.U2q, W.U2s, S.s);
+    // fork: s = a_j U2 on the second stream, beside the down kernel
+    if ((e = cudaEventRecord(L->side_fork, st)) != cudaSuccess) return e;
+    if ((e = cudaStreamWaitEvent(L->side_stream, L->side_fork, 0)) != cudaSuccess) return e;
+    const int nwarp = kSideThreads / 32;
+    lowrank_side_kernel<<<dim3(rows_bound * D.k, (D.r + nwarp - 1) / nwarp), kSideThreads, 0, L->side_stream>>>(
+        S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token, W.U2q, W.U2s, S.s);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    if ((e = cudaEventRecord(L->side_join, L->side_stream)) != cudaSuccess) return e;
   }
   {
     p.Kd = D.d_ff; p.M = D.d; p.ksplit = ts.ksplit;
@@ -522,6 +562,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
     if ((e = launch_stream<false>(ts.mW2, ts.mW1s, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
   }
+  if (D.r > 0 && (e = cudaStreamWaitEvent(st, L->side_join, 0)) != cudaSuccess) return e;     // join
   dim3 fgrid((D.d + 255) / 256, rows_bound);
   launch_chained(stream_final_kernel, dim3(fgrid), dim3(256), 0, st, 1,
       S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
