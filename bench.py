@@ -65,12 +65,14 @@ def stage_work(s, T, stage, active_clusters, active_experts):
 # profiles/ (ncu_gpt2m_tc2_up_down.md, ncu_decode_stream_kernels.md).  The figure is reported only while
 # the kernel sources still have the hash they had at the capture; otherwise "traffic" is null.
 NCU_TRAFFIC = {
-    "gpt2m": {"kernel": "tc2_up_kernel<true,2>", "bytes": 119.380224e6 + 110.086912e6,
-              "sha1": {"tc2_path.cu": "a154d2d232a34cc56ed2e340e6b9af1bc977cfb0",
-                       "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.955200e6 + 9.806848e6,
-               "sha1": {"stream_path.cu": "003cd0de2d54c2059eaa9e7293f25ee4a5ff228d",
-                        "tc_ptx.cuh": "2504442bd80e2e40823dea4fe4299f5d74828528"}},
+    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 135.077120e6 + 110.778368e6,
+              "sha1": {"tc2_up_wide.cu": "0c87ccd7c6e1febe2600e6127b7f11e1eabf767e",
+                       "tc2_common.cuh": "128b12ba3262a9f686454456ca8a42dc3317a939",
+                       "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.946240e6 + 12.473856e6,
+               "sha1": {"stream_path.cu": "2eaf278dd3a1acaeae12cdb44d68bd323491fcd4",
+                        "device_utils.cuh": "daa6a5fc90a4b02a5c17177e8d154044cca709c4",
+                        "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
 }
 
 
