@@ -105,6 +105,17 @@ int cmoe_route(cmoe_layer* layer, const void* x, int32_t T,
  * point atomics, so y is reproducible only up to fp32 summation order. */
 int cmoe_forward(cmoe_layer* layer, const void* x, int32_t T, void* y, void* cuda_stream);
 
+/* The same for HOST buffers: y_host = fp16 [T][d] for x_host = fp16 [T][d] (both host pointers; page-locked
+ * memory makes the copies asynchronous and lets them overlap, pageable memory works but serialises).
+ * x_stage and y_stage are caller-owned DEVICE buffers of T*d fp16 values each (16-byte aligned) that the
+ * call uses as staging.  Tokens are independent (Eq. 9-10 act per token), so the batch is cut into up to
+ * four chunks of at least 2048 tokens and pipelined: chunk c+1 is copied to the device and chunk c-1 back
+ * to the host on two streams owned by the handle while chunk c is computed on the caller's stream.  The
+ * call is asynchronous: when the work queued on cuda_stream has finished, y_host is complete and x_host
+ * may be reused.  0 <= T <= T_max. */
+int cmoe_forward_host(cmoe_layer* layer, const void* x_host, int32_t T, void* y_host,
+                      void* x_stage, void* y_stage, void* cuda_stream);
+
 /* Waits for the stream and returns the device status word of the handle: CMOE_OK, or
  * CMOE_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the output of that call is then
  * undefined; the handle stays usable and the word is cleared). */

@@ -20,7 +20,7 @@ ERRORS = {
     -1: "CMOE_ERR_INVALID_ARG", -2: "CMOE_ERR_UNSUPPORTED_SHAPE", -3: "CMOE_ERR_WORKSPACE_TOO_SMALL",
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
-EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_status",
+EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
            "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
 CMOE_MAX_STAGES = 8
@@ -60,6 +60,7 @@ def lib():
         L.cmoe_create.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_void_p)]
         L.cmoe_route.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.cmoe_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.cmoe_forward_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.cmoe_status.argtypes = [C.c_void_p, C.c_void_p]
         L.cmoe_get_info.argtypes = [C.c_void_p, C.POINTER(cmoe_info)]
         L.cmoe_last_cuda_error.argtypes = [C.c_void_p]
@@ -106,6 +107,10 @@ def cmoe_route(handle, x_ptr: int, T: int, cluster_id_ptr: int, expert_ids_ptr: 
 
 def cmoe_forward(handle, x_ptr: int, T: int, y_ptr: int, stream: int):
     _check(lib().cmoe_forward(handle, x_ptr, T, y_ptr, stream), "cmoe_forward")
+
+
+def cmoe_forward_host(handle, x_host_ptr: int, T: int, y_host_ptr: int, x_stage_ptr: int, y_stage_ptr: int, stream: int):
+    _check(lib().cmoe_forward_host(handle, x_host_ptr, T, y_host_ptr, x_stage_ptr, y_stage_ptr, stream), "cmoe_forward_host")
 
 
 def cmoe_status(handle, stream: int) -> int:
@@ -207,6 +212,20 @@ class ClusteredMoELayer:
         assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.shape[1] == self.shape.d
         y = out if out is not None else torch.empty_like(x)
         cmoe_forward(self.handle, x.data_ptr(), T, y.data_ptr(), self._stream())
+        return y
+
+    def forward_host(self, x_host, out_host=None):
+        """Host tensors in and out (pinned memory lets the copies overlap the kernels); asynchronous on the
+        current stream like forward().  The device staging buffers are kept by the module."""
+        import torch
+        T = x_host.shape[0]
+        assert (not x_host.is_cuda) and x_host.dtype == torch.float16 and x_host.is_contiguous() and x_host.shape[1] == self.shape.d
+        y = out_host if out_host is not None else torch.empty_like(x_host)
+        if getattr(self, "_stage", None) is None or self._stage[0].shape[0] < T:
+            self._stage = (torch.empty((max(T, 1), self.shape.d), dtype=torch.float16, device=self.device),
+                           torch.empty((max(T, 1), self.shape.d), dtype=torch.float16, device=self.device))
+        cmoe_forward_host(self.handle, x_host.data_ptr(), T, y.data_ptr(), self._stage[0].data_ptr(),
+                          self._stage[1].data_ptr(), self._stream())
         return y
 
     def status(self) -> int:

@@ -180,6 +180,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   L->events_created = 0;
   L->events_recorded = 0;
   L->side_created = 0;
+  L->host_created = 0;
   L->n_stages = 5;
   L->stage_names[0] = "router";
   L->stage_names[1] = "permute";
@@ -204,6 +205,21 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   L->side_created = 2;
   if ((e = cudaEventCreateWithFlags(&L->side_join, cudaEventDisableTiming))) return fail(e);
   L->side_created = 3;
+  if ((e = cudaStreamCreateWithFlags(&L->h2d_stream, cudaStreamNonBlocking))) return fail(e);
+  L->host_created = 1;
+  if ((e = cudaStreamCreateWithFlags(&L->d2h_stream, cudaStreamNonBlocking))) return fail(e);
+  L->host_created = 2;
+  {
+    cudaEvent_t* ev[2 + 2 * kMaxHostChunks];
+    int n = 0;
+    ev[n++] = &L->host_fork; ev[n++] = &L->host_join;
+    for (int c = 0; c < kMaxHostChunks; ++c) ev[n++] = &L->chunk_in[c];
+    for (int c = 0; c < kMaxHostChunks; ++c) ev[n++] = &L->chunk_done[c];
+    for (int i = 0; i < n; ++i) {
+      if ((e = cudaEventCreateWithFlags(ev[i], cudaEventDisableTiming))) return fail(e);
+      L->host_created = 3 + i;
+    }
+  }
   // router: C [d][G] -> Ct [G][d];  R [G][d][K] -> Rt [G][K][d]
   if ((e = launch_transpose_f32(desc->C, const_cast<float*>(W.Ct), 1, D.d, D.G, st))) return fail(e);
   if ((e = launch_transpose_f32(desc->R, const_cast<float*>(W.Rt), D.G, D.d, D.K, st))) return fail(e);
@@ -322,6 +338,48 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   return CMOE_OK;
 }
 
+int cmoe_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* y_host,
+                      void* x_stage, void* y_stage, void* cuda_stream) {
+  if (!L) return CMOE_ERR_INVALID_ARG;
+  if (T < 0) return CMOE_ERR_INVALID_ARG;
+  if (T > L->dims.T_max) return CMOE_ERR_T_EXCEEDS_MAX;
+  if (T == 0) return CMOE_OK;
+  if (!x_host || !y_host || !x_stage || !y_stage || !aligned16(x_stage) || !aligned16(y_stage)) return CMOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t row = sizeof(__half) * (size_t)L->dims.d;
+  // chunks of at least 2048 tokens, multiples of 256, at most kMaxHostChunks of them
+  int n_chunks = T / 2048;
+  if (n_chunks < 1) n_chunks = 1;
+  if (n_chunks > kMaxHostChunks) n_chunks = kMaxHostChunks;
+  const int per = ((T + n_chunks - 1) / n_chunks + 255) / 256 * 256;
+  // the copy streams start after what is already queued on the caller's stream (it may still use the buffers)
+  CMOE_CUDA(L, cudaEventRecord(L->host_fork, st));
+  CMOE_CUDA(L, cudaStreamWaitEvent(L->h2d_stream, L->host_fork, 0));
+  CMOE_CUDA(L, cudaStreamWaitEvent(L->d2h_stream, L->host_fork, 0));
+  int n = 0;
+  for (int t0 = 0; t0 < T; t0 += per, ++n) {
+    const int tc = T - t0 < per ? T - t0 : per;
+    CMOE_CUDA(L, cudaMemcpyAsync(static_cast<char*>(x_stage) + row * t0, static_cast<const char*>(x_host) + row * t0,
+                                 row * tc, cudaMemcpyHostToDevice, L->h2d_stream));
+    CMOE_CUDA(L, cudaEventRecord(L->chunk_in[n], L->h2d_stream));
+  }
+  n = 0;
+  for (int t0 = 0; t0 < T; t0 += per, ++n) {
+    const int tc = T - t0 < per ? T - t0 : per;
+    CMOE_CUDA(L, cudaStreamWaitEvent(st, L->chunk_in[n], 0));
+    const int rc = cmoe_forward(L, static_cast<char*>(x_stage) + row * t0, tc, static_cast<char*>(y_stage) + row * t0, st);
+    if (rc != CMOE_OK) return rc;
+    CMOE_CUDA(L, cudaEventRecord(L->chunk_done[n], st));
+    CMOE_CUDA(L, cudaStreamWaitEvent(L->d2h_stream, L->chunk_done[n], 0));
+    CMOE_CUDA(L, cudaMemcpyAsync(static_cast<char*>(y_host) + row * t0, static_cast<char*>(y_stage) + row * t0,
+                                 row * tc, cudaMemcpyDeviceToHost, L->d2h_stream));
+  }
+  // join: the caller's stream ends after the last copy back
+  CMOE_CUDA(L, cudaEventRecord(L->host_join, L->d2h_stream));
+  CMOE_CUDA(L, cudaStreamWaitEvent(st, L->host_join, 0));
+  return CMOE_OK;
+}
+
 int cmoe_status(cmoe_layer* L, void* cuda_stream) {
   if (!L) return CMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -384,6 +442,17 @@ int cmoe_destroy(cmoe_layer* L) {
   if (!L) return CMOE_ERR_INVALID_ARG;
   if (L->events_created)
     for (int i = 0; i <= CMOE_MAX_STAGES; ++i) cudaEventDestroy(L->events[i]);
+  {
+    cudaEvent_t ev[2 + 2 * kMaxHostChunks];
+    int n = 0;
+    ev[n++] = L->host_fork; ev[n++] = L->host_join;
+    for (int c = 0; c < kMaxHostChunks; ++c) ev[n++] = L->chunk_in[c];
+    for (int c = 0; c < kMaxHostChunks; ++c) ev[n++] = L->chunk_done[c];
+    for (int i = 0; i < n; ++i)
+      if (L->host_created >= 3 + i) cudaEventDestroy(ev[i]);
+    if (L->host_created >= 2) { cudaStreamSynchronize(L->d2h_stream); cudaStreamDestroy(L->d2h_stream); }
+    if (L->host_created >= 1) { cudaStreamSynchronize(L->h2d_stream); cudaStreamDestroy(L->h2d_stream); }
+  }
   if (L->side_created >= 3) cudaEventDestroy(L->side_join);
   if (L->side_created >= 2) cudaEventDestroy(L->side_fork);
   if (L->side_created >= 1) { cudaStreamSynchronize(L->side_stream); cudaStreamDestroy(L->side_stream); }

@@ -16,6 +16,7 @@ constexpr int kMaxG = 64;          // clusters
 constexpr int kMaxK = 32;          // experts per cluster (one lane each in the router's top-k)
 constexpr int kMaxKsel = 8;        // k
 constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
+constexpr int kMaxHostChunks = 4; // pipeline depth of cmoe_forward_host
 constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels
 
 enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
@@ -104,6 +105,10 @@ struct cmoe_layer {
   cudaStream_t side_stream;
   cudaEvent_t side_fork, side_join;
   int side_created;
+  // cmoe_forward_host: a stream per copy direction and an event per chunk and direction
+  cudaStream_t h2d_stream, d2h_stream;
+  cudaEvent_t host_fork, host_join, chunk_in[cmoe::kMaxHostChunks], chunk_done[cmoe::kMaxHostChunks];
+  int host_created;     // objects created so far, in the order above
   // tensor-core path: tensor maps and launch shapes (opaque here, see tc_path.cu)
   alignas(128) unsigned char tc_state[2048];
 };

@@ -334,3 +334,49 @@ def test_forward_is_repeatable(name):
         assert float((y - first).abs().max()) <= 2e-3 * scale
     torch.cuda.synchronize()
     assert m.status() == 0
+
+
+# ---- host-buffer entry point: chunked copies overlapped with the kernels ---------------------------------
+@pytest.mark.parametrize("T", [700, 5000, 9000])
+def test_forward_host_equals_forward(T):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=T, d=128, d_ff=256, E=8, G=2, r=16, k=2)
+    L = inputs.make_layer(s, 31)
+    m = ClusteredMoELayer(L)
+    xh = torch.from_numpy(L["x"]).pin_memory()
+    y_dev = m.forward(xh.cuda())
+    yh = torch.empty_like(xh).pin_memory()
+    m.forward_host(xh, yh)
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    a, b = y_dev.float().cpu().numpy(), yh.float().numpy()
+    # the same kernels on chunks of the batch: equal up to the order of the fp32 atomics (and, for a last
+    # chunk below 1024 tokens, the fp32 router instead of the split-fp16 one on near-ties)
+    bad = np.abs(a - b) > 2e-3 * np.abs(a).max() + 1e-3
+    assert bad.any(axis=1).mean() <= 0.002
+    # and against the oracle
+    o = ref.Layer(L)
+    r = o.route(L["x"])
+    idx = np.arange(0, T, 7, dtype=np.int32)
+    y_ref = o.forward(L["x"], idx)
+    cid, eid, gates = m.route(xh.cuda())
+    decided, _ = check_routes(s, r, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+    check_y(b[idx], y_ref, decided[idx])
+    m.close()
+
+
+def test_forward_host_small_batch_on_the_streaming_path():
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=48, d=256, d_ff=512, E=8, G=2, r=8, k=2)
+    L = inputs.make_layer(s, 32)
+    m = ClusteredMoELayer(L)
+    assert m.info.path == 2
+    xh = torch.from_numpy(L["x"]).pin_memory()
+    yh = m.forward_host(xh)
+    y_dev = m.forward(xh.cuda())
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    assert np.abs(yh.float().numpy() - y_dev.float().cpu().numpy()).max() <= 2e-3 * np.abs(y_dev.float().cpu().numpy()).max() + 1e-3
+    m.close()
