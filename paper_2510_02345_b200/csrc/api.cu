@@ -319,7 +319,8 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s
     const size_t rows = (size_t)t_pad_bound(D, T);
     void* zp = L->path == kPathStream ? static_cast<void*>(S.y32) : static_cast<void*>(S.s);
-    const size_t zb = L->path == kPathStream ? sizeof(float) * rows * D.d : sizeof(float) * rows * D.k * D.r;
+    size_t zb = L->path == kPathStream ? sizeof(float) * rows * D.d : sizeof(float) * rows * D.k * D.r;
+    if (L->path == kPathTensor && L->tc_variant == 2) tc2_accum_buffer(L, T, &zp, &zb);
     CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
@@ -401,7 +402,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->launches_route = 1;
   out->launches_forward = 1 + permute_launches(L->dims.T_max) +
                           (L->path == kPathTensor && L->tc_variant == 2
-                               ? tc2_launch_count(L->dims)
+                               ? tc2_launch_count(L)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
   out->memsets_forward = 0;
   out->n_stages = L->n_stages;

@@ -149,7 +149,8 @@ cudaError_t launch_tc_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st
 // tc2_path.cu : the same with the rank-r residual products on the tensor cores as well
 bool tc2_supported(const Dims& D);
 cudaError_t tc2_init(cmoe_layer* L);
-int tc2_launch_count(const Dims& D);
+int tc2_launch_count(const cmoe_layer* L);
+void tc2_accum_buffer(const cmoe_layer* L, int T, void** ptr, size_t* bytes);
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);

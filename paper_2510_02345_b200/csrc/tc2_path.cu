@@ -998,6 +998,32 @@ int pick_unit(int NT, int pt_bound, int pairs) {
 
 int ilog2(int v) { int l = 0; while ((1 << l) < v) ++l; return l; }
 
+// Launch shape of the up kernel for a batch of T tokens.  A unit that is a whole row tile (unit == NT) leaves
+// S complete at its end: the wide kernel then writes the gated rows p_j s_j straight into the down kernel's
+// operand (`direct`), without fp32 reductions into s and without the expansion kernel.  Whole-row units are
+// taken when they keep the pairs as busy as the default units do.
+struct UpPlan {
+  int NT, unit, grid;
+  bool direct;
+};
+UpPlan plan_up(const Tc2State& ts, const Dims& D, int T) {
+  UpPlan u{};
+  const int pt_bound = t_pad_bound(D, T) / (2 * BM), pairs = ts.sm_count / 2;
+  u.NT = D.d_ff / (ts.up_wide ? BN_WIDE : BN_UP);
+  u.unit = pick_unit(u.NT, pt_bound, pairs);
+  if (ts.up_wide && D.r > 0 && u.unit != u.NT) {
+    auto eff = [&](int unit) {
+      const long long n = (long long)pt_bound * (u.NT / unit), rounds = (n + pairs - 1) / pairs;
+      return (double)n / (double)(rounds * pairs);
+    };
+    if (eff(u.NT) >= eff(u.unit) - 0.02) u.unit = u.NT;
+  }
+  u.direct = ts.up_wide && D.r > 0 && u.unit == u.NT;
+  const long long total = (long long)pt_bound * (u.NT / u.unit);
+  u.grid = 2 * (int)(total < pairs ? total : pairs);
+  return u;
+}
+
 }  // namespace
 
 bool tc2_supported(const Dims& D) {
@@ -1054,7 +1080,22 @@ cudaError_t tc2_init(cmoe_layer* L) {
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-int tc2_launch_count(const Dims& D) { return D.r > 0 ? 5 : 2; }
+int tc2_launch_count(const cmoe_layer* L) {
+  const Dims& D = L->dims;
+  if (D.r == 0) return 2;
+  const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
+  return plan_up(ts, D, D.T_max).direct ? 4 : 5;
+}
+
+// The buffer the forward's first kernels clear for this path: the fp32 sums s, or the down kernel's
+// operand As when the up kernel writes it directly.
+void tc2_accum_buffer(const cmoe_layer* L, int T, void** ptr, size_t* bytes) {
+  const Dims& D = L->dims;
+  const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
+  const size_t rows = (size_t)t_pad_bound(D, T);
+  if (D.r > 0 && plan_up(ts, D, T).direct) { *ptr = L->sc.As; *bytes = sizeof(__half) * rows * KE; }
+  else { *ptr = L->sc.s; *bytes = sizeof(float) * rows * D.k * D.r; }
+}
 
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
   const Dims& D = L->dims;
@@ -1094,12 +1135,12 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   up.n_rows = S.n_rows; up.tile_cluster = S.tile_cluster; up.tile_mask = S.tile_mask; up.row_slot = S.row_slot;
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
   up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
+  const UpPlan plan = plan_up(ts, D, T);
   {
-    const int pairs = ts.sm_count / 2;
-    if (ts.up_wide) up.NT = D.d_ff / BN_WIDE;
-    up.unit = pick_unit(up.NT, pt_bound, pairs);
-    const long long total = (long long)pt_bound * (up.NT / up.unit);
-    const int grid = 2 * (int)(total < pairs ? total : pairs);
+    up.NT = plan.NT;
+    up.unit = plan.unit;
+    up.As_direct = plan.direct ? S.As : nullptr;
+    const int grid = plan.grid;
     if (ts.up_wide) {
       const UpWideMaps maps{&ts.mX3, &ts.mB13w, &ts.mA0, &ts.mAd, &ts.mV1w, &ts.mU2};
       e = launch_up_wide(D.r > 0, D.k, maps, up, grid, st);
@@ -1110,7 +1151,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
     if (e != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[2], st);
-  if (D.r > 0) {
+  if (D.r > 0 && !plan.direct) {
     const int threads = rows_bound * 8;
     launch_chained(s_expand_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, 1,
       S.n_rows, S.tile_cluster, S.row_slot, S.row_gate, S.s,

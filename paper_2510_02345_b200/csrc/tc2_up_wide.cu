@@ -383,14 +383,21 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
           const bool real = p.row_token[row] >= 0;
           float* srow = p.s_out + ((size_t)row * KSEL + j) * p.r;
           const int r = p.r;
+          const float gate = j == 0 ? g0f : g1f;
           for (int i = cq & 1; i < p.K; i += 2) {
             const uint32_t ta = taddr + UW_TMEM_S + j * KE + i * r;
             const bool mine = real && e == i;
+            __half* arow = p.As_direct ? p.As_direct + (size_t)row * KE + i * r : nullptr;   // the row's block of the expanded index
             if (r == 16) {
               uint32_t v[16];
               tmem_ld16_nowait(ta, v);
               tmem_ld_wait();
-              if (mine) {
+              if (mine && arow) {
+                uint32_t o[8];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) o[c] = pack_half2(gate * __uint_as_float(v[2 * c]), gate * __uint_as_float(v[2 * c + 1]));
+                st_global_v8(arow, o);
+              } else if (mine) {
 #pragma unroll
                 for (int c = 0; c < 16; c += 4)
                   red_add_v4(srow + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
@@ -399,7 +406,13 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
               uint32_t v[32];
               tmem_ld32_nowait(ta, v);
               tmem_ld_wait();
-              if (mine) {
+              if (mine && arow) {
+                uint32_t o[16];
+#pragma unroll
+                for (int c = 0; c < 16; ++c) o[c] = pack_half2(gate * __uint_as_float(v[2 * c]), gate * __uint_as_float(v[2 * c + 1]));
+                st_global_v8(arow, o);
+                st_global_v8(arow + 16, o + 8);
+              } else if (mine) {
 #pragma unroll
                 for (int c = 0; c < 32; c += 4)
                   red_add_v4(srow + c, __uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
@@ -408,7 +421,13 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
               uint32_t v[8];
               tmem_ld8_nowait(ta, v);
               tmem_ld_wait();
-              if (mine) {
+              if (mine && arow) {
+                *reinterpret_cast<uint4*>(arow) =
+                    make_uint4(pack_half2(gate * __uint_as_float(v[0]), gate * __uint_as_float(v[1])),
+                               pack_half2(gate * __uint_as_float(v[2]), gate * __uint_as_float(v[3])),
+                               pack_half2(gate * __uint_as_float(v[4]), gate * __uint_as_float(v[5])),
+                               pack_half2(gate * __uint_as_float(v[6]), gate * __uint_as_float(v[7])));
+              } else if (mine) {
                 red_add_v4(srow, __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
                 red_add_v4(srow + 4, __uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
               }
@@ -416,7 +435,12 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
               uint32_t v[4];
               tmem_ld4_nowait(ta, v);
               tmem_ld_wait();
-              if (mine) red_add_v4(srow, __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+              if (mine && arow) {
+                *reinterpret_cast<uint2*>(arow) = make_uint2(pack_half2(gate * __uint_as_float(v[0]), gate * __uint_as_float(v[1])),
+                                                             pack_half2(gate * __uint_as_float(v[2]), gate * __uint_as_float(v[3])));
+              } else if (mine) {
+                red_add_v4(srow, __uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+              }
             }
           }
           tc_fence_before();

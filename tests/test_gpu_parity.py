@@ -263,8 +263,11 @@ def test_tensor_path_empty_cluster():
     dict(d=256, d_ff=1024, E=8, G=2, r=16, k=2),     # several units per row tile
     dict(d=128, d_ff=512, E=8, G=2, r=0, k=2),       # no residuals
     dict(d=128, d_ff=512, E=8, G=2, r=8, k=1),       # one kept expert: no second pass
-    dict(d=128, d_ff=256, E=16, G=2, r=8, k=2),      # K = 8
-], ids=["nt3", "units", "r0", "k1", "K8r8"])
+    dict(d=128, d_ff=256, E=16, G=2, r=8, k=2),      # K = 8; one N tile per row tile: S rows written directly
+    dict(d=128, d_ff=256, E=8, G=2, r=4, k=2),       # direct rows, r = 4
+    dict(d=128, d_ff=256, E=4, G=2, r=32, k=2),      # direct rows, r = 32 (K = 2)
+    dict(d=128, d_ff=256, E=8, G=2, r=16, k=1),      # direct rows, one kept expert
+], ids=["nt3", "units", "r0", "k1", "K8r8", "direct_r4", "direct_r32", "direct_k1"])
 @pytest.mark.parametrize("tile", ["256", "128"])
 def test_up_kernel_tile_widths(kw, tile, monkeypatch):
     monkeypatch.setenv("CMOE_UP_TILE", tile)
