@@ -15,6 +15,9 @@
 // touches shared memory: the epilogues store it (fp16 pairs) into spare TMEM columns and the S
 // products read their A operand from there, which leaves shared memory to a ring of three 64 KB
 // stages (two 64-wide K atoms each, 3-D TMA boxes) and the tile's U2f columns.
+// S is accumulated in TMEM over a unit of N tiles; at the unit's end the row's own block of S_j is added
+// to s (fp32 reductions) or, when the unit is a whole row tile, written as fp16(p_j s_j) straight into the
+// down kernel's operand.
 // TMEM columns: P 0..255, S_0 256..319, S_1 320..383, a_j 384..511 (four chunks of 64 activations).
 // Warp roles: 0 and 3 TMA (alternating stages), 1 MMA, 2 S products and U2f loads, 4..19 epilogue
 // (twenty warps: warps are allocated in fours, and 96 registers per thread fit 20 but not 24).
