@@ -62,12 +62,12 @@ def stage_work(s, T, stage, active_clusters, active_experts):
 
 # ------------------------------------------------------------------ DRAM traffic of the dominant kernel
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from the ncu captures summarised under
-# profiles/ (ncu_gpt2m_tc2_up_down.md, ncu_decode_stream_kernels.md).  The figure is reported only while
+# profiles/.  The figure is reported only while
 # the kernel sources still have the hash they had at the capture; otherwise "traffic" is null.
 NCU_TRAFFIC = {
-    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 135.077120e6 + 110.778368e6,
-              "sha1": {"tc2_up_wide.cu": "0c87ccd7c6e1febe2600e6127b7f11e1eabf767e",
-                       "tc2_common.cuh": "128b12ba3262a9f686454456ca8a42dc3317a939",
+    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 125.386752e6 + 113.426944e6,
+              "sha1": {"tc2_up_wide.cu": "6e3a4440cd7724fa75b0e4912f4a4c19c6473d9a",
+                       "tc2_common.cuh": "720891980e6ee01fb474e61a99d1a9eb0baa7553",
                        "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
     "decode": {"kernel": "stream_kernel<up>", "bytes": 955.946240e6 + 12.473856e6,
                "sha1": {"stream_path.cu": "2eaf278dd3a1acaeae12cdb44d68bd323491fcd4",
