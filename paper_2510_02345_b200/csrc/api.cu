@@ -4,6 +4,7 @@
 #include <new>
 
 #include "cmoe_internal.h"
+#include "stage_factors.cuh"
 
 using namespace cmoe;
 
@@ -320,8 +321,12 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     const size_t rows = (size_t)t_pad_bound(D, T);
     void* zp = L->path == kPathStream ? static_cast<void*>(S.y32) : static_cast<void*>(S.s);
     size_t zb = L->path == kPathStream ? sizeof(float) * rows * D.d : sizeof(float) * rows * D.k * D.r;
-    if (L->path == kPathTensor && L->tc_variant == 2) tc2_accum_buffer(L, T, &zp, &zb);
-    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb));
+    FactorStage fs{};                     // nothing to stage unless the pair path has residual factors
+    if (L->path == kPathTensor && L->tc_variant == 2) {
+      tc2_accum_buffer(L, T, &zp, &zb);
+      tc2_factor_stage(L, &fs);
+    }
+    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));

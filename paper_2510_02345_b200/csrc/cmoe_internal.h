@@ -131,8 +131,9 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
                              int* slot_local, cudaStream_t st);
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
+struct FactorStage;   // stage_factors.cuh
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes);
+                           size_t zero_bytes, const FactorStage& fs);
 constexpr int kPermuteLaunches = 4;        // 2 for batches of at most 256 tokens (permute_launches)
 inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
 // generic_path.cu : CUDA-core path for any supported shape
@@ -151,6 +152,7 @@ bool tc2_supported(const Dims& D);
 cudaError_t tc2_init(cmoe_layer* L);
 int tc2_launch_count(const cmoe_layer* L);
 void tc2_accum_buffer(const cmoe_layer* L, int T, void** ptr, size_t* bytes);
+void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs);
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);

@@ -4,7 +4,7 @@
 // cluster, then to experts inside it", Sec. 3.3); the mechanism is this library's.
 //
 //   hist     per-block histogram of the keys (block = 256 consecutive tokens)
-//   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table, and the
+//   scan     block 0: per-key running sums over blocks, cluster segment offsets, tile table, and the
 //            table entries of the padding rows of each segment (no token, zero gates)
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
 //            writes the row tables
@@ -15,6 +15,7 @@
 #include "cmoe_internal.h"
 #include "launch.cuh"
 #include "device_utils.cuh"
+#include "stage_factors.cuh"
 
 namespace cmoe {
 
@@ -78,8 +79,12 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             const int* __restrict__ block_counts, int* __restrict__ block_base,
             int* __restrict__ key_cnt, int* __restrict__ key_off, int* __restrict__ seg_off,
             int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster, int K, int k,
-            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate) {
+            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
+            const FactorStage fs) {
   pdl_wait();
+  // blocks 1.. decode the layer's INT4 factors for the tensor-core residual products (weights only:
+  // independent of the scan, which is one block of latency)
+  if (blockIdx.x > 0) { stage_block(fs, blockIdx.x - 1); return; }
   __shared__ int sh_seg[kMaxG + 1];
   __shared__ int sh_segcnt[kMaxG];
   __shared__ int sh_cnt[kMaxKeys];
@@ -296,12 +301,22 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
   }
 }
 
+// the factor staging alone (batches of at most 256 tokens)
+__global__ void __launch_bounds__(256)
+stage_only_kernel(const FactorStage fs) {
+  pdl_wait();
+  stage_block(fs, blockIdx.x);
+}
+
 }  // namespace
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes) {
+                           size_t zero_bytes, const FactorStage& fs) {
+
   const int rows_bound = t_pad_bound(D, T);
   if (T <= kSmallT) {
+    // (one block of a few microseconds: the factor staging would not hide in it and has its own launch)
+    if (const int extra = stage_blocks(fs, 256)) launch_chained(stage_only_kernel, dim3(extra), dim3(256), 0, st, 1, fs);
     launch_chained(permute_small_kernel, dim3(1), dim3(kSmallT), sizeof(int) * ((size_t)D.nkey + kSmallT), st, 1,
       
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
@@ -315,10 +330,10 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
   launch_chained(hist_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
       T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
                                             S.slot, S.gates, S.keys, S.block_counts);
-  launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
+  launch_chained(scan_kernel, dim3(1 + stage_blocks(fs, 1024)), dim3(1024), 0, st, 1,
       nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
                                   S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
-                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
+                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate, fs);
   launch_chained(scatter_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
       T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,

@@ -5,7 +5,8 @@
 // rank-r product is phrased as a GEMM over an "expanded rank index" c = i*r + p (i = expert of the
 // cluster, p = rank), KE = 64 wide, so that one tile may mix rows routed to different experts:
 //
-//   stage   INT4 factors of the layer -> fp16 operand matrices in scratch (decoded in registers)
+//   stage   INT4 factors of the layer -> fp16 operand matrices in scratch (decoded in registers; stage_factors.cuh:
+//           the blocks ride in the permutation's scan kernel)
 //             U1f [G][KE][d]   V1f [G][d_ff][KE]   U2f [G][KE][d_ff]   V2f [G][d][KE]
 //   t       Tall = x_perm U1f_g^T (128 x KE per tile); row-wise selection writes
 //             A0 [row][c] = t of the row's first kept expert inside that expert's block, else 0
@@ -28,6 +29,7 @@
 // Every device wait is bounded: on expiry the kernel records CMOE_ERR_TIMEOUT in the status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
 #include "tc2_common.cuh"
+#include "stage_factors.cuh"
 
 namespace cmoe {
 
@@ -37,62 +39,6 @@ using namespace tc2c;
 
 constexpr int BN_UP = 128;
 constexpr int kMaxStages = 8;
-
-// ------------------------------------------------------------------------------------------------
-// stage: INT4 factors -> fp16 operand matrices (one thread per 32-bit word = 8 codes)
-// ------------------------------------------------------------------------------------------------
-struct FactorStage {
-  const uint8_t* q[4];     // U1, V1, U2, V2
-  const __half* s[4];
-  __half* dst[4];
-  long long words[4];      // 32-bit words of each packed factor
-  int dim[4];              // non-rank extent: d, d_ff, d_ff, d
-  int K, r;
-};
-
-__global__ void __launch_bounds__(256)
-stage_factors_kernel(const FactorStage fs) {
-  pdl_wait();
-  const int which = blockIdx.y;
-  const long long wd = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (wd >= fs.words[which]) return;
-  const int dim = fs.dim[which], K = fs.K, r = fs.r;
-  const uint32_t word = reinterpret_cast<const uint32_t*>(fs.q[which])[wd];
-  const long long flat0 = wd * 8;
-  const float sc = __half2float(fs.s[which][flat0 >> 5]);
-  __align__(16) __half v[8];
-#pragma unroll
-  for (int n = 0; n < 8; ++n) v[n] = __float2half_rn((float)sext4((int)(word >> (4 * n))) * sc);
-  __half* dst = fs.dst[which];
-  if ((which & 1) == 0) {
-    // U [E][r][dim]: row (e, p) of length dim -> row g*KE + i*r + p
-    const long long row = flat0 / dim;
-    const int c = (int)(flat0 - row * dim);
-    const long long g = row / (K * r);
-    const int n = (int)(row - g * (K * r));
-    *reinterpret_cast<uint4*>(dst + ((g * KE + n) * dim + c)) = *reinterpret_cast<const uint4*>(v);
-  } else if (r >= 8) {
-    // V [E][dim][r]: (e, n, p0..p0+7) -> [g][n][i*r + p0 ..]
-    const long long en = flat0 / r;
-    const int p0 = (int)(flat0 - en * r);
-    const long long e = en / dim;
-    const int n = (int)(en - e * dim);
-    const long long g = e / K;
-    const int i = (int)(e - g * K);
-    *reinterpret_cast<uint4*>(dst + ((g * dim + n) * KE + i * r + p0)) = *reinterpret_cast<const uint4*>(v);
-  } else {
-    // r == 4: the word holds two output columns of four ranks each
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const long long en = (flat0 + 4 * h) / 4;
-      const long long e = en / dim;
-      const int n = (int)(en - e * dim);
-      const long long g = e / K;
-      const int i = (int)(e - g * K);
-      *reinterpret_cast<uint2*>(dst + ((g * dim + n) * KE + i * 4)) = reinterpret_cast<const uint2*>(v)[h];
-    }
-  }
-}
 
 // ------------------------------------------------------------------------------------------------
 // t: Tall = x_perm U1f_g^T, one 128-row tile per CTA, then the row-wise selection into A0 / Ad
@@ -1080,11 +1026,31 @@ cudaError_t tc2_init(cmoe_layer* L) {
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// what the permutation's scan kernel stages beside its own work (tc2 path with residuals; else nothing)
+void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs) {
+  const Dims& D = L->dims;
+  const Weights& W = L->w;
+  const Scratch& S = L->sc;
+  *fs = FactorStage{};
+  if (D.r == 0) return;
+  const uint8_t* q[4] = {W.U1q, W.V1q, W.U2q, W.V2q};
+  const __half* sc[4] = {W.U1s, W.V1s, W.U2s, W.V2s};
+  __half* dst[4] = {S.U1f, S.V1f, S.U2f, S.V2f};
+  const int dim[4] = {D.d, D.d_ff, D.d_ff, D.d};
+  for (int i = 0; i < 4; ++i) {
+    fs->q[i] = q[i]; fs->s[i] = sc[i]; fs->dst[i] = dst[i]; fs->dim[i] = dim[i];
+    fs->words[i] = (long long)D.E * D.r * dim[i] / 8;
+  }
+  fs->K = D.K; fs->r = D.r;
+}
+
 int tc2_launch_count(const cmoe_layer* L) {
   const Dims& D = L->dims;
   if (D.r == 0) return 2;
   const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
-  return plan_up(ts, D, D.T_max).direct ? 4 : 5;
+  // t, up, (expansion,) down; the staging rides in the permutation's scan kernel, except for batches of at most 256
+  // tokens, where it has a launch of its own
+  return (plan_up(ts, D, D.T_max).direct ? 3 : 4) + (D.T_max <= 256 ? 1 : 0);
 }
 
 // The buffer the forward's first kernels clear for this path: the fp32 sums s, or the down kernel's
@@ -1107,22 +1073,6 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   cudaError_t e;
   if (marks) cudaEventRecord(marks[0], st);
   if (D.r > 0) {
-    FactorStage fs{};
-    const uint8_t* q[4] = {W.U1q, W.V1q, W.U2q, W.V2q};
-    const __half* sc[4] = {W.U1s, W.V1s, W.U2s, W.V2s};
-    __half* dst[4] = {S.U1f, S.V1f, S.U2f, S.V2f};
-    const int dim[4] = {D.d, D.d_ff, D.d_ff, D.d};
-    long long maxw = 0;
-    for (int i = 0; i < 4; ++i) {
-      fs.q[i] = q[i]; fs.s[i] = sc[i]; fs.dst[i] = dst[i]; fs.dim[i] = dim[i];
-      fs.words[i] = (long long)D.E * D.r * dim[i] / 8;
-      if (fs.words[i] > maxw) maxw = fs.words[i];
-    }
-    fs.K = D.K; fs.r = D.r;
-    dim3 grid((unsigned)((maxw + 255) / 256), 4);
-    launch_chained(stage_factors_kernel, dim3(grid), dim3(256), 0, st, 1,
-      fs);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
     TParams tp{};
     tp.n_rows = S.n_rows; tp.tile_cluster = S.tile_cluster; tp.row_slot = S.row_slot; tp.row_token = S.row_token;
     tp.A0 = S.A0; tp.Ad = S.Ad; tp.tile_mask = S.tile_mask; tp.status = S.status;
