@@ -5,6 +5,7 @@
 
 #include "cmoe_internal.h"
 #include "stage_factors.cuh"
+#include "lowrank.cuh"
 
 using namespace cmoe;
 
@@ -326,7 +327,9 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
       tc2_accum_buffer(L, T, &zp, &zb);
       tc2_factor_stage(L, &fs);
     }
-    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs));
+    LowrankTok lr{};                      // nothing rides along unless the streaming path has residual factors
+    if (L->path == kPathStream) stream_lowrank_rider(L, xh, T, &lr);
+    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs, lr));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));

@@ -132,8 +132,9 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
 struct FactorStage;   // stage_factors.cuh
+struct LowrankTok;    // lowrank.cuh
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs);
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr);
 constexpr int kPermuteLaunches = 4;        // 2 for batches of at most 256 tokens (permute_launches)
 inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
 // generic_path.cu : CUDA-core path for any supported shape
@@ -158,6 +159,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);
 int stream_launch_count(const Dims& D);
+void stream_lowrank_rider(const cmoe_layer* L, const __half* x, int T, LowrankTok* lr);
 cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 // repack.cu : create-time layout changes
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,

@@ -16,6 +16,7 @@
 #include "launch.cuh"
 #include "device_utils.cuh"
 #include "stage_factors.cuh"
+#include "lowrank.cuh"
 
 namespace cmoe {
 
@@ -226,8 +227,11 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
                      const int* __restrict__ cluster_id, const int* __restrict__ slot, const float* __restrict__ gates,
                      int* __restrict__ seg_off, int* __restrict__ seg_cnt, int* __restrict__ n_rows,
                      int* __restrict__ tile_cluster, int* __restrict__ row_token, int* __restrict__ row_slot,
-                     float* __restrict__ row_gate) {
+                     float* __restrict__ row_gate, const LowrankTok lr) {
   pdl_wait();
+  // blocks 1.. : t = x U1 of every (token, kept expert) on the weight-streaming path: it needs the routes,
+  // not the permutation, and hides in this block's latency
+  if (blockIdx.x > 0) { lowrank_tok_block(lr, blockIdx.x - 1); return; }
   extern __shared__ int sh[];
   int* cnt = sh;                   // [nkey] tokens per key, then first row of the key
   int* keys = cnt + nkey;          // [kSmallT]
@@ -311,16 +315,16 @@ stage_only_kernel(const FactorStage fs) {
 }  // namespace
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs) {
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr) {
 
   const int rows_bound = t_pad_bound(D, T);
   if (T <= kSmallT) {
     // (one block of a few microseconds: the factor staging would not hide in it and has its own launch)
     if (const int extra = stage_blocks(fs, 256)) launch_chained(stage_only_kernel, dim3(extra), dim3(256), 0, st, 1, fs);
-    launch_chained(permute_small_kernel, dim3(1), dim3(kSmallT), sizeof(int) * ((size_t)D.nkey + kSmallT), st, 1,
+    launch_chained(permute_small_kernel, dim3(1 + lowrank_tok_blocks(lr)), dim3(kSmallT), sizeof(int) * ((size_t)D.nkey + kSmallT), st, 1,
       
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
-        S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate);
+        S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate, lr);
     launch_chained(move_rows_kernel, dim3(rows_bound), dim3(128), 0, st, 1,
       D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
     return cudaGetLastError();

@@ -23,6 +23,7 @@
 #include "launch.cuh"
 #include "device_utils.cuh"
 #include "tc_ptx.cuh"
+#include "lowrank.cuh"
 
 namespace cmoe {
 
@@ -238,7 +239,8 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
         for (int c2 = 0; c2 < 4; ++c2) {
           const int c = 4 * c2 + part;
           const int row = row0 + tb + c;
-          const bool real = mine && p.row_token[row] >= 0;
+          const int tok = p.row_token[row];
+          const bool real = mine && tok >= 0;
           const float dv = __uint_as_float(part == 0 ? v[4 * c2] : part == 1 ? v[4 * c2 + 1] : part == 2 ? v[4 * c2 + 2] : v[4 * c2 + 3]);
           if (UP) {
             float ab = 0.f;
@@ -248,7 +250,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
                 float h = dv;
                 if (r > 0) {
                   // h += t_j . V1_e[f, :]: r codes of one scale group, decoded in registers
-                  const float4* tp = reinterpret_cast<const float4*>(p.t + ((size_t)row * k + j) * r);
+                  const float4* tp = reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r);    // t is indexed by token
                   const long long flat = ((long long)e * M + f) * r;
                   const float sc = __half2float(p.V1s[flat >> 5]);
                   float dot0 = 0.f, dot1 = 0.f;
@@ -327,44 +329,8 @@ lowrank_body(const int* __restrict__ seg_off, int G, int k, int r, int len, int 
   }
   const int e = row_slot[item];
   const __half* xin = in + (size_t)(in_per_slot ? item : row) * len;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
-  {
-    // all code lines of this block's first rank rows are requested at once (into L2): the loop below then
-    // meets DRAM latency once, not once per unrolled batch
-    const int lines = len >> 8;                                   // 128-byte lines of one rank row (len / 2 bytes)
-    const int pr0 = blockIdx.y * nwarp, nr = min(nwarp, r - pr0);
-    for (int i = threadIdx.x; i < nr * lines; i += blockDim.x) {
-      const int rr = i / lines, l = i - rr * lines;
-      asm volatile("prefetch.global.L2 [%0];" ::"l"(Uq + ((((long long)e * r + pr0 + rr) * len) >> 1) + (size_t)l * 128));
-    }
-  }
-  for (int pr = blockIdx.y * nwarp + warp; pr < r; pr += gridDim.y * nwarp) {
-    const long long base = ((long long)e * r + pr) * len;
-    float acc = 0.f;
-#pragma unroll 8
-    for (int grp = lane; grp * 32 < len; grp += 32) {
-      const uint4 pk = __ldg(reinterpret_cast<const uint4*>(Uq + ((base + grp * 32) >> 1)));
-      const float sc = __half2float(Us[(base >> 5) + grp]);
-      const uint32_t w[4] = {pk.x, pk.y, pk.z, pk.w};
-      float part = 0.f;
-#pragma unroll
-      for (int qd = 0; qd < 4; ++qd) {
-        const uint4 xv = *reinterpret_cast<const uint4*>(xin + grp * 32 + qd * 8);
-        const __half2* xh = reinterpret_cast<const __half2*>(&xv);
-        float cf[8];
-        int4x8_to_float(w[qd], cf);
-#pragma unroll
-        for (int n = 0; n < 4; ++n) {
-          const float2 xf = __half22float2(xh[n]);
-          part = fmaf(xf.x, cf[2 * n], part);
-          part = fmaf(xf.y, cf[2 * n + 1], part);
-        }
-      }
-      acc = fmaf(part, sc, acc);
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) out[(size_t)item * r + pr] = acc;
-  }
+  const int nwarp = blockDim.x >> 5;
+  lowrank_rows(xin, e, r, len, blockIdx.y * nwarp, gridDim.y * nwarp, Uq, Us, out + (size_t)item * r);
 }
 
 __global__ void __launch_bounds__(256)
@@ -517,7 +483,16 @@ cudaError_t stream_init(cmoe_layer* L) {
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-int stream_launch_count(const Dims& D) { return D.r > 0 ? 5 : 3; }
+int stream_launch_count(const Dims& D) { return D.r > 0 ? 4 : 3; }
+
+// t = x U1 for the blocks that ride in the permutation kernel
+void stream_lowrank_rider(const cmoe_layer* L, const __half* x, int T, LowrankTok* lr) {
+  const Dims& D = L->dims;
+  *lr = LowrankTok{};
+  if (D.r == 0) return;
+  lr->x = x; lr->cluster_id = L->sc.cluster_id; lr->slot = L->sc.slot; lr->Uq = L->w.U1q; lr->Us = L->w.U1s;
+  lr->out = L->sc.t; lr->T = T; lr->K = D.K; lr->k = D.k; lr->r = D.r; lr->len = D.d;
+}
 
 cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
   const Dims& D = L->dims;
@@ -527,12 +502,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   const int rows_bound = t_pad_bound(D, T);
   cudaError_t e;
   if (marks) cudaEventRecord(marks[0], st);
-  if (D.r > 0) {
-    launch_chained(lowrank_kernel, dim3(rows_bound * D.k, (D.r + 7) / 8), dim3(256), 0, st, 1,
-      S.seg_off, D.G, D.k, D.r, D.d, 0, S.x_perm, S.row_slot, S.row_token,
-                                                      W.U1q, W.U1s, S.t);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  }
+  // t = x U1 was computed beside the permutation (stream_lowrank_rider)
   if (marks) cudaEventRecord(marks[1], st);
   StreamParams p{};
   p.seg_off = S.seg_off; p.row_slot = S.row_slot; p.row_gate = S.row_gate; p.row_token = S.row_token;
