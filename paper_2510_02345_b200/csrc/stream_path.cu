@@ -352,6 +352,41 @@ lowrank_side_kernel(const int* __restrict__ seg_off, int G, int k, int r, int le
   lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out);
 }
 
+// Second stream, after s: the rank-r part of the down-projection, y32[row][c] += sum_j p_j s_j . V2_e[c, :],
+// one thread per (row, output column), added with the same fp32 atomics as the K ranges of the down kernel
+// running beside it.
+__global__ void __launch_bounds__(kSideThreads, 16)
+resid_side_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r, float* __restrict__ y32,
+                  const float* __restrict__ s, const int* __restrict__ row_slot, const float* __restrict__ row_gate,
+                  const int* __restrict__ row_token, const uint8_t* __restrict__ V2q, const __half* __restrict__ V2s) {
+  const int row = blockIdx.y;
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= seg_off[G] || c >= d || row_token[row] < 0) return;
+  float v = 0.f;
+  for (int j = 0; j < k; ++j) {
+    const int e = row_slot[(size_t)row * k + j];
+    const float* sj = s + ((size_t)row * k + j) * r;
+    const long long flat = ((long long)e * d + c) * r;      // the r codes of (e, c) share one scale group
+    float u = 0.f;
+    if (r >= 8) {
+      const uint32_t* wq = reinterpret_cast<const uint32_t*>(V2q + (flat >> 1));
+      for (int w8 = 0; w8 < r / 8; ++w8) {
+        float cf[8];
+        int4x8_to_float(wq[w8], cf);
+#pragma unroll
+        for (int n = 0; n < 8; ++n) u = fmaf(sj[w8 * 8 + n], cf[n], u);
+      }
+    } else {
+      float cf[8];
+      int4x8_to_float(*reinterpret_cast<const uint16_t*>(V2q + (flat >> 1)), cf);
+#pragma unroll
+      for (int n = 0; n < 4; ++n) u = fmaf(sj[n], cf[n], u);
+    }
+    v = fmaf(row_gate[(size_t)row * k + j] * __half2float(V2s[flat >> 5]), u, v);
+  }
+  atomicAdd(y32 + (size_t)row * d + c, v);
+}
+
 // y[tok] = fp16(y32[row] + sum_j p_j s_j V2_e), one thread per (row, output column)
 __global__ void __launch_bounds__(256)
 stream_final_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r,
@@ -483,7 +518,7 @@ cudaError_t stream_init(cmoe_layer* L) {
   return ok ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-int stream_launch_count(const Dims& D) { return D.r > 0 ? 4 : 3; }
+int stream_launch_count(const Dims& D) { return D.r > 0 ? 5 : 3; }
 
 // t = x U1 for the blocks that ride in the permutation kernel
 void stream_lowrank_rider(const cmoe_layer* L, const __half* x, int T, LowrankTok* lr) {
@@ -517,12 +552,15 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
-    // fork: s = a_j U2 on the second stream, beside the down kernel
+    // fork: s = a_j U2, then the rank-r part of y, on the second stream beside the down kernel
     if ((e = cudaEventRecord(L->side_fork, st)) != cudaSuccess) return e;
     if ((e = cudaStreamWaitEvent(L->side_stream, L->side_fork, 0)) != cudaSuccess) return e;
     const int nwarp = kSideThreads / 32;
     lowrank_side_kernel<<<dim3(rows_bound * D.k, (D.r + nwarp - 1) / nwarp), kSideThreads, 0, L->side_stream>>>(
         S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token, W.U2q, W.U2s, S.s);
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    resid_side_kernel<<<dim3((D.d + kSideThreads - 1) / kSideThreads, rows_bound), kSideThreads, 0, L->side_stream>>>(
+        S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate, S.row_token, W.V2q, W.V2s);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = cudaEventRecord(L->side_join, L->side_stream)) != cudaSuccess) return e;
   }
@@ -535,7 +573,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   if (D.r > 0 && (e = cudaStreamWaitEvent(st, L->side_join, 0)) != cudaSuccess) return e;     // join
   dim3 fgrid((D.d + 255) / 256, rows_bound);
   launch_chained(stream_final_kernel, dim3(fgrid), dim3(256), 0, st, 1,
-      S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate,
+      S.seg_off, D.G, D.d, D.k, 0 /* the rank-r part is already in y32 */, S.y32, S.s, S.row_slot, S.row_gate,
                                              S.row_token, W.V2q, W.V2s, y);
   return cudaGetLastError();
 }
