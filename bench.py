@@ -69,9 +69,10 @@ NCU_TRAFFIC = {
               "sha1": {"tc2_up_wide.cu": "6e3a4440cd7724fa75b0e4912f4a4c19c6473d9a",
                        "tc2_common.cuh": "720891980e6ee01fb474e61a99d1a9eb0baa7553",
                        "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.946240e6 + 12.473856e6,
-               "sha1": {"stream_path.cu": "2eaf278dd3a1acaeae12cdb44d68bd323491fcd4",
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.926528e6 + 10.317568e6,
+               "sha1": {"stream_path.cu": "a187b05075f992b283ec4221cbc552cf30072f42",
                         "device_utils.cuh": "daa6a5fc90a4b02a5c17177e8d154044cca709c4",
+                        "lowrank.cuh": "269b2967c3b968c508c6afb24186bafe32112f8b",
                         "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
 }
 
