@@ -383,3 +383,12 @@ def test_forward_host_small_batch_on_the_streaming_path():
     assert m.status() == 0
     assert np.abs(yh.float().numpy() - y_dev.float().cpu().numpy()).max() <= 2e-3 * np.abs(y_dev.float().cpu().numpy()).max() + 1e-3
     m.close()
+
+
+def test_headline_shape_at_another_batch_size():
+    """The headline shape with a batch that does not fill whole-row work units evenly (partial units, fp32
+    reductions into s and the expansion kernel instead of the direct rows)."""
+    s = inputs.small_shape(T=20000, d=1024, d_ff=4096, E=32, G=8, r=16, k=2)
+    L = inputs.make_layer(s, 5)
+    got = full_check(L, L["x"], sample=192)
+    assert got["module"].info.path == 1
