@@ -243,6 +243,13 @@ router_token_kernel(const RouterArgs a) {
     const size_t step = (size_t)gridDim.x * blockDim.x * 128;
     for (size_t off = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 128; off < bytes; off += step)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(a.Rt) + off));
+    // the first pass itself: all lines of the cluster prototypes and of this token's row are requested now,
+    // so its unrolled batches of loads meet DRAM latency once
+    const size_t cbytes = (size_t)a.G * d * sizeof(float);
+    for (size_t off = (size_t)threadIdx.x * 128; off < cbytes; off += (size_t)blockDim.x * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(a.Ct) + off));
+    for (size_t off = (size_t)threadIdx.x * 128; off < (size_t)d * sizeof(__half); off += (size_t)blockDim.x * 128)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(xr) + off));
   }
   for (int pass = 0; pass < 2; ++pass) {
     const int n = pass == 0 ? a.G : a.K;
