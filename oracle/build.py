@@ -13,7 +13,8 @@ def build(force: bool = False) -> str:
     deps = [SRC, os.path.join(HERE, "cmoe_oracle.h")]
     if not force and os.path.exists(LIB) and all(os.path.getmtime(LIB) >= os.path.getmtime(p) for p in deps):
         return LIB
-    cmd = ["gcc", "-O2", "-march=native", "-fopenmp", "-shared", "-fPIC", "-Wall", "-Wextra",
+    # no -march=native: the object is built on one machine and may be loaded on another
+    cmd = ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-Wextra",
            "-o", LIB, SRC, "-lm"]
     subprocess.run(cmd, check=True)
     return LIB

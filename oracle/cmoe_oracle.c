@@ -228,3 +228,49 @@ void cmoe_ref_param_count(const cmoe_ref_desc* D, int64_t* stored, int64_t* dens
   *dense = (int64_t)D->E * W;
   *stored = (int64_t)D->G * W + (int64_t)D->E * 2 * D->r * ((int64_t)D->d + D->d_ff);
 }
+
+/* By-products of routing that the clustering of Sec. 3.1 consumes.
+ *   loads[e]  = number of tokens whose kept experts include e              (sum = k T)
+ *   xbar[e]   = (1/N) sum of the N tokens routed to e (text after Eq. 5); zero row when N = 0
+ *   mu[e]    <- (1 - beta) mu[e] + beta xbar[e]   (Eq. 5), unchanged when no token arrived
+ *   cov       = standard deviation of the loads / their mean (Sec. 4.1, expert load balance);
+ *               the population form (divide by E) is this build's reading, the paper does not say which
+ * Sums in double, one rounding to fp32.  xbar, mu and cov may be NULL. */
+int cmoe_ref_expert_stats(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
+                          int32_t* loads, float* xbar, float* mu, float beta, float* cov) {
+  if (!desc_ok(D) || T < 0 || !loads) return -1;
+  const int d = D->d, E = D->E, k = D->k;
+  int32_t* cid = (int32_t*)malloc(sizeof(int32_t) * (size_t)(T + 1));
+  int32_t* slot = (int32_t*)malloc(sizeof(int32_t) * ((size_t)T * k + 1));
+  float* gates = (float*)malloc(sizeof(float) * ((size_t)T * k + 1));
+  if (T > 0 && cmoe_ref_route(D, x, T, cid, slot, gates, NULL, NULL)) { free(cid); free(slot); free(gates); return -1; }
+  for (int e = 0; e < E; ++e) loads[e] = 0;
+  for (int t = 0; t < T; ++t)
+    for (int s = 0; s < k; ++s) loads[slot[(size_t)t * k + s]] += 1;
+  if (xbar || mu) {
+    double* sum = (double*)malloc(sizeof(double) * (size_t)d);
+    for (int e = 0; e < E; ++e) {
+      for (int j = 0; j < d; ++j) sum[j] = 0.0;
+      for (int t = 0; t < T; ++t)
+        for (int s = 0; s < k; ++s)
+          if (slot[(size_t)t * k + s] == e)
+            for (int j = 0; j < d; ++j) sum[j] += (double)cmoe_ref_half_to_float(x[(size_t)t * d + j]);
+      for (int j = 0; j < d; ++j) {
+        const double mean = loads[e] > 0 ? sum[j] / (double)loads[e] : 0.0;
+        if (xbar) xbar[(size_t)e * d + j] = (float)mean;
+        if (mu && loads[e] > 0)
+          mu[(size_t)e * d + j] = (float)((1.0 - (double)beta) * (double)mu[(size_t)e * d + j] + (double)beta * mean);
+      }
+    }
+    free(sum);
+  }
+  if (cov) {
+    double mean = 0.0, var = 0.0;
+    for (int e = 0; e < E; ++e) mean += (double)loads[e];
+    mean /= (double)E;
+    for (int e = 0; e < E; ++e) var += ((double)loads[e] - mean) * ((double)loads[e] - mean);
+    *cov = mean > 0.0 ? (float)(sqrt(var / (double)E) / mean) : 0.f;
+  }
+  free(cid); free(slot); free(gates);
+  return 0;
+}

@@ -23,7 +23,9 @@
  * Pins (tests/test_oracle_pins.py): r = 0 against a library dense FFN; G = E
  * against an independent top-1 MoE; brute-force route enumeration; the factored
  * identity x(B+UV) = xB + (xU)V in fp64; a residual-only layer; exhaustive INT4
- * codec; the parameter-count closed form (Eq. 8); equivariance invariants.
+ * codec; the parameter-count closed form (Eq. 8); equivariance invariants;
+ * for the routing by-products (loads, x-bar, Eq. 5, load CoV): conservation
+ * sums, a hand-counted example and numpy bincount / mean on the routes.
  * The paper prints no numeric layer output, so the absolute value of y on
  * random weights is otherwise "parity unpinned".
  */
@@ -71,6 +73,12 @@ int cmoe_ref_forward(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
 /* Stored parameter elements of the compressed layer and of the E dense experts it replaces
  * (routers excluded): the ingredients of the compression ratio of Eq. 8. */
 void cmoe_ref_param_count(const cmoe_ref_desc* D, int64_t* stored, int64_t* dense);
+
+/* Routing by-products for the clustering of Sec. 3.1: tokens per expert slot, the mean routed token
+ * x-bar_i, the EMA centroid update of Eq. 5 applied in place to mu (NULL = skip), and the coefficient of
+ * variation of the loads (population standard deviation / mean; Sec. 4.1).  loads [E]; xbar, mu [E][d]. */
+int cmoe_ref_expert_stats(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
+                          int32_t* loads, float* xbar, float* mu, float beta, float* cov);
 
 int cmoe_ref_num_threads(void);
 

@@ -40,6 +40,9 @@ def load(path: str):
         L.cmoe_ref_forward.argtypes = [C.POINTER(_Desc), C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         L.cmoe_ref_param_count.restype = None
         L.cmoe_ref_param_count.argtypes = [C.POINTER(_Desc), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.cmoe_ref_expert_stats.restype = C.c_int
+        L.cmoe_ref_expert_stats.argtypes = [C.POINTER(_Desc), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_float, C.c_void_p]
         L.cmoe_ref_num_threads.restype = C.c_int
     return L
 
@@ -111,6 +114,21 @@ class Layer:
         if rc:
             raise ValueError("oracle rejected its arguments")
         return W
+
+    def expert_stats(self, x: np.ndarray, mu: np.ndarray | None = None, beta: float = 0.05):
+        """-> loads [E] int32, xbar [E][d] fp32, cov (float); `mu` ([E][d] fp32, contiguous) is updated in place."""
+        s = self.shape
+        x = np.ascontiguousarray(x, dtype=np.float16)
+        loads = np.zeros(s.E, np.int32)
+        xbar = np.zeros((s.E, s.d), np.float32)
+        cov = np.zeros(1, np.float32)
+        if mu is not None:
+            assert mu.dtype == np.float32 and mu.flags.c_contiguous and mu.shape == (s.E, s.d)
+        rc = lib().cmoe_ref_expert_stats(C.byref(self.desc), _ptr(x), x.shape[0], _ptr(loads), _ptr(xbar),
+                                         None if mu is None else mu.ctypes.data, beta, _ptr(cov))
+        if rc:
+            raise ValueError("oracle rejected its arguments")
+        return loads, xbar, float(cov[0])
 
     def param_count(self):
         a, b = C.c_int64(), C.c_int64()

@@ -35,6 +35,14 @@ MUTANTS = [
     ("gate dropped in combine", "(double)gate[(size_t)n * k + s] *", ""),
     ("only first slot combined", "for (int s = 0; s < k; ++s)\n        acc += (double)gate", "for (int s = 0; s < 1; ++s)\n        acc += (double)gate"),
     ("param count", "(int64_t)D->E * 2 * D->r", "(int64_t)D->E * D->r"),
+    ("loads count the first kept expert only", "for (int s = 0; s < k; ++s) loads[slot[(size_t)t * k + s]] += 1;",
+     "for (int s = 0; s < 1; ++s) loads[slot[(size_t)t * k + s]] += 1;"),
+    ("mean over all tokens", "sum[j] / (double)loads[e] : 0.0;", "sum[j] / (double)T : 0.0;"),
+    ("EMA weights swapped", "(1.0 - (double)beta) * (double)mu[(size_t)e * d + j] + (double)beta * mean",
+     "(double)beta * (double)mu[(size_t)e * d + j] + (1.0 - (double)beta) * mean"),
+    ("EMA applied without tokens", "if (mu && loads[e] > 0)", "if (mu)"),
+    ("sample variance", "sqrt(var / (double)E) / mean", "sqrt(var / (double)(E - 1)) / mean"),
+    ("variance instead of deviation", "sqrt(var / (double)E) / mean", "(var / (double)E) / mean"),
 ]
 
 PINS = [
@@ -50,6 +58,8 @@ PINS = [
     pins.test_residual_only_layer,
     pins.test_formed_weights_orientation,
     pins.test_invariants,
+    pins.test_expert_stats_hand_counted,
+    pins.test_expert_stats_conservation_and_numpy_counts,
 ]
 
 

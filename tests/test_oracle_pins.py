@@ -15,9 +15,18 @@ GOLD = os.path.join(os.path.dirname(__file__), "golden")
 NIBBLE_VALUE = [0, 1, 2, 3, 4, 5, 6, 7, -8, -7, -6, -5, -4, -3, -2, -1]  # two's complement, by hand
 
 
+def unpack_codes(packed: np.ndarray) -> np.ndarray:
+    """Inverse of the nibble packing (even flat index in the low nibble, two's complement), codes as int8."""
+    table = np.array(NIBBLE_VALUE, np.int8)
+    out = np.empty(packed.size * 2, np.int8)
+    out[0::2] = table[packed & 0xF]
+    out[1::2] = table[packed >> 4]
+    return out
+
+
 def np_dequant(q, s, shape):
     """Independent decoder (numpy): codes from the packing inverse times the per-32 scale, fp64."""
-    codes = inputs.unpack_codes(q).astype(np.float64)
+    codes = unpack_codes(q).astype(np.float64)
     scale = np.repeat(s.astype(np.float64), 32)
     return (codes * scale).reshape(shape)
 
@@ -308,3 +317,59 @@ def test_bad_descriptor_rejected():
     s = inputs.LayerShape("bad", T=1, d=4, d_ff=4, E=6, G=4, r=0, k=1)
     with pytest.raises(ValueError):
         ref.Layer(dict(shape=s, C=np.zeros((4, 4), np.float32))).route(np.zeros((1, 4), np.float16))
+
+
+# ---- routing by-products: loads, mean routed token, Eq. 5, load CoV ------------------------------------
+def _hand_stats_layer():
+    s = inputs.small_shape(T=5, d=4, d_ff=2, E=4, G=2, r=0, k=1)
+    C = np.zeros((4, 2), np.float32); C[0, 0] = 1; C[1, 1] = 1
+    R = np.zeros((2, 4, 2), np.float32); R[:, 2, 0] = 1; R[:, 3, 1] = 1
+    L = dict(shape=s, C=C, R=R, b_c=None, b_e=None, B1=np.zeros((2, 4, 2), np.float16), B2=np.zeros((2, 2, 4), np.float16))
+    x = np.array([[2, 0, 1, 0], [4, 0, 3, 0], [1, 0, 0, 2], [0, 1, 2, 0], [1, 0, 0, 4]], np.float16)
+    return L, x
+
+
+def test_expert_stats_hand_counted():
+    gold = {}
+    for line in open(os.path.join(GOLD, "hand_worked_stats.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *vals = line.split()
+        gold[key] = np.array([float(v) for v in vals])
+    L, x = _hand_stats_layer()
+    mu = np.ones((4, 4), np.float32)
+    loads, xbar, cov = ref.Layer(L).expert_stats(x, mu=mu, beta=0.25)
+    assert np.array_equal(loads, gold["loads"].astype(np.int32))
+    assert np.allclose(xbar.reshape(-1), gold["xbar"], atol=1e-6)
+    assert np.allclose(mu.reshape(-1), gold["mu"], atol=1e-6)
+    assert abs(cov - gold["cov"][0]) < 1e-6
+
+
+def test_expert_stats_conservation_and_numpy_counts():
+    L = inputs.make_layer(inputs.small_shape(T=301, d=64, d_ff=32, E=12, G=3, r=0, k=2), 51)
+    s, x = L["shape"], L["x"]
+    o = ref.Layer(L)
+    mu0 = np.random.default_rng(0).standard_normal((s.E, s.d)).astype(np.float32)
+    mu = mu0.copy()
+    loads, xbar, cov = o.expert_stats(x, mu=mu, beta=0.05)
+    # every token is counted once per kept expert
+    assert loads.sum() == s.k * s.T
+    # sum_e load_e xbar_e = k * (sum of all tokens): every token enters k expert means
+    lhs = (loads[:, None].astype(np.float64) * xbar.astype(np.float64)).sum(0)
+    rhs = s.k * x.astype(np.float64).sum(0)
+    assert np.allclose(lhs, rhs, atol=1e-3)
+    # counts and means again from the routes with numpy
+    slots = o.route(x)["expert_slot"]
+    assert np.array_equal(loads, np.bincount(slots.reshape(-1), minlength=s.E))
+    for e in range(s.E):
+        rows = np.nonzero((slots == e).any(axis=1))[0]
+        want = x[rows].astype(np.float64).mean(0) if rows.size else np.zeros(s.d)
+        assert np.allclose(xbar[e], want, atol=1e-6)
+        want_mu = 0.95 * mu0[e].astype(np.float64) + 0.05 * want if rows.size else mu0[e]
+        assert np.allclose(mu[e], want_mu, atol=1e-6)
+    assert abs(cov - np.std(loads.astype(np.float64)) / np.mean(loads)) < 1e-6
+    # an expert without tokens keeps its centroid: close cluster 1
+    L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)
+    mu = mu0.copy()
+    loads, xbar, _ = ref.Layer(L).expert_stats(x, mu=mu, beta=0.5)
+    assert loads[s.K:2 * s.K].sum() == 0 and np.array_equal(mu[s.K:2 * s.K], mu0[s.K:2 * s.K]) and not xbar[s.K:2 * s.K].any()
