@@ -4,7 +4,8 @@
 A step is one pass of the whole hot path (router, permutation, expert FFNs with the fused
 residuals, gated combine, un-permute) over one batch of synthetic tokens.  Default workload: the
 GPT-2-medium-shaped layer (T=16384, d=1024, d_ff=4096, E=32, G=8, r=16, top-2), the compute-bound
-headline configuration; `--all` adds one short line per other workload under "workloads".
+headline configuration; the decode-shaped memory-bound workload is timed too and reported under "workloads"
+(`--all` adds the other three).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--all] [--impl reference]
 
@@ -147,7 +148,8 @@ def load_peaks():
 
 
 # ------------------------------------------------------------------ the CUDA arm
-def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks, dev_index, sync_ranks=True):
+def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks, dev_index, sync_ranks=True,
+                  sustained_s=0.0, keep_outputs=False):
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer, cmoe_profile_enable, cmoe_profile_read
     s = inputs.CONFIGS[name]
@@ -162,12 +164,13 @@ def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks,
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
     stream = torch.cuda.current_stream(dev)
 
-    cid, eid, _ = m.route(x)
+    cid, eid, gates = m.route(x)
+    loads, _, cov = m.expert_stats(x)          # the library's own by-products: tokens per expert, load CoV
     torch.cuda.synchronize(dev)
     active_clusters = int(torch.unique(cid).numel())
-    active_experts = int(torch.unique(eid).numel())
-    loads = torch.bincount(eid.flatten().long(), minlength=s.E).float()
-    i_load = float(loads.std(unbiased=False) / loads.mean())
+    active_experts = int((loads > 0).sum())
+    i_load = float(cov)
+    routes = (cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy()) if keep_outputs else None
 
     for _ in range(max(3, warmup)):
         flush.zero_()
@@ -210,6 +213,30 @@ def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks,
             stage_ms[k_] = stage_ms.get(k_, 0.0) + v / steps
     cmoe_profile_enable(m.handle, False)
 
+    # sustained pass: the same forward called back to back (no flush, no host round trip) for sustained_s
+    # seconds with the clock sampler running: what a forward costs once the board is under load
+    sustained = None
+    if sustained_s > 0:
+        per = max(dev_ms / steps, 1e-3)
+        n_sus = int(max(50, sustained_s * 1e3 / per))
+        for _ in range(20):
+            m.forward(x, out=y)
+        torch.cuda.synchronize(dev)
+        sam = ClockSampler(dev_index)
+        sam.__enter__()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(n_sus):
+            m.forward(x, out=y)
+        s1.record(stream)
+        s1.synchronize()
+        sam.__exit__()
+        assert m.status() == 0
+        sustained = {"forwards": n_sus, "seconds": s0.elapsed_time(s1) * 1e-3, "ms_per_forward": s0.elapsed_time(s1) / n_sus,
+                     "clocks": sam.summary(), "l2": "not flushed: inputs and weights of this workload exceed L2" if name != "tiny" else "not flushed"}
+
+    y_host = y.float().cpu().numpy() if keep_outputs else None
+
     e2e = None
     if want_e2e:
         xh = torch.from_numpy(x_np).pin_memory()
@@ -233,7 +260,8 @@ def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks,
 
     res = dict(name=name, shape=s, T=T, dev_ms=dev_ms, steps=steps, wall_s=wall, per_step=per_step,
                stage_ms=stage_ms, active_clusters=active_clusters, active_experts=active_experts,
-               i_load=i_load, info=m.info, e2e=e2e, clocks=sampler.summary() if sampler else None)
+               i_load=i_load, info=m.info, e2e=e2e, clocks=sampler.summary() if sampler else None,
+               sustained=sustained, routes=routes, y=y_host, x=x_np if keep_outputs else None)
     m.close()
     del m, x, y, flush
     torch.cuda.empty_cache()
@@ -264,36 +292,57 @@ def replicas_value(world, tokens_per_rank, ms_per_step):
 
 
 def roofline_for(res, peaks, peaks_kind):
+    """Roofline entry of the dominant kernel.  Its time is the stage's CUDA-event interval in a pass whose steps
+    are separated by an L2 flush and a host round trip: a kernel timed alone, so `frac` divides by the BURST
+    peak; the sustained and nominal fractions are printed beside it."""
     s, T = res["shape"], res["T"]
     stage = max(("up", "down"), key=lambda n: res["stage_ms"].get(n, 0.0))
     ms = res["stage_ms"][stage]
     flops, nbytes = stage_work(s, T, stage, res["active_clusters"], res["active_experts"])
     intensity = flops / max(nbytes, 1.0)
+    traffic = ncu_traffic(res["name"]) if stage == "up" else None
     if intensity > 300:           # ridge of the B200 is ~250 flop/B
-        peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        burst = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+        sust = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
         ach = flops / (ms * 1e-3) / 1e12
-        return {"bound": "tensor", "kernel": stage, "achieved": ach, "peak": peak, "unit": "TFLOP/s",
-                "frac": ach / peak, "traffic": ncu_traffic(res["name"]) if stage == "up" else None, "peak_kind": f"{peaks_kind} cuBLAS bf16 sustained (fp16 has the same rate)",
+        return {"bound": "tensor", "kernel": stage, "achieved": ach, "peak": burst, "unit": "TFLOP/s",
+                "frac": ach / burst, "traffic": traffic,
+                "peak_kind": f"{peaks_kind} cuBLAS bf16 burst (kernel timed alone; fp16 has the same rate)",
+                "fracs": {"of_burst": ach / burst, "of_sustained": ach / sust, "of_nominal_2250": ach / NOMINAL_FP16_TFLOPS},
                 "kernel_ms": ms, "flops_per_launch": flops}
     peak = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
     ach = nbytes / (ms * 1e-3) / 1e9
     return {"bound": "hbm", "kernel": stage, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-            "traffic": ncu_traffic(res["name"]) if stage == "up" else None, "peak_kind": f"{peaks_kind} copy bandwidth", "kernel_ms": ms,
-            "bytes_per_launch": nbytes}
+            "traffic": traffic, "peak_kind": f"{peaks_kind} copy bandwidth",
+            "fracs": {"of_measured_copy": ach / peak, "of_nominal_8000": ach / NOMINAL_HBM_GBS},
+            "kernel_ms": ms, "bytes_per_launch": nbytes}
 
 
-def whole_layer_fractions(res, n_gpus):
+def whole_layer_fractions(res, n_gpus, peaks=None):
     s, T = res["shape"], res["T"]
     flops, nbytes = algorithmic_work(s, T, res["active_clusters"], res["active_experts"])
     sec = res["dev_ms"] / res["steps"] * 1e-3
-    return {"algorithmic_tflops": flops / sec / 1e12, "algorithmic_gbs": nbytes / sec / 1e9,
-            "frac_of_nominal_fp16_2250T": flops / sec / 1e12 / NOMINAL_FP16_TFLOPS,
-            "frac_of_nominal_hbm_8TBs": nbytes / sec / 1e9 / NOMINAL_HBM_GBS}
+    out = {"algorithmic_tflops": flops / sec / 1e12, "algorithmic_gbs": nbytes / sec / 1e9,
+           "frac_of_nominal_fp16_2250T": flops / sec / 1e12 / NOMINAL_FP16_TFLOPS,
+           "frac_of_nominal_hbm_8TBs": nbytes / sec / 1e9 / NOMINAL_HBM_GBS}
+    if peaks:
+        out["frac_of_measured_bf16_burst"] = flops / sec / 1e12 / float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+        out["frac_of_measured_hbm_copy"] = nbytes / sec / 1e9 / float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+    if res.get("sustained"):
+        sus = res["sustained"]["ms_per_forward"] * 1e-3
+        out["sustained"] = {"ms_per_forward": res["sustained"]["ms_per_forward"], "algorithmic_tflops": flops / sus / 1e12,
+                            "frac_of_nominal_fp16_2250T": flops / sus / 1e12 / NOMINAL_FP16_TFLOPS,
+                            "frac_of_nominal_hbm_8TBs": nbytes / sus / 1e9 / NOMINAL_HBM_GBS}
+        if peaks:
+            out["sustained"]["frac_of_measured_bf16_sustained"] = flops / sus / 1e12 / float(
+                peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+    return out
 
 
 # ------------------------------------------------------------------ the CPU oracle arm
-def oracle_rate(name, target_s=15.0, max_tokens=None):
-    """tokens/s of the CPU oracle on a bounded sample (first n tokens) of the workload."""
+def oracle_rate(name, target_s=15.0, max_tokens=None, gpu=None):
+    """tokens/s of the CPU oracle on a bounded sample (first n tokens) of the workload.  With `gpu` (the CUDA arm's
+    routes and output rows of the same batch) the sample's rows are also compared: the second returned dict."""
     from oracle import ref
     s = inputs.CONFIGS[name]
     L = inputs.make_layer(s, seed=0)
@@ -310,9 +359,39 @@ def oracle_rate(name, target_s=15.0, max_tokens=None):
     if max_tokens:
         n = min(n, max_tokens)
     n = max(1, n)
-    t0 = time.perf_counter(); o.forward(L["x"][:n]); dt = time.perf_counter() - t0
-    return {"value": n / dt, "unit": UNIT, "cores": ref.num_threads(), "kind": "oracle",
+    t0 = time.perf_counter(); y_ref = o.forward(L["x"][:n]); dt = time.perf_counter() - t0
+    base = {"value": n / dt, "unit": UNIT, "cores": ref.num_threads(), "kind": "oracle",
             "sample": f"first {n} of {T} tokens of '{name}', one call, {dt:.1f} s, expert weights formed explicitly inside the timed call"}
+    parity = None
+    if gpu is not None:
+        parity = parity_on_sample(s, o.route(L["x"][:n]), y_ref, gpu, n)
+    return base, parity
+
+
+def parity_on_sample(s, r, y_ref, gpu, n):
+    """The CUDA arm's routes and output rows against the oracle's on the first n tokens: routes must agree wherever
+    the oracle's logit margins exceed 1e-4 (tokens inside that band are counted and left out of the row check);
+    rows within max|y - y_ref| <= 1e-2 max|y_ref| + 1e-3."""
+    cid, eid, _ = (a[:n] for a in gpu["routes"])
+    z = np.sort(r["z"].astype(np.float64), axis=1)[:, ::-1]
+    l = np.sort(r["l"].astype(np.float64), axis=1)[:, ::-1]
+    cm = z[:, 0] - z[:, 1] if z.shape[1] > 1 else np.full(n, np.inf)
+    last = min(s.k, l.shape[1] - 1)
+    em = np.min(l[:, :last] - l[:, 1:last + 1], axis=1) if last >= 1 else np.full(n, np.inf)
+    c_ok = cm > 1e-4
+    e_ok = c_ok & (em > 1e-4)
+    bad = int((cid[c_ok] != r["cluster_id"][c_ok]).sum() + (eid[e_ok] != r["expert_slot"][e_ok]).any(axis=1).sum())
+    err = float(np.abs(gpu["y"][:n][e_ok] - y_ref[e_ok]).max()) if e_ok.any() else 0.0
+    tol = 1e-2 * float(np.abs(y_ref).max()) + 1e-3
+    return {"rows_checked": int(e_ok.sum()), "of_tokens": int(gpu["y"].shape[0]), "max_abs_err": err, "tolerance": tol,
+            "within_tolerance": bool(err <= tol), "route_mismatches_outside_band": bad,
+            "cluster_near_ties": int((~c_ok).sum()), "expert_near_ties": int((c_ok & ~e_ok).sum()), "band": 1e-4}
+
+
+def config_of(name, s, T, world):
+    """The workload's description: the same keys in both arms."""
+    return {"workload": name, "T_per_gpu": T, "d": s.d, "d_ff": s.d_ff, "E": s.E, "G": s.G, "r": s.r, "k": s.k,
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
 
 
 def run_reference(args, rank):
@@ -339,10 +418,9 @@ def run_reference(args, rank):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": name, "T": T, "d": s.d, "d_ff": s.d_ff, "E": s.E, "G": s.G, "r": s.r, "k": s.k,
-                       "sample_tokens_per_step": n},
+            "config": config_of(name, s, T, 1),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": ref.num_threads(), "kind": "oracle",
-                             "sample": f"first {n} of {T} tokens per step"},
+                             "sample": f"first {n} of {T} tokens per step ({args.steps} steps)"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -359,6 +437,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--all", action="store_true", help="also time the other four workloads (short runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="leave the decode workload out of the default line")
+    ap.add_argument("--sustained", type=float, default=2.0,
+                    help="seconds of back-to-back forwards for the sustained figure (0: skip)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -379,7 +460,8 @@ def main():
 
     steps, warmup = args.steps, max(3, args.warmup)
     res = time_workload(args.workload, steps, warmup, rank, seed_offset=rank, want_e2e=True,
-                        want_clocks=True, dev_index=local_rank)
+                        want_clocks=True, dev_index=local_rank, sustained_s=args.sustained,
+                        keep_outputs=(rank == 0 and not args.no_cpu_baseline))
     dev_ms = res["dev_ms"]
     e2e_ms = res["e2e"]["ms_per_step"]
     if world > 1:
@@ -395,37 +477,41 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f16", "data": "synthetic",
-            "config": {"workload": args.workload, "T_per_gpu": T, "d": s.d, "d_ff": s.d_ff, "E": s.E, "G": s.G,
-                       "r": s.r, "k": s.k, "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": "flushed between steps by a 256 MB write outside the per-step CUDA events",
-                       "timing": "sum of per-step CUDA-event intervals on the launch stream",
-                       "path": int(res["info"].path),
-                       "active_clusters": res["active_clusters"], "active_experts": res["active_experts"],
-                       "expert_load_cov": res["i_load"]},
+            "config": config_of(args.workload, s, T, world),
+            "run": {"l2": "flushed between steps by a 256 MB write outside the per-step CUDA events",
+                    "timing": "sum of per-step CUDA-event intervals on the launch stream",
+                    "path": int(res["info"].path), "launches_per_forward": int(res["info"].launches_forward),
+                    "active_clusters": res["active_clusters"], "active_experts": res["active_experts"],
+                    "expert_load_cov": res["i_load"]},
             "clocks": res["clocks"],
             "e2e": {"value": world * T / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": res["e2e"]["h2d_bytes_per_step"],
                     "d2h_bytes_per_step": res["e2e"]["d2h_bytes_per_step"], "ms_per_step": e2e_ms},
             "gpu_launches": int(res["info"].launches_forward) * steps,
             "roofline": roof,
-            "layer": whole_layer_fractions(res, world),
+            "layer": whole_layer_fractions(res, world, peaks),
+            "sustained": res["sustained"],
             "stage_ms": res["stage_ms"],
             "wall_ms_per_step_incl_flush": res["wall_s"] / steps * 1e3,
         }
-        if args.all:
-            others = {}
-            for name in inputs.CONFIG_ORDER:
-                if name == args.workload:
-                    continue
-                r2 = time_workload(name, max(5, steps // 3), 3, rank, 0, False, False, local_rank, sync_ranks=False)
-                ms2 = r2["dev_ms"] / r2["steps"]
-                others[name] = {"tokens_per_s": r2["T"] / (ms2 * 1e-3), "ms_per_step": ms2,
-                                "roofline": roofline_for(r2, peaks, kind), "layer": whole_layer_fractions(r2, 1),
-                                "stage_ms": r2["stage_ms"], "path": int(r2["info"].path),
-                                "active_clusters": r2["active_clusters"], "active_experts": r2["active_experts"]}
+        # the memory-bound target (decode) rides in every default line; --all adds the other workloads
+        extra = [n for n in inputs.CONFIG_ORDER if n != args.workload and (args.all or (n == "decode" and not args.no_decode))]
+        others = {}
+        for name in extra:
+            r2 = time_workload(name, max(10, steps // 3), 3, rank, 0, name == "decode", False, local_rank, sync_ranks=False,
+                               sustained_s=min(args.sustained, 1.0) if name == "decode" else 0.0)
+            ms2 = r2["dev_ms"] / r2["steps"]
+            others[name] = {"tokens_per_s": r2["T"] / (ms2 * 1e-3), "ms_per_step": ms2, "config": config_of(name, r2["shape"], r2["T"], 1),
+                            "roofline": roofline_for(r2, peaks, kind), "layer": whole_layer_fractions(r2, 1, peaks),
+                            "stage_ms": r2["stage_ms"], "path": int(r2["info"].path),
+                            "launches_per_forward": int(r2["info"].launches_forward),
+                            "active_clusters": r2["active_clusters"], "active_experts": r2["active_experts"]}
+            if r2["e2e"]:
+                others[name]["e2e_ms_per_step"] = r2["e2e"]["ms_per_step"]
+        if others:
             line["workloads"] = others
         if not args.no_cpu_baseline:
-            line["cpu_baseline"] = oracle_rate(args.workload)
+            line["cpu_baseline"], line["parity"] = oracle_rate(args.workload, gpu=res if res.get("y") is not None else None)
         print(json.dumps(line), flush=True)
     if world > 1:
         _dist.barrier()

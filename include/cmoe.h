@@ -13,6 +13,13 @@
  *             computed once per token and shared by the token's k experts (text after Eq. 7).
  *   combine   y = sum_{e in top-k} p_e GELU(x W1_e) W2_e, GELU(u) = u/2 (1 + erf(u / sqrt 2)).
  *
+ * Arithmetic.  Activations, bases and outputs are fp16, all products accumulate in fp32.  The paths for
+ * small batches (T_max <= 128) and the CUDA-core path evaluate GELU in the erf form in fp32.  The
+ * tensor-core path for large batches rounds h to fp16 and evaluates u/2 (1 + tanh(u (0.80015708 +
+ * 0.03470089 u^2))) in packed fp16 with the hardware tanh: the two coefficients are fitted to the erf
+ * form (largest deviation 2.7e-4, at |u| near 1.7), of the size of the fp16 rounding of the stored
+ * activation.  On every path max|y - y_exact| <= 1e-2 max|y_exact| + 1e-3 for the layer as defined above.
+ *
  * Conventions
  *   - Every pointer below is a DEVICE pointer on the current CUDA device unless it says "host".
  *   - All arrays are dense, row-major, last index fastest.  fp16 values are IEEE binary16 bits.
@@ -21,9 +28,13 @@
  *     cmoe_workspace_bytes() says how large it must be for a descriptor.
  *   - Every function returns CMOE_OK (0) or a negative cmoe_error; nothing throws or aborts.
  *     Argument errors are found on the host before anything is launched.
- *   - cmoe_route / cmoe_forward are asynchronous on the given stream, issue only kernel launches and
- *     cudaMemsetAsync on it, never synchronise, and touch only the arena and the given outputs.
- *     They are not re-entrant on one handle (the arena holds the call's scratch).
+ *   - cmoe_route / cmoe_forward are asynchronous on the given stream, issue only kernel launches (no
+ *     memsets, no copies), never synchronise, and touch only the arena and the given outputs.
+ *     For handles with T_max <= 128 and r > 0, cmoe_forward forks two of its kernels onto a second
+ *     stream that the handle owns and joins them back with two events (created with the handle): the
+ *     work is complete when the given stream reaches the end of the call, as for any other call.
+ *     They are not re-entrant on one handle (the arena holds the call's scratch, and the handle's second
+ *     stream and events serve one call at a time): use one handle per concurrent caller.
  */
 #ifndef CMOE_H
 #define CMOE_H
@@ -84,12 +95,24 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes);
  * default stream and waits for them; work queued by the caller on other non-blocking streams that
  * produces the weights must have finished.  After it returns the source weight buffers may be
  * freed; the arena must outlive the handle and must not be written by the caller. */
-/* Three environment variables, read by cmoe_create, exist for A/B measurements: CMOE_FORCE_PATH=0 keeps
- * the generic CUDA-core path for every shape; CMOE_ROUTER_FP32=1 keeps batches of 1024 tokens and more
- * on the fp32 CUDA-core router instead of the tensor-core router (split fp16 router matrices, logit
- * error about 1e-6); CMOE_UP_TILE=128 keeps the up projection of large batches on 128-column tiles
- * where d_ff would allow 256-column tiles. */
 int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
+
+/* cmoe_create with kernel-selection switches for A/B measurements and tests (NULL options = cmoe_create).
+ * Results stay within the same tolerances whatever is chosen; only speed changes.
+ *   force_path   -1 automatic (default); 0 keeps the generic CUDA-core path for every shape
+ *   router_fp32   1 keeps batches of 1024 tokens and more on the fp32 CUDA-core router instead of the
+ *                 tensor-core router (which splits the fp32 router matrices into two fp16 pieces; logit error
+ *                 about 1e-6)
+ *   up_tile       0 automatic; 128 keeps the up projection of large batches on 128-column tiles where d_ff
+ *                 would allow 256-column tiles
+ * Other values: CMOE_ERR_INVALID_ARG.  reserved must be zero. */
+typedef struct {
+  int32_t force_path;
+  int32_t router_fp32;
+  int32_t up_tile;
+  int32_t reserved[5];
+} cmoe_options;
+int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
 
 /* Two-stage routing only (Sec. 3.3, Eq. 9-10) for x = fp16 [T][d]:
  *   cluster_id [T]     chosen cluster g*
@@ -120,6 +143,28 @@ int cmoe_forward_host(cmoe_layer* layer, const void* x_host, int32_t T, void* y_
  * CMOE_ERR_TIMEOUT if a bounded wait inside a kernel gave up (the output of that call is then
  * undefined; the handle stays usable and the word is cleared). */
 int cmoe_status(cmoe_layer* layer, void* cuda_stream);
+
+/* Test hook for the error path of the bounded device waits.  Every wait inside the kernels (on an mbarrier
+ * fed by TMA, by the tensor cores or by another warp) gives up after a cycle limit, records
+ * CMOE_ERR_TIMEOUT in the handle's status word and lets the kernel return normally.  This call launches a
+ * one-block kernel that waits, with the same primitive and a limit of limit_cycles SM clocks (1 .. 2^31),
+ * on a barrier nothing ever arrives on: it returns after about limit_cycles, nothing faults, and the next
+ * cmoe_status reports CMOE_ERR_TIMEOUT once.  Asynchronous on the given stream. */
+int cmoe_selftest_wait_timeout(cmoe_layer* layer, int64_t limit_cycles, void* cuda_stream);
+
+/* By-products of routing that the training-side clustering consumes (Sec. 3.1, Eq. 5; Sec. 4.1's expert load
+ * balance), for x = fp16 [T][d].  Routes x with the same kernels as cmoe_route and writes
+ *   loads   [E]     int32  tokens routed to each expert slot (sum = k*T)
+ *   xbar    [E][d]  fp32   mean of the tokens routed to the expert (Eq. 5's x-bar_i); rows of experts without
+ *                          tokens are zero.  May be NULL.
+ *   mu      [E][d]  fp32   in/out, or NULL: activation centroids, updated in place by Eq. 5,
+ *                          mu_i <- (1 - beta) mu_i + beta xbar_i, unchanged for experts without tokens
+ *   cov     [1]     fp32   coefficient of variation of the loads, population standard deviation / mean.  May be NULL.
+ * All four are device pointers.  Uses the handle's scratch like cmoe_route / cmoe_forward (not re-entrant
+ * with them); asynchronous on the given stream; 0 <= T <= T_max (T == 0: loads, xbar, cov are zeroed, mu
+ * untouched). */
+int cmoe_expert_stats(cmoe_layer* layer, const void* x, int32_t T, int32_t* loads, float* xbar,
+                      float* mu, float beta, float* cov, void* cuda_stream);
 
 /* Per-handle facts for tests and benchmarks (host struct, filled by cmoe_get_info). */
 typedef struct {

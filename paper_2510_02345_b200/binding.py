@@ -20,7 +20,7 @@ ERRORS = {
     -1: "CMOE_ERR_INVALID_ARG", -2: "CMOE_ERR_UNSUPPORTED_SHAPE", -3: "CMOE_ERR_WORKSPACE_TOO_SMALL",
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
-EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
+EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
            "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
 CMOE_MAX_STAGES = 8
@@ -37,6 +37,10 @@ class cmoe_desc(C.Structure):
         (n, C.c_void_p) for n in ("C", "R", "b_c", "b_e", "B1", "B2", "U1q", "V1q", "U2q", "V2q",
                                   "U1s", "V1s", "U2s", "V2s", "expert_global_id", "workspace")
     ] + [("workspace_bytes", C.c_size_t)]
+
+
+class cmoe_options(C.Structure):
+    _fields_ = [("force_path", C.c_int32), ("router_fp32", C.c_int32), ("up_tile", C.c_int32), ("reserved", C.c_int32 * 5)]
 
 
 class cmoe_info(C.Structure):
@@ -58,6 +62,10 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.cmoe_workspace_bytes.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_size_t)]
         L.cmoe_create.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_void_p)]
+        L.cmoe_create_ex.argtypes = [C.POINTER(cmoe_desc), C.POINTER(cmoe_options), C.POINTER(C.c_void_p)]
+        L.cmoe_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
+        L.cmoe_expert_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
+                                        C.c_void_p, C.c_void_p]
         L.cmoe_route.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.cmoe_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.cmoe_forward_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -99,6 +107,21 @@ def cmoe_create(desc: cmoe_desc) -> C.c_void_p:
     handle = C.c_void_p()
     _check(lib().cmoe_create(C.byref(desc), C.byref(handle)), "cmoe_create")
     return handle
+
+
+def cmoe_create_ex(desc: cmoe_desc, options: "cmoe_options | None") -> C.c_void_p:
+    handle = C.c_void_p()
+    _check(lib().cmoe_create_ex(C.byref(desc), C.byref(options) if options is not None else None, C.byref(handle)),
+           "cmoe_create_ex")
+    return handle
+
+
+def cmoe_selftest_wait_timeout(handle, limit_cycles: int, stream: int):
+    _check(lib().cmoe_selftest_wait_timeout(handle, limit_cycles, stream), "cmoe_selftest_wait_timeout")
+
+
+def cmoe_expert_stats(handle, x_ptr: int, T: int, loads_ptr: int, xbar_ptr, mu_ptr, beta: float, cov_ptr, stream: int):
+    _check(lib().cmoe_expert_stats(handle, x_ptr, T, loads_ptr, xbar_ptr, mu_ptr, beta, cov_ptr, stream), "cmoe_expert_stats")
 
 
 def cmoe_route(handle, x_ptr: int, T: int, cluster_id_ptr: int, expert_ids_ptr: int, gates_ptr: int, stream: int):
@@ -160,7 +183,11 @@ class ClusteredMoELayer:
                   ("U1s", np.float16), ("V1s", np.float16), ("U2s", np.float16), ("V2s", np.float16),
                   ("expert_global_id", np.int32))
 
-    def __init__(self, layer: dict, T_max: int | None = None, device: str = "cuda:0", keep_source: bool = False):
+    def __init__(self, layer: dict, T_max: int | None = None, device: str = "cuda:0", keep_source: bool = False,
+                 options: dict | None = None, guard_bytes: int = 0, fill_byte: int | None = None):
+        """`options`: fields of cmoe_options (force_path, router_fp32, up_tile) for cmoe_create_ex.
+        `guard_bytes` / `fill_byte` (tests): the arena is allocated with that many bytes of a canary pattern
+        before and after it, and filled with `fill_byte` before the library sees it."""
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
@@ -182,12 +209,28 @@ class ClusteredMoELayer:
         for name, _ in self._NP_FIELDS:
             setattr(desc, name, None if src[name] is None else src[name].data_ptr())
         nbytes = cmoe_workspace_bytes(desc)
-        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
-        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        guard = (int(guard_bytes) + 255) // 256 * 256
+        self.workspace = torch.empty(nbytes + 256 + 2 * guard, dtype=torch.uint8, device=self.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256 + guard
+        off = base - self.workspace.data_ptr()
+        if fill_byte is not None:
+            self.workspace[off:off + nbytes] = int(fill_byte)
+        self._guards = None
+        if guard:
+            self._guards = (self.workspace[off - guard:off], self.workspace[off + nbytes:off + nbytes + guard])
+            for gbuf in self._guards:
+                gbuf.fill_(0xA5)
         desc.workspace, desc.workspace_bytes = base, nbytes
         self.workspace_bytes = nbytes
         torch.cuda.synchronize(self.device)
-        self.handle = cmoe_create(desc)
+        if options:
+            o = cmoe_options()
+            o.force_path = -1
+            for key, val in options.items():
+                setattr(o, key, int(val))
+            self.handle = cmoe_create_ex(desc, o)
+        else:
+            self.handle = cmoe_create(desc)
         self.info = cmoe_get_info(self.handle)
         self._src = src if keep_source else None   # the library holds its own copies in the arena
 
@@ -227,6 +270,24 @@ class ClusteredMoELayer:
         cmoe_forward_host(self.handle, x_host.data_ptr(), T, y.data_ptr(), self._stage[0].data_ptr(),
                           self._stage[1].data_ptr(), self._stream())
         return y
+
+    def expert_stats(self, x, mu=None, beta: float = 0.05):
+        """loads [E] int32, xbar [E][d] fp32, cov (0-d fp32) of routing x; `mu` ([E][d] fp32) is updated in place by Eq. 5."""
+        import torch
+        s = self.shape
+        assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.shape[1] == s.d
+        loads = torch.empty(s.E, dtype=torch.int32, device=x.device)
+        xbar = torch.empty((s.E, s.d), dtype=torch.float32, device=x.device)
+        cov = torch.empty((), dtype=torch.float32, device=x.device)
+        if mu is not None:
+            assert mu.is_cuda and mu.dtype == torch.float32 and mu.is_contiguous() and tuple(mu.shape) == (s.E, s.d)
+        cmoe_expert_stats(self.handle, x.data_ptr(), x.shape[0], loads.data_ptr(), xbar.data_ptr(),
+                          None if mu is None else mu.data_ptr(), beta, cov.data_ptr(), self._stream())
+        return loads, xbar, cov
+
+    def guards_intact(self) -> bool:
+        """True if the canary bytes around the arena (guard_bytes) still hold their pattern."""
+        return self._guards is None or all(bool((gbuf == 0xA5).all()) for gbuf in self._guards)
 
     def status(self) -> int:
         return cmoe_status(self.handle, self._stream())

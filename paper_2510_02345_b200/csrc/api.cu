@@ -6,6 +6,7 @@
 #include "cmoe_internal.h"
 #include "stage_factors.cuh"
 #include "lowrank.cuh"
+#include "perm_keys.cuh"
 
 using namespace cmoe;
 
@@ -64,7 +65,7 @@ int validate_dims(const cmoe_desc* desc, Dims* D) {
 void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r, k = D.k;
   const size_t T = D.T_max, P = D.T_pad_max;
-  const size_t nblk = (T + kPermBlock - 1) / kPermBlock;
+  const size_t nblk = (T + kMinCountTile - 1) / kMinCountTile;
   Weights w{};
   Scratch s{};
   w.Ct = A.take<float>(G * d);
@@ -155,7 +156,9 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) {
   return CMOE_OK;
 }
 
-int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
+int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) { return cmoe_create_ex(desc, nullptr, out_layer); }
+
+int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** out_layer) {
   if (!out_layer) return CMOE_ERR_INVALID_ARG;
   *out_layer = nullptr;
   Dims D{};
@@ -173,9 +176,19 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   cmoe_workspace_bytes(desc, &need);
   if (desc->workspace_bytes < need) return CMOE_ERR_WORKSPACE_TOO_SMALL;
 
+  cmoe_options o{};
+  o.force_path = -1;
+  if (opt) o = *opt;
+  if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256)) return CMOE_ERR_INVALID_ARG;
+  {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return CMOE_ERR_CUDA;
+  }
   cmoe_layer* L = new (std::nothrow) cmoe_layer();
   if (!L) return CMOE_ERR_INVALID_ARG;
   L->dims = D;
+  L->opt = o;
   L->path = kPathGeneric;
   L->last_cuda_error = 0;
   L->profiling = 0;
@@ -256,9 +269,8 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
   if ((e = cudaMemsetAsync(L->sc.status, 0, sizeof(int), st))) return fail(e);
   if ((e = cudaStreamSynchronize(st))) return fail(e);
   // path choice: tensor-core grouped GEMMs when the shape allows and there are enough tokens to
-  // fill 128-row tiles; CMOE_FORCE_PATH=0 keeps the generic path (for A/B checks)
-  const char* force = std::getenv("CMOE_FORCE_PATH");
-  const int forced = force ? std::atoi(force) : -1;
+  // fill 128-row tiles; cmoe_options.force_path = 0 keeps the generic path (for A/B checks)
+  const int forced = o.force_path;
   L->tc_variant = 0;
   if (D.tc2 && forced != kPathGeneric) {
     if ((e = tc2_init(L))) return fail(e);
@@ -273,7 +285,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer) {
     L->tc_variant = 1;
   }
   L->router_tc = 0;
-  if (router_tc_supported(D) && !std::getenv("CMOE_ROUTER_FP32")) {
+  if (router_tc_supported(D) && !o.router_fp32) {
     if ((e = router_tc_init(L))) return fail(e);
     L->router_tc = 1;
   }
@@ -312,24 +324,30 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     ++stage;                                                               \
   } while (0)
   CMOE_MARK();
-  if (L->router_tc && T >= 1024)
-    CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
-  else
-    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  FactorStage fs{};                     // nothing to stage unless the pair path has residual factors
+  if (L->path == kPathTensor && L->tc_variant == 2) tc2_factor_stage(L, &fs);
+  // batches of at least 1024 tokens: the router counts the permutation keys of its token tiles as it goes
+  KeyCount kc{};
+  kc.keys = S.keys; kc.block_counts = S.block_counts; kc.nsub = D.nsub; kc.nkey = D.nkey; kc.sub_is_combo = D.sub_is_combo;
+  int counted_tile = 0;
+  if (L->router_tc && T >= 1024) {
+    CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc));
+    counted_tile = router_tc_tile_tokens();
+  } else {
+    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc, &fs));
+    counted_tile = router_tile_tokens(T);
+  }
+  if (T < 1024) fs = FactorStage{};     // staged beside the per-token router
   CMOE_MARK();
   {
     // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s
     const size_t rows = (size_t)t_pad_bound(D, T);
     void* zp = L->path == kPathStream ? static_cast<void*>(S.y32) : static_cast<void*>(S.s);
     size_t zb = L->path == kPathStream ? sizeof(float) * rows * D.d : sizeof(float) * rows * D.k * D.r;
-    FactorStage fs{};                     // nothing to stage unless the pair path has residual factors
-    if (L->path == kPathTensor && L->tc_variant == 2) {
-      tc2_accum_buffer(L, T, &zp, &zb);
-      tc2_factor_stage(L, &fs);
-    }
+    if (L->path == kPathTensor && L->tc_variant == 2) tc2_accum_buffer(L, T, &zp, &zb);
     LowrankTok lr{};                      // nothing rides along unless the streaming path has residual factors
     if (L->path == kPathStream) stream_lowrank_rider(L, xh, T, &lr);
-    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs, lr));
+    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs, lr, counted_tile));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));

@@ -17,7 +17,8 @@ constexpr int kMaxK = 32;          // experts per cluster (one lane each in the 
 constexpr int kMaxKsel = 8;        // k
 constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
 constexpr int kMaxHostChunks = 4; // pipeline depth of cmoe_forward_host
-constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels
+constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels (when they count the keys themselves)
+constexpr int kMinCountTile = 64;  // smallest token tile of a router kernel that counts keys
 
 enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
 
@@ -31,6 +32,7 @@ struct Dims {
   int sub_is_combo;
   int tc2;         // the shape takes the tensor-core path with tensor-core residuals (tc2_path.cu)
   int stream;      // the shape takes the weight-streaming path (stream_path.cu)
+  int sm_count;    // multiprocessors of the handle's device (set by cmoe_create; 0 in pure host queries)
 };
 
 // Weights as re-laid-out in the arena by cmoe_create.
@@ -88,6 +90,7 @@ struct cmoe_layer {
   cmoe::Dims dims;
   cmoe::Weights w;
   cmoe::Scratch sc;
+  cmoe_options opt;  // what cmoe_create_ex was given (defaults otherwise)
   int path;
   int tc_variant;   // 1: tc_path.cu, 2: tc2_path.cu (when path == kPathTensor)
   int router_tc;    // batches of at least 1024 tokens are routed by router_tc.cu
@@ -120,23 +123,30 @@ inline int t_pad_bound(const Dims& D, int T) { return round_up(T, D.row_align) +
 
 // ---- launchers (each returns the cudaError_t of its launches) ----------------------------------
 // router.cu
+// kc (or null): the kernel also writes every token's permutation key and, for batches of at least 1024 tokens, the
+// key counts of its token tiles (router_tile_tokens(T) tokens each; 0: it counts nothing).  fs (or null): factor
+// staging that rides in the per-token kernel's grid (batches below 1024 tokens).
+struct KeyCount;      // perm_keys.cuh
+struct FactorStage;   // stage_factors.cuh
+struct LowrankTok;    // lowrank.cuh
 cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int T,
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
-                          cudaStream_t st);
+                          cudaStream_t st, const KeyCount* kc = nullptr, const FactorStage* fs = nullptr);
+int router_tile_tokens(int T);
 // router_tc.cu : the same routing on the tensor cores (split fp16 router matrices), for large batches
 int router_tc_rp(const Dims& D);
 bool router_tc_supported(const Dims& D);
 cudaError_t router_tc_init(cmoe_layer* L);
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
-                             int* slot_local, cudaStream_t st);
+                             int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr);
+int router_tc_tile_tokens();
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
-struct FactorStage;   // stage_factors.cuh
-struct LowrankTok;    // lowrank.cuh
+// counted_tile > 0: the router kernel has already written the keys and the key counts of its tiles of that many tokens
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr);
-constexpr int kPermuteLaunches = 4;        // 2 for batches of at most 256 tokens (permute_launches)
-inline int permute_launches(int T) { return T <= 256 ? 2 : kPermuteLaunches; }
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile);
+// kernels of the permutation: 2 for batches of at most 256 tokens, 4 below 1024 tokens, else 3 (the router counts the keys)
+inline int permute_launches(int T) { return T <= 256 ? 2 : (T < 1024 ? 4 : 3); }
 // generic_path.cu : CUDA-core path for any supported shape
 // `marks` (or null): three events recorded before the residual-t, up and down stages
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,

@@ -192,7 +192,8 @@ cudaError_t launch_residual_t(const Dims& D, const Weights& W, const Scratch& S,
   if (D.r <= 0) return cudaSuccess;
   const int rows_bound = t_pad_bound(D, T);
   int blocks = (rows_bound * D.k + 7) / 8;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  const int cap = (D.sm_count > 0 ? D.sm_count : 148) * 16;      // grid-stride loop: a few resident rounds
+  if (blocks > cap) blocks = cap;
   launch_chained(residual_t_kernel, dim3(blocks), dim3(256), 0, st, 1,
       D.d, D.k, D.r, S.n_rows, S.x_perm, S.row_slot, W.U1q,
                                             W.U1s, S.t);

@@ -5,9 +5,27 @@
 // dozen short kernels of one forward.
 #pragma once
 
+#include <atomic>
+
 #include <cuda_runtime.h>
 
 namespace cmoe {
+
+// The dynamic shared-memory limit of a kernel is a per-device attribute: `done` is the calling site's record
+// (one bit per device ordinal) of the devices it has been set on.  The current device is the one the launch
+// that follows goes to.
+template <typename Kern>
+inline cudaError_t ensure_dynamic_smem(Kern kern, size_t bytes, std::atomic<unsigned long long>& done) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  const unsigned long long bit = 1ull << (dev & 63);
+  if (done.load(std::memory_order_relaxed) & bit) return cudaSuccess;
+  e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e != cudaSuccess) return e;
+  done.fetch_or(bit, std::memory_order_relaxed);
+  return cudaSuccess;
+}
 
 // Blocks until the kernels this one depends on have completed (a no-op for an ordinary launch).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -3,8 +3,9 @@
 // never straddle two clusters.  The paper only implies this step ("tokens are assigned to a
 // cluster, then to experts inside it", Sec. 3.3); the mechanism is this library's.
 //
-//   hist     per-block histogram of the keys (block = 256 consecutive tokens)
-//   scan     block 0: per-key running sums over blocks, cluster segment offsets, tile table, and the
+//   hist     per-block histogram of the keys (block = 256 consecutive tokens); for batches of 1024 tokens and
+//            more the router kernel has counted the keys of its token tiles itself and this kernel is not launched
+//   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table, and the
 //            table entries of the padding rows of each segment (no token, zero gates)
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
 //            writes the row tables
@@ -17,41 +18,11 @@
 #include "device_utils.cuh"
 #include "stage_factors.cuh"
 #include "lowrank.cuh"
+#include "perm_keys.cuh"
 
 namespace cmoe {
 
 namespace {
-
-__device__ __forceinline__ int binom(int n, int m) {
-  if (m > n) return 0;
-  long long r = 1;
-  for (int i = 1; i <= m; ++i) r = r * (n - m + i) / i;
-  return (int)r;
-}
-
-// Sort the token's k local expert indices ascending (gates follow) and return the sub-key.
-__device__ __forceinline__ int canonical_slots(const int* __restrict__ slot, const float* __restrict__ gate,
-                                               int k, int sub_is_combo, int* cs, float* cg) {
-#pragma unroll
-  for (int j = 0; j < kMaxKsel; ++j)
-    if (j < k) { cs[j] = slot[j]; cg[j] = gate[j]; }
-#pragma unroll
-  for (int a = 1; a < kMaxKsel; ++a)
-    if (a < k) {
-#pragma unroll
-      for (int b = kMaxKsel - 1; b > 0; --b)
-        if (b <= a && cs[b] < cs[b - 1]) {
-          int ti = cs[b]; cs[b] = cs[b - 1]; cs[b - 1] = ti;
-          float tg = cg[b]; cg[b] = cg[b - 1]; cg[b - 1] = tg;
-        }
-    }
-  if (!sub_is_combo) return cs[0];
-  int rank = 0;                    // combinatorial number system: sum_i C(c_i, i+1)
-#pragma unroll
-  for (int j = 0; j < kMaxKsel; ++j)
-    if (j < k) rank += binom(cs[j], j + 1);
-  return rank;
-}
 
 __global__ void __launch_bounds__(kPermBlock)
 hist_kernel(int T, int k, int nsub, int nkey, int sub_is_combo,
@@ -80,12 +51,8 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
             const int* __restrict__ block_counts, int* __restrict__ block_base,
             int* __restrict__ key_cnt, int* __restrict__ key_off, int* __restrict__ seg_off,
             int* __restrict__ seg_cnt, int* __restrict__ n_rows, int* __restrict__ tile_cluster, int K, int k,
-            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
-            const FactorStage fs) {
+            int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate) {
   pdl_wait();
-  // blocks 1.. decode the layer's INT4 factors for the tensor-core residual products (weights only:
-  // independent of the scan, which is one block of latency)
-  if (blockIdx.x > 0) { stage_block(fs, blockIdx.x - 1); return; }
   __shared__ int sh_seg[kMaxG + 1];
   __shared__ int sh_segcnt[kMaxG];
   __shared__ int sh_cnt[kMaxKeys];
@@ -150,21 +117,24 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
   }
 }
 
-__global__ void __launch_bounds__(kPermBlock)
+__global__ void __launch_bounds__(kPermBlock)      // 64, 128 or 256 threads: the token tile of the kernel that counted the keys
 scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
                const __half* __restrict__ x, const int* __restrict__ cluster_id,
                const int* __restrict__ slot, const float* __restrict__ gates,
                const int* __restrict__ keys, const int* __restrict__ block_base,
                const int* __restrict__ key_off,
                int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
-               __half* __restrict__ x_perm) {
+               __half* __restrict__ x_perm, int nblk, const FactorStage fs) {
   pdl_wait();
+  // blocks nblk.. decode the layer's INT4 factors for the tensor-core residual products (weights only: they
+  // fill the SMs beside the few, latency-bound scatter blocks)
+  if ((int)blockIdx.x >= nblk) { stage_block(fs, blockIdx.x - nblk); return; }
   extern __shared__ int sh_next[];   // next free row of each key for this block
   for (int i = threadIdx.x; i < nkey; i += blockDim.x)
     sh_next[i] = key_off[i] + block_base[(size_t)blockIdx.x * nkey + i];
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.x * kPermBlock + threadIdx.x;
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;        // a block takes the tokens one counting block took
   const bool live = t < T;
   const int key = live ? keys[t] : -1 - lane;     // dead lanes get unique keys: groups of one
   const unsigned peers = __match_any_sync(0xffffffffu, key);
@@ -172,7 +142,7 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
   const bool leader = rank_in_warp == 0;
   int row = -1;
   // warps take their rows in warp order, so rows of a key stay in token order
-  for (int w = 0; w < kPermBlock / 32; ++w) {
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
     if (warp == w && live) {
       row = sh_next[key] + rank_in_warp;
     }
@@ -305,22 +275,14 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
   }
 }
 
-// the factor staging alone (batches of at most 256 tokens)
-__global__ void __launch_bounds__(256)
-stage_only_kernel(const FactorStage fs) {
-  pdl_wait();
-  stage_block(fs, blockIdx.x);
-}
-
 }  // namespace
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr) {
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile) {
 
   const int rows_bound = t_pad_bound(D, T);
   if (T <= kSmallT) {
-    // (one block of a few microseconds: the factor staging would not hide in it and has its own launch)
-    if (const int extra = stage_blocks(fs, 256)) launch_chained(stage_only_kernel, dim3(extra), dim3(256), 0, st, 1, fs);
+    // (the factor staging rode in the router kernel)
     launch_chained(permute_small_kernel, dim3(1 + lowrank_tok_blocks(lr)), dim3(kSmallT), sizeof(int) * ((size_t)D.nkey + kSmallT), st, 1,
       
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
@@ -329,21 +291,26 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
       D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
     return cudaGetLastError();
   }
-  const int nblk = (T + kPermBlock - 1) / kPermBlock;
+  // counting blocks: the router's token tiles when it counted the keys itself (counted_tile tokens each), else
+  // blocks of 256 tokens counted here
+  const int tile = counted_tile > 0 ? counted_tile : kPermBlock;
+  const int nblk = (T + tile - 1) / tile;
   const size_t sh = sizeof(int) * (size_t)D.nkey;
-  launch_chained(hist_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
-      T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
-                                            S.slot, S.gates, S.keys, S.block_counts);
-  launch_chained(scan_kernel, dim3(1 + stage_blocks(fs, 1024)), dim3(1024), 0, st, 1,
+  if (counted_tile <= 0)
+    launch_chained(hist_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
+        T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
+                                              S.slot, S.gates, S.keys, S.block_counts);
+  launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
       nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
                                   S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
-                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate, fs);
-  launch_chained(scatter_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
+                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
+  launch_chained(scatter_kernel, dim3(nblk + stage_blocks(fs, tile)), dim3(tile), sh, st, 1,
       T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
-                                               S.x_perm);
-  const int move_grid = rows_bound < 148 * 32 ? rows_bound : 148 * 32;
+                                               S.x_perm, nblk, fs);
+  const int move_max = (D.sm_count > 0 ? D.sm_count : 148) * 32;      // resident blocks of 128 threads
+  const int move_grid = rows_bound < move_max ? rows_bound : move_max;
   launch_chained(move_rows_kernel, dim3(move_grid), dim3(128), 0, st, 1,
       D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
   return cudaGetLastError();

@@ -14,6 +14,7 @@
 #include "device_utils.cuh"
 #include "launch.cuh"
 #include "tc_ptx.cuh"
+#include "perm_keys.cuh"
 
 namespace cmoe {
 
@@ -37,6 +38,7 @@ struct RtcParams {
   float* gates;
   int* slot_local;
   int* status;
+  KeyCount kc;     // key counting for the permutation (keys == nullptr: routing only)
 };
 
 // fp32 router rows -> the two fp16 pieces, rows [hi_0 .. hi_{rp-1}, lo_0 .. lo_{rp-1}] x d (padding rows zero)
@@ -70,6 +72,8 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 17);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   float* lg = reinterpret_cast<float*>(sm);              // [128][N + 1] logits, reusing the operand ring after the main loop
+  int* key_of = reinterpret_cast<int*>(lg + (size_t)RBM * (N + 1));   // [128] keys of the tile's tokens, then [nkey] counts
+  int* cnt = key_of + RBM;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x;
   const int KC = p.d / (RBK * RKA);
@@ -128,6 +132,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
     const int trow = q * 32 + lane;
     const int tok = tile * RBM + trow;
     const bool ok = mbar_wait(tfull, 0, abort_flag);
+    int key = -1;
     if (__all_sync(0xffffffffu, ok)) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -172,14 +177,22 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         float sum = 0.f;
         for (int s = 0; s < p.k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
         for (int s = 0; s < p.k; ++s) {
-          if (p.gates) p.gates[(size_t)tok * p.k + s] = ev[s] / sum;
+          ev[s] = ev[s] / sum;
+          if (p.gates) p.gates[(size_t)tok * p.k + s] = ev[s];
           if (p.expert_ids) p.expert_ids[(size_t)tok * p.k + s] = p.label[gs * K + seli[s]];
           if (p.slot_local) p.slot_local[(size_t)tok * p.k + s] = seli[s];
+        }
+        if (p.kc.keys) {
+          int cs[kMaxKsel];
+          float cg[kMaxKsel];
+          key = gs * p.kc.nsub + canonical_slots(seli, ev, p.k, p.kc.sub_is_combo, cs, cg);
+          p.kc.keys[tok] = key;
         }
       }
     } else {
       failed = true;
     }
+    if (p.kc.keys) key_of[trow] = key;       // (its own logits row is no longer read; the key table lies past all rows)
     tc_fence_before();
   }
 
@@ -196,6 +209,14 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   tc_fence_after();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+  if (p.kc.keys) {
+    // keys of this tile counted in shared memory: the permutation's histogram, for free
+    for (int i = threadIdx.x; i < p.kc.nkey; i += blockDim.x) cnt[i] = 0;
+    __syncthreads();
+    if (threadIdx.x < RBM && key_of[threadIdx.x] >= 0) atomicAdd(&cnt[key_of[threadIdx.x]], 1);
+    __syncthreads();
+    for (int i = threadIdx.x; i < p.kc.nkey; i += blockDim.x) p.kc.block_counts[(size_t)tile * p.kc.nkey + i] = cnt[i];
+  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -231,7 +252,7 @@ bool make_map3(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
 
 size_t rtc_smem(int N) {
   const size_t ring = (size_t)R_STAGES * RKA * (RBM + N) * RBK * 2;
-  const size_t logits = (size_t)RBM * (N + 1) * 4;
+  const size_t logits = (size_t)RBM * (N + 1) * 4 + (size_t)(RBM + kMaxKeys) * 4;   // logits, keys of the tile, key counts
   return 1024 + (ring > logits ? ring : logits) + 32 * 8;
 }
 
@@ -257,8 +278,10 @@ cudaError_t router_tc_init(cmoe_layer* L) {
   return cudaDeviceSynchronize();
 }
 
+int router_tc_tile_tokens() { return RBM; }
+
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
-                             int* slot_local, cudaStream_t st) {
+                             int* slot_local, cudaStream_t st, const KeyCount* kc) {
   const Dims& D = L->dims;
   CUtensorMap mx;
   if (!make_map3(&mx, x, (uint64_t)T, D.d, RBM)) return cudaErrorInvalidValue;   // x is the caller's buffer: a map per call
@@ -266,6 +289,7 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
   p.T = T; p.d = D.d; p.G = D.G; p.K = D.K; p.k = D.k; p.E = D.E; p.rp = router_tc_rp(D);
   p.bc = L->w.bc; p.be = L->w.be; p.label = L->w.label;
   p.cluster_id = cluster_id; p.expert_ids = expert_ids; p.gates = gates; p.slot_local = slot_local; p.status = L->sc.status;
+  if (kc) p.kc = *kc;
   return launch_chained(router_tc_kernel, dim3((unsigned)((T + RBM - 1) / RBM)), dim3(R_THREADS), rtc_smem(2 * p.rp), st, 1, mx,
                         L->router_map_w, p);
 }

@@ -472,12 +472,8 @@ cudaError_t launch_stream(const CUtensorMap& mW, const SliceMaps& mWs, const CUt
   auto kern = stream_kernel<UP>;
   constexpr size_t sm = SCfg<128>::SMEM;
   static_assert(sm <= 232448, "stream kernel shared memory");
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   launch_chained(kern, dim3(grid), dim3(S_THREADS), sm, st, 1,
       mW, mWs, mTok, p);
   return cudaGetLastError();

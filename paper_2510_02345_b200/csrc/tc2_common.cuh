@@ -66,11 +66,6 @@ struct Up2Params {
                        // end and the gated rows p_j s_j go straight into the down kernel's operand (zeroed by the caller)
 };
 
-template <typename Kern>
-inline cudaError_t set_smem(Kern kern, size_t bytes) {
-  return cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-}
-
 // launch as thread-block clusters of two CTAs (grid = 2 x pairs)
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pairs(void (*kern)(KArgs...), int grid, int threads, size_t smem, cudaStream_t st, Args... args) {

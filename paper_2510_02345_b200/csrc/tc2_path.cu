@@ -895,12 +895,8 @@ cudaError_t launch_up(const Tc2State& ts, const Up2Params& p, int grid, cudaStre
   auto kern = tc2_up_kernel<HAS_R, KSEL>;
   constexpr size_t sm = UpCfg<HAS_R, KSEL>::SMEM;
   static_assert(sm <= kSmemLimit, "up kernel shared memory");
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = set_smem(kern, sm);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   return launch_pairs(kern, grid, UP_THREADS, sm, st, ts.mX3, ts.mB13, ts.mA0, ts.mAd, ts.mV1, ts.mU2, p);
 }
 
@@ -909,12 +905,8 @@ cudaError_t launch_down(const Tc2State& ts, const Down2Params& p, int grid, cuda
   auto kern = tc2_down_kernel<BN, HAS_R>;
   constexpr size_t sm = DownCfg<BN, HAS_R>::SMEM;
   static_assert(sm <= kSmemLimit, "down kernel shared memory");
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = set_smem(kern, sm);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   return launch_pairs(kern, grid, DN_THREADS, sm, st, ts.mAbar3, ts.mB23, ts.mAs, ts.mV2, p);
 }
 
@@ -922,12 +914,8 @@ template <int KSEL>
 cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_t st) {
   auto kern = tc2_t_kernel<KSEL>;
   constexpr size_t sm = 1024 + (size_t)T_STAGES * T_STAGE_BYTES + 32 * 8;
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = set_smem(kern, sm);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   launch_chained(kern, dim3(grid), dim3(T_THREADS), sm, st, 1,
       ts.mX, ts.mU1, p);
   return cudaGetLastError();
@@ -985,16 +973,10 @@ cudaError_t tc2_init(cmoe_layer* L) {
   const Scratch& S = L->sc;
   Tc2State* ts = reinterpret_cast<Tc2State*>(L->tc_state);
   ts->bn_down = (D.d % 256 == 0) ? 256 : 128;
-  {
-    const char* tile = getenv("CMOE_UP_TILE");
-    ts->up_wide = (D.d_ff % BN_WIDE == 0 && !(tile && atoi(tile) == 128)) ? 1 : 0;
-  }
+  ts->up_wide = (D.d_ff % BN_WIDE == 0 && L->opt.up_tile != 128) ? 1 : 0;
   ts->log2r = D.r > 0 ? ilog2(D.r) : 0;
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
-  if (e != cudaSuccess) return e;
+  ts->sm_count = D.sm_count;
+  cudaError_t e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mX3, S.x_perm, P, D.d, BM) &&
@@ -1048,9 +1030,8 @@ int tc2_launch_count(const cmoe_layer* L) {
   const Dims& D = L->dims;
   if (D.r == 0) return 2;
   const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
-  // t, up, (expansion,) down; the staging rides in the permutation's scan kernel, except for batches of at most 256
-  // tokens, where it has a launch of its own
-  return (plan_up(ts, D, D.T_max).direct ? 3 : 4) + (D.T_max <= 256 ? 1 : 0);
+  // t, up, (expansion,) down; the factor staging rides in the router's or the permutation's grid
+  return plan_up(ts, D, D.T_max).direct ? 3 : 4;
 }
 
 // The buffer the forward's first kernels clear for this path: the fp32 sums s, or the down kernel's

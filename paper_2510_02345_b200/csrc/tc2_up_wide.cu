@@ -477,12 +477,8 @@ cudaError_t launch_w(const UpWideMaps& m, const Up2Params& p, int grid, cudaStre
   auto kern = tc2_up_wide_kernel<HAS_R, KSEL>;
   constexpr size_t sm = WideCfg<HAS_R, KSEL>::SMEM;
   static_assert(sm <= kSmemLimit, "wide up kernel shared memory");
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = set_smem(kern, sm);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   return launch_pairs(kern, grid, UW_THREADS, sm, st, *m.x3, *m.b13, *m.a0, *m.ad, *m.v1, *m.u2, p);
 }
 

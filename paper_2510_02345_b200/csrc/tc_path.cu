@@ -16,6 +16,7 @@
 #include <cuda.h>
 
 #include "cmoe_internal.h"
+#include "launch.cuh"
 #include "device_utils.cuh"
 
 namespace cmoe {
@@ -425,12 +426,8 @@ template <int BN, int R, int KSEL, bool UP>
 cudaError_t launch_one(const TcState& ts, const TcParams& p, int grid, cudaStream_t st) {
   auto kern = tc_ffn_kernel<BN, R, KSEL, UP>;
   const size_t sm = smem_bytes(BN, p.K, R, UP, p.stages);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
+  static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
+  if (cudaError_t e = ensure_dynamic_smem(kern, kSmemLimit, smem_set)) return e;
   kern<<<grid, kThreads, sm, st>>>(UP ? ts.mapA_up : ts.mapA_dn, UP ? ts.mapB_up : ts.mapB_dn, p);
   return cudaGetLastError();
 }

@@ -92,18 +92,6 @@ def quantize_int4(w: np.ndarray) -> tuple[np.ndarray, np.ndarray]:
     return packed, scale
 
 
-def unpack_codes(packed: np.ndarray) -> np.ndarray:
-    """Inverse of the nibble packing only (codes as int8, no scaling)."""
-    lo = (packed & 0xF).astype(np.int8)
-    hi = (packed >> 4).astype(np.int8)
-    lo = np.where(lo > 7, lo - 16, lo).astype(np.int8)
-    hi = np.where(hi > 7, hi - 16, hi).astype(np.int8)
-    out = np.empty(packed.size * 2, np.int8)
-    out[0::2] = lo
-    out[1::2] = hi
-    return out
-
-
 def zipf_shares(G: int, s: float = 1.2) -> np.ndarray:
     w = 1.0 / np.arange(1, G + 1, dtype=np.float64) ** s
     return w / w.sum()
@@ -128,7 +116,8 @@ def _calibrate_cluster_bias(x16: np.ndarray, C: np.ndarray, target: np.ndarray) 
     return b.astype(np.float32)
 
 
-def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None) -> dict:
+def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None, base_scale: float = 1.0,
+               factor_std: float = 0.02) -> dict:
     """Draw one layer and one token batch.
 
     Draw order (float32 standard normals from numpy PCG64(seed)):
@@ -136,7 +125,9 @@ def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None) -> dict:
     in the workload description is a standard deviation.
     Passing ``T`` overrides the number of tokens (x is drawn first, so the
     weights of a shape depend on T; use :func:`make_tokens` for extra batches
-    against fixed weights).
+    against fixed weights).  ``base_scale`` multiplies both shared bases (0 gives a layer whose experts
+    are their low-rank residuals alone) and ``factor_std`` replaces the 0.02 of the residual factors: test
+    layers in which the residual terms, a few percent of the activations in the workloads, dominate.
     """
     T = shape.T if T is None else T
     d, d_ff, E, G, r, k = shape.d, shape.d_ff, shape.E, shape.G, shape.r, shape.k
@@ -151,11 +142,11 @@ def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None) -> dict:
     x = normal((T, d), 1.0).astype(np.float16)
     C = normal((d, G), 0.02)
     R = normal((G, d, K), 0.02)
-    B1 = normal((G, d, d_ff), 1.0 / math.sqrt(d)).astype(np.float16)
-    B2 = normal((G, d_ff, d), 1.0 / math.sqrt(d_ff)).astype(np.float16)
+    B1 = normal((G, d, d_ff), base_scale / math.sqrt(d)).astype(np.float16)
+    B2 = normal((G, d_ff, d), base_scale / math.sqrt(d_ff)).astype(np.float16)
     out = dict(shape=shape, T=T, seed=seed, x=x, C=C, R=R, B1=B1, B2=B2, b_c=None, b_e=None)
     for name, dims in (("U1", (E, r, d)), ("V1", (E, d_ff, r)), ("U2", (E, r, d_ff)), ("V2", (E, d, r))):
-        w = normal(dims, 0.02)
+        w = normal(dims, factor_std)
         q, s = quantize_int4(w)
         out[name + "q"] = q
         out[name + "s"] = s

@@ -1,12 +1,12 @@
 """GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element on
-the same seeded inputs.  Small and ragged cases in full; the large workloads on all routes and on
-sampled output rows."""
+the same seeded inputs: all routes and every output row of the five workloads and of the small, ragged
+and degenerate cases (a few very large extra shapes on sampled rows)."""
 import numpy as np
 import pytest
 
 from oracle import ref
 from paper_2510_02345_b200 import inputs
-from parity import check_routes, check_y
+from parity import check_routes, check_y, compare
 
 pytestmark = pytest.mark.gpu
 
@@ -21,10 +21,10 @@ def layer_for(name, seed=0):
     return _cache[key]
 
 
-def run_gpu(L, x_np, T_max=None):
+def run_gpu(L, x_np, T_max=None, options=None):
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer
-    m = ClusteredMoELayer(L, T_max=T_max if T_max is not None else max(1, x_np.shape[0]))
+    m = ClusteredMoELayer(L, T_max=T_max if T_max is not None else max(1, x_np.shape[0]), options=options)
     x = torch.from_numpy(x_np).cuda()
     cid, eid, gates = m.route(x)
     y = m.forward(x)
@@ -35,20 +35,16 @@ def run_gpu(L, x_np, T_max=None):
     return out
 
 
-def full_check(L, x_np, sample=None, seed=0):
+def full_check(L, x_np, sample=None, seed=0, label=None, options=None):
     s = L["shape"]
     o = ref.Layer(L)
-    got = run_gpu(L, x_np)
-    r = o.route(x_np)
-    decided, ties = check_routes(s, r, got["cid"], got["eid"], got["gates"])
+    got = run_gpu(L, x_np, options=options)
     T = x_np.shape[0]
-    if sample is None or sample >= T:
-        idx = np.arange(T, dtype=np.int32)
-    else:
+    idx = None
+    if sample is not None and sample < T:
         idx = np.sort(np.random.default_rng(seed).choice(T, sample, replace=False)).astype(np.int32)
-    y_ref = o.forward(x_np, idx)
-    err, tol = check_y(got["y"][idx], y_ref, decided[idx])
-    print(f"{s.name}: T={T} near-ties {ties} checked {idx.size} rows, max err {err:.3e} (tol {tol:.3e})")
+    err, tol, ties = compare(L, o, x_np, got["cid"], got["eid"], got["gates"], got["y"], idx=idx, label=label)
+    print(f"{s.name}: T={T} near-ties {ties} checked {T if idx is None else idx.size} rows, max err {err:.3e} (tol {tol:.3e})")
     return got
 
 
@@ -64,17 +60,17 @@ def test_bert_full():
 
 
 @pytest.mark.parametrize("name", ["gpt2m", "skew"])
-def test_large_sampled(name):
+def test_large_full(name):
     L = layer_for(name)
-    got = full_check(L, L["x"], sample=192)
+    got = full_check(L, L["x"])
     if name == "skew":
         share = np.bincount(got["cid"], minlength=8) / L["x"].shape[0]
         assert abs(share[0] - 0.429) < 0.02 and share[-1] < 0.06
 
 
-def test_decode_sampled():
+def test_decode_full():
     L = layer_for("decode")
-    full_check(L, L["x"], sample=12)
+    full_check(L, L["x"])
 
 
 @pytest.mark.parametrize("T", [1, 2, 127, 129, 257, 300])
@@ -105,12 +101,8 @@ def test_empty_cluster_and_labels():
     L["b_e"] = np.zeros((3, 3), np.float32)
     label = (np.arange(9, dtype=np.int32) * 7 + 100)
     L["expert_global_id"] = label
-    o = ref.Layer(L)
-    got = run_gpu(L, L["x"])
+    got = full_check(L, L["x"], label=label)
     assert not np.any(got["cid"] == 1)
-    r = o.route(L["x"])
-    decided, _ = check_routes(s, r, got["cid"], got["eid"], got["gates"], label=label)
-    check_y(got["y"], o.forward(L["x"]), decided)
 
 
 def test_zero_tokens_and_reuse():
@@ -129,8 +121,7 @@ def test_zero_tokens_and_reuse():
         cid, eid, gates = m.route(x)
         y = m.forward(x)
         torch.cuda.synchronize()
-        decided, _ = check_routes(s, o.route(x_np), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
-        check_y(y.float().cpu().numpy(), o.forward(x_np), decided)
+        compare(L, o, x_np, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy())
     assert m.status() == 0
 
 
@@ -168,21 +159,21 @@ def test_permutation_equivariance_on_gpu():
     dict(T=1500, d=160, d_ff=64, E=10, G=2, r=0, k=3),      # K = 5: a ragged group of expert rows
     dict(T=1027, d=1056, d_ff=32, E=8, G=8, r=0, k=1),      # d not a multiple of 256, one expert per cluster
     dict(T=2048, d=2304, d_ff=32, E=64, G=2, r=0, k=8),     # prototypes staged in several chunks, K = 32
-], ids=["G12", "K5", "d1056", "d2304_K32"])
-def test_router_tile_kernel_shapes(kw, monkeypatch):
+    dict(T=1024, d=4096, d_ff=32, E=4, G=2, r=0, k=2),      # two clusters, rows of 16 KB: staged in two pieces
+], ids=["G12", "K5", "d1056", "d2304_K32", "G2_d4096"])
+def test_router_tile_kernel_shapes(kw):
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer
-    monkeypatch.setenv("CMOE_ROUTER_FP32", "1")          # the CUDA-core kernels, also for these large batches
     s = inputs.small_shape(**kw)
     L = inputs.make_layer(s, 17)
     rng = np.random.default_rng(1)
     L["b_c"] = (rng.standard_normal(s.G) * 0.2).astype(np.float32)
     L["b_e"] = (rng.standard_normal((s.G, s.K)) * 0.2).astype(np.float32)
-    m = ClusteredMoELayer(L)
+    m = ClusteredMoELayer(L, options=dict(router_fp32=1))      # the CUDA-core kernels, also for these large batches
     x = torch.from_numpy(L["x"]).cuda()
     cid, eid, gates = m.route(x)
     torch.cuda.synchronize()
-    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), layer=L, x=L["x"])
 
 
 @pytest.mark.parametrize("kw", [
@@ -205,18 +196,17 @@ def test_router_tensor_core_shapes(kw):
     cid, eid, gates = m.route(x)
     torch.cuda.synchronize()
     assert m.status() == 0
-    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
+    check_routes(s, ref.Layer(L).route(L["x"]), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), layer=L, x=L["x"])
 
 
-def test_route_does_not_depend_on_the_batch(monkeypatch):
-    """With the fp32 CUDA-core router kernels (CMOE_ROUTER_FP32=1 keeps large batches off the tensor-core
+def test_route_does_not_depend_on_the_batch():
+    """With the fp32 CUDA-core router kernels (the router_fp32 option keeps large batches off the tensor-core
     router) a token's route is bit-identical whether it arrives in a large batch (tiled kernel) or in a
     small one (per-token kernel): both sum every dot product in the same order."""
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer
-    monkeypatch.setenv("CMOE_ROUTER_FP32", "1")
     L = layer_for("bert")
-    m = ClusteredMoELayer(L)
+    m = ClusteredMoELayer(L, options=dict(router_fp32=1))
     x = torch.from_numpy(L["x"]).cuda()
     big = [t.clone() for t in m.route(x)]
     small = m.route(x[1000:1300].contiguous())
@@ -257,7 +247,7 @@ def test_tensor_path_empty_cluster():
 
 
 # The up kernel has two tile widths: 256 columns (one accumulator updated in place for the second
-# expert) where d_ff allows, else 128 columns (two accumulators).  CMOE_UP_TILE=128 keeps the narrow one.
+# expert) where d_ff allows, else 128 columns (two accumulators).  The up_tile option keeps the narrow one.
 @pytest.mark.parametrize("kw", [
     dict(d=128, d_ff=768, E=8, G=2, r=16, k=2),      # three N tiles: a unit of three
     dict(d=256, d_ff=1024, E=8, G=2, r=16, k=2),     # several units per row tile
@@ -269,18 +259,16 @@ def test_tensor_path_empty_cluster():
     dict(d=128, d_ff=256, E=8, G=2, r=16, k=1),      # direct rows, one kept expert
 ], ids=["nt3", "units", "r0", "k1", "K8r8", "direct_r4", "direct_r32", "direct_k1"])
 @pytest.mark.parametrize("tile", ["256", "128"])
-def test_up_kernel_tile_widths(kw, tile, monkeypatch):
-    monkeypatch.setenv("CMOE_UP_TILE", tile)
+def test_up_kernel_tile_widths(kw, tile):
     s = inputs.small_shape(T=1500, **kw)
     L = inputs.make_layer(s, 21)
-    got = full_check(L, L["x"])
+    got = full_check(L, L["x"], options=dict(up_tile=int(tile)))
     assert got["module"].info.path == 1
 
 
-def test_bert_with_the_narrow_up_kernel(monkeypatch):
-    monkeypatch.setenv("CMOE_UP_TILE", "128")
+def test_bert_with_the_narrow_up_kernel():
     L = layer_for("bert")
-    full_check(L, L["x"], sample=512)
+    full_check(L, L["x"], options=dict(up_tile=128))
 
 
 # ---- shapes that take the weight-streaming path (T_max <= 128, d and d_ff multiples of 128) ---------
@@ -315,8 +303,7 @@ def test_stream_path_empty_cluster_and_reuse():
         cid, eid, gates = m.route(x)
         y = m.forward(x)
         torch.cuda.synchronize()
-        decided, _ = check_routes(s, o.route(x_np), cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
-        check_y(y.float().cpu().numpy(), o.forward(x_np), decided)
+        compare(L, o, x_np, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy())
     assert m.status() == 0
 
 
@@ -359,13 +346,14 @@ def test_forward_host_equals_forward(T):
     bad = np.abs(a - b) > 2e-3 * np.abs(a).max() + 1e-3
     assert bad.any(axis=1).mean() <= 0.002
     # and against the oracle
+    # and against the oracle (rows of tokens whose near-tie a chunk's router may have settled the other way are left out)
     o = ref.Layer(L)
     r = o.route(L["x"])
-    idx = np.arange(0, T, 7, dtype=np.int32)
-    y_ref = o.forward(L["x"], idx)
     cid, eid, gates = m.route(xh.cuda())
-    decided, _ = check_routes(s, r, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy())
-    check_y(b[idx], y_ref, decided[idx])
+    decided, _, _ = check_routes(s, r, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), layer=L, x=L["x"])
+    idx = np.arange(0, T, 7, dtype=np.int32)
+    idx = idx[decided[idx]]
+    check_y(b[idx], o.forward(L["x"], idx))
     m.close()
 
 
@@ -390,5 +378,183 @@ def test_headline_shape_at_another_batch_size():
     reductions into s and the expansion kernel instead of the direct rows)."""
     s = inputs.small_shape(T=20000, d=1024, d_ff=4096, E=32, G=8, r=16, k=2)
     L = inputs.make_layer(s, 5)
-    got = full_check(L, L["x"], sample=192)
+    got = full_check(L, L["x"])
     assert got["module"].info.path == 1
+
+
+# ---- layers in which the rank-r residual terms dominate (Eq. 7) ---------------------------------------------
+# In the workloads the residual moves h and y by a few percent, so a partial mistake in it (a neighbouring
+# scale group, one factor's scale, a wrong block of the expanded rank index) could hide inside the tolerance.
+# Here the bases are zero, or a quarter of their size beside factors twelve times larger, on every path that
+# evaluates the residual.
+_RESID_CASES = [
+    # generic CUDA-core path (d, d_ff not multiples of 128)
+    ("generic_r4_k2", dict(T=200, d=96, d_ff=224, E=8, G=2, r=4, k=2), None),
+    ("generic_r32_k3", dict(T=200, d=96, d_ff=224, E=16, G=2, r=32, k=3), None),
+    # first tensor-core path: K * r > 64, rank-r terms in the epilogue
+    ("tc1_K8_r32", dict(T=700, d=384, d_ff=256, E=16, G=2, r=32, k=2), None),
+    ("tc1_K8_r16_k1", dict(T=700, d=256, d_ff=384, E=16, G=2, r=16, k=1), None),
+    # pair path, 256-column up tiles: several units per row tile, whole-row units (direct rows), both k
+    ("pair_wide_units", dict(T=1500, d=256, d_ff=1024, E=8, G=2, r=16, k=2), None),
+    ("pair_wide_direct_r4", dict(T=1500, d=128, d_ff=256, E=8, G=2, r=4, k=2), None),
+    ("pair_wide_direct_r8_K8", dict(T=1500, d=128, d_ff=256, E=16, G=2, r=8, k=2), None),
+    ("pair_wide_direct_r32", dict(T=1500, d=128, d_ff=256, E=4, G=2, r=32, k=2), None),
+    ("pair_wide_k1", dict(T=1500, d=128, d_ff=512, E=8, G=2, r=8, k=1), None),
+    # pair path, 128-column up tiles
+    ("pair_narrow_r16", dict(T=1500, d=128, d_ff=768, E=8, G=2, r=16, k=2), dict(up_tile=128)),
+    ("pair_narrow_dff384", dict(T=700, d=256, d_ff=384, E=8, G=2, r=8, k=2), None),
+    # weight-streaming path
+    ("stream_r4", dict(T=64, d=128, d_ff=256, E=8, G=2, r=4, k=2), None),
+    ("stream_r16_k1", dict(T=100, d=256, d_ff=128, E=4, G=1, r=16, k=1), None),
+    ("stream_r32_k3", dict(T=64, d=128, d_ff=256, E=16, G=2, r=32, k=3), None),
+]
+
+
+@pytest.mark.parametrize("mode", ["zero_bases", "large_factors"])
+@pytest.mark.parametrize("name,kw,options", _RESID_CASES, ids=[c[0] for c in _RESID_CASES])
+def test_residual_dominated_layers(name, kw, options, mode):
+    s = inputs.small_shape(**kw)
+    if mode == "zero_bases":
+        L = inputs.make_layer(s, 61, base_scale=0.0, factor_std=0.2)
+    else:
+        L = inputs.make_layer(s, 62, base_scale=0.25, factor_std=0.25)
+    # the residual really dominates: U V is several times B
+    o = ref.Layer(L)
+    W = o.weight(0, 1).astype(np.float64)
+    Bpart = L["B1"][0].astype(np.float64)
+    assert (W - Bpart).std() > 2.0 * Bpart.std()
+    full_check(L, L["x"], options=options)
+
+
+# ---- canaries around the arena and the outputs; scratch not assumed to start at zero ----------------------
+@pytest.mark.parametrize("kw", [
+    dict(d=96, d_ff=224, E=8, G=2, r=4, k=2),          # generic path
+    dict(d=384, d_ff=256, E=16, G=2, r=32, k=2),       # first tensor-core path
+    dict(d=128, d_ff=256, E=8, G=2, r=16, k=2),        # pair path, wide tiles
+    dict(d=256, d_ff=384, E=8, G=2, r=8, k=2),         # pair path, narrow tiles
+], ids=["generic", "tc1", "pair_wide", "pair_narrow"])
+@pytest.mark.parametrize("T", [1, 127, 129, 257, 1500])
+def test_nothing_is_written_outside_the_arena_or_y(kw, T):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=1500, **kw)
+    L = inputs.make_layer(s, 71)
+    # arena pre-filled with 0xFF (NaN as fp16 / fp32, -1 as int32): nothing may rely on zeroed scratch
+    m = ClusteredMoELayer(L, T_max=1500, guard_bytes=1 << 16, fill_byte=0xFF)
+    x_np = inputs.make_tokens(s, T, seed=T)
+    band = 4096
+    buf = torch.full((T * s.d + 2 * band,), float("nan"), dtype=torch.float16, device="cuda")
+    y = buf[band:band + T * s.d].view(T, s.d)
+    x = torch.from_numpy(x_np).cuda()
+    cid, eid, gates = m.route(x)
+    m.forward(x, out=y)
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    assert m.guards_intact(), "bytes around the arena were overwritten"
+    assert bool(torch.isnan(buf[:band]).all()) and bool(torch.isnan(buf[band + T * s.d:]).all()), "bytes around y were overwritten"
+    assert bool(torch.isfinite(y).all())
+    compare(L, ref.Layer(L), x_np, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy())
+    m.close()
+
+
+@pytest.mark.parametrize("T", [1, 17, 64, 128])
+def test_nothing_is_written_outside_the_arena_or_y_streaming(T):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=128, d=256, d_ff=384, E=8, G=2, r=16, k=2)
+    L = inputs.make_layer(s, 72)
+    m = ClusteredMoELayer(L, T_max=128, guard_bytes=1 << 16, fill_byte=0xFF)
+    assert m.info.path == 2
+    x_np = inputs.make_tokens(s, T, seed=T)
+    band = 4096
+    buf = torch.full((T * s.d + 2 * band,), float("nan"), dtype=torch.float16, device="cuda")
+    y = buf[band:band + T * s.d].view(T, s.d)
+    x = torch.from_numpy(x_np).cuda()
+    cid, eid, gates = m.route(x)
+    m.forward(x, out=y)
+    torch.cuda.synchronize()
+    assert m.status() == 0 and m.guards_intact()
+    assert bool(torch.isnan(buf[:band]).all()) and bool(torch.isnan(buf[band + T * s.d:]).all())
+    compare(L, ref.Layer(L), x_np, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy())
+    m.close()
+
+
+# ---- the bounded waits' error path ---------------------------------------------------------------------------
+def test_wait_timeout_is_reported_once_and_the_handle_stays_usable():
+    """A wait that runs into its cycle limit (a barrier nothing arrives on, a limit of about a millisecond) sets the
+    status word and the kernel returns normally: cmoe_status says CMOE_ERR_TIMEOUT once, then CMOE_OK, and the next
+    forward on the same handle is right."""
+    import torch
+    from paper_2510_02345_b200 import binding
+    L = layer_for("tiny")
+    m = binding.ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    m.forward(x)
+    assert m.status() == 0
+    binding.cmoe_selftest_wait_timeout(m.handle, 2_000_000, torch.cuda.current_stream().cuda_stream)
+    assert m.status() == -6
+    assert m.status() == 0
+    cid, eid, gates = m.route(x)
+    y = m.forward(x)
+    torch.cuda.synchronize()
+    assert m.status() == 0
+    compare(L, ref.Layer(L), L["x"], cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), y.float().cpu().numpy())
+    with pytest.raises(binding.CmoeError):
+        binding.cmoe_selftest_wait_timeout(m.handle, 0, 0)
+    m.close()
+
+
+# ---- routing by-products (Eq. 5, load CoV) -------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["tiny", "bert", "skew", "decode"])
+def test_expert_stats_match_the_oracle(name):
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    L = layer_for(name)
+    s = L["shape"]
+    m = ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    mu0 = np.random.default_rng(5).standard_normal((s.E, s.d)).astype(np.float32)
+    mu = torch.from_numpy(mu0.copy()).cuda()
+    loads, xbar, cov = m.expert_stats(x, mu=mu, beta=0.05)
+    torch.cuda.synchronize()
+    o = ref.Layer(L)
+    mu_ref = mu0.copy()
+    loads_ref, xbar_ref, cov_ref = o.expert_stats(L["x"], mu=mu_ref, beta=0.05)
+    r = o.route(L["x"])
+    cid, eid, gates = m.route(x)
+    decided, ties, _ = check_routes(s, r, cid.cpu().numpy(), eid.cpu().numpy(), gates.cpu().numpy(), layer=L, x=L["x"])
+    n_band = int((~decided).sum())
+    got = loads.cpu().numpy()
+    assert got.sum() == s.k * s.T
+    # integer counts: equal, up to the tokens inside the near-tie band (each may move one unit between two experts per slot)
+    assert np.abs(got - loads_ref).sum() <= 2 * s.k * n_band
+    if n_band == 0:
+        assert np.array_equal(got, loads_ref)
+        assert np.allclose(xbar.cpu().numpy(), xbar_ref, atol=2e-5, rtol=1e-5)
+        assert np.allclose(mu.cpu().numpy(), mu_ref, atol=2e-5, rtol=1e-5)
+        assert abs(float(cov) - cov_ref) < 1e-6
+    else:
+        bound = 4.0 * n_band / max(1, loads_ref.min())          # a few banded tokens move a mean by at most this much
+        assert np.abs(xbar.cpu().numpy() - xbar_ref).max() <= 8.0 * bound + 2e-5
+        assert abs(float(cov) - cov_ref) < 1e-3
+    m.close()
+
+
+def test_expert_stats_empty_batch_and_untouched_centroids():
+    import torch
+    from paper_2510_02345_b200.binding import ClusteredMoELayer
+    s = inputs.small_shape(T=150, d=64, d_ff=96, E=9, G=3, r=4, k=2)
+    L = inputs.make_layer(s, 6)
+    L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)        # cluster 1 never wins: its experts get no tokens
+    m = ClusteredMoELayer(L)
+    x = torch.from_numpy(L["x"]).cuda()
+    mu0 = torch.ones((s.E, s.d), dtype=torch.float32, device="cuda")
+    mu = mu0.clone()
+    loads, xbar, cov = m.expert_stats(x, mu=mu, beta=0.5)
+    torch.cuda.synchronize()
+    assert int(loads[3:6].sum()) == 0 and bool((mu[3:6] == 1).all()) and not bool(xbar[3:6].any())
+    assert int(loads.sum()) == s.k * s.T
+    loads0, xbar0, cov0 = m.expert_stats(x[:0], mu=mu, beta=0.5)
+    torch.cuda.synchronize()
+    assert int(loads0.sum()) == 0 and not bool(xbar0.any()) and float(cov0) == 0.0
+    m.close()
