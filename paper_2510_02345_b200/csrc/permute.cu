@@ -6,7 +6,8 @@
 //   hist     per-block histogram of the keys (block = 256 consecutive tokens); for batches of 1024 tokens and
 //            more the router kernel has counted the keys of its token tiles itself and this kernel is not launched
 //   scan     one block: per-key running sums over blocks, cluster segment offsets, tile table, and the
-//            table entries of the padding rows of each segment (no token, zero gates)
+//            table entries of the padding rows of each segment (no token, zero gates); when the table of counts
+//            is small every scatter block does these sums for itself and this kernel is not launched either
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
 //            writes the row tables
 //   move     copies every token's activations to its row with 16-byte vectors (a block per row;
@@ -117,6 +118,15 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
   }
 }
 
+// What the scan computes, for the scatter kernel to work out itself when the count table is small (ScanInline.counts
+// not null): every scatter block then sums the table for its own keys - the keys' totals and the counts of the blocks
+// before it - and block 0 also writes the segment tables; one kernel and one launch gap less.
+struct ScanInline {
+  const int* counts;      // [nblk][nkey], or null: block_base / key_off come from the scan kernel
+  int nblk, G, nsub, row_align, max_tiles;
+  int *seg_off, *seg_cnt, *n_rows, *tile_cluster;
+};
+
 __global__ void __launch_bounds__(kPermBlock)      // 64, 128 or 256 threads: the token tile of the kernel that counted the keys
 scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
                const __half* __restrict__ x, const int* __restrict__ cluster_id,
@@ -124,14 +134,81 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
                const int* __restrict__ keys, const int* __restrict__ block_base,
                const int* __restrict__ key_off,
                int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
-               __half* __restrict__ x_perm, int nblk, const FactorStage fs) {
+               __half* __restrict__ x_perm, const ScanInline si) {
   pdl_wait();
-  // blocks nblk.. decode the layer's INT4 factors for the tensor-core residual products (weights only: they
-  // fill the SMs beside the few, latency-bound scatter blocks)
-  if ((int)blockIdx.x >= nblk) { stage_block(fs, blockIdx.x - nblk); return; }
   extern __shared__ int sh_next[];   // next free row of each key for this block
-  for (int i = threadIdx.x; i < nkey; i += blockDim.x)
-    sh_next[i] = key_off[i] + block_base[(size_t)blockIdx.x * nkey + i];
+  if (si.counts) {
+    int* sh_tot = sh_next + nkey;    // [nkey] tokens of each key in the whole batch
+    __shared__ int sh_seg[kMaxG + 1];
+    __shared__ int sh_segcnt[kMaxG];
+    for (int key = threadIdx.x; key < nkey; key += blockDim.x) {
+      int tot = 0, before = 0;
+      for (int b = 0; b < si.nblk; ++b) {
+        const int c = si.counts[(size_t)b * nkey + key];
+        tot += c;
+        before += b < (int)blockIdx.x ? c : 0;
+      }
+      sh_tot[key] = tot;
+      sh_next[key] = before;
+    }
+    __syncthreads();
+    if (threadIdx.x < si.G) {
+      // tokens of this thread's cluster, then (thread 0) the padded segment offsets
+      int cnt = 0;
+      for (int sb = 0; sb < si.nsub; ++sb) cnt += sh_tot[threadIdx.x * si.nsub + sb];
+      sh_segcnt[threadIdx.x] = cnt;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      int off = 0;
+      for (int g = 0; g < si.G; ++g) {
+        sh_seg[g] = off;
+        off += (sh_segcnt[g] + si.row_align - 1) / si.row_align * si.row_align;
+      }
+      sh_seg[si.G] = off;
+    }
+    __syncthreads();
+    if (threadIdx.x < si.G) {
+      // first row of every key of this thread's cluster, plus the rows of the blocks before this one
+      int off = sh_seg[threadIdx.x];
+      for (int sb = 0; sb < si.nsub; ++sb) {
+        const int key = threadIdx.x * si.nsub + sb;
+        sh_next[key] += off;
+        off += sh_tot[key];
+      }
+    }
+    if (blockIdx.x == 0) {
+      // block 0 also writes the tables the later kernels read
+      for (int g = threadIdx.x; g <= si.G; g += blockDim.x) {
+        si.seg_off[g] = sh_seg[g];
+        if (g < si.G) si.seg_cnt[g] = sh_segcnt[g];
+      }
+      if (threadIdx.x == 0) *si.n_rows = sh_seg[si.G];
+      for (int g = 0; g < si.G; ++g) {
+        const int first = sh_seg[g] + sh_segcnt[g], last = sh_seg[g + 1];
+        for (int row = first + (int)threadIdx.x; row < last; row += blockDim.x) {
+          row_token[row] = -1;
+          for (int j = 0; j < k; ++j) {
+            row_slot[(size_t)row * k + j] = g * K + j;       // any valid experts of the cluster
+            row_gate[(size_t)row * k + j] = 0.f;
+          }
+        }
+      }
+      const int ntile = sh_seg[si.G] / si.row_align;
+      for (int tile = threadIdx.x; tile < si.max_tiles; tile += blockDim.x) {
+        int g = -1;
+        if (tile < ntile) {
+          const int row = tile * si.row_align;
+          g = 0;
+          while (g + 1 < si.G && sh_seg[g + 1] <= row) ++g;
+        }
+        si.tile_cluster[tile] = g;
+      }
+    }
+  } else {
+    for (int i = threadIdx.x; i < nkey; i += blockDim.x)
+      sh_next[i] = key_off[i] + block_base[(size_t)blockIdx.x * nkey + i];
+  }
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = blockIdx.x * blockDim.x + threadIdx.x;        // a block takes the tokens one counting block took
@@ -168,10 +245,14 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
 // x_perm[row] = x[row_token[row]], zeros for padding rows; a block per row, 16 bytes per thread
 __global__ void __launch_bounds__(128)
 move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ row_token,
-                 const __half* __restrict__ x, __half* __restrict__ x_perm, uint4* __restrict__ zero_ptr, size_t zero_n) {
+                 const __half* __restrict__ x, __half* __restrict__ x_perm, uint4* __restrict__ zero_ptr, size_t zero_n,
+                 int n_move, const FactorStage fs) {
   pdl_wait();
+  // blocks n_move.. decode the layer's INT4 factors for the tensor-core residual products (weights only; a few MB
+  // more for a kernel that is bound by memory bandwidth anyway)
+  if ((int)blockIdx.x >= n_move) { stage_block(fs, blockIdx.x - n_move); return; }
   const int vec_per_row = d / 8;
-  for (int row = blockIdx.x; row < *n_rows; row += gridDim.x) {
+  for (int row = blockIdx.x; row < *n_rows; row += n_move) {
     const int tok = row_token[row];
     uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
     if (tok >= 0) {
@@ -182,7 +263,7 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
     }
   }
   // the accumulation buffer of the later stages starts at zero
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += (size_t)gridDim.x * blockDim.x)
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < zero_n; i += (size_t)n_move * blockDim.x)
     zero_ptr[i] = make_uint4(0, 0, 0, 0);
 }
 
@@ -275,7 +356,16 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
   }
 }
 
+// the count table is small enough for every scatter block to sum it itself
+bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk * D.nkey <= 16384 && D.G <= tile; }
+
 }  // namespace
+
+int permute_launches(const Dims& D, int T, int counted_tile) {
+  if (T <= kSmallT) return 2;
+  if (counted_tile <= 0) return 4;
+  return inline_scan_ok(D, (T + counted_tile - 1) / counted_tile, counted_tile) ? 2 : 3;
+}
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
                            size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile) {
@@ -288,7 +378,7 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
         S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate, lr);
     launch_chained(move_rows_kernel, dim3(rows_bound), dim3(128), 0, st, 1,
-      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, rows_bound, FactorStage{});
     return cudaGetLastError();
   }
   // counting blocks: the router's token tiles when it counted the keys itself (counted_tile tokens each), else
@@ -300,19 +390,28 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
     launch_chained(hist_kernel, dim3(nblk), dim3(kPermBlock), sh, st, 1,
         T, D.k, D.nsub, D.nkey, D.sub_is_combo, S.cluster_id,
                                               S.slot, S.gates, S.keys, S.block_counts);
-  launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
-      nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
-                                  S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
-                                  S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
-  launch_chained(scatter_kernel, dim3(nblk + stage_blocks(fs, tile)), dim3(tile), sh, st, 1,
+  // a small count table: every scatter block sums it for itself and the scan kernel is not launched
+  ScanInline si{};
+  const bool inline_scan = counted_tile > 0 && inline_scan_ok(D, nblk, tile);
+  if (inline_scan) {
+    si.counts = S.block_counts; si.nblk = nblk; si.G = D.G; si.nsub = D.nsub; si.row_align = D.row_align;
+    si.max_tiles = D.T_pad_max / D.row_align;
+    si.seg_off = S.seg_off; si.seg_cnt = S.seg_cnt; si.n_rows = S.n_rows; si.tile_cluster = S.tile_cluster;
+  } else {
+    launch_chained(scan_kernel, dim3(1), dim3(1024), 0, st, 1,
+        nblk, D.G, D.nsub, D.nkey, D.row_align, D.T_pad_max / D.row_align,
+                                    S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
+                                    S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
+  }
+  launch_chained(scatter_kernel, dim3(nblk), dim3(tile), sh * (inline_scan ? 2 : 1), st, 1,
       T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
-                                               S.x_perm, nblk, fs);
+                                               S.x_perm, si);
   const int move_max = (D.sm_count > 0 ? D.sm_count : 148) * 32;      // resident blocks of 128 threads
   const int move_grid = rows_bound < move_max ? rows_bound : move_max;
-  launch_chained(move_rows_kernel, dim3(move_grid), dim3(128), 0, st, 1,
-      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16);
+  launch_chained(move_rows_kernel, dim3(move_grid + stage_blocks(fs, 128)), dim3(128), 0, st, 1,
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, move_grid, fs);
   return cudaGetLastError();
 }
 

@@ -256,7 +256,7 @@ router_tile_kernel(const RouterArgs a) {
 __global__ void __launch_bounds__(256)
 router_token_kernel(const RouterArgs a) {
   pdl_wait();
-  if ((int)blockIdx.x >= a.n_route_blocks) { stage_rider(a.fs, blockIdx.x - a.n_route_blocks, a.n_riders); return; }
+  if ((int)blockIdx.x >= a.n_route_blocks) { stage_block(a.fs, blockIdx.x - a.n_route_blocks); return; }
   __shared__ float lg[kMaxG];           // cluster logits, then the expert logits (kMaxK <= kMaxG)
   __shared__ int s_g;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
@@ -317,9 +317,9 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
   if (T <= 0) return cudaSuccess;
   RouterArgs a{};
   // (the staging of the tensor-core residual factors rides here for batches below 1024 tokens, else in the
-  // permutation's scatter kernel)
+  // permutation's row-move kernel)
   if (fs && T < 1024) a.fs = *fs;
-  a.n_riders = stage_riders(a.fs, 256, (D.sm_count > 0 ? D.sm_count : 148) * 4);
+  a.n_riders = stage_blocks(a.fs, 256);          // one 32-bit word of packed codes per thread
   a.x = x; a.T = T; a.d = D.d; a.G = D.G; a.K = D.K; a.k = D.k;
   a.Ct = W.Ct; a.Rt = W.Rt; a.bc = W.bc; a.be = W.be; a.label = W.label;
   a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;

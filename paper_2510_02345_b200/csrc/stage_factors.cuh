@@ -85,27 +85,4 @@ __device__ __forceinline__ void stage_block(const FactorStage& fs, int b) {
   }
 }
 
-// The same work as `n_riders` blocks of another kernel's grid, each thread striding over the words of the four
-// factors (for kernels whose blocks are too expensive to spend on one word per thread).
-inline long long stage_words(const FactorStage& fs) { return fs.words[0] + fs.words[1] + fs.words[2] + fs.words[3]; }
-
-inline int stage_riders(const FactorStage& fs, int threads, int max_blocks) {
-  const long long per_block = (long long)threads * 8;          // about eight words per thread
-  const long long n = (stage_words(fs) + per_block - 1) / per_block;
-  return (int)(n < max_blocks ? n : max_blocks);
-}
-
-__device__ __forceinline__ void stage_rider(const FactorStage& fs, int rider, int n_riders) {
-  const long long total = fs.words[0] + fs.words[1] + fs.words[2] + fs.words[3];
-  const long long stride = (long long)n_riders * blockDim.x;
-  for (long long i = (long long)rider * blockDim.x + threadIdx.x; i < total; i += stride) {
-    long long wd = i;
-    int which = 0;
-#pragma unroll
-    for (int f = 0; f < 3; ++f)
-      if (which == f && wd >= fs.words[f]) { wd -= fs.words[f]; which = f + 1; }
-    stage_word(fs, which, wd);
-  }
-}
-
 }  // namespace cmoe
