@@ -141,15 +141,23 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
     int* sh_tot = sh_next + nkey;    // [nkey] tokens of each key in the whole batch
     __shared__ int sh_seg[kMaxG + 1];
     __shared__ int sh_segcnt[kMaxG];
-    for (int key = threadIdx.x; key < nkey; key += blockDim.x) {
-      int tot = 0, before = 0;
-      for (int b = 0; b < si.nblk; ++b) {
-        const int c = si.counts[(size_t)b * nkey + key];
-        tot += c;
-        before += b < (int)blockIdx.x ? c : 0;
+    // a warp per key, lanes over the counting blocks: the key's total and the part of the blocks before this one
+    {
+      const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5, nwarp_ = blockDim.x >> 5;
+      for (int key = warp_; key < nkey; key += nwarp_) {
+        int tot = 0, before = 0;
+        for (int b = lane_; b < si.nblk; b += 32) {
+          const int c = si.counts[(size_t)b * nkey + key];
+          tot += c;
+          before += b < (int)blockIdx.x ? c : 0;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          tot += __shfl_xor_sync(0xffffffffu, tot, o);
+          before += __shfl_xor_sync(0xffffffffu, before, o);
+        }
+        if (lane_ == 0) { sh_tot[key] = tot; sh_next[key] = before; }
       }
-      sh_tot[key] = tot;
-      sh_next[key] = before;
     }
     __syncthreads();
     if (threadIdx.x < si.G) {

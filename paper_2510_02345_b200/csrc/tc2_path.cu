@@ -1021,7 +1021,7 @@ void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs) {
   const int dim[4] = {D.d, D.d_ff, D.d_ff, D.d};
   for (int i = 0; i < 4; ++i) {
     fs->q[i] = q[i]; fs->s[i] = sc[i]; fs->dst[i] = dst[i]; fs->dim[i] = dim[i];
-    fs->words[i] = (long long)D.E * D.r * dim[i] / 8;
+    fs->words[i] = (long long)D.E * D.r * dim[i] / 32;      // scale groups of 32 codes
   }
   fs->K = D.K; fs->r = D.r;
 }
