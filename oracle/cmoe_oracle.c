@@ -29,6 +29,14 @@ float cmoe_ref_half_to_float(uint16_t h) {
   return v;
 }
 
+/* bfloat16 -> binary32, exact: the 16 bits are the upper half of the binary32 pattern. */
+float cmoe_ref_bf16_to_float(uint16_t h) {
+  uint32_t bits = (uint32_t)h << 16;
+  float v;
+  memcpy(&v, &bits, sizeof v);
+  return v;
+}
+
 /* INT4 storage format of the residual factors (Sec. 3.4 "Precision and Memory
  * Management"): two's-complement 4-bit code, even flat index in the low nibble,
  * times the fp16 scale shared by its group of 32 consecutive flat elements. */
@@ -134,7 +142,8 @@ int cmoe_ref_form_weight(const cmoe_ref_desc* D, int32_t e, int32_t which, float
     double* acc = (double*)malloc(sizeof(double) * (size_t)dout);
 #pragma omp for schedule(static)
     for (int64_t a = 0; a < din; ++a) {
-      for (int64_t b = 0; b < dout; ++b) acc[b] = (double)cmoe_ref_half_to_float(B[a * dout + b]);
+      for (int64_t b = 0; b < dout; ++b)
+        acc[b] = (double)(D->base_is_bf16 ? cmoe_ref_bf16_to_float(B[a * dout + b]) : cmoe_ref_half_to_float(B[a * dout + b]));
       for (int p = 0; p < r; ++p) {
         double u = (double)Ud[a * r + p];
         for (int64_t b = 0; b < dout; ++b) acc[b] += u * (double)Vd[p * dout + b];

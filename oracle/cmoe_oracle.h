@@ -47,10 +47,13 @@ typedef struct {
   const uint16_t* B2;   /* [G][d_ff][d] fp16 bits      */
   const uint8_t *U1q, *V1q, *U2q, *V2q;   /* packed INT4: U1 [E][r][d], V1 [E][d_ff][r], U2 [E][r][d_ff], V2 [E][d][r] */
   const uint16_t *U1s, *V1s, *U2s, *V2s;  /* fp16 scale per 32 consecutive flat elements */
+  int32_t base_is_bf16; /* 0: B1, B2 hold fp16 bits (the paper's storage format, Sec. 3.4); 1: bfloat16 bits (a variant) */
 } cmoe_ref_desc;
 
 /* fp16 bits -> fp32 value (exact). */
 float cmoe_ref_half_to_float(uint16_t h);
+/* bfloat16 bits -> fp32 value (exact). */
+float cmoe_ref_bf16_to_float(uint16_t h);
 
 /* Element `idx` of a packed INT4 factor: code * scale of its 32-group (exact in fp32). */
 float cmoe_ref_dequant(const uint8_t* q, const uint16_t* s, int64_t idx);

@@ -18,6 +18,7 @@ class _Desc(C.Structure):
         ("B1", C.c_void_p), ("B2", C.c_void_p),
         ("U1q", C.c_void_p), ("V1q", C.c_void_p), ("U2q", C.c_void_p), ("V2q", C.c_void_p),
         ("U1s", C.c_void_p), ("V1s", C.c_void_p), ("U2s", C.c_void_p), ("V2s", C.c_void_p),
+        ("base_is_bf16", C.c_int32),
     ]
 
 
@@ -30,6 +31,8 @@ def load(path: str):
         L = C.CDLL(path)
         L.cmoe_ref_half_to_float.restype = C.c_float
         L.cmoe_ref_half_to_float.argtypes = [C.c_uint16]
+        L.cmoe_ref_bf16_to_float.restype = C.c_float
+        L.cmoe_ref_bf16_to_float.argtypes = [C.c_uint16]
         L.cmoe_ref_dequant.restype = C.c_float
         L.cmoe_ref_dequant.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.cmoe_ref_route.restype = C.c_int
@@ -65,15 +68,16 @@ class Layer:
         s = layer["shape"]
         self.shape = s
         keep = {}
+        bf16 = layer.get("base_dtype", "fp16") == "bf16"      # B1, B2 then hold bfloat16 bit patterns as uint16
         for name, dt in (("C", np.float32), ("R", np.float32), ("b_c", np.float32), ("b_e", np.float32),
-                         ("B1", np.float16), ("B2", np.float16),
+                         ("B1", np.uint16 if bf16 else np.float16), ("B2", np.uint16 if bf16 else np.float16),
                          ("U1q", np.uint8), ("V1q", np.uint8), ("U2q", np.uint8), ("V2q", np.uint8),
                          ("U1s", np.float16), ("V1s", np.float16), ("U2s", np.float16), ("V2s", np.float16)):
             a = layer.get(name)
             keep[name] = None if a is None else np.ascontiguousarray(a, dtype=dt)
         self._keep = keep
         self.desc = _Desc(s.d, s.d_ff, s.E, s.G, s.r, s.k, *[_ptr(keep[n]) for n in (
-            "C", "R", "b_c", "b_e", "B1", "B2", "U1q", "V1q", "U2q", "V2q", "U1s", "V1s", "U2s", "V2s")])
+            "C", "R", "b_c", "b_e", "B1", "B2", "U1q", "V1q", "U2q", "V2q", "U1s", "V1s", "U2s", "V2s")], 1 if bf16 else 0)
 
     def route(self, x: np.ndarray):
         """-> dict(cluster_id [T], expert_slot [T][k], gates [T][k], z [T][G], l [T][K])."""
@@ -134,6 +138,10 @@ class Layer:
         a, b = C.c_int64(), C.c_int64()
         lib().cmoe_ref_param_count(C.byref(self.desc), C.byref(a), C.byref(b))
         return a.value, b.value
+
+
+def bf16_to_float(bits: int) -> float:
+    return float(lib().cmoe_ref_bf16_to_float(bits))
 
 
 def half_to_float(bits: int) -> float:

@@ -116,8 +116,15 @@ def _calibrate_cluster_bias(x16: np.ndarray, C: np.ndarray, target: np.ndarray) 
     return b.astype(np.float32)
 
 
+def to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    """float32 -> bfloat16 bit patterns (uint16), round to nearest even (an encoding of the drawn data)."""
+    u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
+    rounded = u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))
+    return (rounded >> np.uint32(16)).astype(np.uint16)
+
+
 def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None, base_scale: float = 1.0,
-               factor_std: float = 0.02) -> dict:
+               factor_std: float = 0.02, base_dtype: str = "fp16") -> dict:
     """Draw one layer and one token batch.
 
     Draw order (float32 standard normals from numpy PCG64(seed)):
@@ -128,6 +135,7 @@ def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None, base_scal
     against fixed weights).  ``base_scale`` multiplies both shared bases (0 gives a layer whose experts
     are their low-rank residuals alone) and ``factor_std`` replaces the 0.02 of the residual factors: test
     layers in which the residual terms, a few percent of the activations in the workloads, dominate.
+    ``base_dtype`` "bf16" stores the two bases as bfloat16 bit patterns (uint16 arrays) instead of fp16.
     """
     T = shape.T if T is None else T
     d, d_ff, E, G, r, k = shape.d, shape.d_ff, shape.E, shape.G, shape.r, shape.k
@@ -142,9 +150,13 @@ def make_layer(shape: LayerShape, seed: int = 0, T: int | None = None, base_scal
     x = normal((T, d), 1.0).astype(np.float16)
     C = normal((d, G), 0.02)
     R = normal((G, d, K), 0.02)
-    B1 = normal((G, d, d_ff), base_scale / math.sqrt(d)).astype(np.float16)
-    B2 = normal((G, d_ff, d), base_scale / math.sqrt(d_ff)).astype(np.float16)
-    out = dict(shape=shape, T=T, seed=seed, x=x, C=C, R=R, B1=B1, B2=B2, b_c=None, b_e=None)
+    B1 = normal((G, d, d_ff), base_scale / math.sqrt(d))
+    B2 = normal((G, d_ff, d), base_scale / math.sqrt(d_ff))
+    if base_dtype == "bf16":
+        B1, B2 = to_bf16_bits(B1), to_bf16_bits(B2)
+    else:
+        B1, B2 = B1.astype(np.float16), B2.astype(np.float16)
+    out = dict(shape=shape, T=T, seed=seed, x=x, C=C, R=R, B1=B1, B2=B2, b_c=None, b_e=None, base_dtype=base_dtype)
     for name, dims in (("U1", (E, r, d)), ("V1", (E, d_ff, r)), ("U2", (E, r, d_ff)), ("V2", (E, d, r))):
         w = normal(dims, factor_std)
         q, s = quantize_int4(w)

@@ -35,6 +35,9 @@ MUTANTS = [
     ("gate dropped in combine", "(double)gate[(size_t)n * k + s] *", ""),
     ("only first slot combined", "for (int s = 0; s < k; ++s)\n        acc += (double)gate", "for (int s = 0; s < 1; ++s)\n        acc += (double)gate"),
     ("param count", "(int64_t)D->E * 2 * D->r", "(int64_t)D->E * D->r"),
+    ("bf16 read as the low half", "uint32_t bits = (uint32_t)h << 16;", "uint32_t bits = (uint32_t)h;"),
+    ("bf16 flag ignored", "D->base_is_bf16 ? cmoe_ref_bf16_to_float(B[a * dout + b]) : cmoe_ref_half_to_float(B[a * dout + b])",
+     "cmoe_ref_half_to_float(B[a * dout + b])"),
     ("loads count the first kept expert only", "for (int s = 0; s < k; ++s) loads[slot[(size_t)t * k + s]] += 1;",
      "for (int s = 0; s < 1; ++s) loads[slot[(size_t)t * k + s]] += 1;"),
     ("mean over all tokens", "sum[j] / (double)loads[e] : 0.0;", "sum[j] / (double)T : 0.0;"),
@@ -58,6 +61,8 @@ PINS = [
     pins.test_residual_only_layer,
     pins.test_formed_weights_orientation,
     pins.test_invariants,
+    pins.test_bf16_decode_all_bit_patterns,
+    pins.test_bf16_bases_are_decoded_as_bf16,
     pins.test_expert_stats_hand_counted,
     pins.test_expert_stats_conservation_and_numpy_counts,
 ]

@@ -373,3 +373,45 @@ def test_expert_stats_conservation_and_numpy_counts():
     mu = mu0.copy()
     loads, xbar, _ = ref.Layer(L).expert_stats(x, mu=mu, beta=0.5)
     assert loads[s.K:2 * s.K].sum() == 0 and np.array_equal(mu[s.K:2 * s.K], mu0[s.K:2 * s.K]) and not xbar[s.K:2 * s.K].any()
+
+
+# ---- bfloat16 bases (a variant of the paper's FP16 storage) ---------------------------------------------------
+def test_bf16_decode_all_bit_patterns():
+    """All 65536 bfloat16 patterns against the format's definition worked out with Python integers: sign, 8
+    exponent bits (bias 127), 7 mantissa bits; subnormals, infinities and NaNs included."""
+    for bits in range(65536):
+        sign = -1.0 if bits >> 15 else 1.0
+        expo = (bits >> 7) & 0xFF
+        mant = bits & 0x7F
+        got = ref.bf16_to_float(bits)
+        if expo == 255:
+            if mant:
+                assert math.isnan(got)
+            else:
+                assert got == sign * math.inf
+            continue
+        want = sign * (mant / 128.0) * 2.0 ** -126 if expo == 0 else sign * (1.0 + mant / 128.0) * 2.0 ** (expo - 127)
+        assert got == want, (bits, got, want)
+
+
+def test_bf16_bases_are_decoded_as_bf16():
+    """A layer with bf16 bases and r = 0 is the dense FFN of the decoded bases (torch fp64): the decode path of the
+    base and nothing else differs from the fp16 layer."""
+    s = inputs.small_shape(T=9, d=32, d_ff=64, E=4, G=2, r=0, k=2)
+    L = inputs.make_layer(s, 77, base_dtype="bf16")
+    o = ref.Layer(L)
+    y = o.forward(L["x"])
+    r = o.route(L["x"])
+    dec = lambda a: torch.from_numpy((a.astype(np.uint32) << 16).view(np.float32).astype(np.float64))
+    B1, B2 = dec(L["B1"]), dec(L["B2"])
+    x = torch.from_numpy(L["x"].astype(np.float64))
+    for t in range(s.T):
+        g = int(r["cluster_id"][t])
+        h = x[t] @ B1[g]
+        a = 0.5 * h * (1.0 + torch.erf(h / math.sqrt(2.0)))
+        want = (a @ B2[g]).numpy()
+        assert np.allclose(y[t], want, atol=1e-5, rtol=1e-5)
+    # the same bits read as fp16 give something else: the flag matters
+    L16 = dict(L, base_dtype="fp16", B1=L["B1"].view(np.float16), B2=L["B2"].view(np.float16))
+    y16 = ref.Layer(L16).forward(L["x"])
+    assert np.isnan(y16).any() or np.abs(np.nan_to_num(y16) - y).max() > 1e-3
