@@ -105,12 +105,19 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *                 about 1e-6)
  *   up_tile       0 automatic; 128 keeps the up projection of large batches on 128-column tiles where d_ff
  *                 would allow 256-column tiles
+ * and one switch that changes what the descriptor means:
+ *   base_dtype    0: desc.B1 / desc.B2 hold fp16 bits (the paper's storage format, Sec. 3.4); 1: they hold bfloat16
+ *                 bits.  The tensor cores take both operands of a product in one 16-bit type and the activations
+ *                 are fp16, so bf16 bases are converted to fp16 while cmoe_create re-lays them out: exact for
+ *                 magnitudes from 2^-14 to 65504 (fp16 has the wider significand), rounded to the fp16 subnormal
+ *                 grid below, overflowing above.
  * Other values: CMOE_ERR_INVALID_ARG.  reserved must be zero. */
 typedef struct {
   int32_t force_path;
   int32_t router_fp32;
   int32_t up_tile;
-  int32_t reserved[5];
+  int32_t base_dtype;
+  int32_t reserved[4];
 } cmoe_options;
 int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
 
@@ -176,7 +183,8 @@ typedef struct {
   int32_t T_pad_max;         /* rows of the permuted activations buffers                           */
   int32_t memsets_forward;   /* cudaMemsetAsync calls one cmoe_forward enqueues                    */
   int32_t n_stages;          /* stages cmoe_profile_read reports for this handle                   */
-  int32_t reserved[1];
+  int32_t pruned_blocks;     /* residual blocks (an expert's U V for one of its two matrices) that cmoe_create
+                                found entirely zero - pruned by the cosine gate of Sec. 3.4; their work is skipped */
 } cmoe_info;
 int cmoe_get_info(const cmoe_layer* layer, cmoe_info* out);
 

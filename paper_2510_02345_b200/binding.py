@@ -40,12 +40,13 @@ class cmoe_desc(C.Structure):
 
 
 class cmoe_options(C.Structure):
-    _fields_ = [("force_path", C.c_int32), ("router_fp32", C.c_int32), ("up_tile", C.c_int32), ("reserved", C.c_int32 * 5)]
+    _fields_ = [("force_path", C.c_int32), ("router_fp32", C.c_int32), ("up_tile", C.c_int32), ("base_dtype", C.c_int32),
+                ("reserved", C.c_int32 * 4)]
 
 
 class cmoe_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max",
-                                         "memsets_forward", "n_stages")] + [("reserved", C.c_int32 * 1)]
+                                         "memsets_forward", "n_stages", "pruned_blocks")]
 
 
 _lib = None
@@ -193,6 +194,8 @@ class ClusteredMoELayer:
             raise RuntimeError("a CUDA device is required (there is no CPU path)")
         s = layer["shape"]
         self.shape = s
+        if layer.get("base_dtype", "fp16") == "bf16":         # B1, B2 are uint16 arrays of bfloat16 bits
+            options = dict(options or {}, base_dtype=1)
         self.device = torch.device(device)
         self.T_max = int(T_max if T_max is not None else layer.get("T", s.T))
         torch.cuda.set_device(self.device)
@@ -201,6 +204,8 @@ class ClusteredMoELayer:
             a = layer.get(name)
             if a is None or a.size == 0:
                 src[name] = None
+            elif name in ("B1", "B2") and a.dtype == np.uint16:
+                src[name] = torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).to(self.device)   # bit patterns
             else:
                 src[name] = torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(self.device)
         desc = cmoe_desc()

@@ -73,6 +73,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   w.bc = A.take<float>(G);
   w.be = A.take<float>(E);
   w.label = A.take<int>(E);
+  w.live = A.take<int>(E);
   w.B1t = A.take<__half>(G * d * f);
   w.B2t = A.take<__half>(G * d * f);
   w.U1q = A.take<uint8_t>(E * r * d / 2 + 16);
@@ -112,6 +113,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
     s.Ad = A.take<__half>(P * 64);
     s.As = A.take<__half>(P * 64);
     s.tile_mask = A.take<int>(P / 128 * 2);
+    s.tile_mask_dn = A.take<int>(P / 128);
   }
   if (router_tc_supported(D)) s.Wsplit = A.take<__half>((size_t)2 * router_tc_rp(D) * d);
   if (D.stream) {
@@ -179,7 +181,8 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   cmoe_options o{};
   o.force_path = -1;
   if (opt) o = *opt;
-  if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256)) return CMOE_ERR_INVALID_ARG;
+  if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
+      o.base_dtype < 0 || o.base_dtype > 1) return CMOE_ERR_INVALID_ARG;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -255,8 +258,8 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   }
   if (e) return fail(e);
   // bases: B1 [G][d][d_ff] -> B1t [G][d_ff][d];  B2 [G][d_ff][d] -> B2t [G][d][d_ff]
-  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B1), const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st))) return fail(e);
-  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B2), const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st))) return fail(e);
+  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B1), const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
+  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B2), const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
   if (r > 0) {
     struct { const void* src; const void* dst; size_t bytes; } cp[] = {
         {desc->U1q, W.U1q, E * r * d / 2}, {desc->V1q, W.V1q, E * f * r / 2},
@@ -266,8 +269,18 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
     for (auto& c : cp)
       if ((e = cudaMemcpyAsync(const_cast<void*>(c.dst), c.src, c.bytes, cudaMemcpyDeviceToDevice, st))) return fail(e);
   }
+  if ((e = launch_residual_live(D, W, st))) return fail(e);
   if ((e = cudaMemsetAsync(L->sc.status, 0, sizeof(int), st))) return fail(e);
   if ((e = cudaStreamSynchronize(st))) return fail(e);
+  {
+    int* live_h = new (std::nothrow) int[E];
+    if (!live_h) { cmoe_destroy(L); return CMOE_ERR_INVALID_ARG; }
+    e = cudaMemcpy(live_h, W.live, E * sizeof(int), cudaMemcpyDeviceToHost);
+    L->pruned_blocks = 0;
+    for (size_t i = 0; i < E && r > 0; ++i) L->pruned_blocks += ((live_h[i] & 1) ? 0 : 1) + ((live_h[i] & 2) ? 0 : 1);
+    delete[] live_h;
+    if (e) return fail(e);
+  }
   // path choice: tensor-core grouped GEMMs when the shape allows and there are enough tokens to
   // fill 128-row tiles; cmoe_options.force_path = 0 keeps the generic path (for A/B checks)
   const int forced = o.force_path;
@@ -434,6 +447,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;
   out->T_pad_max = L->dims.T_pad_max;
+  out->pruned_blocks = L->pruned_blocks;
   return CMOE_OK;
 }
 

@@ -46,6 +46,7 @@ struct Weights {
   const __half* B2t; // [G][d][d_ff]   base of the down-projection, reduction index fastest
   const uint8_t *U1q, *V1q, *U2q, *V2q;  // packed INT4 in the boundary layouts
   const __half *U1s, *V1s, *U2s, *V2s;   // fp16 scale per 32 flat elements
+  const int* live;   // [E]  bit 0: the residual U1_e V1_e is not a zero block, bit 1: U2_e V2_e is not (Sec. 3.4's pruned blocks)
 };
 
 // Per-call scratch in the arena.
@@ -76,7 +77,8 @@ struct Scratch {
   // tensor-core path with tensor-core residuals only (see tc2_path.cu)
   __half *U1f, *V1f, *U2f, *V2f;   // INT4 factors decoded to fp16 operand matrices, per call
   __half *A0, *Ad, *As;            // [T_pad][64] expanded-rank-index operands
-  int* tile_mask;                  // [T_pad / 128][2]
+  int* tile_mask;                  // [T_pad / 128][2]  16-wide steps of the expanded index the up projection needs
+  int* tile_mask_dn;               // [T_pad / 128]     the same for the down projection
   // weight-streaming path only (see stream_path.cu)
   __half* a_slot;                  // [T_pad][k][d_ff]  GELU(h_j) of every kept expert
   float* y32;                      // [T_pad][d]        fp32 sum of the K ranges of the down-projection
@@ -94,6 +96,7 @@ struct cmoe_layer {
   int path;
   int tc_variant;   // 1: tc_path.cu, 2: tc2_path.cu (when path == kPathTensor)
   int router_tc;    // batches of at least 1024 tokens are routed by router_tc.cu
+  int pruned_blocks; // residual blocks (an expert's U V of one matrix) found to be entirely zero at create time
   CUtensorMap router_map_w;
   int last_cuda_error;
   // optional stage timing (cmoe_profile_*)
@@ -172,9 +175,12 @@ cudaError_t stream_init(cmoe_layer* L);
 int stream_launch_count(const Dims& D);
 void stream_lowrank_rider(const cmoe_layer* L, const __half* x, int T, LowrankTok* lr);
 cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
-// repack.cu : create-time layout changes
+// repack.cu : create-time layout changes; residual blocks that are entirely zero
+cudaError_t launch_residual_live(const Dims& D, const Weights& W, cudaStream_t st);
+
+// src_is_bf16: the source holds bfloat16 bit patterns, converted to fp16 on the way
 cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int rows, int cols,
-                                  cudaStream_t st);
+                                  cudaStream_t st, bool src_is_bf16 = false);
 cudaError_t launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols,
                                  cudaStream_t st);
 

@@ -64,6 +64,7 @@ struct LowrankTok {
   const uint8_t* Uq;
   const __half* Us;
   float* out;               // [T][k][r]
+  const int* live;          // [E] bit 0: the expert's up residual block is not zero (else t is not needed)
   int T, K, k, r, len;      // T == 0: nothing to do
 };
 
@@ -87,6 +88,7 @@ __device__ __forceinline__ void lowrank_tok_block(const LowrankTok& a, int b) {
 #pragma unroll
   for (int i = 1; i < kMaxKsel; ++i) if (i == j) mine = sl[i];
   const int e = a.cluster_id[tok] * a.K + mine;
+  if (!(a.live[e] & 1)) return;                 // zero residual block: the epilogue does not read this t
   const int nwarp = blockDim.x >> 5;
   lowrank_rows(a.x + (size_t)tok * a.len, e, a.r, a.len, by * nwarp, ny * nwarp, a.Uq, a.Us, a.out + (size_t)item * a.r);
 }

@@ -47,6 +47,7 @@ struct StreamParams {
   // up
   const float* t;            // [rows][k][r]
   const uint8_t* V1q;        // packed INT4 in the boundary layout
+  const int* live;           // [E] bit 0 / 1: the expert's up / down residual block is not zero
   const __half* V1s;
   __half* a_slot;            // [rows][k][d_ff]  GELU(h_j) of every kept expert
   __half* abar;              // [rows][d_ff]
@@ -248,7 +249,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
               for (int j = 0; j < k; ++j) {
                 const int e = p.row_slot[(size_t)row * k + j];
                 float h = dv;
-                if (r > 0) {
+                if (r > 0 && (p.live[e] & 1)) {      // (a zero residual block is skipped: Sec. 3.4)
                   // h += t_j . V1_e[f, :]: r codes of one scale group, decoded in registers
                   const float4* tp = reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r);    // t is indexed by token
                   const long long flat = ((long long)e * M + f) * r;
@@ -320,10 +321,12 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
 __device__ __forceinline__ void
 lowrank_body(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
              const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
-             const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+             const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out,
+             const int* __restrict__ live, int live_bit) {
   const int item = blockIdx.x;
   const int row = item / k;
-  if (row >= seg_off[G] || row_token[row] < 0) {
+  // padding rows and rows whose expert's residual block is zero: the projection is zero
+  if (row >= seg_off[G] || row_token[row] < 0 || !(live[row_slot[item]] & live_bit)) {
     if (row < seg_off[G] && blockIdx.y == 0) for (int pr = threadIdx.x; pr < r; pr += blockDim.x) out[(size_t)item * r + pr] = 0.f;
     return;
   }
@@ -336,9 +339,10 @@ lowrank_body(const int* __restrict__ seg_off, int G, int k, int r, int len, int 
 __global__ void __launch_bounds__(256)
 lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
                const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
-               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
+               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out,
+               const int* __restrict__ live, int live_bit) {
   pdl_wait();
-  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out);
+  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out, live, live_bit);
 }
 
 // The same for the second stream: s = a_j U2 is not needed before the last kernel of the forward, so it
@@ -348,8 +352,9 @@ constexpr int kSideThreads = 128;
 __global__ void __launch_bounds__(kSideThreads, 16)
 lowrank_side_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
                     const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
-                    const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out) {
-  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out);
+                    const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out,
+                    const int* __restrict__ live, int live_bit) {
+  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out, live, live_bit);
 }
 
 // Second stream, after s: the rank-r part of the down-projection, y32[row][c] += sum_j p_j s_j . V2_e[c, :],
@@ -358,13 +363,15 @@ lowrank_side_kernel(const int* __restrict__ seg_off, int G, int k, int r, int le
 __global__ void __launch_bounds__(kSideThreads, 16)
 resid_side_kernel(const int* __restrict__ seg_off, int G, int d, int k, int r, float* __restrict__ y32,
                   const float* __restrict__ s, const int* __restrict__ row_slot, const float* __restrict__ row_gate,
-                  const int* __restrict__ row_token, const uint8_t* __restrict__ V2q, const __half* __restrict__ V2s) {
+                  const int* __restrict__ row_token, const uint8_t* __restrict__ V2q, const __half* __restrict__ V2s,
+                  const int* __restrict__ live) {
   const int row = blockIdx.y;
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= seg_off[G] || c >= d || row_token[row] < 0) return;
   float v = 0.f;
   for (int j = 0; j < k; ++j) {
     const int e = row_slot[(size_t)row * k + j];
+    if (!(live[e] & 2)) continue;                            // zero residual block
     const float* sj = s + ((size_t)row * k + j) * r;
     const long long flat = ((long long)e * d + c) * r;      // the r codes of (e, c) share one scale group
     float u = 0.f;
@@ -522,7 +529,7 @@ void stream_lowrank_rider(const cmoe_layer* L, const __half* x, int T, LowrankTo
   *lr = LowrankTok{};
   if (D.r == 0) return;
   lr->x = x; lr->cluster_id = L->sc.cluster_id; lr->slot = L->sc.slot; lr->Uq = L->w.U1q; lr->Us = L->w.U1s;
-  lr->out = L->sc.t; lr->T = T; lr->K = D.K; lr->k = D.k; lr->r = D.r; lr->len = D.d;
+  lr->out = L->sc.t; lr->live = L->w.live; lr->T = T; lr->K = D.K; lr->k = D.k; lr->r = D.r; lr->len = D.d;
 }
 
 cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
@@ -537,7 +544,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   if (marks) cudaEventRecord(marks[1], st);
   StreamParams p{};
   p.seg_off = S.seg_off; p.row_slot = S.row_slot; p.row_gate = S.row_gate; p.row_token = S.row_token;
-  p.t = S.t; p.V1q = W.V1q; p.V1s = W.V1s; p.a_slot = S.a_slot; p.abar = S.abar; p.y32 = S.y32; p.status = S.status;
+  p.t = S.t; p.V1q = W.V1q; p.V1s = W.V1s; p.live = W.live; p.a_slot = S.a_slot; p.abar = S.abar; p.y32 = S.y32; p.status = S.status;
   p.G = D.G; p.K = D.K; p.k = D.k; p.r = D.r;
   const int seg_bound = D.G + rows_bound / SNB;
   {
@@ -553,10 +560,10 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     if ((e = cudaStreamWaitEvent(L->side_stream, L->side_fork, 0)) != cudaSuccess) return e;
     const int nwarp = kSideThreads / 32;
     lowrank_side_kernel<<<dim3(rows_bound * D.k, (D.r + nwarp - 1) / nwarp), kSideThreads, 0, L->side_stream>>>(
-        S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token, W.U2q, W.U2s, S.s);
+        S.seg_off, D.G, D.k, D.r, D.d_ff, 1, S.a_slot, S.row_slot, S.row_token, W.U2q, W.U2s, S.s, W.live, 2);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     resid_side_kernel<<<dim3((D.d + kSideThreads - 1) / kSideThreads, rows_bound), kSideThreads, 0, L->side_stream>>>(
-        S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate, S.row_token, W.V2q, W.V2s);
+        S.seg_off, D.G, D.d, D.k, D.r, S.y32, S.s, S.row_slot, S.row_gate, S.row_token, W.V2q, W.V2s, W.live);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     if ((e = cudaEventRecord(L->side_join, L->side_stream)) != cudaSuccess) return e;
   }

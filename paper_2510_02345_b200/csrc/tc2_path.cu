@@ -50,7 +50,9 @@ struct TParams {
   const int* row_token;
   __half* A0;          // [rows][KE]
   __half* Ad;          // [rows][KE]  (k == 2 only)
-  int* tile_mask;      // [tiles][2]  16-wide steps of the expanded index used by slot 0 / slot 1
+  int* tile_mask;      // [tiles][2]  16-wide steps of the expanded index used by slot 0 / slot 1 (up projection)
+  int* tile_mask_dn;   // [tiles]     steps the down projection needs
+  const int* live;     // [E]         bit 0 / 1: the expert's up / down residual block is not zero
   int* status;
   int KC, K, r;
 };
@@ -74,14 +76,14 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kMaxStages), tfull = smem_u32(bars + 2 * kMaxStages);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
-  int* sh_mask = reinterpret_cast<int*>(tmem_holder + 2);     // [2]
+  int* sh_mask = reinterpret_cast<int*>(tmem_holder + 2);     // [3]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
-    sh_mask[0] = 0; sh_mask[1] = 0;
+    sh_mask[0] = 0; sh_mask[1] = 0; sh_mask[2] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -132,6 +134,9 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
     const int lo0 = (p.row_slot[(size_t)row * KSEL] - g * p.K) * r;
     const int lo1 = KSEL == 2 ? (p.row_slot[(size_t)row * KSEL + 1] - g * p.K) * r : -1;
     const bool real = p.row_token[row] >= 0;
+    // residual blocks that are zero (pruned) need no step: bit 0 up, bit 1 down, per kept expert
+    const int live0 = p.live[p.row_slot[(size_t)row * KSEL]];
+    const int live1 = KSEL == 2 ? p.live[p.row_slot[(size_t)row * KSEL + 1]] : 0;
     if (warp_wait(tfull, 0, abort_flag)) {
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -166,15 +171,22 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
         }
       }
       // 16-wide steps of the expanded index that rows of this tile use
-      int m0 = 0, m1 = 0;
+      int m0 = 0, m1 = 0, md = 0;
       if (real) {
-        for (int c = lo0; c < lo0 + r; c += (r < 16 ? r : 16)) m0 |= 1 << (c >> 4);
+        int s0 = 0, s1 = 0;
+        for (int c = lo0; c < lo0 + r; c += (r < 16 ? r : 16)) s0 |= 1 << (c >> 4);
         if (KSEL == 2)
-          for (int c = lo1; c < lo1 + r; c += (r < 16 ? r : 16)) m1 |= 1 << (c >> 4);
+          for (int c = lo1; c < lo1 + r; c += (r < 16 ? r : 16)) s1 |= 1 << (c >> 4);
+        if (live0 & 1) m0 = s0;
+        if (live1 & 1) m1 = s1;
+        // Ad carries -t of the first expert inside that expert's block: its steps are needed whenever the second pass runs
+        if (KSEL == 2 && (live0 & 1)) m1 |= s0;
+        md = ((live0 & 2) ? s0 : 0) | ((live1 & 2) ? s1 : 0);
       }
       m0 = __reduce_or_sync(0xffffffffu, (unsigned)m0);
       m1 = __reduce_or_sync(0xffffffffu, (unsigned)m1);
-      if (lane == 0) { atomicOr(&sh_mask[0], m0); atomicOr(&sh_mask[1], m1); }
+      md = __reduce_or_sync(0xffffffffu, (unsigned)md);
+      if (lane == 0) { atomicOr(&sh_mask[0], m0); atomicOr(&sh_mask[1], m1); atomicOr(&sh_mask[2], md); }
     } else {
       failed = true;
     }
@@ -186,7 +198,7 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
     atomicExch(p.status, (int)CMOE_ERR_TIMEOUT);
   }
   __syncthreads();
-  if (threadIdx.x == 64) { p.tile_mask[2 * mt] = sh_mask[0]; p.tile_mask[2 * mt + 1] = sh_mask[1]; }
+  if (threadIdx.x == 64) { p.tile_mask[2 * mt] = sh_mask[0]; p.tile_mask[2 * mt + 1] = sh_mask[1]; p.tile_mask_dn[mt] = sh_mask[2]; }
   if (*abort_flag) {
     const unsigned long long t0 = global_ns();
     while (global_ns() - t0 < 200000ull) { }    // let copies already issued land
@@ -648,7 +660,7 @@ s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_clu
 struct Down2Params {
   const int* n_rows;
   const int* tile_cluster;   // per 256-row tile
-  const int* tile_mask;      // per 128-row tile, two words
+  const int* tile_mask;      // per 128-row tile: 16-wide steps of As V2f^T in use
   const int* row_token;
   __half* y;           // [T][N], original token order
   int* status;
@@ -769,7 +781,7 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
             }
           } else {
             const uint64_t adesc = umma_desc(a_src), bdesc = umma_desc(b_src);
-            const int m = p.tile_mask[4 * pt] | p.tile_mask[4 * pt + 1] | p.tile_mask[4 * pt + 2] | p.tile_mask[4 * pt + 3];
+            const int m = p.tile_mask[2 * pt] | p.tile_mask[2 * pt + 1];        // (the down projection's own table)
 #pragma unroll
             for (int ks = 0; ks < KE / 16; ++ks)
               if ((m >> ks) & 1) umma2_f16(d_tmem, adesc + 2 * ks, bdesc + 2 * ks, IDESC, 1u);
@@ -1056,7 +1068,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
   if (D.r > 0) {
     TParams tp{};
     tp.n_rows = S.n_rows; tp.tile_cluster = S.tile_cluster; tp.row_slot = S.row_slot; tp.row_token = S.row_token;
-    tp.A0 = S.A0; tp.Ad = S.Ad; tp.tile_mask = S.tile_mask; tp.status = S.status;
+    tp.A0 = S.A0; tp.Ad = S.Ad; tp.tile_mask = S.tile_mask; tp.tile_mask_dn = S.tile_mask_dn; tp.live = L->w.live; tp.status = S.status;
     tp.KC = D.d / BK; tp.K = D.K; tp.r = D.r;
     e = D.k == 2 ? launch_t<2>(ts, tp, mt_bound, st) : launch_t<1>(ts, tp, mt_bound, st);
     if (e != cudaSuccess) return e;
@@ -1090,7 +1102,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
   }
   Down2Params dn{};
-  dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask; dn.row_token = S.row_token;
+  dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask_dn; dn.row_token = S.row_token;
   dn.y = y; dn.status = S.status; dn.KC = D.d_ff / (BK * KA); dn.NT = D.d / ts.bn_down; dn.N = D.d;
   {
     const int pairs = ts.sm_count / 2;

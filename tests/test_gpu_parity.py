@@ -558,3 +558,71 @@ def test_expert_stats_empty_batch_and_untouched_centroids():
     torch.cuda.synchronize()
     assert int(loads0.sum()) == 0 and not bool(xbar0.any()) and float(cov0) == 0.0
     m.close()
+
+
+# ---- variants of the same path: bfloat16 bases, and the headline shape at other ranks / k / expert counts ------
+@pytest.mark.parametrize("kw", [
+    dict(T=200, d=96, d_ff=224, E=8, G=2, r=4, k=2),          # generic path
+    dict(T=1500, d=256, d_ff=1024, E=8, G=2, r=16, k=2),      # pair path
+    dict(T=64, d=256, d_ff=384, E=8, G=2, r=8, k=2),          # weight-streaming path
+], ids=["generic", "pair", "stream"])
+def test_bf16_bases(kw):
+    s = inputs.small_shape(**kw)
+    L = inputs.make_layer(s, 81, base_dtype="bf16")
+    full_check(L, L["x"])
+
+
+@pytest.mark.parametrize("kw", [
+    dict(r=4, k=2, E=32, G=8),
+    dict(r=8, k=1, E=32, G=8),
+    dict(r=32, k=2, E=16, G=8),       # K = 2: the widest rank the pair path takes
+    dict(r=16, k=2, E=64, G=16),      # K = 4 with sixteen clusters
+    dict(r=8, k=2, E=64, G=8),        # K = 8
+], ids=["r4", "r8_k1", "r32_K2", "G16", "K8_r8"])
+def test_headline_shape_variants(kw):
+    """T = 16384, d = 1024, d_ff = 4096 with other ranks, k and expert counts, all on the pair path; every row."""
+    s = inputs.small_shape(T=16384, d=1024, d_ff=4096, **kw)
+    L = inputs.make_layer(s, 7)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1
+
+
+def test_many_experts_beyond_the_pair_path():
+    """E = 128 in G = 16 clusters with r = 16 (K r = 128 > 64): the first tensor-core path with the rank-r terms in
+    its epilogue takes it; sampled rows."""
+    s = inputs.small_shape(T=4096, d=1024, d_ff=4096, E=128, G=16, r=16, k=2)
+    L = inputs.make_layer(s, 8)
+    got = full_check(L, L["x"], sample=512)
+    assert got["module"].info.path == 1
+
+
+# ---- zero residual blocks (Sec. 3.4: blocks pruned by the cosine gate) are found at create time and skipped ----
+def _prune(L, which, experts, via):
+    """Zero one factor of the residual block `which` (1: up, 2: down) of the listed experts: `via` = "U" or "V",
+    by its codes ("q") or by its scales ("s")."""
+    s = L["shape"]
+    fac, how = via[0], via[1]
+    name = f"{fac}{which}{how}"
+    a = L[name].copy()
+    per = a.size // s.E
+    for e in experts:
+        a[e * per:(e + 1) * per] = 0
+    L[name] = a
+
+
+@pytest.mark.parametrize("kw", [
+    dict(T=1500, d=256, d_ff=1024, E=8, G=2, r=16, k=2),      # pair path, 256-column up tiles
+    dict(T=1500, d=128, d_ff=768, E=8, G=2, r=16, k=2),       # pair path, whole-row units
+    dict(T=700, d=256, d_ff=384, E=16, G=2, r=8, k=2),        # pair path, 128-column up tiles, two experts per step
+    dict(T=64, d=256, d_ff=384, E=8, G=2, r=8, k=2),          # weight-streaming path
+    dict(T=200, d=96, d_ff=224, E=8, G=2, r=4, k=2),          # generic path
+], ids=["pair_wide", "pair_direct", "pair_narrow_r8", "stream", "generic"])
+def test_zero_residual_blocks_are_skipped_and_change_nothing(kw):
+    s = inputs.small_shape(**kw)
+    L = inputs.make_layer(s, 91, base_scale=0.25, factor_std=0.25)      # residual-dominated: a wrongly skipped block shows
+    _prune(L, 1, [0, 1], "Vq")          # up blocks of experts 0, 1: all codes of V1 zero
+    _prune(L, 1, [2], "Us")             # up block of expert 2: all scales of U1 zero
+    _prune(L, 2, [1, 3], "Uq")          # down blocks of experts 1, 3
+    _prune(L, 2, list(range(s.K, 2 * s.K)), "Vs")      # every down block of cluster 1
+    got = full_check(L, L["x"])
+    assert got["module"].info.pruned_blocks == 3 + 2 + s.K
