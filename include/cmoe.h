@@ -105,6 +105,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *                 about 1e-6)
  *   up_tile       0 automatic; 128 keeps the up projection of large batches on 128-column tiles where d_ff
  *                 would allow 256-column tiles
+ *   host_chunks   0 automatic; 1..8: the most chunks cmoe_forward_host cuts a batch into (chunks stay >= 2048 tokens)
  * and one switch that changes what the descriptor means:
  *   base_dtype    0: desc.B1 / desc.B2 hold fp16 bits (the paper's storage format, Sec. 3.4); 1: they hold bfloat16
  *                 bits.  The tensor cores take both operands of a product in one 16-bit type and the activations
@@ -117,7 +118,8 @@ typedef struct {
   int32_t router_fp32;
   int32_t up_tile;
   int32_t base_dtype;
-  int32_t reserved[4];
+  int32_t host_chunks;
+  int32_t reserved[3];
 } cmoe_options;
 int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
 

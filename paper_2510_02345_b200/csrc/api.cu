@@ -12,6 +12,8 @@ using namespace cmoe;
 
 namespace {
 
+constexpr int kDefaultHostChunks = 4;   // chunks of a large batch in cmoe_forward_host unless the options say otherwise
+
 struct Arena {
   size_t used = 0;
   char* base = nullptr;
@@ -182,7 +184,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   o.force_path = -1;
   if (opt) o = *opt;
   if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
-      o.base_dtype < 0 || o.base_dtype > 1) return CMOE_ERR_INVALID_ARG;
+      o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks) return CMOE_ERR_INVALID_ARG;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -389,8 +391,9 @@ int cmoe_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* y_host
   const size_t row = sizeof(__half) * (size_t)L->dims.d;
   // chunks of at least 2048 tokens, multiples of 256, at most kMaxHostChunks of them
   int n_chunks = T / 2048;
+  const int most = L->opt.host_chunks > 0 ? L->opt.host_chunks : kDefaultHostChunks;
   if (n_chunks < 1) n_chunks = 1;
-  if (n_chunks > kMaxHostChunks) n_chunks = kMaxHostChunks;
+  if (n_chunks > most) n_chunks = most;
   const int per = ((T + n_chunks - 1) / n_chunks + 255) / 256 * 256;
   // the copy streams start after what is already queued on the caller's stream (it may still use the buffers)
   CMOE_CUDA(L, cudaEventRecord(L->host_fork, st));

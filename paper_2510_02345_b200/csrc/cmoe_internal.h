@@ -16,7 +16,7 @@ constexpr int kMaxG = 64;          // clusters
 constexpr int kMaxK = 32;          // experts per cluster (one lane each in the router's top-k)
 constexpr int kMaxKsel = 8;        // k
 constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
-constexpr int kMaxHostChunks = 4; // pipeline depth of cmoe_forward_host
+constexpr int kMaxHostChunks = 8; // most chunks cmoe_forward_host cuts a batch into
 constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels (when they count the keys themselves)
 constexpr int kMinCountTile = 64;  // smallest token tile of a router kernel that counts keys
 

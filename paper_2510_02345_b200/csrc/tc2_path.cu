@@ -15,8 +15,9 @@
 //           epilogue: a_j = GELU(h_j), abar = sum_j p_j a_j (fp16 to HBM), a_j (fp16) to shared
 //           memory as the A operand of  S_j += a_j U2f^T  (accumulated in TMEM over the N tiles of
 //           a row tile, then the row's own block is added to s with fp32 atomics)
-//   expand  As [row][c] = p_j s_j inside the block of expert e_j (fp16)
-//   down    y = abar B2_g^T + As V2f^T, stored un-permuted
+//   down    y = abar B2_g^T + As V2f^T, stored un-permuted, with As [row][c] = p_j s_j inside the block of expert
+//           e_j (fp16): written by the up kernel when its work units are whole row tiles, else by this kernel's
+//           epilogue warps from the fp32 sums s while they wait for a tile's main loop
 //
 // The up and down kernels run as CTA pairs (thread-block clusters of two, tcgen05 cta_group::2) on
 // 256-row tiles: each CTA loads its 128 rows of A and half of the B tile, the leader CTA issues the
@@ -631,30 +632,6 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
 }
 
 // ------------------------------------------------------------------------------------------------
-// expand: As[row][c] = sum_j [c in block of e_j] p_j s_j[c mod r]   (fp16)
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-s_expand_kernel(const int* __restrict__ n_rows, const int* __restrict__ tile_cluster,
-                const int* __restrict__ row_slot, const float* __restrict__ row_gate,
-                const float* __restrict__ s, __half* __restrict__ As, int K, int k, int r, int log2r) {
-  pdl_wait();
-  const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-  const int row = idx >> 3, c0 = (idx & 7) * 8;
-  if (row >= *n_rows) return;
-  const int g = tile_cluster[row / (2 * BM)];
-  __align__(16) __half out[8];
-#pragma unroll
-  for (int n = 0; n < 8; ++n) {
-    const int c = c0 + n, i = c >> log2r, pr = c & (r - 1);
-    float v = 0.f;
-    for (int j = 0; j < k; ++j)
-      if (row_slot[(size_t)row * k + j] - g * K == i) v = fmaf(row_gate[(size_t)row * k + j], s[((size_t)row * k + j) * r + pr], v);
-    out[n] = __float2half_rn(v);
-  }
-  *reinterpret_cast<uint4*>(As + (size_t)row * KE + c0) = *reinterpret_cast<const uint4*>(out);
-}
-
-// ------------------------------------------------------------------------------------------------
 // down: CTA pairs on 256 x BN tiles
 // ------------------------------------------------------------------------------------------------
 struct Down2Params {
@@ -665,6 +642,14 @@ struct Down2Params {
   __half* y;           // [T][N], original token order
   int* status;
   int KC, NT, N;
+  // Not null: the up kernel left the sums s = a_j U2_e in fp32 (its work units were parts of a row tile) and this
+  // kernel turns them into its own operand As[row][block of e_j] = fp16(p_j s_j), row tile by row tile, in the
+  // epilogue warps while they wait for the tile's main loop.
+  const float* s;            // [rows][k][r]
+  const int* row_slot;       // [rows][k]
+  const float* row_gate;     // [rows][k]
+  __half* As;                // [rows][KE]
+  int K, k, r;
 };
 
 constexpr int DN_THREADS = 224;   // warps 0 and 6 TMA (alternating stages), warp 1 MMA, warps 2..5 epilogue
@@ -697,6 +682,7 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
   const uint32_t bar0 = smem_u32(bars);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 20);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+  constexpr int B_ASREADY = 24;       // this CTA's rows of As have been written (four epilogue warps arrive)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const bool leader = rank == 0;
@@ -708,6 +694,7 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(local(B_FULL + s), 1); mbar_init(local(B_EMPTY + s), 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(local(B_TFULL + a), 1); mbar_init(local(B_TEMPTY + a), 8); }
+    mbar_init(local(B_ASREADY), 4);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -750,6 +737,8 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
           tma2_load_3d(a_dst, &tmA3, lead(B_FULL + s), 0, arow, c * KA);
           tma2_load_3d(b_dst, &tmB23, lead(B_FULL + s), 0, brow, c * KA);
         } else {
+          // (this CTA's epilogue warps have written the tile's rows of As, if that is this kernel's job)
+          if (p.s && !mbar_wait(local(B_ASREADY), (uint32_t)ti & 1u, abort_flag)) { failed = true; break; }
           if (leader) mbar_expect_tx(local(B_FULL + s), 2 * (Cfg::A_ATOM + Cfg::B_ATOM));
           tma2_load_2d(a_dst, &tmAs, lead(B_FULL + s), 0, arow);
           tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, brow);
@@ -800,6 +789,35 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
       const int pt = w / NT, nt = w - pt * NT;
       const uint32_t acc = tile_i & 1u, aph = (tile_i >> 1) & 1u;
       const int tok = p.row_token[(2 * pt + (int)rank) * BM + q * 32 + lane];
+      if (HAS_R && p.s) {
+        // As of this thread's row: fp16(p_j s_j) inside the block of e_j, zeros elsewhere (the whole row is written,
+        // so As needs no clearing; tiles of the same row tile write the same values again)
+        const int row = (2 * pt + (int)rank) * BM + q * 32 + lane;
+        const int g = p.tile_cluster[pt];
+        uint4* arow = reinterpret_cast<uint4*>(p.As + (size_t)row * KE);
+#pragma unroll
+        for (int u = 0; u < KE / 8; ++u) {
+          float f[8];
+#pragma unroll
+          for (int n = 0; n < 8; ++n) f[n] = 0.f;
+          if (tok >= 0) {
+            for (int j = 0; j < p.k; ++j) {
+              const int lo = (p.row_slot[(size_t)row * p.k + j] - g * p.K) * p.r;      // first column of the block of e_j
+              const float gate = p.row_gate[(size_t)row * p.k + j];
+              const float* sj = p.s + ((size_t)row * p.k + j) * p.r;
+#pragma unroll
+              for (int n = 0; n < 8; ++n) {
+                const int c = 8 * u + n - lo;
+                if (c >= 0 && c < p.r) f[n] = gate * __ldcg(sj + c);
+              }
+            }
+          }
+          arow[u] = make_uint4(pack_half2(f[0], f[1]), pack_half2(f[2], f[3]), pack_half2(f[4], f[5]), pack_half2(f[6], f[7]));
+        }
+        asm volatile("fence.proxy.async.global;" ::: "memory");      // the tile load of As (async proxy) comes after these writes
+        __syncwarp();
+        if (lane == 0) mbar_arrive(local(B_ASREADY));
+      }
       {
         const bool ok = mbar_wait_cluster(local(B_TFULL + acc), aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -1042,8 +1060,8 @@ int tc2_launch_count(const cmoe_layer* L) {
   const Dims& D = L->dims;
   if (D.r == 0) return 2;
   const Tc2State& ts = *reinterpret_cast<const Tc2State*>(L->tc_state);
-  // t, up, (expansion,) down; the factor staging rides in the router's or the permutation's grid
-  return plan_up(ts, D, D.T_max).direct ? 3 : 4;
+  // t, up, down; the factor staging rides in the router's or the permutation's grid
+  return 3;
 }
 
 // The buffer the forward's first kernels clear for this path: the fp32 sums s, or the down kernel's
@@ -1094,16 +1112,12 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
     if (e != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[2], st);
-  if (D.r > 0 && !plan.direct) {
-    const int threads = rows_bound * 8;
-    launch_chained(s_expand_kernel, dim3((threads + 255) / 256), dim3(256), 0, st, 1,
-      S.n_rows, S.tile_cluster, S.row_slot, S.row_gate, S.s,
-                                                           S.As, D.K, D.k, D.r, ts.log2r);
-    if ((e = cudaGetLastError()) != cudaSuccess) return e;
-  }
   Down2Params dn{};
   dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask_dn; dn.row_token = S.row_token;
   dn.y = y; dn.status = S.status; dn.KC = D.d_ff / (BK * KA); dn.NT = D.d / ts.bn_down; dn.N = D.d;
+  if (D.r > 0 && !plan.direct) {
+    dn.s = S.s; dn.row_slot = S.row_slot; dn.row_gate = S.row_gate; dn.As = S.As; dn.K = D.K; dn.k = D.k; dn.r = D.r;
+  }
   {
     const int pairs = ts.sm_count / 2;
     const long long total = (long long)pt_bound * dn.NT;
