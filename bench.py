@@ -66,15 +66,15 @@ def stage_work(s, T, stage, active_clusters, active_experts):
 # profiles/.  The figure is reported only while
 # the kernel sources still have the hash they had at the capture; otherwise "traffic" is null.
 NCU_TRAFFIC = {
-    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 125.386752e6 + 113.426944e6,
-              "sha1": {"tc2_up_wide.cu": "6e3a4440cd7724fa75b0e4912f4a4c19c6473d9a",
-                       "tc2_common.cuh": "720891980e6ee01fb474e61a99d1a9eb0baa7553",
-                       "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.926528e6 + 10.317568e6,
-               "sha1": {"stream_path.cu": "a187b05075f992b283ec4221cbc552cf30072f42",
+    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 123.953664e6 + 116.289024e6,
+              "sha1": {"tc2_up_wide.cu": "23425974743ca4b7062c11e72b2631012d941af8",
+                       "tc2_common.cuh": "cc74b43ead519c31205497b0115ec5e167d791e0",
+                       "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.886592e6 + 10.025728e6,
+               "sha1": {"stream_path.cu": "c310f832f6387ba82754967036ad94c30024fc45",
                         "device_utils.cuh": "daa6a5fc90a4b02a5c17177e8d154044cca709c4",
-                        "lowrank.cuh": "269b2967c3b968c508c6afb24186bafe32112f8b",
-                        "tc_ptx.cuh": "b87be374de4016935d5b96aaf3dc20e4446ac208"}},
+                        "lowrank.cuh": "698889609319931f08fc77e7b2de29ef206fc1c8",
+                        "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
 }
 
 
@@ -148,12 +148,26 @@ def load_peaks():
 
 
 # ------------------------------------------------------------------ the CUDA arm
+# Variants of the headline shape (the paper sweeps r over {4, 8, 16, 32} and lists E = 128 in G = 16 clusters): timed
+# with `--variants`, reported under "variants" (parity of the same shapes: tests/test_gpu_parity.py).
+VARIANTS = {
+    "gpt2m_r4": dict(r=4), "gpt2m_r8": dict(r=8), "gpt2m_r32_K2": dict(r=32, E=16), "gpt2m_k1": dict(k=1),
+    "gpt2m_G16_K4": dict(E=64, G=16), "gpt2m_K8_r8": dict(E=64, r=8), "gpt2m_E128_G16": dict(E=128, G=16),
+    "gpt2m_bf16_bases": dict(),
+}
+
+
+def variant_shape(name):
+    import dataclasses
+    return dataclasses.replace(inputs.CONFIGS["gpt2m"], name=name, **VARIANTS[name])
+
+
 def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks, dev_index, sync_ranks=True,
                   sustained_s=0.0, keep_outputs=False):
     import torch
     from paper_2510_02345_b200.binding import ClusteredMoELayer, cmoe_profile_enable, cmoe_profile_read
-    s = inputs.CONFIGS[name]
-    L = inputs.make_layer(s, seed=0)
+    s = inputs.CONFIGS[name] if name in inputs.CONFIGS else variant_shape(name)
+    L = inputs.make_layer(s, seed=0, base_dtype="bf16" if name.endswith("bf16_bases") else "fp16")
     x_np = L["x"] if seed_offset == 0 else inputs.make_tokens(s, s.T, seed=seed_offset)
     dev = torch.device(f"cuda:{dev_index}")
     torch.cuda.set_device(dev)
@@ -436,6 +450,7 @@ def main():
     ap.add_argument("--workload", default="gpt2m", choices=list(inputs.CONFIGS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--all", action="store_true", help="also time the other four workloads (short runs)")
+    ap.add_argument("--variants", action="store_true", help="also time the headline shape at other ranks, k and expert counts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true", help="leave the decode workload out of the default line")
     ap.add_argument("--sustained", type=float, default=2.0,
@@ -510,6 +525,15 @@ def main():
                 others[name]["e2e_ms_per_step"] = r2["e2e"]["ms_per_step"]
         if others:
             line["workloads"] = others
+        if args.variants:
+            var = {}
+            for name in VARIANTS:
+                r3 = time_workload(name, 10, 3, rank, 0, False, False, local_rank, sync_ranks=False)
+                ms3 = r3["dev_ms"] / r3["steps"]
+                var[name] = {"tokens_per_s": r3["T"] / (ms3 * 1e-3), "ms_per_step": ms3, "config": config_of(name, r3["shape"], r3["T"], 1),
+                             "layer": whole_layer_fractions(r3, 1, peaks), "stage_ms": r3["stage_ms"], "path": int(r3["info"].path),
+                             "launches_per_forward": int(r3["info"].launches_forward)}
+            line["variants"] = var
         if not args.no_cpu_baseline:
             line["cpu_baseline"], line["parity"] = oracle_rate(args.workload, gpu=res if res.get("y") is not None else None)
         print(json.dumps(line), flush=True)

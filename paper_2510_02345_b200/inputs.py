@@ -180,3 +180,29 @@ def make_tokens(shape: LayerShape, T: int, seed: int) -> np.ndarray:
 def small_shape(name="s", T=37, d=64, d_ff=96, E=6, G=3, r=4, k=2, skew=False) -> LayerShape:
     """Helper for tests: an arbitrary small layer shape."""
     return LayerShape(name, T=T, d=d, d_ff=d_ff, E=E, G=G, r=r, k=k, skew=skew)
+
+
+def make_dense_experts(E: int, G: int, d_in: int, d_out: int, seed: int = 0, spectrum=None, noise: float = 0.0,
+                       base_std: float | None = None) -> np.ndarray:
+    """Dense expert matrices [E][d_in][d_out] (fp32) that are correlated inside each cluster, the input of the offline
+    compressor: W_e = C_g + sum_j spectrum[j] * p_j q_j^T + noise, with a cluster matrix C_g ~ N(0, base_std)
+    (default 1/sqrt(d_in)), orthonormal p_j, q_j per expert (QR of seeded Gaussians) and `spectrum` the singular
+    values of the expert's own part (default: 24 values decaying geometrically from 0.5).  The own parts of a cluster
+    are centred (their mean over the cluster is removed) so that C_g is the cluster's mean up to the noise."""
+    rng = np.random.Generator(np.random.PCG64([seed, 0xC0DE]))
+    K = E // G
+    spectrum = np.asarray(spectrum if spectrum is not None else 0.5 * 0.8 ** np.arange(24), np.float64)
+    n = spectrum.size
+    base_std = 1.0 / math.sqrt(d_in) if base_std is None else base_std
+    W = np.empty((E, d_in, d_out), np.float32)
+    for g in range(G):
+        C = rng.standard_normal((d_in, d_out)) * base_std
+        own = []
+        for _ in range(K):
+            P, _r = np.linalg.qr(rng.standard_normal((d_in, n)))
+            Q, _r = np.linalg.qr(rng.standard_normal((d_out, n)))
+            own.append((P * spectrum[None, :]) @ Q.T + noise * rng.standard_normal((d_in, d_out)))
+        mean_own = sum(own) / K
+        for i in range(K):
+            W[g * K + i] = (C + own[i] - mean_own).astype(np.float32)
+    return W
