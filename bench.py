@@ -358,8 +358,8 @@ def oracle_rate(name, target_s=15.0, max_tokens=None, gpu=None):
     """tokens/s of the CPU oracle on a bounded sample (first n tokens) of the workload.  With `gpu` (the CUDA arm's
     routes and output rows of the same batch) the sample's rows are also compared: the second returned dict."""
     from oracle import ref
-    s = inputs.CONFIGS[name]
-    L = inputs.make_layer(s, seed=0)
+    s = inputs.CONFIGS[name] if name in inputs.CONFIGS else variant_shape(name)
+    L = inputs.make_layer(s, seed=0, base_dtype="bf16" if name.endswith("bf16_bases") else "fp16")
     o = ref.Layer(L)
     T = L["x"].shape[0]
     # every call forms the expert weights first (a fixed cost) and then works per token: two probes
@@ -413,8 +413,8 @@ def run_reference(args, rank):
         return
     from oracle import ref
     name = args.workload
-    s = inputs.CONFIGS[name]
-    L = inputs.make_layer(s, seed=0)
+    s = inputs.CONFIGS[name] if name in inputs.CONFIGS else variant_shape(name)
+    L = inputs.make_layer(s, seed=0, base_dtype="bf16" if name.endswith("bf16_bases") else "fp16")
     o = ref.Layer(L)
     T = L["x"].shape[0]
     # size the per-step sample so that the whole run stays within a few minutes
@@ -447,7 +447,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="gpt2m", choices=list(inputs.CONFIGS))
+    ap.add_argument("--workload", default="gpt2m", choices=list(inputs.CONFIGS) + list(VARIANTS))
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--all", action="store_true", help="also time the other four workloads (short runs)")
     ap.add_argument("--variants", action="store_true", help="also time the headline shape at other ranks, k and expert counts")

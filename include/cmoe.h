@@ -231,6 +231,52 @@ int cmoe_route_static(int32_t d, int32_t E, int32_t G, int32_t k,
                       const void* x, int32_t T,
                       int32_t* cluster_id, int32_t* expert_ids, float* gates, void* cuda_stream);
 
+/* Offline compressor (Sec. 3.2, Eq. 6-7; Sec. 3.4): from E dense expert matrices W_e (d_in x d_out, row-vector
+ * convention; expert slot e = g*K + i belongs to cluster g) to the stored form of one of the layer's two matrices:
+ *   B   [G][d_in][d_out]  fp16  W_base^g = mean of the cluster's experts (Eq. 6)
+ *   Uq  [E][r][d_in], Vq [E][d_out][r]  packed INT4 + fp16 scales Us, Vs (one per 32 consecutive elements), with
+ *       deq(U_e)^T deq(V_e)^T ~ W_e - W_base^g: the rank-r truncated SVD of the residual against the base as stored
+ *       (Eq. 7; singular values split evenly over the two factors), quantised as Sec. 3.4 stores them
+ * so that the outputs of two calls (W1: d_in = d, d_out = d_ff; W2: d_in = d_ff, d_out = d) are the B1, U1q, V1q ... /
+ * B2, U2q, V2q ... fields of cmoe_desc.  The SVD is a randomised range finder with subspace iteration; its Gaussian
+ * test matrices are the caller's input:
+ *   omega [E][d_out][r + oversample] fp32 (standard normal draws), r + oversample <= 48
+ * gamma > 0 switches the cosine gate of Sec. 3.4 on: a residual whose cosine similarity to its base,
+ * <dW, B>_F / (|dW|_F |B|_F), is below gamma becomes a zero block (all codes and scales zero).
+ * Optional outputs (NULL = not wanted): sigma [E][r] singular values, rel_err [E] = |dW - A B^T|_F / |dW|_F before
+ * quantisation, cosine [E], pruned [E], and the fp32 factors A_out [E][d_in][r], Bt_out [E][r][d_out].
+ * All pointers are device pointers; workspace (256-byte aligned) of cmoe_compress_workspace_bytes() bytes is the
+ * caller's; asynchronous on the given stream.  Shapes: E % G == 0, K <= 32, d_in % 32 == d_out % 32 == 0,
+ * r in {4, 8, 16, 32}, power_iters <= 8. */
+typedef struct {
+  int32_t d_in, d_out, E, G, r;
+  int32_t oversample;
+  int32_t power_iters;
+  float gamma;
+  const float* W;
+  const float* omega;
+  uint16_t* B;
+  uint8_t* Uq;
+  uint16_t* Us;
+  uint8_t* Vq;
+  uint16_t* Vs;
+  float* sigma;
+  float* rel_err;
+  float* cosine;
+  int32_t* pruned;
+  float* A_out;
+  float* Bt_out;
+  void* workspace;
+  size_t workspace_bytes;
+} cmoe_compress_desc;
+int cmoe_compress_workspace_bytes(const cmoe_compress_desc* desc, size_t* out_bytes);
+int cmoe_compress(const cmoe_compress_desc* desc, void* cuda_stream);
+
+/* The INT4 quantiser of the stored factors on its own (Sec. 3.4): w [n] fp32 in the stored order, n a multiple of 32
+ * -> q [n / 2] packed codes (16-byte aligned), s [n / 32] fp16 scales; scale = fp16(absmax / 7), code =
+ * clamp(round-half-even(w / scale), -8, 7), even index in the low nibble.  Device pointers; asynchronous. */
+int cmoe_quantize_int4(const float* w, int64_t n, uint8_t* q, uint16_t* s, void* cuda_stream);
+
 /* Frees the host object.  The arena is the caller's. */
 int cmoe_destroy(cmoe_layer* layer);
 

@@ -20,7 +20,8 @@ ERRORS = {
     -1: "CMOE_ERR_INVALID_ARG", -2: "CMOE_ERR_UNSUPPORTED_SHAPE", -3: "CMOE_ERR_WORKSPACE_TOO_SMALL",
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
-EXPORTS = ["cmoe_workspace_bytes", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
+EXPORTS = ["cmoe_compress_workspace_bytes", "cmoe_compress", "cmoe_quantize_int4",
+           "cmoe_workspace_bytes", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
            "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
 CMOE_MAX_STAGES = 8
@@ -44,6 +45,12 @@ class cmoe_options(C.Structure):
                 ("host_chunks", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
+class cmoe_compress_desc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("d_in", "d_out", "E", "G", "r", "oversample", "power_iters")] + [("gamma", C.c_float)] + [
+        (n, C.c_void_p) for n in ("W", "omega", "B", "Uq", "Us", "Vq", "Vs", "sigma", "rel_err", "cosine", "pruned",
+                                  "A_out", "Bt_out", "workspace")] + [("workspace_bytes", C.c_size_t)]
+
+
 class cmoe_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max",
                                          "memsets_forward", "n_stages", "pruned_blocks")]
@@ -63,6 +70,9 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.cmoe_workspace_bytes.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_size_t)]
         L.cmoe_create.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_void_p)]
+        L.cmoe_compress_workspace_bytes.argtypes = [C.POINTER(cmoe_compress_desc), C.POINTER(C.c_size_t)]
+        L.cmoe_compress.argtypes = [C.POINTER(cmoe_compress_desc), C.c_void_p]
+        L.cmoe_quantize_int4.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
         L.cmoe_create_ex.argtypes = [C.POINTER(cmoe_desc), C.POINTER(cmoe_options), C.POINTER(C.c_void_p)]
         L.cmoe_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
         L.cmoe_expert_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
@@ -169,6 +179,53 @@ def cmoe_route_static(d: int, E: int, G: int, k: int, C_ptr, R_ptr, b_c_ptr, b_e
 
 def cmoe_destroy(handle):
     _check(lib().cmoe_destroy(handle), "cmoe_destroy")
+
+
+def compress(W, G: int, r: int, omega, gamma: float = 0.0, power_iters: int = 2):
+    """cmoe_compress on CUDA tensors: W [E][d_in][d_out] fp32, omega [E][d_out][l] fp32 (l = r + oversample).
+    Returns a dict of CUDA tensors: B (fp16), Uq, Us, Vq, Vs, sigma, rel_err, cosine, pruned, A, Bt."""
+    import torch
+    E, d_in, d_out = W.shape
+    l = omega.shape[2]
+    assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+    assert omega.is_cuda and omega.dtype == torch.float32 and omega.is_contiguous() and tuple(omega.shape) == (E, d_out, l)
+    dev = W.device
+    out = dict(B=torch.empty((G, d_in, d_out), dtype=torch.float16, device=dev),
+               Uq=torch.empty((E, r * d_in // 2), dtype=torch.uint8, device=dev),
+               Us=torch.empty((E, r * d_in // 32), dtype=torch.float16, device=dev),
+               Vq=torch.empty((E, d_out * r // 2), dtype=torch.uint8, device=dev),
+               Vs=torch.empty((E, d_out * r // 32), dtype=torch.float16, device=dev),
+               sigma=torch.empty((E, r), dtype=torch.float32, device=dev),
+               rel_err=torch.empty(E, dtype=torch.float32, device=dev),
+               cosine=torch.empty(E, dtype=torch.float32, device=dev),
+               pruned=torch.empty(E, dtype=torch.int32, device=dev),
+               A=torch.empty((E, d_in, r), dtype=torch.float32, device=dev),
+               Bt=torch.empty((E, r, d_out), dtype=torch.float32, device=dev))
+    d = cmoe_compress_desc()
+    d.d_in, d.d_out, d.E, d.G, d.r, d.oversample, d.power_iters, d.gamma = d_in, d_out, E, G, r, l - r, power_iters, gamma
+    d.W, d.omega = W.data_ptr(), omega.data_ptr()
+    for name, field in (("B", "B"), ("Uq", "Uq"), ("Us", "Us"), ("Vq", "Vq"), ("Vs", "Vs"), ("sigma", "sigma"),
+                        ("rel_err", "rel_err"), ("cosine", "cosine"), ("pruned", "pruned"), ("A", "A_out"), ("Bt", "Bt_out")):
+        setattr(d, field, out[name].data_ptr())
+    need = C.c_size_t(0)
+    _check(lib().cmoe_compress_workspace_bytes(C.byref(d), C.byref(need)), "cmoe_compress_workspace_bytes")
+    ws = torch.empty(need.value + 256, dtype=torch.uint8, device=dev)
+    d.workspace = (ws.data_ptr() + 255) // 256 * 256
+    d.workspace_bytes = need.value
+    _check(lib().cmoe_compress(C.byref(d), torch.cuda.current_stream(dev).cuda_stream), "cmoe_compress")
+    out["_workspace"] = ws          # keeps the scratch alive until the caller has synchronised
+    return out
+
+
+def quantize_int4(w):
+    """cmoe_quantize_int4 on a CUDA fp32 tensor (size a multiple of 32) -> (packed uint8, fp16 scales)."""
+    import torch
+    assert w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and w.numel() % 32 == 0
+    q = torch.empty(w.numel() // 2, dtype=torch.uint8, device=w.device)
+    s = torch.empty(w.numel() // 32, dtype=torch.float16, device=w.device)
+    _check(lib().cmoe_quantize_int4(w.data_ptr(), w.numel(), q.data_ptr(), s.data_ptr(),
+                                    torch.cuda.current_stream(w.device).cuda_stream), "cmoe_quantize_int4")
+    return q, s
 
 
 # ---- convenience owner of the device buffers ---------------------------------------------------

@@ -349,10 +349,9 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc));
     counted_tile = router_tc_tile_tokens();
   } else {
-    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc, &fs));
-    counted_tile = router_tile_tokens(T);
+    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &fs));
   }
-  if (T < 1024) fs = FactorStage{};     // staged beside the per-token router
+  if (T < 1024) fs = FactorStage{};     // staged beside the per-token router (else by the row-move kernel)
   CMOE_MARK();
   {
     // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s
@@ -442,7 +441,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   *out = cmoe_info{};
   out->path = L->path;
   out->launches_route = 1;
-  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, L->dims.T_max < 1024 ? 0 : (L->router_tc ? router_tc_tile_tokens() : router_tile_tokens(L->dims.T_max))) +
+  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));

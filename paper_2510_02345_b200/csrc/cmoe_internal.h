@@ -18,7 +18,7 @@ constexpr int kMaxKsel = 8;        // k
 constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
 constexpr int kMaxHostChunks = 8; // most chunks cmoe_forward_host cuts a batch into
 constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels (when they count the keys themselves)
-constexpr int kMinCountTile = 64;  // smallest token tile of a router kernel that counts keys
+constexpr int kMinCountTile = 128; // token tile of the router kernel that counts keys (router_tc.cu)
 
 enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
 
@@ -126,20 +126,18 @@ inline int t_pad_bound(const Dims& D, int T) { return round_up(T, D.row_align) +
 
 // ---- launchers (each returns the cudaError_t of its launches) ----------------------------------
 // router.cu
-// kc (or null): the kernel also writes every token's permutation key and, for batches of at least 1024 tokens, the
-// key counts of its token tiles (router_tile_tokens(T) tokens each; 0: it counts nothing).  fs (or null): factor
-// staging that rides in the per-token kernel's grid (batches below 1024 tokens).
+// fs (or null): factor staging that rides in the per-token kernel's grid (batches below 1024 tokens)
 struct KeyCount;      // perm_keys.cuh
 struct FactorStage;   // stage_factors.cuh
 struct LowrankTok;    // lowrank.cuh
 cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int T,
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
-                          cudaStream_t st, const KeyCount* kc = nullptr, const FactorStage* fs = nullptr);
-int router_tile_tokens(int T);
+                          cudaStream_t st, const FactorStage* fs = nullptr);
 // router_tc.cu : the same routing on the tensor cores (split fp16 router matrices), for large batches
 int router_tc_rp(const Dims& D);
 bool router_tc_supported(const Dims& D);
 cudaError_t router_tc_init(cmoe_layer* L);
+// kc (or null): the kernel also writes every token's permutation key and the key counts of its 128-token tiles
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
                              int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr);
 int router_tc_tile_tokens();

@@ -1,6 +1,6 @@
 // The permutation key of a token: cluster * nsub + (rank of its set of kept experts among the k-subsets of the
-// cluster's K experts, or its lowest kept expert when there are too many subsets).  Shared by the router kernels,
-// which count the keys of their token tile, and the permutation kernels.  Also: what a router kernel is handed
+// cluster's K experts, or its lowest kept expert when there are too many subsets).  Shared by the tensor-core router
+// kernel, which counts the keys of its token tile, and the permutation kernels.  Also: what a router kernel is handed
 // when it runs as the first kernel of a forward (key counts, and the factor-staging work that rides in its grid).
 #pragma once
 

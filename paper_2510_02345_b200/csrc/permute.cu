@@ -61,17 +61,26 @@ scan_kernel(int nblk, int G, int nsub, int nkey, int row_align, int max_tiles,
   const int lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   for (int key = threadIdx.x >> 5; key < nkey; key += nwarp) {
     int run = 0;
-    for (int b0 = 0; b0 < nblk; b0 += 32) {
-      const int b = b0 + lane;
-      const int c = b < nblk ? block_counts[(size_t)b * nkey + key] : 0;
-      int incl = c;
+    for (int b0 = 0; b0 < nblk; b0 += 256) {
+      // eight loads per lane in flight (blocks b0 + 32 i + lane), then eight warp scans
+      int c[8];
 #pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
+      for (int i = 0; i < 8; ++i) {
+        const int b = b0 + 32 * i + lane;
+        c[i] = b < nblk ? block_counts[(size_t)b * nkey + key] : 0;
       }
-      if (b < nblk) block_base[(size_t)b * nkey + key] = run + incl - c;
-      run += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int b = b0 + 32 * i + lane;
+        int incl = c[i];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int up = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += up;
+        }
+        if (b < nblk) block_base[(size_t)b * nkey + key] = run + incl - c[i];
+        run += __shfl_sync(0xffffffffu, incl, 31);
+      }
     }
     if (lane == 0) { key_cnt[key] = run; sh_cnt[key] = run; }
   }
@@ -127,8 +136,8 @@ struct ScanInline {
   int *seg_off, *seg_cnt, *n_rows, *tile_cluster;
 };
 
-__global__ void __launch_bounds__(kPermBlock)      // 64, 128 or 256 threads: the token tile of the kernel that counted the keys
-scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
+__global__ void __launch_bounds__(512)      // at least `tile` threads: the token tile of the kernel that counted the keys
+scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
                const __half* __restrict__ x, const int* __restrict__ cluster_id,
                const int* __restrict__ slot, const float* __restrict__ gates,
                const int* __restrict__ keys, const int* __restrict__ block_base,
@@ -141,22 +150,30 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
     int* sh_tot = sh_next + nkey;    // [nkey] tokens of each key in the whole batch
     __shared__ int sh_seg[kMaxG + 1];
     __shared__ int sh_segcnt[kMaxG];
-    // a warp per key, lanes over the counting blocks: the key's total and the part of the blocks before this one
+    // Column sums of the count table, read along its rows: lanes over the keys (four columns of 32 keys per pass),
+    // warps over the counting blocks; a key's total and the part of the blocks before this one.
+    for (int key = threadIdx.x; key < nkey; key += blockDim.x) { sh_tot[key] = 0; sh_next[key] = 0; }
+    __syncthreads();
     {
       const int lane_ = threadIdx.x & 31, warp_ = threadIdx.x >> 5, nwarp_ = blockDim.x >> 5;
-      for (int key = warp_; key < nkey; key += nwarp_) {
-        int tot = 0, before = 0;
-        for (int b = lane_; b < si.nblk; b += 32) {
-          const int c = si.counts[(size_t)b * nkey + key];
-          tot += c;
-          before += b < (int)blockIdx.x ? c : 0;
+      for (int k0 = 0; k0 < nkey; k0 += 128) {
+        int tot[4] = {0, 0, 0, 0}, bef[4] = {0, 0, 0, 0};
+#pragma unroll 4
+        for (int b = warp_; b < si.nblk; b += nwarp_) {
+          const bool before = b < (int)blockIdx.x;
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int key = k0 + 32 * j + lane_;
+            const int c = key < nkey ? si.counts[(size_t)b * nkey + key] : 0;
+            tot[j] += c;
+            bef[j] += before ? c : 0;
+          }
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          tot += __shfl_xor_sync(0xffffffffu, tot, o);
-          before += __shfl_xor_sync(0xffffffffu, before, o);
+        for (int j = 0; j < 4; ++j) {
+          const int key = k0 + 32 * j + lane_;
+          if (key < nkey) { atomicAdd(&sh_tot[key], tot[j]); atomicAdd(&sh_next[key], bef[j]); }
         }
-        if (lane_ == 0) { sh_tot[key] = tot; sh_next[key] = before; }
       }
     }
     __syncthreads();
@@ -219,15 +236,15 @@ scatter_kernel(int T, int d, int K, int k, int nkey, int sub_is_combo,
   }
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;        // a block takes the tokens one counting block took
-  const bool live = t < T;
+  const int t = blockIdx.x * tile + threadIdx.x;              // a block takes the tokens one counting block took,
+  const bool live = (int)threadIdx.x < tile && t < T;         // a thread each (the block may have more threads: they help with the sums above)
   const int key = live ? keys[t] : -1 - lane;     // dead lanes get unique keys: groups of one
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
   const bool leader = rank_in_warp == 0;
   int row = -1;
   // warps take their rows in warp order, so rows of a key stay in token order
-  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) {
+  for (int w = 0; w < (tile >> 5); ++w) {
     if (warp == w && live) {
       row = sh_next[key] + rank_in_warp;
     }
@@ -365,7 +382,7 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
 }
 
 // the count table is small enough for every scatter block to sum it itself
-bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk * D.nkey <= 16384 && D.G <= tile; }
+bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk * D.nkey <= 65536 && D.G <= tile; }
 
 }  // namespace
 
@@ -411,8 +428,8 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                                     S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
                                     S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
   }
-  launch_chained(scatter_kernel, dim3(nblk), dim3(tile), sh * (inline_scan ? 2 : 1), st, 1,
-      T, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
+  launch_chained(scatter_kernel, dim3(nblk), dim3(inline_scan ? 512 : tile), sh * (inline_scan ? 2 : 1), st, 1,
+      T, tile, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
                                                S.x_perm, si);

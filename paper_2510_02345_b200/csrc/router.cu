@@ -16,7 +16,7 @@
 #include "cmoe_internal.h"
 #include "launch.cuh"
 #include "device_utils.cuh"
-#include "perm_keys.cuh"
+#include "stage_factors.cuh"
 
 namespace cmoe {
 
@@ -39,11 +39,9 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& xv, const float4& 
 
 // Top-k of K logits (ties: lowest index), gates = softmax over the kept logits (Eq. 10
 // renormalised over the kept experts); one thread per token, logits read from `lg`.
-// Returns the token's permutation key when kc asks for keys (else -1).
-__device__ __forceinline__ int select_and_store(const float* lg, int K, int k, int g, int t,
-                                                const int* __restrict__ label, int* __restrict__ expert_ids,
-                                                float* __restrict__ gates, int* __restrict__ slot_local,
-                                                const KeyCount& kc) {
+__device__ __forceinline__ void select_and_store(const float* lg, int K, int k, int g, int t,
+                                                 const int* __restrict__ label, int* __restrict__ expert_ids,
+                                                 float* __restrict__ gates, int* __restrict__ slot_local) {
   unsigned taken = 0;
   float selv[kMaxKsel];
   int seli[kMaxKsel];
@@ -65,17 +63,10 @@ __device__ __forceinline__ int select_and_store(const float* lg, int K, int k, i
   float sum = 0.f;
   for (int s = 0; s < k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
   for (int s = 0; s < k; ++s) {
-    ev[s] = ev[s] / sum;
-    if (gates) gates[(size_t)t * k + s] = ev[s];
+    if (gates) gates[(size_t)t * k + s] = ev[s] / sum;
     if (expert_ids) expert_ids[(size_t)t * k + s] = label[g * K + seli[s]];
     if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
   }
-  if (!kc.keys) return -1;
-  int cs[kMaxKsel];
-  float cg[kMaxKsel];
-  const int key = g * kc.nsub + canonical_slots(seli, ev, k, kc.sub_is_combo, cs, cg);
-  kc.keys[t] = key;
-  return key;
 }
 
 struct RouterArgs {
@@ -87,7 +78,6 @@ struct RouterArgs {
   int* expert_ids;
   float* gates;
   int* slot_local;
-  KeyCount kc;     // key counting for the permutation (keys == nullptr: routing only)
   FactorStage fs;  // per-token kernel only: factor staging that rides in the blocks past the router's own (all words zero: none)
   int n_route_blocks, n_riders;
   int dc;          // columns of the cluster prototypes staged in shared memory at a time
@@ -235,20 +225,9 @@ router_tile_kernel(const RouterArgs a) {
   __syncthreads();
 
   // ---- top-k and gates: one thread per token
-  int key = -1;
   if (threadIdx.x < kTileTokens && tok0 + threadIdx.x < a.T)
-    key = select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
-                           a.expert_ids, a.gates, a.slot_local, a.kc);
-  if (a.kc.keys) {
-    // keys of this tile counted in shared memory (over the prototype buffer, which is no longer read)
-    int* cnt = reinterpret_cast<int*>(sm_f);
-    __syncthreads();
-    for (int i = threadIdx.x; i < a.kc.nkey; i += blockDim.x) cnt[i] = 0;
-    __syncthreads();
-    if (key >= 0) atomicAdd(&cnt[key], 1);
-    __syncthreads();
-    for (int i = threadIdx.x; i < a.kc.nkey; i += blockDim.x) a.kc.block_counts[(size_t)blockIdx.x * a.kc.nkey + i] = cnt[i];
-  }
+    select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
+                     a.expert_ids, a.gates, a.slot_local);
 }
 
 // One block per token; warp w computes the rows w, w + nwarp, ... of the router matrix, each over all of d
@@ -304,16 +283,14 @@ router_token_kernel(const RouterArgs a) {
       __syncthreads();
     }
   }
-  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, KeyCount{});
+  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local);
 }
 
 }  // namespace
 
-int router_tile_tokens(int T) { return T < 1024 ? 0 : kTileTokens; }
-
 cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int T,
                           int* cluster_id, int* expert_ids, float* gates, int* slot_local,
-                          cudaStream_t st, const KeyCount* kc, const FactorStage* fs) {
+                          cudaStream_t st, const FactorStage* fs) {
   if (T <= 0) return cudaSuccess;
   RouterArgs a{};
   // (the staging of the tensor-core residual factors rides here for batches below 1024 tokens, else in the
@@ -330,15 +307,13 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
       a);
     return cudaGetLastError();
   }
-  if (kc) a.kc = *kc;
   // chunk of the prototypes staged at a time: at most 32 KB for a group of eight clusters
   const int rows = D.G < kGroup ? D.G : kGroup;
   int dc = 32768 / (4 * rows) / 256 * 256;
   if (dc > D.d) dc = D.d;
   a.dc = dc;
   a.crows = rows;
-  size_t sh = sizeof(float) * ((size_t)rows * dc + (size_t)kTileTokens * D.K);      // at most 32 KB + 8 KB
-  if (a.kc.keys && sh < sizeof(int) * (size_t)a.kc.nkey) sh = sizeof(int) * (size_t)a.kc.nkey;   // the key counts reuse the buffer
+  const size_t sh = sizeof(float) * ((size_t)rows * dc + (size_t)kTileTokens * D.K);      // at most 32 KB + 8 KB
   static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
   if (cudaError_t e = ensure_dynamic_smem(router_tile_kernel, 64 * 1024, smem_set)) return e;
   launch_chained(router_tile_kernel, dim3((T + kTileTokens - 1) / kTileTokens), dim3(kTileWarps * 32), sh, st, 1,

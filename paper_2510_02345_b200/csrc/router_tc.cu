@@ -26,7 +26,7 @@ constexpr int RBM = 128;          // tokens per tile
 constexpr int RBK = 64;           // halves per K atom
 constexpr int RKA = 2;            // K atoms per stage
 constexpr int R_THREADS = 224;    // warps 0, 6 TMA (alternating stages), 1 MMA, 2..5 epilogue
-constexpr int R_STAGES = 4;
+constexpr int R_MAX_STAGES = 4;    // stages of the operand ring: as many as shared memory allows for the router's width (2..4)
 
 struct RtcParams {
   int T, d, G, K, k, E;
@@ -39,6 +39,7 @@ struct RtcParams {
   int* slot_local;
   int* status;
   KeyCount kc;     // key counting for the permutation (keys == nullptr: routing only)
+  int stages;      // stages of the operand ring
 };
 
 // fp32 router rows -> the two fp16 pieces, rows [hi_0 .. hi_{rp-1}, lo_0 .. lo_{rp-1}] x d (padding rows zero)
@@ -67,6 +68,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   const int N = 2 * p.rp;
   const uint32_t a_atom = RBM * RBK * 2, b_atom = (uint32_t)N * RBK * 2;
   const uint32_t a_bytes = RKA * a_atom, b_bytes = RKA * b_atom, st_bytes = a_bytes + b_bytes;   // b_atom is a multiple of 1024
+  const int R_STAGES = p.stages;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sm + (size_t)R_STAGES * st_bytes);
   const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + 8), tfull = smem_u32(bars + 16);
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 17);
@@ -250,10 +252,17 @@ bool make_map3(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, 
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-size_t rtc_smem(int N) {
-  const size_t ring = (size_t)R_STAGES * RKA * (RBM + N) * RBK * 2;
+size_t rtc_smem(int N, int stages) {
+  const size_t ring = (size_t)stages * RKA * (RBM + N) * RBK * 2;
   const size_t logits = (size_t)RBM * (N + 1) * 4 + (size_t)(RBM + kMaxKeys) * 4;   // logits, keys of the tile, key counts
   return 1024 + (ring > logits ? ring : logits) + 32 * 8;
+}
+
+// the deepest ring that fits (0: the router is too wide for this kernel)
+int rtc_stages(int N) {
+  for (int st = R_MAX_STAGES; st >= 2; --st)
+    if (rtc_smem(N, st) <= 232448) return st;
+  return 0;
 }
 
 }  // namespace
@@ -262,7 +271,7 @@ int router_tc_rp(const Dims& D) { return (D.G + D.E + 7) / 8 * 8; }
 
 bool router_tc_supported(const Dims& D) {
   const int N = 2 * router_tc_rp(D);
-  return D.d % (RBK * RKA) == 0 && N <= 256 && D.T_max >= 1024 && rtc_smem(N) <= 232448;
+  return D.d % (RBK * RKA) == 0 && N <= 256 && D.T_max >= 1024 && rtc_stages(N) > 0;
 }
 
 cudaError_t router_tc_init(cmoe_layer* L) {
@@ -273,7 +282,7 @@ cudaError_t router_tc_init(cmoe_layer* L) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (!make_map3(&L->router_map_w, L->sc.Wsplit, (uint64_t)2 * rp, D.d, (uint32_t)(2 * rp))) return cudaErrorInvalidValue;
-  e = cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rtc_smem(2 * rp));
+  e = cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rtc_smem(2 * rp, rtc_stages(2 * rp)));
   if (e != cudaSuccess) return e;
   return cudaDeviceSynchronize();
 }
@@ -290,7 +299,8 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
   p.bc = L->w.bc; p.be = L->w.be; p.label = L->w.label;
   p.cluster_id = cluster_id; p.expert_ids = expert_ids; p.gates = gates; p.slot_local = slot_local; p.status = L->sc.status;
   if (kc) p.kc = *kc;
-  return launch_chained(router_tc_kernel, dim3((unsigned)((T + RBM - 1) / RBM)), dim3(R_THREADS), rtc_smem(2 * p.rp), st, 1, mx,
+  p.stages = rtc_stages(2 * p.rp);
+  return launch_chained(router_tc_kernel, dim3((unsigned)((T + RBM - 1) / RBM)), dim3(R_THREADS), rtc_smem(2 * p.rp, p.stages), st, 1, mx,
                         L->router_map_w, p);
 }
 
