@@ -336,16 +336,7 @@ lowrank_body(const int* __restrict__ seg_off, int G, int k, int r, int len, int 
   lowrank_rows(xin, e, r, len, blockIdx.y * nwarp, gridDim.y * nwarp, Uq, Us, out + (size_t)item * r);
 }
 
-__global__ void __launch_bounds__(256)
-lowrank_kernel(const int* __restrict__ seg_off, int G, int k, int r, int len, int in_per_slot,
-               const __half* __restrict__ in, const int* __restrict__ row_slot, const int* __restrict__ row_token,
-               const uint8_t* __restrict__ Uq, const __half* __restrict__ Us, float* __restrict__ out,
-               const int* __restrict__ live, int live_bit) {
-  pdl_wait();
-  lowrank_body(seg_off, G, k, r, len, in_per_slot, in, row_slot, row_token, Uq, Us, out, live, live_bit);
-}
-
-// The same for the second stream: s = a_j U2 is not needed before the last kernel of the forward, so it
+// On the second stream: s = a_j U2 is not needed before the last kernel of the forward, so it
 // runs beside the down kernel.  That kernel holds 640 threads x 96 registers of every SM; four warps of
 // 32 registers are what fits next to it.
 constexpr int kSideThreads = 128;
