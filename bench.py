@@ -70,8 +70,8 @@ NCU_TRAFFIC = {
               "sha1": {"tc2_up_wide.cu": "23425974743ca4b7062c11e72b2631012d941af8",
                        "tc2_common.cuh": "cc74b43ead519c31205497b0115ec5e167d791e0",
                        "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.886592e6 + 10.025728e6,
-               "sha1": {"stream_path.cu": "c310f832f6387ba82754967036ad94c30024fc45",
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.824896e6 + 9.873408e6,
+               "sha1": {"stream_path.cu": "56f3a492ae638749f58a73aa07eeb29bb207b097",
                         "device_utils.cuh": "daa6a5fc90a4b02a5c17177e8d154044cca709c4",
                         "lowrank.cuh": "698889609319931f08fc77e7b2de29ef206fc1c8",
                         "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
