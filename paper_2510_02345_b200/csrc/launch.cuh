@@ -1,8 +1,11 @@
-// Kernel launches of the forward chain.  Every kernel of the chain starts with pdl_wait() and is
-// launched with programmatic stream serialization: the next kernel's blocks may be scheduled while
-// the previous kernel is still draining, and wait at their first instruction until it has completed
-// and its writes are visible.  Nothing else overlaps; what is saved is the launch gap between the
-// dozen short kernels of one forward.
+// Kernel launches of the forward chain.  Every kernel of the chain is launched with programmatic
+// stream serialization and calls pdl_wait() before it touches anything an earlier kernel wrote: its
+// blocks may be scheduled while the previous kernel is still draining, and wait there until that
+// kernel has completed and its writes are visible.  The persistent kernels (grids of at most one block
+// per SM) put the wait after their set-up (barriers, tensor-memory allocation) and then call
+// pdl_release_dependents(), so that the next kernel's blocks take each SM as soon as a block of this
+// grid leaves it and have their own set-up done by the time the grid has finished.  Nothing else
+// overlaps; what is saved is the launch gap and the set-up between the kernels of one forward.
 #pragma once
 
 #include <atomic>
@@ -29,6 +32,17 @@ inline cudaError_t ensure_dynamic_smem(Kern kern, size_t bytes, std::atomic<unsi
 
 // Blocks until the kernels this one depends on have completed (a no-op for an ordinary launch).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Lets the next kernel of the chain be scheduled before this grid has finished (its blocks still wait in
+// pdl_wait() for this grid's completion).  Called after this kernel's own pdl_wait(), so at most two kernels
+// of the chain are on the device, and only by grids that are resident as a whole (no more blocks than SMs):
+// every block of such a grid already has its SM, so a dependent block can only take an SM that a block of this
+// grid has left, never one that a block of this grid still waits for.
+__device__ __forceinline__ void pdl_release_dependents() {
+  uint32_t nsm;
+  asm("mov.u32 %0, %%nsmid;" : "=r"(nsm));
+  if (gridDim.x * gridDim.y * gridDim.z <= nsm) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // cluster = 2 launches thread-block clusters of two CTAs (grid.x must be even)
 template <typename... KArgs, typename... Args>

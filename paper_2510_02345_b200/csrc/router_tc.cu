@@ -61,6 +61,7 @@ router_split_kernel(const float* __restrict__ Ct, const float* __restrict__ Rt, 
 __global__ void __launch_bounds__(R_THREADS, 1)
 router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, const RtcParams p) {
   pdl_wait();
+  pdl_release_dependents();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;

@@ -80,7 +80,6 @@ template <bool UP>
 __global__ void __launch_bounds__(S_THREADS, 1)
 stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ SliceMaps tmWs,
               const __grid_constant__ CUtensorMap tmTok, const StreamParams p) {
-  pdl_wait();
   constexpr int MROWS = 128;
   using Cfg = SCfg<MROWS>;
   constexpr int STAGES = Cfg::STAGES;
@@ -106,21 +105,35 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
     for (int a = 0; a < 2; ++a) { mbar_init(tfull0 + 8 * a, 1); mbar_init(tempty0 + 8 * a, kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    // segments of at most SNB rows
-    int n = 0;
-    for (int g = 0; g < p.G; ++g) {
-      const int r0 = p.seg_off[g], r1 = p.seg_off[g + 1];
-      for (int r = r0; r < r1 && n < SMAXSEG; r += SNB) {
-        seg_row0[n] = r; seg_rows[n] = min(SNB, r1 - r); seg_g[n] = g; ++n;
-      }
-    }
-    *n_seg_p = n;
   }
   if (warp == 2) {
-    __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_holder)), "r"(S_TMEM_COLS) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  pdl_wait();                  // nothing above reads what an earlier kernel wrote
+  pdl_release_dependents();
+  if (warp == 0) {
+    // segments of at most SNB rows, in cluster order: a lane per cluster (32 at a time), so that the reads of
+    // the offsets table are one round trip instead of G dependent ones
+    __syncwarp();
+    int n = 0;
+    for (int g0 = 0; g0 < p.G; g0 += 32) {
+      const int g = g0 + lane;
+      int r0 = 0, r1 = 0;
+      if (g < p.G) { r0 = p.seg_off[g]; r1 = p.seg_off[g + 1]; }
+      const int cnt = (r1 - r0 + SNB - 1) / SNB;
+      int incl = cnt;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      int at = n + incl - cnt;
+      for (int r = r0; r < r1 && at < SMAXSEG; r += SNB, ++at) { seg_row0[at] = r; seg_rows[at] = min(SNB, r1 - r); seg_g[at] = g; }
+      n += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) *n_seg_p = min(n, SMAXSEG);
   }
   tc_fence_before();
   __syncthreads();
@@ -227,12 +240,87 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
       const int row0 = seg_row0[seg], nrows = q * 32 < srows ? seg_rows[seg] : 0;
       const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
       const int f = mt * MROWS + (slice < 0 ? 0 : slice * srows) + q * 32 + lane;   // output feature (up) / output column (down)
+      // Residual operands of one block of 16 token columns: for each of this warp's four columns and up to two
+      // kept experts, the r INT4 codes and the scale of this thread's feature row of V1.  The first block is
+      // requested before the accumulator is complete, so that the latency of these scattered reads (three
+      // dependent table lookups, then HBM) hides behind the tile's weight stream instead of adding up, column
+      // after column, between two tiles.
+      constexpr int PJ = 2;
+      const bool pre = UP && r > 0 && k <= PJ;
+      uint32_t wq[4][PJ][4];
+      float wsc[4][PJ];
+      auto load_codes = [&](int e, uint32_t (&w)[4], float& sc) {
+        const long long flat = ((long long)e * M + f) * r;           // the r codes of (e, f) are one scale group
+        const uint8_t* src = p.V1q + (flat >> 1);
+        sc = __half2float(p.V1s[flat >> 5]);
+        w[1] = w[2] = w[3] = 0u;
+        if (r == 32) {
+          const uint4 v4 = *reinterpret_cast<const uint4*>(src);
+          w[0] = v4.x; w[1] = v4.y; w[2] = v4.z; w[3] = v4.w;
+        } else if (r == 16) {
+          const uint2 v2 = *reinterpret_cast<const uint2*>(src);
+          w[0] = v2.x; w[1] = v2.y;
+        } else if (r == 8) {
+          w[0] = *reinterpret_cast<const uint32_t*>(src);
+        } else {
+          w[0] = *reinterpret_cast<const uint16_t*>(src);
+        }
+      };
+      auto preload = [&](int tb) {
+#pragma unroll
+        for (int c2 = 0; c2 < 4; ++c2) {
+          const int row = row0 + tb + 4 * c2 + part;
+          const bool real = mine && p.row_token[row] >= 0;
+#pragma unroll
+          for (int j = 0; j < PJ; ++j) {
+            wsc[c2][j] = 0.f;
+            wq[c2][j][0] = wq[c2][j][1] = wq[c2][j][2] = wq[c2][j][3] = 0u;
+            if (real && j < k) {
+              const int e = p.row_slot[(size_t)row * k + j];
+              if (p.live[e] & 1) load_codes(e, wq[c2][j], wsc[c2][j]);      // (a zero residual block is skipped: Sec. 3.4)
+            }
+          }
+        }
+      };
+      // h = dv + sc (t_j . codes): the r codes decoded in registers
+      auto residual = [&](float dv, const float4* tp, const uint32_t (&w)[4], float sc) -> float {
+        float dot0 = 0.f, dot1 = 0.f;
+        if (r >= 8) {
+#pragma unroll
+          for (int w8 = 0; w8 < 4; ++w8) {
+            if (w8 < r / 8) {
+              float cf[8];
+              int4x8_to_float(w[w8], cf);
+              const float4 ta = tp[2 * w8], tb4 = tp[2 * w8 + 1];
+              dot0 = fmaf(ta.x, cf[0], dot0);
+              dot1 = fmaf(ta.y, cf[1], dot1);
+              dot0 = fmaf(ta.z, cf[2], dot0);
+              dot1 = fmaf(ta.w, cf[3], dot1);
+              dot0 = fmaf(tb4.x, cf[4], dot0);
+              dot1 = fmaf(tb4.y, cf[5], dot1);
+              dot0 = fmaf(tb4.z, cf[6], dot0);
+              dot1 = fmaf(tb4.w, cf[7], dot1);
+            }
+          }
+        } else {
+          float cf[8];
+          int4x8_to_float(w[0], cf);
+          const float4 ta = tp[0];
+          dot0 = fmaf(ta.x, cf[0], dot0);
+          dot1 = fmaf(ta.y, cf[1], dot1);
+          dot0 = fmaf(ta.z, cf[2], dot0);
+          dot1 = fmaf(ta.w, cf[3], dot1);
+        }
+        return fmaf(sc, dot0 + dot1, dv);
+      };
+      if (pre && nrows > 0) preload(0);
       {
         const bool ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       }
       tc_fence_after();
       for (int tb = 0; tb < nrows; tb += 16) {
+        if (pre && tb > 0) preload(tb);
         uint32_t v[16];
         tmem_ld16_nowait(taddr + acc * SNB + tb, v);
         tmem_ld_wait();
@@ -245,40 +333,26 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
           const float dv = __uint_as_float(part == 0 ? v[4 * c2] : part == 1 ? v[4 * c2 + 1] : part == 2 ? v[4 * c2 + 2] : v[4 * c2 + 3]);
           if (UP) {
             float ab = 0.f;
-            if (real) {
+            if (real && pre) {
+#pragma unroll
+              for (int j = 0; j < PJ; ++j) {
+                if (j < k) {
+                  // a zero residual block has scale and codes 0 here: h = dv
+                  const float h = residual(dv, reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r), wq[c2][j], wsc[c2][j]);
+                  const float a = gelu_erf(h);
+                  ab = fmaf(p.row_gate[(size_t)row * k + j], a, ab);
+                  p.a_slot[((size_t)row * k + j) * M + f] = __float2half_rn(a);
+                }
+              }
+            } else if (real) {
               for (int j = 0; j < k; ++j) {
                 const int e = p.row_slot[(size_t)row * k + j];
                 float h = dv;
-                if (r > 0 && (p.live[e] & 1)) {      // (a zero residual block is skipped: Sec. 3.4)
-                  // h += t_j . V1_e[f, :]: r codes of one scale group, decoded in registers
-                  const float4* tp = reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r);    // t is indexed by token
-                  const long long flat = ((long long)e * M + f) * r;
-                  const float sc = __half2float(p.V1s[flat >> 5]);
-                  float dot0 = 0.f, dot1 = 0.f;
-                  if (r >= 8) {
-                    const uint32_t* wq = reinterpret_cast<const uint32_t*>(p.V1q + (flat >> 1));
-                    for (int w8 = 0; w8 < r / 8; ++w8) {
-                      float cf[8];
-                      int4x8_to_float(wq[w8], cf);
-                      const float4 ta = tp[2 * w8], tb4 = tp[2 * w8 + 1];
-                      dot0 = fmaf(ta.x, cf[0], dot0);
-                      dot1 = fmaf(ta.y, cf[1], dot1);
-                      dot0 = fmaf(ta.z, cf[2], dot0);
-                      dot1 = fmaf(ta.w, cf[3], dot1);
-                      dot0 = fmaf(tb4.x, cf[4], dot0);
-                      dot1 = fmaf(tb4.y, cf[5], dot1);
-                      dot0 = fmaf(tb4.z, cf[6], dot0);
-                      dot1 = fmaf(tb4.w, cf[7], dot1);
-                    }
-                  } else {
-                    const uint32_t word = *reinterpret_cast<const uint16_t*>(p.V1q + (flat >> 1));
-                    const float4 ta = tp[0];
-                    dot0 = fmaf(ta.x, (float)sext4((int)word), dot0);
-                    dot1 = fmaf(ta.y, (float)sext4((int)(word >> 4)), dot1);
-                    dot0 = fmaf(ta.z, (float)sext4((int)(word >> 8)), dot0);
-                    dot1 = fmaf(ta.w, (float)sext4((int)(word >> 12)), dot1);
-                  }
-                  h = fmaf(sc, dot0 + dot1, h);
+                if (r > 0 && (p.live[e] & 1)) {
+                  uint32_t w[4];
+                  float sc;
+                  load_codes(e, w, sc);
+                  h = residual(dv, reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r), w, sc);      // t is indexed by token
                 }
                 const float a = gelu_erf(h);
                 ab = fmaf(p.row_gate[(size_t)row * k + j], a, ab);

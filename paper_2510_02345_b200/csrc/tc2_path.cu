@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(T_THREADS, 1)
 tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU1,
              const TParams p) {
   pdl_wait();
+  pdl_release_dependents();
   const int mt = blockIdx.x;
   if (mt >= *p.n_rows / BM) return;
   extern __shared__ uint8_t smem_raw[];
@@ -670,7 +671,6 @@ __global__ void __launch_bounds__(DN_THREADS, 1)
 tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant__ CUtensorMap tmB23,
                 const __grid_constant__ CUtensorMap tmAs, const __grid_constant__ CUtensorMap tmV2,
                 const Down2Params p) {
-  pdl_wait();
   using Cfg = DownCfg<BN, HAS_R>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr uint32_t STAGE_BYTES = Cfg::STAGE_BYTES;
@@ -709,6 +709,8 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
   cluster_sync_all();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  pdl_wait();                  // nothing above reads what an earlier kernel wrote
+  pdl_release_dependents();
 
   const int NT = p.NT, KC = p.KC;
   const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;

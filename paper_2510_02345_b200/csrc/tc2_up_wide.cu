@@ -63,7 +63,6 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
                    const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmAd,
                    const __grid_constant__ CUtensorMap tmV1, const __grid_constant__ CUtensorMap tmU2,
                    const Up2Params p) {
-  pdl_wait();
   using Cfg = WideCfg<HAS_R, KSEL>;
   constexpr int STAGES = Cfg::STAGES;
   constexpr bool TWO = HAS_R && KSEL == 2;                 // a second pass over P for the second expert
@@ -111,6 +110,8 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
   const uint32_t tmem_s = tmem_base + UW_TMEM_S, tmem_a = tmem_base + UW_TMEM_A;
+  pdl_wait();                  // nothing above reads what an earlier kernel wrote
+  pdl_release_dependents();
 
   const int NT = p.NT, KC = p.KC;
   // Work units of `unit` consecutive N tiles of one 256-row tile, dealt round-robin to the CTA pairs:
