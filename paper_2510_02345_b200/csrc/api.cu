@@ -259,9 +259,18 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
     delete[] ids;
   }
   if (e) return fail(e);
-  // bases: B1 [G][d][d_ff] -> B1t [G][d_ff][d];  B2 [G][d_ff][d] -> B2t [G][d][d_ff]
-  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B1), const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
-  if ((e = launch_transpose_fp16(reinterpret_cast<const __half*>(desc->B2), const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
+  // bases: B1 [G][d][d_ff] -> B1t [G][d_ff][d];  B2 [G][d_ff][d] -> B2t [G][d][d_ff]; the weight-streaming path
+  // reads them stage by stage instead: [d / 128][G d_ff][128] and [d_ff / 128][G d][128]
+  const bool streamed = D.stream && o.force_path != kPathGeneric;
+  const __half* B1src = reinterpret_cast<const __half*>(desc->B1);
+  const __half* B2src = reinterpret_cast<const __half*>(desc->B2);
+  if (streamed) {
+    if ((e = launch_stage_major_fp16(B1src, const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_stage_major_fp16(B2src, const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
+  } else {
+    if ((e = launch_transpose_fp16(B1src, const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_transpose_fp16(B2src, const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
+  }
   if (r > 0) {
     struct { const void* src; const void* dst; size_t bytes; } cp[] = {
         {desc->U1q, W.U1q, E * r * d / 2}, {desc->V1q, W.V1q, E * f * r / 2},

@@ -116,7 +116,7 @@ struct cmoe_layer {
   cudaEvent_t host_fork, host_join, chunk_in[cmoe::kMaxHostChunks], chunk_done[cmoe::kMaxHostChunks];
   int host_created;     // objects created so far, in the order above
   // tensor-core path: tensor maps and launch shapes (opaque here, see tc_path.cu)
-  alignas(128) unsigned char tc_state[2048];
+  alignas(128) unsigned char tc_state[4096];
 };
 
 namespace cmoe {
@@ -181,5 +181,9 @@ cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int
                                   cudaStream_t st, bool src_is_bf16 = false);
 cudaError_t launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols,
                                  cudaStream_t st);
+// src [batch][rows][cols] -> dst [rows / 128][batch * cols][128] (rows a multiple of 128): the layout the
+// weight-streaming path reads its bases in
+cudaError_t launch_stage_major_fp16(const __half* src, __half* dst, int batch, int rows, int cols, cudaStream_t st,
+                                    bool src_is_bf16 = false);
 
 }  // namespace cmoe

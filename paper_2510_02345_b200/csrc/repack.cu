@@ -37,6 +37,30 @@ transpose_kernel(const T* __restrict__ src, T* __restrict__ dst, int rows, int c
   }
 }
 
+// Base matrices of the weight-streaming path: src [batch][rows][cols] (rows = reduction index) ->
+// dst [rows / 128][batch * cols][128], i.e. for every 128 reduction indices (one pipeline stage of the kernel)
+// the slab of all output features, 256 bytes each: the rows a CTA loads per stage are one contiguous piece of
+// memory, and the CTAs of a launch, which walk the reduction index in step, read neighbouring pieces.
+template <typename Conv>
+__global__ void __launch_bounds__(256)
+stage_major_kernel(const __half* __restrict__ src, __half* __restrict__ dst, int batch, int rows, int cols) {
+  __shared__ __half tile[32][33];
+  const size_t mat = (size_t)blockIdx.z * rows * cols;
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;       // rows is a multiple of 128: a tile stays inside one stage
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // 32 x 8
+  for (int i = ty; i < 32; i += 8) {
+    const int r = r0 + i, c = c0 + tx;
+    if (r < rows && c < cols) tile[i][tx] = src[mat + (size_t)r * cols + c];
+  }
+  __syncthreads();
+  const size_t slab = (size_t)batch * cols * 128;
+  for (int i = ty; i < 32; i += 8) {
+    const int c = c0 + i, r = r0 + tx;
+    if (r < rows && c < cols)
+      dst[(size_t)(r >> 7) * slab + ((size_t)blockIdx.z * cols + c) * 128 + (r & 127)] = Conv::apply(tile[tx][i]);
+  }
+}
+
 template <typename T, typename Conv = KeepBits>
 cudaError_t launch_t(const T* src, T* dst, int batch, int rows, int cols, cudaStream_t st) {
   // grid.y and grid.z are limited to 65535: fold large batches / row counts by looping on the host
@@ -94,6 +118,15 @@ cudaError_t launch_transpose_fp16(const __half* src, __half* dst, int batch, int
                                   cudaStream_t st, bool src_is_bf16) {
   if (src_is_bf16) return launch_t<__half, Bf16ToHalf>(src, dst, batch, rows, cols, st);
   return launch_t<__half>(src, dst, batch, rows, cols, st);
+}
+cudaError_t launch_stage_major_fp16(const __half* src, __half* dst, int batch, int rows, int cols, cudaStream_t st,
+                                    bool src_is_bf16) {
+  const int gx = (cols + 31) / 32, gy = (rows + 31) / 32;
+  if (rows % 128 != 0 || gy > 65535 || batch > 65535 || gx <= 0) return cudaErrorInvalidValue;
+  dim3 grid(gx, gy, batch);
+  if (src_is_bf16) stage_major_kernel<Bf16ToHalf><<<grid, 256, 0, st>>>(src, dst, batch, rows, cols);
+  else             stage_major_kernel<KeepBits><<<grid, 256, 0, st>>>(src, dst, batch, rows, cols);
+  return cudaGetLastError();
 }
 cudaError_t launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols,
                                  cudaStream_t st) {

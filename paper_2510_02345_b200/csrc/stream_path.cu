@@ -5,7 +5,9 @@
 // The roles of the two GEMM operands are swapped with respect to the large-batch path: the WEIGHTS
 // are the 128-row A operand (a tile of output features, streamed once), the cluster's few tokens
 // are the narrow B operand (N = 16..64, re-read from L2), and the accumulator holds
-// D[feature][token].  Tensor-core rows cost nothing here; bytes do.
+// D[feature][token].  Tensor-core rows cost nothing here; bytes do.  The bases are stored for this
+// path stage by stage, [reduction index / 128][feature][128], so that what a CTA loads per pipeline
+// stage is one contiguous piece of memory.
 //
 //   t      t_j = x U1_e for every (row, kept expert)                 (CUDA cores, tiny)
 //   up     D = B1t_g[f-tile] x_g^T; epilogue per feature f (one thread each): h_j = D + t_j V1_e[f],
@@ -38,6 +40,17 @@ constexpr int SMAXSEG = 160;       // segments: at most G + T_pad / 64
 constexpr int S_THREADS = 640;     // warps 0, 3 TMA (alternating stages), 1 MMA, 2 TMEM allocation, 4..19 epilogue
 constexpr uint32_t S_B_ATOM = SNB * SBK * 2;             // 8 KB
 constexpr uint32_t S_TMEM_COLS = 128;                    // two accumulators of up to 64 columns
+constexpr int S_EPI_WARPS = 16;
+constexpr int S_PJ = 2;            // kept experts per token the up epilogue stages operands for (more: read in place)
+
+// What an epilogue warp needs of its four token columns of one block of 16, staged in shared memory by the
+// warp itself before the accumulator is complete: token, expert slots, gates and (up) the rows of t.
+struct __align__(16) WarpStage {
+  float t[4][S_PJ][32];
+  int tok[4];
+  int slot[4][S_PJ];
+  float gate[4][S_PJ];
+};
 
 struct StreamParams {
   const int* seg_off;        // [G+1] first permuted row of each cluster (multiples of 16)
@@ -67,18 +80,21 @@ struct SCfg {
   static constexpr uint32_t B_BYTES = SKA * S_B_ATOM;
   static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
   static constexpr int STAGES = 4;                                   // 48 KB each
-  static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + 64 * 8 + SMAXSEG * 12 + 64;
+  static constexpr size_t TABLES = 64 * 8 + SMAXSEG * 12 + 64;         // barriers, segment table
+  static constexpr size_t SMEM = 1024 + (size_t)STAGES * STAGE_BYTES + TABLES + S_EPI_WARPS * sizeof(WarpStage);
 };
 
-// Tiles have 128 feature rows.  In the up kernel the tiles of the last, incomplete round of the
-// round-robin are cut into 2, 4, 8 or 16 slices of 64 ... 8 rows (loaded with the boxes of tmWs; the
-// MMA still spans 128 rows and the rest of the accumulator is not read), as many as still fit one
-// slice per CTA, so that the tail occupies all SMs for a fraction of a tile time.  The down kernel
-// gets its granularity from the K ranges.
-struct SliceMaps { CUtensorMap m[4]; };      // boxes of 64, 32, 16, 8 weight rows
+// The down kernel's tiles have 128 feature rows and its granularity comes from the K ranges.  The up kernel
+// cannot split K (GELU needs the complete h), so it picks the tile height R, a multiple of 8 up to 128, for
+// which the round-robin over the CTAs ends soonest: with 896 tiles of 128 rows on 148 CTAs the last of seven
+// rounds would hold 8 tiles, with 1024 tiles of 112 rows all seven rounds are nearly full and an eighth
+// shorter.  Tiles of R rows are loaded with the box of tmRows.m[R / 8 - 1]; the MMA still spans 128 rows and
+// the rest of the accumulator is not read.  A tile that reaches past the cluster's last feature loads rows
+// of the next cluster (or the fill value past the matrix) into accumulator lanes that are not read either.
+struct RowMaps { CUtensorMap m[16]; };       // boxes of 8, 16, ..., 128 weight rows
 template <bool UP>
 __global__ void __launch_bounds__(S_THREADS, 1)
-stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ SliceMaps tmWs,
+stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ RowMaps tmRows,
               const __grid_constant__ CUtensorMap tmTok, const StreamParams p) {
   constexpr int MROWS = 128;
   using Cfg = SCfg<MROWS>;
@@ -96,9 +112,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
   int* seg_row0 = reinterpret_cast<int*>(bars + 64);       // [SMAXSEG]
   int* seg_rows = seg_row0 + SMAXSEG;
   int* seg_g = seg_rows + SMAXSEG;
+  WarpStage* stage_area = reinterpret_cast<WarpStage*>(sm + (size_t)STAGES * Cfg::STAGE_BYTES + Cfg::TABLES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  constexpr int kEpiWarps = 16;      // four warps per TMEM lane quadrant: token columns c with c mod 4 = 0, 1, 2, 3
+  constexpr int kEpiWarps = S_EPI_WARPS;      // four warps per TMEM lane quadrant: token columns c with c mod 4 = 0, 1, 2, 3
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
@@ -141,26 +158,24 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
   const uint32_t tmem_base = *tmem_holder;
 
   // work units: u = (seg * n_mt + mt) * ksplit + ks
-  const int n_mt = p.M / MROWS;
   const int ksplit = UP ? 1 : p.ksplit;
   const int KCH = p.Kd / (SBK * SKA);                    // stages in the whole reduction
-  const int n_tiles = *n_seg_p * n_mt * ksplit;
-  int n_whole = n_tiles;                                 // units [0, n_whole) are whole tiles, the rest slices
-  int lg_f = 0;                                          // log2 of the slices per tail tile
+  int R = MROWS;                                         // feature rows per tile
   if (UP) {
-    const int tail = n_tiles % (int)gridDim.x;
-    if (tail > 0) {
-      while (lg_f < 4 && (tail << (lg_f + 1)) <= (int)gridDim.x) ++lg_f;
-      if (lg_f > 0) n_whole = n_tiles - tail;
+    // time ~ rounds x rows per tile; below about 64 rows a stage is too small to keep the memory pipe full
+    // and a round costs as much as one of 64 rows.  Ties go to the taller tile.
+    long long best = 0;
+    for (int cand = MROWS; cand >= 8; cand -= 8) {
+      const long long tiles = (long long)*n_seg_p * ((p.M + cand - 1) / cand);
+      const long long cost = ((tiles + gridDim.x - 1) / gridDim.x) * (cand > 64 ? cand : 64);
+      if (cand == MROWS || cost < best) { best = cost; R = cand; }
     }
   }
-  const int n_units = n_whole + ((n_tiles - n_whole) << lg_f);
+  const int n_mt = (p.M + R - 1) / R;
+  const int n_units = *n_seg_p * n_mt * ksplit;
   const int my_units = (int)blockIdx.x < n_units ? (n_units - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  // slice: -1 for a whole tile, else which (128 >> lg_f) rows of the tile
-  auto unit_of = [&](int i, int& seg, int& mt, int& slice, int& c_begin, int& c_end) {
-    int u = blockIdx.x + i * gridDim.x;
-    slice = -1;
-    if (u >= n_whole) { slice = (u - n_whole) & ((1 << lg_f) - 1); u = n_whole + ((u - n_whole) >> lg_f); }
+  auto unit_of = [&](int i, int& seg, int& mt, int& c_begin, int& c_end) {
+    const int u = blockIdx.x + i * gridDim.x;
     const int ks = u % ksplit, sm_ = u / ksplit;
     mt = sm_ % n_mt;
     seg = sm_ / n_mt;
@@ -175,19 +190,19 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
       uint32_t it = 0;                                     // stage counter over all units
       const uint32_t mine = warp == 0 ? 0u : 1u;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, slice, c0, c1;
-        unit_of(i, seg, mt, slice, c0, c1);
+        int seg, mt, c0, c1;
+        unit_of(i, seg, mt, c0, c1);
         const int g = seg_g[seg], row0 = seg_row0[seg], nb = seg_rows[seg] / 16;
-        const int srows = slice < 0 ? MROWS : MROWS >> lg_f;          // weight rows this unit loads
-        const int wrow = g * p.M + mt * MROWS + (slice < 0 ? 0 : slice * srows);
-        const uint32_t a_bytes = (uint32_t)srows * SBK * 2 * SKA;
+        const int wrow = g * p.M + mt * R;
+        const uint32_t a_bytes = (uint32_t)R * SBK * 2 * SKA;
+        const CUtensorMap* wmap = UP ? &tmRows.m[R / 8 - 1] : &tmW;
         for (int c = c0; c < c1; ++c, ++it) {
           if ((it & 1u) != mine) continue;
           const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
           if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
           const uint32_t a_dst = base + s * Cfg::STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
           mbar_expect_tx(full0 + 8 * s, a_bytes + (uint32_t)nb * SKA * 16 * SBK * 2);
-          tma_load_3d(a_dst, slice < 0 ? &tmW : &tmWs.m[lg_f - 1], full0 + 8 * s, 0, wrow, c * SKA);
+          tma_load_4d(a_dst, wmap, full0 + 8 * s, 0, wrow, 0, c);     // stage c of the weights: rows wrow .., both K atoms
           // the tokens: 16 rows per box; atom a of block b lands at atom a, rows 16 b .. of the B tile
           for (int b = 0; b < nb; ++b)
             for (int a = 0; a < SKA; ++a)
@@ -200,10 +215,10 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
       for (int i = 0; i < my_units && !failed; ++i) {
-        int seg, mt, slice, c0, c1;
-        unit_of(i, seg, mt, slice, c0, c1);
+        int seg, mt, c0, c1;
+        unit_of(i, seg, mt, c0, c1);
         const uint32_t idesc = idesc_f16(128, seg_rows[seg]);
-        const uint32_t a_atom16 = (slice < 0 ? Cfg::A_ATOM : Cfg::A_ATOM >> lg_f) >> 4;   // second K atom, in 16-byte units
+        const uint32_t a_atom16 = (uint32_t)(R * SBK * 2) >> 4;        // second K atom of the R-row box, in 16-byte units
         const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
         if (!mbar_wait(tempty0 + 8 * acc, aph ^ 1u, abort_flag)) { failed = true; break; }
         tc_fence_after();
@@ -232,20 +247,21 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
     const int part = (warp - 4) >> 2;                    // which token columns of the accumulator this warp takes
     const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16);
     const int r = p.r, k = p.k, M = p.M;
+    WarpStage* ws = stage_area + (warp - 4);
     for (int i = 0; i < my_units; ++i) {
-      int seg, mt, slice, c0, c1;
-      unit_of(i, seg, mt, slice, c0, c1);
-      const int srows = slice < 0 ? MROWS : MROWS >> lg_f;
-      const bool mine = q * 32 + lane < srows;             // slices: only the first srows accumulator lanes are real
-      const int row0 = seg_row0[seg], nrows = q * 32 < srows ? seg_rows[seg] : 0;
+      int seg, mt, c0, c1;
+      unit_of(i, seg, mt, c0, c1);
+      const int f = mt * R + q * 32 + lane;                // output feature (up) / output column (down)
+      const bool mine = q * 32 + lane < R && f < M;        // only the tile's own accumulator lanes are real
+      const int row0 = seg_row0[seg], nrows = q * 32 < R ? seg_rows[seg] : 0;
       const uint32_t acc = (uint32_t)i & 1u, aph = ((uint32_t)i >> 1) & 1u;
-      const int f = mt * MROWS + (slice < 0 ? 0 : slice * srows) + q * 32 + lane;   // output feature (up) / output column (down)
-      // Residual operands of one block of 16 token columns: for each of this warp's four columns and up to two
-      // kept experts, the r INT4 codes and the scale of this thread's feature row of V1.  The first block is
-      // requested before the accumulator is complete, so that the latency of these scattered reads (three
-      // dependent table lookups, then HBM) hides behind the tile's weight stream instead of adding up, column
-      // after column, between two tiles.
-      constexpr int PJ = 2;
+      // Everything the warp needs of one block of 16 token columns besides the accumulator is fetched before
+      // the accumulator is complete, so that the latency of these reads (dependent table lookups, then scattered
+      // reads of V1 from HBM) hides behind the tile's weight stream instead of adding up, column after column,
+      // between two tiles and at the kernel's end: tokens, slots, gates and the rows of t go into the warp's
+      // staging area (lanes in parallel), the r INT4 codes and the scale of this thread's feature row of V1, for
+      // each of the four columns and up to two kept experts, into registers.
+      constexpr int PJ = S_PJ;
       const bool pre = UP && r > 0 && k <= PJ;
       uint32_t wq[4][PJ][4];
       float wsc[4][PJ];
@@ -267,20 +283,42 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
         }
       };
       auto preload = [&](int tb) {
+        __syncwarp();                                      // the warp has finished with the previous block's stage
+        const int rowb = row0 + tb + part;                 // column c2 of this warp is row rowb + 4 c2
+        if (lane < 4) ws->tok[lane] = p.row_token[rowb + 4 * lane];
+        if (pre && lane < 4 * PJ) {
+          const int c2 = lane / PJ, j = lane % PJ;
+          if (j < k) {
+            ws->slot[c2][j] = p.row_slot[(size_t)(rowb + 4 * c2) * k + j];       // (padding rows hold valid slots and gate 0)
+            ws->gate[c2][j] = p.row_gate[(size_t)(rowb + 4 * c2) * k + j];
+          }
+        }
+        __syncwarp();
+        if (pre) {
+          // the rows of t (indexed by token): k r floats per column, four floats per lane and step
+          const int per_col = k * r / 4;
+          for (int idx = lane; idx < 4 * per_col; idx += 32) {
+            const int c2 = idx / per_col, rem = idx - c2 * per_col;
+            const int j = rem / (r / 4), q4 = rem - j * (r / 4);
+            const int tok = ws->tok[c2];
+            if (tok >= 0)
+              *reinterpret_cast<float4*>(&ws->t[c2][j][4 * q4]) = *reinterpret_cast<const float4*>(p.t + (size_t)tok * k * r + 4 * rem);
+          }
 #pragma unroll
-        for (int c2 = 0; c2 < 4; ++c2) {
-          const int row = row0 + tb + 4 * c2 + part;
-          const bool real = mine && p.row_token[row] >= 0;
+          for (int c2 = 0; c2 < 4; ++c2) {
+            const bool real = mine && ws->tok[c2] >= 0;
 #pragma unroll
-          for (int j = 0; j < PJ; ++j) {
-            wsc[c2][j] = 0.f;
-            wq[c2][j][0] = wq[c2][j][1] = wq[c2][j][2] = wq[c2][j][3] = 0u;
-            if (real && j < k) {
-              const int e = p.row_slot[(size_t)row * k + j];
-              if (p.live[e] & 1) load_codes(e, wq[c2][j], wsc[c2][j]);      // (a zero residual block is skipped: Sec. 3.4)
+            for (int j = 0; j < PJ; ++j) {
+              wsc[c2][j] = 0.f;
+              wq[c2][j][0] = wq[c2][j][1] = wq[c2][j][2] = wq[c2][j][3] = 0u;
+              if (real && j < k) {
+                const int e = ws->slot[c2][j];
+                if (p.live[e] & 1) load_codes(e, wq[c2][j], wsc[c2][j]);      // (a zero residual block is skipped: Sec. 3.4)
+              }
             }
           }
         }
+        __syncwarp();
       };
       // h = dv + sc (t_j . codes): the r codes decoded in registers
       auto residual = [&](float dv, const float4* tp, const uint32_t (&w)[4], float sc) -> float {
@@ -313,14 +351,14 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
         }
         return fmaf(sc, dot0 + dot1, dv);
       };
-      if (pre && nrows > 0) preload(0);
+      if (nrows > 0) preload(0);
       {
         const bool ok = mbar_wait(tfull0 + 8 * acc, aph, abort_flag);
         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
       }
       tc_fence_after();
       for (int tb = 0; tb < nrows; tb += 16) {
-        if (pre && tb > 0) preload(tb);
+        if (tb > 0) preload(tb);
         uint32_t v[16];
         tmem_ld16_nowait(taddr + acc * SNB + tb, v);
         tmem_ld_wait();
@@ -328,7 +366,7 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
         for (int c2 = 0; c2 < 4; ++c2) {
           const int c = 4 * c2 + part;
           const int row = row0 + tb + c;
-          const int tok = p.row_token[row];
+          const int tok = ws->tok[c2];
           const bool real = mine && tok >= 0;
           const float dv = __uint_as_float(part == 0 ? v[4 * c2] : part == 1 ? v[4 * c2 + 1] : part == 2 ? v[4 * c2 + 2] : v[4 * c2 + 3]);
           if (UP) {
@@ -338,9 +376,9 @@ stream_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ S
               for (int j = 0; j < PJ; ++j) {
                 if (j < k) {
                   // a zero residual block has scale and codes 0 here: h = dv
-                  const float h = residual(dv, reinterpret_cast<const float4*>(p.t + ((size_t)tok * k + j) * r), wq[c2][j], wsc[c2][j]);
+                  const float h = residual(dv, reinterpret_cast<const float4*>(ws->t[c2][j]), wq[c2][j], wsc[c2][j]);
                   const float a = gelu_erf(h);
-                  ab = fmaf(p.row_gate[(size_t)row * k + j], a, ab);
+                  ab = fmaf(ws->gate[c2][j], a, ab);
                   p.a_slot[((size_t)row * k + j) * M + f] = __float2half_rn(a);
                 }
               }
@@ -516,30 +554,44 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
-// fp16 matrix [rows][cols]; katoms == 0: 2-D box of box_rows x 64 halves; otherwise the matrix is seen
-// as [cols / 64][rows][64] and the box takes katoms K atoms (consecutive swizzled tiles in shared memory)
-bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t katoms) {
+// the token operand: fp16 matrix [rows][cols], boxes of 16 rows x 64 halves (one K atom of one block of 16 tokens)
+bool make_token_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols) {
   EncodeTiledFn enc = get_encode();
   if (!enc) return false;
-  cuuint64_t gdim[3] = {katoms ? (cuuint64_t)SBK : cols, rows, cols / SBK};
-  cuuint64_t gstride[2] = {cols * 2, (cuuint64_t)SBK * 2};
-  cuuint32_t box[3] = {(cuuint32_t)SBK, box_rows, katoms};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, katoms ? 3 : 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)SBK, 16};
+  cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(ptr), gdim, gstride, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The bases as the streaming kernels read them, [Kd / 128][rows][128] fp16 (stage-major): a 4-D view
+// {64 halves, rows, 2 K atoms, Kd / 128 stages} whose box (64, box_rows, 2, 1) lands in shared memory as two
+// consecutive swizzled [box_rows][64] tiles, read from one contiguous piece of box_rows x 256 bytes.
+bool make_weight_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t Kd, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) return false;
+  cuuint64_t gdim[4] = {(cuuint64_t)SBK, rows, (cuuint64_t)SKA, Kd / (SBK * SKA)};
+  cuuint64_t gstride[3] = {(cuuint64_t)SBK * SKA * 2, (cuuint64_t)SBK * 2, rows * SBK * SKA * 2};
+  cuuint32_t box[4] = {(cuuint32_t)SBK, box_rows, (cuuint32_t)SKA, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4, const_cast<void*>(ptr), gdim, gstride, box, estr,
              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct StreamState {
   CUtensorMap mW1, mX, mW2, mAbar;
-  SliceMaps mW1s;
+  RowMaps mW1r;
   int sm_count;
   int ksplit;
 };
 static_assert(sizeof(StreamState) <= sizeof(((cmoe_layer*)nullptr)->tc_state), "tc_state too small");
 
 template <bool UP>
-cudaError_t launch_stream(const CUtensorMap& mW, const SliceMaps& mWs, const CUtensorMap& mTok, const StreamParams& p, int grid,
+cudaError_t launch_stream(const CUtensorMap& mW, const RowMaps& mWs, const CUtensorMap& mTok, const StreamParams& p, int grid,
                           cudaStream_t st) {
   auto kern = stream_kernel<UP>;
   constexpr size_t sm = SCfg<128>::SMEM;
@@ -567,11 +619,10 @@ cudaError_t stream_init(cmoe_layer* L) {
   e = cudaDeviceGetAttribute(&ts->sm_count, cudaDevAttrMultiProcessorCount, dev);
   if (e != cudaSuccess) return e;
   const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
-  const bool ok = make_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 128, SKA) && make_map(&ts->mW1s.m[0], L->w.B1t, G * D.d_ff, D.d, 64, SKA) &&
-                  make_map(&ts->mW1s.m[1], L->w.B1t, G * D.d_ff, D.d, 32, SKA) && make_map(&ts->mW1s.m[2], L->w.B1t, G * D.d_ff, D.d, 16, SKA) &&
-                  make_map(&ts->mW1s.m[3], L->w.B1t, G * D.d_ff, D.d, 8, SKA) &&
-                  make_map(&ts->mX, S.x_perm, P, D.d, 16, 0) &&
-                  make_map(&ts->mW2, L->w.B2t, G * D.d, D.d_ff, 128, SKA) && make_map(&ts->mAbar, S.abar, P, D.d_ff, 16, 0);
+  bool ok = make_weight_map(&ts->mW1, L->w.B1t, G * D.d_ff, D.d, 128);
+  for (int i = 0; i < 16 && ok; ++i) ok = make_weight_map(&ts->mW1r.m[i], L->w.B1t, G * D.d_ff, D.d, 8 * (i + 1));
+  ok = ok && make_token_map(&ts->mX, S.x_perm, P, D.d) &&
+                  make_weight_map(&ts->mW2, L->w.B2t, G * D.d, D.d_ff, 128) && make_token_map(&ts->mAbar, S.abar, P, D.d_ff);
   // K ranges per down tile: fill the SMs evenly, keep at least four stages per range
   const int kch = D.d_ff / (SBK * SKA);
   const long long tiles = (long long)D.G * (D.d / 128);
@@ -614,9 +665,9 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
   const int seg_bound = D.G + rows_bound / SNB;
   {
     p.Kd = D.d; p.M = D.d_ff; p.ksplit = 1;
-    const long long units = (long long)seg_bound * (D.d_ff / 128);
+    const long long units = (long long)seg_bound * (D.d_ff / 8);       // the kernel may choose tiles as low as 8 rows
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<true>(ts.mW1, ts.mW1s, ts.mX, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<true>(ts.mW1, ts.mW1r, ts.mX, p, grid, st)) != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[2], st);
   if (D.r > 0) {
@@ -636,7 +687,7 @@ cudaError_t launch_stream_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_
     p.Kd = D.d_ff; p.M = D.d; p.ksplit = ts.ksplit;
     const long long units = (long long)seg_bound * (D.d / 128) * ts.ksplit;
     const int grid = (int)(units < ts.sm_count ? units : ts.sm_count);
-    if ((e = launch_stream<false>(ts.mW2, ts.mW1s, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
+    if ((e = launch_stream<false>(ts.mW2, ts.mW1r, ts.mAbar, p, grid, st)) != cudaSuccess) return e;
   }
   if (D.r > 0 && (e = cudaStreamWaitEvent(st, L->side_join, 0)) != cudaSuccess) return e;     // join
   dim3 fgrid((D.d + 255) / 256, rows_bound);
