@@ -70,11 +70,11 @@ NCU_TRAFFIC = {
               "sha1": {"tc2_up_wide.cu": "23425974743ca4b7062c11e72b2631012d941af8",
                        "tc2_common.cuh": "cc74b43ead519c31205497b0115ec5e167d791e0",
                        "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
-    "decode": {"kernel": "stream_kernel<up>", "bytes": 955.824896e6 + 9.873408e6,
-               "sha1": {"stream_path.cu": "56f3a492ae638749f58a73aa07eeb29bb207b097",
+    "decode": {"kernel": "stream_kernel<up>", "bytes": 956.045056e6 + 10.527744e6,
+               "sha1": {"stream_path.cu": "232f8c53b14c361c003fef805982308b22b73f54",
                         "device_utils.cuh": "daa6a5fc90a4b02a5c17177e8d154044cca709c4",
                         "lowrank.cuh": "698889609319931f08fc77e7b2de29ef206fc1c8",
-                        "tc_ptx.cuh": "497c14e72f4384fbbb6a1d12d67ecfacf3e23b33"}},
+                        "tc_ptx.cuh": "1049d28657994901f1d99952835b95fa9d50fa8d"}},
 }
 
 
@@ -441,6 +441,32 @@ def run_reference(args, rank):
 
 
 # ------------------------------------------------------------------ main
+def time_similarity(peaks, E=32, n=1024 * 4096, d=1024, reps=10):
+    """The Gram kernel of cmoe_expert_similarity (Eq. 2) on the headline layer's up matrices: E x n fp32 weights read
+    once, so its roofline is the HBM stream (4 E n bytes per call)."""
+    import torch
+    from paper_2510_02345_b200 import binding
+    W = torch.randn((E, n), dtype=torch.float32, device="cuda")
+    mu = torch.randn((E, d), dtype=torch.float32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    out = binding.expert_similarity(W, mu, 0.7)
+    for _ in range(3):
+        binding.expert_similarity(W, mu, 0.7, out)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in ev:
+        flush.zero_()
+        a.record()
+        binding.expert_similarity(W, mu, 0.7, out)       # results into the same tensors: no allocation in the timed region
+        b.record()
+    torch.cuda.synchronize()
+    assert int(out["status"].item()) == 0
+    ms = sum(a.elapsed_time(b) for a, b in ev) / reps
+    gbs = 4.0 * E * n / (ms * 1e-3) / 1e9
+    return {"E": E, "weights_per_expert": n, "ms_per_call": ms, "achieved_gbs": gbs, "bound": "hbm",
+            "frac_of_measured_copy": gbs / float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])), "frac_of_nominal_8000": gbs / 8000.0,
+            "l2": "flushed between calls", "launches_per_call": 3}
+
+
 def main():
     global _dist
     ap = argparse.ArgumentParser()
@@ -452,6 +478,7 @@ def main():
     ap.add_argument("--all", action="store_true", help="also time the other four workloads (short runs)")
     ap.add_argument("--variants", action="store_true", help="also time the headline shape at other ranks, k and expert counts")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--similarity", action="store_true", help="time only cmoe_expert_similarity (Eq. 2-4) and print its line")
     ap.add_argument("--no-decode", action="store_true", help="leave the decode workload out of the default line")
     ap.add_argument("--sustained", type=float, default=2.0,
                     help="seconds of back-to-back forwards for the sustained figure (0: skip)")
@@ -467,6 +494,11 @@ def main():
     import torch
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    if args.similarity:
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            print(json.dumps({"similarity": time_similarity(load_peaks()[0])}), flush=True)
+        return
     if world > 1:
         import torch.distributed as dist
         torch.cuda.set_device(local_rank)
@@ -534,6 +566,8 @@ def main():
                              "layer": whole_layer_fractions(r3, 1, peaks), "stage_ms": r3["stage_ms"], "path": int(r3["info"].path),
                              "launches_per_forward": int(r3["info"].launches_forward)}
             line["variants"] = var
+        if args.all:
+            line["similarity"] = time_similarity(peaks)
         if not args.no_cpu_baseline:
             line["cpu_baseline"], line["parity"] = oracle_rate(args.workload, gpu=res if res.get("y") is not None else None)
         print(json.dumps(line), flush=True)

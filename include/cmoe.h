@@ -231,6 +231,34 @@ int cmoe_route_static(int32_t d, int32_t E, int32_t G, int32_t k,
                       const void* x, int32_t T,
                       int32_t* cluster_id, int32_t* expert_ids, float* gates, void* cuda_stream);
 
+/* Expert similarity that the clustering step consumes (Sec. 3.1, Eq. 2-4), for E experts:
+ *   S_param [E][E] fp32  cosine similarity of the experts' flattened weight matrices (Eq. 2),
+ *                        W = fp32 [E][n], n = number of weights per expert (n % 32 == 0, W 16-byte aligned)
+ *   S_task  [E][E] fp32  cosine similarity of the activation centroids (Eq. 3), mu = fp32 [E][d]
+ *                        (the mu that cmoe_expert_stats maintains)
+ *   S       [E][E] fp32  alpha S_param + (1 - alpha) S_task (Eq. 4), 0 <= alpha <= 1
+ * W == NULL skips S_param, mu == NULL skips S_task; S needs both (else it must be NULL).  A vector of norm zero has
+ * similarity 0 to every other vector and 1 to itself.  The dot products of S_param run on the tensor cores with the
+ * weights cut to tf32 (10 mantissa bits) and fp32 accumulation, partial sums of different ranges of the flattened
+ * index combined with atomic additions: results agree with exact arithmetic to about 1e-4 and may differ in the
+ * last bits between calls.  status: optional device word (caller zeroes it) that receives CMOE_ERR_TIMEOUT if a
+ * bounded wait inside the kernel expires (the outputs are then undefined); may be NULL.
+ * All pointers are device pointers; 1 <= E <= 128; needs no workspace (S_param doubles as the accumulation
+ * buffer); asynchronous on the given stream. */
+typedef struct {
+  int32_t E;
+  int32_t d;
+  int64_t n;
+  float alpha;
+  const float* W;
+  const float* mu;
+  float* S_param;
+  float* S_task;
+  float* S;
+  int32_t* status;
+} cmoe_similarity_desc;
+int cmoe_expert_similarity(const cmoe_similarity_desc* desc, void* cuda_stream);
+
 /* Offline compressor (Sec. 3.2, Eq. 6-7; Sec. 3.4): from E dense expert matrices W_e (d_in x d_out, row-vector
  * convention; expert slot e = g*K + i belongs to cluster g) to the stored form of one of the layer's two matrices:
  *   B   [G][d_in][d_out]  fp16  W_base^g = mean of the cluster's experts (Eq. 6)

@@ -20,7 +20,7 @@ ERRORS = {
     -1: "CMOE_ERR_INVALID_ARG", -2: "CMOE_ERR_UNSUPPORTED_SHAPE", -3: "CMOE_ERR_WORKSPACE_TOO_SMALL",
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
-EXPORTS = ["cmoe_compress_workspace_bytes", "cmoe_compress", "cmoe_quantize_int4",
+EXPORTS = ["cmoe_compress_workspace_bytes", "cmoe_compress", "cmoe_quantize_int4", "cmoe_expert_similarity",
            "cmoe_workspace_bytes", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
            "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
@@ -51,6 +51,11 @@ class cmoe_compress_desc(C.Structure):
                                   "A_out", "Bt_out", "workspace")] + [("workspace_bytes", C.c_size_t)]
 
 
+class cmoe_similarity_desc(C.Structure):
+    _fields_ = [("E", C.c_int32), ("d", C.c_int32), ("n", C.c_int64), ("alpha", C.c_float)] + [
+        (n, C.c_void_p) for n in ("W", "mu", "S_param", "S_task", "S", "status")]
+
+
 class cmoe_info(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("path", "launches_route", "launches_forward", "row_align", "T_pad_max",
                                          "memsets_forward", "n_stages", "pruned_blocks")]
@@ -73,6 +78,7 @@ def lib():
         L.cmoe_compress_workspace_bytes.argtypes = [C.POINTER(cmoe_compress_desc), C.POINTER(C.c_size_t)]
         L.cmoe_compress.argtypes = [C.POINTER(cmoe_compress_desc), C.c_void_p]
         L.cmoe_quantize_int4.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.cmoe_expert_similarity.argtypes = [C.POINTER(cmoe_similarity_desc), C.c_void_p]
         L.cmoe_create_ex.argtypes = [C.POINTER(cmoe_desc), C.POINTER(cmoe_options), C.POINTER(C.c_void_p)]
         L.cmoe_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
         L.cmoe_expert_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
@@ -226,6 +232,35 @@ def quantize_int4(w):
     _check(lib().cmoe_quantize_int4(w.data_ptr(), w.numel(), q.data_ptr(), s.data_ptr(),
                                     torch.cuda.current_stream(w.device).cuda_stream), "cmoe_quantize_int4")
     return q, s
+
+
+def expert_similarity(W=None, mu=None, alpha: float = 0.7, out: dict | None = None):
+    """cmoe_expert_similarity on CUDA fp32 tensors: W [E][...] (flattened per expert) and / or mu [E][d].
+    Returns a dict of CUDA tensors [E][E]: S_param (if W), S_task (if mu), S (if both), and the int32 status word;
+    `out` = the dict of an earlier call with the same arguments' shapes, to write into its tensors again."""
+    import torch
+    ref = W if W is not None else mu
+    E, dev = ref.shape[0], ref.device
+    q = cmoe_similarity_desc()
+    q.E, q.alpha = E, alpha
+    if out is None:
+        out = {"status": torch.zeros(1, dtype=torch.int32, device=dev)}
+        for name, need in (("S_param", W is not None), ("S_task", mu is not None), ("S", W is not None and mu is not None)):
+            if need:
+                out[name] = torch.empty((E, E), dtype=torch.float32, device=dev)
+    q.status = out["status"].data_ptr()
+    if W is not None:
+        assert W.is_cuda and W.dtype == torch.float32 and W.is_contiguous()
+        q.W, q.n = W.data_ptr(), W[0].numel()
+        q.S_param = out["S_param"].data_ptr()
+    if mu is not None:
+        assert mu.is_cuda and mu.dtype == torch.float32 and mu.is_contiguous() and mu.shape[0] == E
+        q.mu, q.d = mu.data_ptr(), mu.shape[1]
+        q.S_task = out["S_task"].data_ptr()
+    if W is not None and mu is not None:
+        q.S = out["S"].data_ptr()
+    _check(lib().cmoe_expert_similarity(C.byref(q), torch.cuda.current_stream(dev).cuda_stream), "cmoe_expert_similarity")
+    return out
 
 
 # ---- convenience owner of the device buffers ---------------------------------------------------
