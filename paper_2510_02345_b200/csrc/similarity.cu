@@ -92,15 +92,16 @@ gram_kernel(const __grid_constant__ CUtensorMap tmW, const GramParams p) {
   tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
 
-  // this CTA's range of stages
-  const long long s0 = p.n_stages * blockIdx.x / gridDim.x, s1 = p.n_stages * (blockIdx.x + 1) / gridDim.x;
+  // This CTA's stages: s0, s0 + grid, s0 + 2 grid, ...  Dealt round-robin, the CTAs of the launch read, at any
+  // time, one contiguous window of every expert's row between them.
+  const long long s0 = blockIdx.x, s1 = p.n_stages, sstep = gridDim.x;
   const uint32_t atom_bytes = (uint32_t)p.rows * 128u, stage_bytes = atom_bytes * (uint32_t)p.KA;
   bool failed = false;
 
   if (warp == 0) {
     if (lane == 0) {
       uint32_t s = 0, ph = 0;
-      for (long long st = s0; st < s1; ++st) {
+      for (long long st = s0; st < s1; st += sstep) {
         if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
         mbar_expect_tx(full0 + 8 * s, stage_bytes);
         // KA atoms of 32 floats x `rows` experts; past the end of the flattened index the fill value (zero)
@@ -113,7 +114,7 @@ gram_kernel(const __grid_constant__ CUtensorMap tmW, const GramParams p) {
       const int N = (p.stack * p.rows + 15) & ~15;
       const uint32_t idesc = idesc_tf32(128, N);
       uint32_t s = 0, ph = 0;
-      for (long long st = s0; st < s1; ++st) {
+      for (long long st = s0; st < s1; st += sstep) {
         if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
         tc_fence_after();
         const uint64_t desc0 = umma_desc(base + s * GR_STAGE_BYTES);      // A and B are the same tile
