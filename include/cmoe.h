@@ -106,6 +106,10 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *   up_tile       0 automatic; 128 keeps the up projection of large batches on 128-column tiles where d_ff
  *                 would allow 256-column tiles
  *   host_chunks   0 automatic; 1..8: the most chunks cmoe_forward_host cuts a batch into (chunks stay >= 2048 tokens)
+ *   row_gather    0 (default): a copy kernel permutes the rows of x; 1: on the CTA-pair path with residual factors
+ *                 the kernel that projects the tokens onto U1 reads them from x by TMA row gather (four rows of 128
+ *                 bytes per instruction) and writes the permuted copy as it goes: one pass over x less, but slower
+ *                 as measured (the gathers are issued at a fraction of the rate of tiled loads)
  * and one switch that changes what the descriptor means:
  *   base_dtype    0: desc.B1 / desc.B2 hold fp16 bits (the paper's storage format, Sec. 3.4); 1: they hold bfloat16
  *                 bits.  The tensor cores take both operands of a product in one 16-bit type and the activations
@@ -119,7 +123,8 @@ typedef struct {
   int32_t up_tile;
   int32_t base_dtype;
   int32_t host_chunks;
-  int32_t reserved[3];
+  int32_t row_gather;
+  int32_t reserved[2];
 } cmoe_options;
 int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
 

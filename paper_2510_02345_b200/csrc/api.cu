@@ -184,7 +184,8 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   o.force_path = -1;
   if (opt) o = *opt;
   if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
-      o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks) return CMOE_ERR_INVALID_ARG;
+      o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks || o.row_gather < 0 || o.row_gather > 1 ||
+      o.reserved[0] != 0 || o.reserved[1] != 0) return CMOE_ERR_INVALID_ARG;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -370,10 +371,11 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
     if (L->path == kPathTensor && L->tc_variant == 2) tc2_accum_buffer(L, T, &zp, &zb);
     LowrankTok lr{};                      // nothing rides along unless the streaming path has residual factors
     if (L->path == kPathStream) stream_lowrank_rider(L, xh, T, &lr);
-    CMOE_CUDA(L, launch_permute(D, S, xh, T, st, zp, zb, fs, lr, counted_tile));
+    const bool gather = L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L);
+    CMOE_CUDA(L, launch_permute(D, S, gather ? nullptr : xh, T, st, zp, zb, fs, lr, counted_tile));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
-    CMOE_CUDA(L, launch_tc2_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
+    CMOE_CUDA(L, launch_tc2_ffn(L, tc2_gathers_rows(L) ? xh : nullptr, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else if (L->path == kPathStream)
     CMOE_CUDA(L, launch_stream_ffn(L, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
   else if (L->path == kPathTensor)

@@ -166,7 +166,9 @@ cudaError_t tc2_init(cmoe_layer* L);
 int tc2_launch_count(const cmoe_layer* L);
 void tc2_accum_buffer(const cmoe_layer* L, int T, void** ptr, size_t* bytes);
 void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs);
-cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
+// x_src: not null when the t kernel gathers the rows of x itself (tc2_gathers_rows)
+cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
+bool tc2_gathers_rows(const cmoe_layer* L);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);

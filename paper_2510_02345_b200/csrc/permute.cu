@@ -277,7 +277,7 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
   // more for a kernel that is bound by memory bandwidth anyway)
   if ((int)blockIdx.x >= n_move) { stage_block(fs, blockIdx.x - n_move); return; }
   const int vec_per_row = d / 8;
-  for (int row = blockIdx.x; row < *n_rows; row += n_move) {
+  for (int row = blockIdx.x; x != nullptr && row < *n_rows; row += n_move) {      // (no x: a later kernel gathers the rows)
     const int tok = row_token[row];
     uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
     if (tok >= 0) {

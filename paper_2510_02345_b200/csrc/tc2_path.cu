@@ -56,16 +56,20 @@ struct TParams {
   const int* live;     // [E]         bit 0 / 1: the expert's up / down residual block is not zero
   int* status;
   int KC, K, r;
+  int x_rows;          // gather mode: rows of x (the first row index that reads zeros)
 };
 
 constexpr int T_THREADS = 224;      // warps 0 and 6 TMA (alternating stages), 1 MMA, 2..5 epilogue
 constexpr int T_STAGES = 6;
 constexpr uint32_t T_STAGE_BYTES = BM * BK * 2 + KE * BK * 2;   // 24 KB
 
-template <int KSEL>
+// GATHER: the kernel reads the tile's rows from x itself (TMA gather by row_token, zeros for padding rows) and, as
+// each K chunk passes through shared memory, stores it to x_perm for the up kernel: the permuted copy of x is a
+// by-product of this kernel instead of a pass of its own over x.
+template <int KSEL, bool GATHER>
 __global__ void __launch_bounds__(T_THREADS, 1)
 tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmU1,
-             const TParams p) {
+             const __grid_constant__ CUtensorMap tmXsrc, const TParams p) {
   pdl_wait();
   pdl_release_dependents();
   const int mt = blockIdx.x;
@@ -79,8 +83,13 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(bars + 2 * kMaxStages + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   int* sh_mask = reinterpret_cast<int*>(tmem_holder + 2);     // [3]
+  int* s_tok = sh_mask + 4;                                   // [BM] gather mode: source row of every row of the tile
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
+  if (GATHER && threadIdx.x < BM) {
+    const int tok = p.row_token[mt * BM + threadIdx.x];
+    s_tok[threadIdx.x] = tok >= 0 ? tok : p.x_rows;           // padding rows: outside the tensor, i.e. zeros
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < T_STAGES; ++s) { mbar_init(full0 + 8 * s, 1); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(tfull, 1);
@@ -109,7 +118,15 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
         if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) { failed = true; break; }
         const uint32_t a_dst = base + s * T_STAGE_BYTES, b_dst = a_dst + BM * BK * 2;
         mbar_expect_tx(full0 + 8 * s, T_STAGE_BYTES);
-        tma_load_2d(a_dst, &tmX, full0 + 8 * s, kc * BK, mt * BM);
+        if (GATHER) {
+          // four rows (512 bytes of the swizzled tile) per instruction
+          for (int r4 = 0; r4 < BM; r4 += 4) {
+            const int4 t4 = *reinterpret_cast<const int4*>(s_tok + r4);
+            tma_gather4_2d(a_dst + r4 * (BK * 2), &tmXsrc, full0 + 8 * s, kc * BK, t4.x, t4.y, t4.z, t4.w);
+          }
+        } else {
+          tma_load_2d(a_dst, &tmX, full0 + 8 * s, kc * BK, mt * BM);
+        }
         tma_load_2d(b_dst, &tmU1, full0 + 8 * s, kc * BK, g * KE);
       }
     }
@@ -125,7 +142,22 @@ tc2_t_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CU
 #pragma unroll
         for (int ks = 0; ks < BK / 16; ++ks)
           umma_f16(tmem_base, adesc + 2 * ks, bdesc + 2 * ks, IDESC, (kc | ks) != 0 ? 1u : 0u);
-        umma_commit(empty0 + 8 * s);
+        if (GATHER) {
+          // The chunk of x rows goes out to x_perm.  A stage is handed back once its store has read it: two
+          // stores stay in flight, so the stage of chunk kc - 2 is released here (the commit also covers its MMAs,
+          // issued long before).
+          tma_store_2d(&tmX, a_src, kc * BK, mt * BM);
+          bulk_commit_group();
+          bulk_wait_read_but2();
+          if (kc >= 2) umma_commit(empty0 + 8 * ((kc - 2) % T_STAGES));
+        } else {
+          umma_commit(empty0 + 8 * s);
+        }
+      }
+      if (GATHER) {
+        bulk_wait_read_all();
+        // (the last two stages are not refilled: nothing waits for their release)
+        bulk_wait_all();
       }
       if (!failed) umma_commit(tfull);
     }
@@ -942,14 +974,14 @@ cudaError_t launch_down(const Tc2State& ts, const Down2Params& p, int grid, cuda
   return launch_pairs(kern, grid, DN_THREADS, sm, st, ts.mAbar3, ts.mB23, ts.mAs, ts.mV2, p);
 }
 
-template <int KSEL>
-cudaError_t launch_t(const Tc2State& ts, const TParams& p, int grid, cudaStream_t st) {
-  auto kern = tc2_t_kernel<KSEL>;
-  constexpr size_t sm = 1024 + (size_t)T_STAGES * T_STAGE_BYTES + 32 * 8;
+template <int KSEL, bool GATHER>
+cudaError_t launch_t(const Tc2State& ts, const CUtensorMap& x_src, const TParams& p, int grid, cudaStream_t st) {
+  auto kern = tc2_t_kernel<KSEL, GATHER>;
+  constexpr size_t sm = 1024 + (size_t)T_STAGES * T_STAGE_BYTES + 32 * 8 + BM * sizeof(int);
   static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
   if (cudaError_t e = ensure_dynamic_smem(kern, sm, smem_set)) return e;
   launch_chained(kern, dim3(grid), dim3(T_THREADS), sm, st, 1,
-      ts.mX, ts.mU1, p);
+      ts.mX, ts.mU1, x_src, p);
   return cudaGetLastError();
 }
 
@@ -1058,6 +1090,9 @@ void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs) {
   fs->K = D.K; fs->r = D.r;
 }
 
+// (option) the t kernel reads x by row_token and writes x_perm itself: the permutation then moves no rows
+bool tc2_gathers_rows(const cmoe_layer* L) { return L->dims.r > 0 && L->opt.row_gather == 1; }
+
 int tc2_launch_count(const cmoe_layer* L) {
   const Dims& D = L->dims;
   if (D.r == 0) return 2;
@@ -1076,7 +1111,7 @@ void tc2_accum_buffer(const cmoe_layer* L, int T, void** ptr, size_t* bytes) {
   else { *ptr = L->sc.s; *bytes = sizeof(float) * rows * D.k * D.r; }
 }
 
-cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
+cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __half* y, cudaStream_t st, cudaEvent_t* marks) {
   const Dims& D = L->dims;
   const Weights& W = L->w;
   const Scratch& S = L->sc;
@@ -1089,8 +1124,15 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, int T, __half* y, cudaStream_t s
     TParams tp{};
     tp.n_rows = S.n_rows; tp.tile_cluster = S.tile_cluster; tp.row_slot = S.row_slot; tp.row_token = S.row_token;
     tp.A0 = S.A0; tp.Ad = S.Ad; tp.tile_mask = S.tile_mask; tp.tile_mask_dn = S.tile_mask_dn; tp.live = L->w.live; tp.status = S.status;
-    tp.KC = D.d / BK; tp.K = D.K; tp.r = D.r;
-    e = D.k == 2 ? launch_t<2>(ts, tp, mt_bound, st) : launch_t<1>(ts, tp, mt_bound, st);
+    tp.KC = D.d / BK; tp.K = D.K; tp.r = D.r; tp.x_rows = T;
+    if (x_src) {
+      // the t kernel gathers the rows of x itself (and writes x_perm): a map of this call's x, boxes of one row
+      CUtensorMap mx;
+      if (!make_map(&mx, x_src, (uint64_t)T, D.d, 1)) return cudaErrorInvalidValue;
+      e = D.k == 2 ? launch_t<2, true>(ts, mx, tp, mt_bound, st) : launch_t<1, true>(ts, mx, tp, mt_bound, st);
+    } else {
+      e = D.k == 2 ? launch_t<2, false>(ts, ts.mX, tp, mt_bound, st) : launch_t<1, false>(ts, ts.mX, tp, mt_bound, st);
+    }
     if (e != cudaSuccess) return e;
   }
   if (marks) cudaEventRecord(marks[1], st);

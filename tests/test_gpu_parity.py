@@ -271,6 +271,24 @@ def test_bert_with_the_narrow_up_kernel():
     full_check(L, L["x"], options=dict(up_tile=128))
 
 
+@pytest.mark.parametrize("T,kw", [
+    (129, dict(d=128, d_ff=256, E=8, G=2, r=16, k=2)),        # ragged: most rows of the last tiles are padding
+    (1111, dict(d=256, d_ff=256, E=6, G=3, r=8, k=1)),
+    (1500, dict(d=384, d_ff=512, E=16, G=2, r=4, k=2)),       # K = 8, r = 4
+], ids=["ragged", "k1", "K8r4"])
+def test_rows_gathered_by_the_projection_kernel(T, kw):
+    # option row_gather: the kernel of t = x U1 reads x by TMA row gather and writes the permuted copy itself
+    s = inputs.small_shape(T=T, **kw)
+    L = inputs.make_layer(s, 31)
+    got = full_check(L, L["x"], options=dict(row_gather=1))
+    assert got["module"].info.path == 1
+
+
+def test_bert_with_gathered_rows():
+    L = layer_for("bert")
+    full_check(L, L["x"], options=dict(row_gather=1))
+
+
 # ---- shapes that take the weight-streaming path (T_max <= 128, d and d_ff multiples of 128) ---------
 @pytest.mark.parametrize("kw", [
     dict(T=1, d=128, d_ff=128, E=8, G=2, r=4, k=2),
