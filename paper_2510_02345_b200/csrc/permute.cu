@@ -277,14 +277,24 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
   // more for a kernel that is bound by memory bandwidth anyway)
   if ((int)blockIdx.x >= n_move) { stage_block(fs, blockIdx.x - n_move); return; }
   const int vec_per_row = d / 8;
-  for (int row = blockIdx.x; x != nullptr && row < *n_rows; row += n_move) {      // (no x: a later kernel gathers the rows)
-    const int tok = row_token[row];
-    uint4* dst = reinterpret_cast<uint4*>(x_perm + (size_t)row * d);
-    if (tok >= 0) {
-      const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)tok * d);
-      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = src[v];
-    } else {
-      for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) dst[v] = make_uint4(0, 0, 0, 0);
+  const int rows = x != nullptr ? *n_rows : 0;                 // (no x: a later kernel gathers the rows)
+  // four rows at a time: their token lookups, then their loads, are in flight together instead of one row's
+  // lookup - load - store chain after the other
+  for (int row0 = blockIdx.x; row0 < rows; row0 += 4 * n_move) {
+    int tok[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int row = row0 + i * n_move;
+      tok[i] = row < rows ? row_token[row] : -2;               // -2: no such row
+    }
+    for (int v = threadIdx.x; v < vec_per_row; v += blockDim.x) {
+      uint4 val[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        val[i] = tok[i] >= 0 ? reinterpret_cast<const uint4*>(x + (size_t)tok[i] * d)[v] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (tok[i] != -2) reinterpret_cast<uint4*>(x_perm + (size_t)(row0 + i * n_move) * d)[v] = val[i];
     }
   }
   // the accumulation buffer of the later stages starts at zero
