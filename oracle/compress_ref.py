@@ -12,7 +12,7 @@ From E dense expert matrices W_i (d_in x d_out, row-vector convention y = x W) g
     Sec. 3.4   optional cosine gate: a residual block whose cosine similarity to the base matrix is below gamma is
                zeroed
 
-Readings (the paper leaves them open; they are listed in the design doc): the residual is taken against the base AS STORED
+Readings (the paper leaves them open): the residual is taken against the base AS STORED
 (the fp16-rounded mean), so that the factors also absorb the rounding of the base; the singular values are split
 evenly, A = U_r sqrt(S_r), B^T = sqrt(S_r) V_r^T; the gate compares <Delta W, W_base>_F / (|Delta W|_F |W_base|_F)
 with gamma literally (gamma = 0 switches it off); quantiser: scale = fp16(absmax / 7) (0 for an all-zero group),
