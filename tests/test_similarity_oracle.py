@@ -73,3 +73,34 @@ def test_fused_score_eq4():
     assert ref.fused_similarity(W2, mu2, 0.7)["S"][0, 1] == pytest.approx(0.05, abs=1e-12)
     with pytest.raises(AssertionError):
         ref.fused_similarity(W, mu, 1.5)
+
+
+# ---- planted mistakes: each must make one of the pins above fail ------------------------------------------------
+_MUTANTS = {
+    "norm_without_root": ("norm = np.sqrt((V * V).sum(axis=1))", "norm = (V * V).sum(axis=1)"),
+    "one_norm_only": ("/ (norm[i] * norm[j])", "/ (norm[i] * norm[i])"),
+    "alpha_swapped": ("S=alpha * S_param + (1.0 - alpha) * S_task", "S=(1.0 - alpha) * S_param + alpha * S_task"),
+    "task_from_weights": ("S_task = cosine_matrix(mu)", "S_task = cosine_matrix(W)"),
+    "matrices_not_flattened": ("V = np.asarray(V, dtype=np.float64).reshape(V.shape[0], -1)", "V = np.asarray(V, dtype=np.float64)[:, 0] if np.ndim(V) == 3 else np.asarray(V, dtype=np.float64)"),
+    "zero_vector_gives_one": ("out[i, j] = 1.0 if i == j else 0.0", "out[i, j] = 1.0"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(_MUTANTS))
+def test_planted_mistakes_are_caught(name, monkeypatch):
+    import inspect
+    import types
+    src = inspect.getsource(ref)
+    old, new = _MUTANTS[name]
+    assert src.count(old) == 1
+    mutant = types.ModuleType("similarity_mutant")
+    exec(compile(src.replace(old, new), "similarity_mutant", "exec"), mutant.__dict__)
+    monkeypatch.setattr(ref, "cosine_matrix", mutant.cosine_matrix)
+    monkeypatch.setattr(ref, "fused_similarity", mutant.fused_similarity)
+    caught = 0
+    for pin in (test_hand_worked_angles, test_against_sklearn, test_invariants, test_zero_vector_reading, test_fused_score_eq4):
+        try:
+            pin()
+        except (AssertionError, ValueError, IndexError):
+            caught += 1
+    assert caught >= 1, f"no pin notices the planted mistake {name}"
