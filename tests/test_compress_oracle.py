@@ -110,3 +110,39 @@ def test_cosine_gate():
     assert not c["pruned"].any() and c["Uq"].any()
     c = cr.compress(W, 1, 4, gamma=0.5 * cos)                            # expert 0 stays, expert 1 (negative cosine) goes
     assert list(c["pruned"]) == [0, 1] and c["Uq"][0].any() and not c["Uq"][1].any() and not c["Vs"][1].any()
+
+
+# ---- planted mistakes: each must make one of the pins above fail ------------------------------------------------
+_MUTANTS = {
+    "sum_instead_of_mean": (".mean(axis=1).astype(np.float16)", ".sum(axis=1).astype(np.float16)"),
+    "base_of_the_wrong_cluster": ("base = B[e // K].astype(np.float64)", "base = B[(e // K + 1) % G].astype(np.float64)"),
+    "residual_sign": ("dW = W[e].astype(np.float64) - base", "dW = base - W[e].astype(np.float64)"),
+    "smallest_singular_values": ("root = np.sqrt(S[:r])\n    return U[:, :r] * root[None, :], root[:, None] * Vt[:r], S[:r]",
+                                 "root = np.sqrt(S[-r:])\n    return U[:, -r:] * root[None, :], root[:, None] * Vt[-r:], S[-r:]"),
+    "singular_values_not_split": ("root = np.sqrt(S[:r])", "root = S[:r]"),
+    "scale_over_8": ("scale = (absmax / np.float32(7.0)).astype(np.float16)", "scale = (absmax / np.float32(8.0)).astype(np.float16)"),
+    "nibbles_swapped": ("packed = (nib[0::2] | (nib[1::2] << 4)).astype(np.uint8)", "packed = (nib[1::2] | (nib[0::2] << 4)).astype(np.uint8)"),
+    "gate_keeps_what_it_should_prune": ("if gamma > 0.0 and cos < gamma:", "if gamma > 0.0 and cos > gamma:"),
+    "factor_layouts_swapped": ("quantize_int4_groups(A.T)          # U layout [r][d_in]: d_in fastest", "quantize_int4_groups(A)"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(_MUTANTS))
+def test_planted_mistakes_are_caught(name, monkeypatch):
+    import inspect
+    import types
+    src = inspect.getsource(cr)
+    old, new = _MUTANTS[name]
+    assert src.count(old) == 1, name
+    mutant = types.ModuleType("compress_mutant")
+    exec(compile(src.replace(old, new), "compress_mutant", "exec"), mutant.__dict__)
+    for fn in ("quantize_int4_groups", "dequantize_int4_groups", "shared_base", "truncated_factors", "compress", "reconstruct"):
+        monkeypatch.setattr(cr, fn, getattr(mutant, fn))
+    caught = 0
+    for pin in (test_mean_and_residual_by_hand, test_prescribed_singular_values_give_the_eckart_young_error,
+                test_known_low_rank_residuals_are_recovered, test_quantiser_format_and_round_trip, test_cosine_gate):
+        try:
+            pin()
+        except (AssertionError, ValueError, IndexError):
+            caught += 1
+    assert caught >= 1, f"no pin notices the planted mistake {name}"
