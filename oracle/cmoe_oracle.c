@@ -283,3 +283,134 @@ int cmoe_ref_expert_stats(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
   free(cid); free(slot); free(gates);
   return 0;
 }
+
+/* ---------------------------------------------------------------------------------------------------------
+ * More than one cluster per token (Sec. 3.3: "We select the Top-g1 groups (typically g1 = 1)").
+ * The paper gives the second stage for one selected cluster only.  Reading taken here: the g1 clusters with the
+ * largest p_g of Eq. 9 (= largest z_g; lowest index first on ties) are kept; inside each the second stage runs
+ * exactly as for g1 = 1 (top-k of the cluster's K logits, Eq. 10 renormalised over the kept experts); the
+ * clusters' outputs are mixed with p_g renormalised over the kept clusters, i.e. expert i of kept cluster g
+ * weighs p~_g p~_{i|g}, and all g1 k weights of a token sum to one.  g1 = 1 gives cmoe_ref_route's result.
+ * --------------------------------------------------------------------------------------------------------- */
+int cmoe_ref_route_g1(const cmoe_ref_desc* D, const uint16_t* x, int32_t T, int32_t g1,
+                      int32_t* cluster_id, int32_t* expert_slot, float* gates) {
+  if (!desc_ok(D) || g1 < 1 || g1 > D->G || D->E / D->G > 64) return -1;
+  const int d = D->d, G = D->G, K = D->E / D->G, k = D->k;
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    float* z = (float*)malloc(sizeof(float) * (size_t)G);
+    float* l = (float*)malloc(sizeof(float) * (size_t)K);
+    char* gone = (char*)calloc((size_t)G, 1);
+    int* gsel = (int*)malloc(sizeof(int) * (size_t)g1);
+    for (int g = 0; g < G; ++g) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j)
+        acc += (double)cmoe_ref_half_to_float(x[(size_t)t * d + j]) * (double)D->C[(size_t)j * G + g];
+      if (D->b_c) acc += (double)D->b_c[g];
+      z[g] = (float)acc;
+    }
+    /* the g1 largest z_g by repeated argmax */
+    for (int c = 0; c < g1; ++c) {
+      int best = -1;
+      for (int g = 0; g < G; ++g)
+        if (!gone[g] && (best < 0 || z[g] > z[best])) best = g;
+      gone[best] = 1;
+      gsel[c] = best;
+      cluster_id[(size_t)t * g1 + c] = best;
+    }
+    /* p_g of Eq. 9 renormalised over the kept clusters */
+    double zden = 0.0;
+    for (int c = 0; c < g1; ++c) zden += exp((double)z[gsel[c]] - (double)z[gsel[0]]);
+    for (int c = 0; c < g1; ++c) {
+      const int gs = gsel[c];
+      const double pg = exp((double)z[gs] - (double)z[gsel[0]]) / zden;
+      for (int i = 0; i < K; ++i) {
+        double acc = 0.0;
+        for (int j = 0; j < d; ++j)
+          acc += (double)cmoe_ref_half_to_float(x[(size_t)t * d + j]) *
+                 (double)D->R[((size_t)gs * d + j) * K + i];
+        if (D->b_e) acc += (double)D->b_e[(size_t)gs * K + i];
+        l[i] = (float)acc;
+      }
+      char taken[64];
+      int sel[64];
+      memset(taken, 0, sizeof(taken));
+      for (int s = 0; s < k; ++s) {
+        int best = -1;
+        for (int i = 0; i < K; ++i)
+          if (!taken[i] && (best < 0 || l[i] > l[best])) best = i;
+        taken[best] = 1;
+        sel[s] = best;
+        expert_slot[((size_t)t * g1 + c) * k + s] = gs * K + best;
+      }
+      double lmax = (double)l[sel[0]], denom = 0.0;
+      for (int s = 0; s < k; ++s) denom += exp((double)l[sel[s]] - lmax);
+      for (int s = 0; s < k; ++s)
+        gates[((size_t)t * g1 + c) * k + s] = (float)(pg * (exp((double)l[sel[s]] - lmax) / denom));
+    }
+    free(z); free(l); free(gone); free(gsel);
+  }
+  return 0;
+}
+
+/* Layer output with g1 clusters per token: y = sum over the g1 k routed experts of weight * FFN_e(x), the
+ * expert FFNs formed and applied exactly as in cmoe_ref_forward. */
+int cmoe_ref_forward_g1(const cmoe_ref_desc* D, const uint16_t* x, int32_t T, int32_t g1,
+                        const int32_t* token_idx, int32_t n_idx, float* y) {
+  if (!desc_ok(D) || g1 < 1 || g1 > D->G) return -1;
+  const int d = D->d, d_ff = D->d_ff, kk = g1 * D->k, E = D->E;
+  if (n_idx <= 0) return 0;
+  uint16_t* xs = (uint16_t*)malloc(sizeof(uint16_t) * (size_t)n_idx * d);
+  for (int n = 0; n < n_idx; ++n) {
+    int t = token_idx ? token_idx[n] : n;
+    if (t < 0 || t >= T) { free(xs); return -1; }
+    memcpy(xs + (size_t)n * d, x + (size_t)t * d, sizeof(uint16_t) * (size_t)d);
+  }
+  int32_t* cid = (int32_t*)malloc(sizeof(int32_t) * (size_t)n_idx * g1);
+  int32_t* slot = (int32_t*)malloc(sizeof(int32_t) * (size_t)n_idx * kk);
+  float* gate = (float*)malloc(sizeof(float) * (size_t)n_idx * kk);
+  if (cmoe_ref_route_g1(D, xs, n_idx, g1, cid, slot, gate)) { free(xs); free(cid); free(slot); free(gate); return -1; }
+
+  float* W1 = (float*)malloc(sizeof(float) * (size_t)d * d_ff);
+  float* W2 = (float*)malloc(sizeof(float) * (size_t)d_ff * d);
+  double* ysum = (double*)calloc((size_t)n_idx * d, sizeof(double));
+  for (int e = 0; e < E; ++e) {
+    int used = 0;
+    for (int64_t i = 0; i < (int64_t)n_idx * kk; ++i) if (slot[i] == e) { used = 1; break; }
+    if (!used) continue;
+    cmoe_ref_form_weight(D, e, 1, W1);
+    cmoe_ref_form_weight(D, e, 2, W2);
+#pragma omp parallel
+    {
+      double* acc = (double*)malloc(sizeof(double) * (size_t)(d_ff > d ? d_ff : d));
+      float* a = (float*)malloc(sizeof(float) * (size_t)d_ff);
+#pragma omp for schedule(dynamic, 1)
+      for (int n = 0; n < n_idx; ++n) {
+        for (int s = 0; s < kk; ++s) {
+          if (slot[(size_t)n * kk + s] != e) continue;
+          const uint16_t* xt = xs + (size_t)n * d;
+          for (int f = 0; f < d_ff; ++f) acc[f] = 0.0;
+          for (int j = 0; j < d; ++j) {
+            double xj = (double)cmoe_ref_half_to_float(xt[j]);
+            const float* w = W1 + (size_t)j * d_ff;
+            for (int f = 0; f < d_ff; ++f) acc[f] += xj * (double)w[f];
+          }
+          for (int f = 0; f < d_ff; ++f) a[f] = gelu_erf((float)acc[f]);
+          for (int c = 0; c < d; ++c) acc[c] = 0.0;
+          for (int f = 0; f < d_ff; ++f) {
+            double af = (double)a[f];
+            const float* w = W2 + (size_t)f * d;
+            for (int c = 0; c < d; ++c) acc[c] += af * (double)w[c];
+          }
+          /* an expert's output is an fp32 value, as in cmoe_ref_forward; the weighted sum runs in double */
+          for (int c = 0; c < d; ++c)
+            ysum[(size_t)n * d + c] += (double)gate[(size_t)n * kk + s] * (double)(float)acc[c];
+        }
+      }
+      free(acc); free(a);
+    }
+  }
+  for (int64_t i = 0; i < (int64_t)n_idx * d; ++i) y[i] = (float)ysum[i];
+  free(xs); free(cid); free(slot); free(gate); free(W1); free(W2); free(ysum);
+  return 0;
+}

@@ -83,6 +83,14 @@ void cmoe_ref_param_count(const cmoe_ref_desc* D, int64_t* stored, int64_t* dens
 int cmoe_ref_expert_stats(const cmoe_ref_desc* D, const uint16_t* x, int32_t T,
                           int32_t* loads, float* xbar, float* mu, float beta, float* cov);
 
+/* More than one cluster per token (Sec. 3.3, "Top-g1 groups"; the reading is stated above the functions in
+ * cmoe_oracle.c): cluster_id [T][g1] by descending z, expert_slot and gates [T][g1][k]; a token's g1 k gates
+ * sum to one.  g1 = 1 reproduces cmoe_ref_route / cmoe_ref_forward. */
+int cmoe_ref_route_g1(const cmoe_ref_desc* D, const uint16_t* x, int32_t T, int32_t g1,
+                      int32_t* cluster_id, int32_t* expert_slot, float* gates);
+int cmoe_ref_forward_g1(const cmoe_ref_desc* D, const uint16_t* x, int32_t T, int32_t g1,
+                        const int32_t* token_idx, int32_t n_idx, float* y);
+
 int cmoe_ref_num_threads(void);
 
 #ifdef __cplusplus

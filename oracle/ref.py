@@ -46,6 +46,10 @@ def load(path: str):
         L.cmoe_ref_expert_stats.restype = C.c_int
         L.cmoe_ref_expert_stats.argtypes = [C.POINTER(_Desc), C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_float, C.c_void_p]
+        L.cmoe_ref_route_g1.restype = C.c_int
+        L.cmoe_ref_route_g1.argtypes = [C.POINTER(_Desc), C.c_void_p, C.c_int32, C.c_int32] + [C.c_void_p] * 3
+        L.cmoe_ref_forward_g1.restype = C.c_int
+        L.cmoe_ref_forward_g1.argtypes = [C.POINTER(_Desc), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         L.cmoe_ref_num_threads.restype = C.c_int
     return L
 
@@ -107,6 +111,33 @@ class Layer:
         y = np.zeros((n, s.d), np.float32)
         rc = lib().cmoe_ref_forward(C.byref(self.desc), _ptr(x), T, _ptr(idx), n, _ptr(y))
         if rc:
+            raise ValueError("oracle rejected its arguments")
+        return y
+
+    def route_g1(self, x: np.ndarray, g1: int):
+        """g1 clusters per token -> dict(cluster_id [T][g1], expert_slot [T][g1][k], gates [T][g1][k])."""
+        s = self.shape
+        x = np.ascontiguousarray(x, dtype=np.float16)
+        T = x.shape[0]
+        cid = np.empty((T, g1), np.int32)
+        slot = np.empty((T, g1, s.k), np.int32)
+        gates = np.empty((T, g1, s.k), np.float32)
+        if lib().cmoe_ref_route_g1(C.byref(self.desc), _ptr(x), T, g1, _ptr(cid), _ptr(slot), _ptr(gates)):
+            raise ValueError("oracle rejected its arguments")
+        return dict(cluster_id=cid, expert_slot=slot, gates=gates)
+
+    def forward_g1(self, x: np.ndarray, g1: int, token_idx=None) -> np.ndarray:
+        """y (fp32) with g1 clusters per token, for all tokens or for the listed ones."""
+        s = self.shape
+        x = np.ascontiguousarray(x, dtype=np.float16)
+        T = x.shape[0]
+        if token_idx is None:
+            idx, n = None, T
+        else:
+            idx = np.ascontiguousarray(token_idx, dtype=np.int32)
+            n = idx.size
+        y = np.zeros((n, s.d), np.float32)
+        if lib().cmoe_ref_forward_g1(C.byref(self.desc), _ptr(x), T, g1, _ptr(idx), n, _ptr(y)):
             raise ValueError("oracle rejected its arguments")
         return y
 

@@ -8,6 +8,7 @@ import pytest
 
 from oracle import ref
 import test_oracle_pins as pins
+import test_oracle_g1 as g1pins
 
 SRC = os.path.join(os.path.dirname(ref.__file__), "cmoe_oracle.c")
 
@@ -46,6 +47,15 @@ MUTANTS = [
     ("EMA applied without tokens", "if (mu && loads[e] > 0)", "if (mu)"),
     ("sample variance", "sqrt(var / (double)E) / mean", "sqrt(var / (double)(E - 1)) / mean"),
     ("variance instead of deviation", "sqrt(var / (double)E) / mean", "(var / (double)E) / mean"),
+    ("g1: least probable clusters", "z[g] > z[best]", "z[g] < z[best]"),
+    ("g1: a cluster may be kept twice", "gone[best] = 1;", ";"),
+    ("g1: cluster weights not renormalised", "const double pg = exp((double)z[gs] - (double)z[gsel[0]]) / zden;",
+     "const double pg = exp((double)z[gs] - (double)z[gsel[0]]);"),
+    ("g1: cluster weights dropped", "(float)(pg * (exp((double)l[sel[s]] - lmax) / denom))", "(float)((exp((double)l[sel[s]] - lmax) / denom))"),
+    ("g1: only the last expert's output kept", "ysum[(size_t)n * d + c] += (double)gate[(size_t)n * kk + s] *",
+     "ysum[(size_t)n * d + c] = (double)gate[(size_t)n * kk + s] *"),
+    ("g1: expert bias of the first kept cluster", "if (D->b_e) acc += (double)D->b_e[(size_t)gs * K + i];\n        l[i] = (float)acc;\n      }\n      char taken[64];",
+     "if (D->b_e) acc += (double)D->b_e[(size_t)gsel[0] * K + i];\n        l[i] = (float)acc;\n      }\n      char taken[64];"),
 ]
 
 PINS = [
@@ -65,6 +75,12 @@ PINS = [
     pins.test_bf16_bases_are_decoded_as_bf16,
     pins.test_expert_stats_hand_counted,
     pins.test_expert_stats_conservation_and_numpy_counts,
+    g1pins.test_one_cluster_is_the_pinned_routing_and_forward,
+    lambda: g1pins.test_routes_by_enumeration(dict(E=12, G=3, k=2), 2),
+    g1pins.test_forward_against_a_dense_evaluation,
+    g1pins.test_all_clusters_and_all_experts_is_the_full_soft_mixture,
+    g1pins.test_hand_worked_token,
+    g1pins.test_ties_and_bad_arguments,
 ]
 
 
