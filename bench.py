@@ -154,7 +154,9 @@ VARIANTS = {
     "gpt2m_r4": dict(r=4), "gpt2m_r8": dict(r=8), "gpt2m_r32_K2": dict(r=32, E=16), "gpt2m_k1": dict(k=1),
     "gpt2m_G16_K4": dict(E=64, G=16), "gpt2m_K8_r8": dict(E=64, r=8), "gpt2m_E128_G16": dict(E=128, G=16),
     "gpt2m_bf16_bases": dict(),
+    "gpt2m_two_clusters": dict(T=8192),      # Sec. 3.3 "Top-g1 groups", g1 = 2: 8192 tokens, two clusters each
 }
+VARIANT_OPTIONS = {"gpt2m_two_clusters": dict(clusters_per_token=2)}
 
 
 def variant_shape(name):
@@ -171,7 +173,7 @@ def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks,
     x_np = L["x"] if seed_offset == 0 else inputs.make_tokens(s, s.T, seed=seed_offset)
     dev = torch.device(f"cuda:{dev_index}")
     torch.cuda.set_device(dev)
-    m = ClusteredMoELayer(L, device=str(dev))
+    m = ClusteredMoELayer(L, device=str(dev), options=VARIANT_OPTIONS.get(name))
     T = x_np.shape[0]
     x = torch.from_numpy(x_np).to(dev)
     y = torch.empty_like(x)
@@ -275,7 +277,8 @@ def time_workload(name, steps, warmup, rank, seed_offset, want_e2e, want_clocks,
     res = dict(name=name, shape=s, T=T, dev_ms=dev_ms, steps=steps, wall_s=wall, per_step=per_step,
                stage_ms=stage_ms, active_clusters=active_clusters, active_experts=active_experts,
                i_load=i_load, info=m.info, e2e=e2e, clocks=sampler.summary() if sampler else None,
-               sustained=sustained, routes=routes, y=y_host, x=x_np if keep_outputs else None)
+               sustained=sustained, routes=routes, y=y_host, x=x_np if keep_outputs else None,
+               clusters_per_token=(VARIANT_OPTIONS.get(name) or {}).get("clusters_per_token", 1))
     m.close()
     del m, x, y, flush
     torch.cuda.empty_cache()
@@ -312,7 +315,7 @@ def roofline_for(res, peaks, peaks_kind):
     s, T = res["shape"], res["T"]
     stage = max(("up", "down"), key=lambda n: res["stage_ms"].get(n, 0.0))
     ms = res["stage_ms"][stage]
-    flops, nbytes = stage_work(s, T, stage, res["active_clusters"], res["active_experts"])
+    flops, nbytes = stage_work(s, T * res.get("clusters_per_token", 1), stage, res["active_clusters"], res["active_experts"])
     intensity = flops / max(nbytes, 1.0)
     traffic = ncu_traffic(res["name"]) if stage == "up" else None
     if intensity > 300:           # ridge of the B200 is ~250 flop/B
@@ -334,7 +337,8 @@ def roofline_for(res, peaks, peaks_kind):
 
 def whole_layer_fractions(res, n_gpus, peaks=None):
     s, T = res["shape"], res["T"]
-    flops, nbytes = algorithmic_work(s, T, res["active_clusters"], res["active_experts"])
+    # (two clusters per token: the expert FFNs run once per kept cluster)
+    flops, nbytes = algorithmic_work(s, T * res.get("clusters_per_token", 1), res["active_clusters"], res["active_experts"])
     sec = res["dev_ms"] / res["steps"] * 1e-3
     out = {"algorithmic_tflops": flops / sec / 1e12, "algorithmic_gbs": nbytes / sec / 1e9,
            "frac_of_nominal_fp16_2250T": flops / sec / 1e12 / NOMINAL_FP16_TFLOPS,

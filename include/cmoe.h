@@ -116,6 +116,17 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *                 are fp16, so bf16 bases are converted to fp16 while cmoe_create re-lays them out: exact for
  *                 magnitudes from 2^-14 to 65504 (fp16 has the wider significand), rounded to the fp16 subnormal
  *                 grid below, overflowing above.
+ *   clusters_per_token  0 or 1: one cluster per token (Eq. 9's top-1, the paper's "typically g1 = 1"); 2: the paper's
+ *                 "Top-g1 groups" with g1 = 2 (needs G >= 2).  The paper spells out the second stage for one
+ *                 selected cluster only; the reading implemented: the two clusters with the largest p_g of Eq. 9
+ *                 (largest z_g, lowest index first on ties) are kept, the second stage runs in each exactly as for
+ *                 one cluster (top-k of its K logits, Eq. 10 renormalised over the kept experts), and the two
+ *                 clusters' outputs are mixed with p_g renormalised over the kept clusters: expert i of kept cluster g
+ *                 has gate p~_g p~_{i|g}, and a token's 2k gates sum to one.  cmoe_route then writes
+ *                 cluster_id [T][2] (most probable first), expert_ids and gates [T][2][k].  Internally the layer runs
+ *                 on two virtual tokens per token (2 T rows through router, permutation and expert FFNs, then one
+ *                 sum per token), so a call costs about what one of 2 T tokens costs, and the workspace must be sized
+ *                 with cmoe_workspace_bytes_ex.
  * Other values: CMOE_ERR_INVALID_ARG.  reserved must be zero. */
 typedef struct {
   int32_t force_path;
@@ -124,9 +135,13 @@ typedef struct {
   int32_t base_dtype;
   int32_t host_chunks;
   int32_t row_gather;
-  int32_t reserved[2];
+  int32_t clusters_per_token;
+  int32_t reserved[1];
 } cmoe_options;
 int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
+/* cmoe_workspace_bytes for a handle that cmoe_create_ex will make with these options (NULL = cmoe_workspace_bytes):
+ * clusters_per_token = 2 needs a larger arena. */
+int cmoe_workspace_bytes_ex(const cmoe_desc* desc, const cmoe_options* options, size_t* out_bytes);
 
 /* Two-stage routing only (Sec. 3.3, Eq. 9-10) for x = fp16 [T][d]:
  *   cluster_id [T]     chosen cluster g*

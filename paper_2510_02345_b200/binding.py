@@ -21,7 +21,7 @@ ERRORS = {
     -4: "CMOE_ERR_T_EXCEEDS_MAX", -5: "CMOE_ERR_CUDA", -6: "CMOE_ERR_TIMEOUT",
 }
 EXPORTS = ["cmoe_compress_workspace_bytes", "cmoe_compress", "cmoe_quantize_int4", "cmoe_expert_similarity",
-           "cmoe_workspace_bytes", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
+           "cmoe_workspace_bytes", "cmoe_workspace_bytes_ex", "cmoe_create", "cmoe_create_ex", "cmoe_selftest_wait_timeout", "cmoe_expert_stats", "cmoe_route", "cmoe_forward", "cmoe_forward_host", "cmoe_status",
            "cmoe_get_info", "cmoe_last_cuda_error", "cmoe_destroy", "cmoe_strerror",
            "cmoe_profile_enable", "cmoe_profile_read", "cmoe_stage_name", "cmoe_route_static"]
 CMOE_MAX_STAGES = 8
@@ -42,7 +42,7 @@ class cmoe_desc(C.Structure):
 
 class cmoe_options(C.Structure):
     _fields_ = [("force_path", C.c_int32), ("router_fp32", C.c_int32), ("up_tile", C.c_int32), ("base_dtype", C.c_int32),
-                ("host_chunks", C.c_int32), ("row_gather", C.c_int32), ("reserved", C.c_int32 * 2)]
+                ("host_chunks", C.c_int32), ("row_gather", C.c_int32), ("clusters_per_token", C.c_int32), ("reserved", C.c_int32 * 1)]
 
 
 class cmoe_compress_desc(C.Structure):
@@ -75,6 +75,7 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.cmoe_workspace_bytes.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_size_t)]
         L.cmoe_create.argtypes = [C.POINTER(cmoe_desc), C.POINTER(C.c_void_p)]
+        L.cmoe_workspace_bytes_ex.argtypes = [C.POINTER(cmoe_desc), C.POINTER(cmoe_options), C.POINTER(C.c_size_t)]
         L.cmoe_compress_workspace_bytes.argtypes = [C.POINTER(cmoe_compress_desc), C.POINTER(C.c_size_t)]
         L.cmoe_compress.argtypes = [C.POINTER(cmoe_compress_desc), C.c_void_p]
         L.cmoe_quantize_int4.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -278,7 +279,7 @@ class ClusteredMoELayer:
 
     def __init__(self, layer: dict, T_max: int | None = None, device: str = "cuda:0", keep_source: bool = False,
                  options: dict | None = None, guard_bytes: int = 0, fill_byte: int | None = None):
-        """`options`: fields of cmoe_options (force_path, router_fp32, up_tile) for cmoe_create_ex.
+        """`options`: fields of cmoe_options (force_path, router_fp32, up_tile, clusters_per_token, ...) for cmoe_create_ex.
         `guard_bytes` / `fill_byte` (tests): the arena is allocated with that many bytes of a canary pattern
         before and after it, and filled with `fill_byte` before the library sees it."""
         import torch
@@ -305,7 +306,17 @@ class ClusteredMoELayer:
         desc.quant_group, desc.T_max = 32, self.T_max
         for name, _ in self._NP_FIELDS:
             setattr(desc, name, None if src[name] is None else src[name].data_ptr())
-        nbytes = cmoe_workspace_bytes(desc)
+        opts = None
+        if options:
+            opts = cmoe_options()
+            opts.force_path = -1
+            for key, val in options.items():
+                setattr(opts, key, int(val))
+        self.g1 = max(1, int(opts.clusters_per_token)) if opts is not None else 1
+        need = C.c_size_t(0)
+        _check(lib().cmoe_workspace_bytes_ex(C.byref(desc), C.byref(opts) if opts is not None else None, C.byref(need)),
+               "cmoe_workspace_bytes_ex")
+        nbytes = need.value
         guard = (int(guard_bytes) + 255) // 256 * 256
         self.workspace = torch.empty(nbytes + 256 + 2 * guard, dtype=torch.uint8, device=self.device)
         base = (self.workspace.data_ptr() + 255) // 256 * 256 + guard
@@ -320,12 +331,8 @@ class ClusteredMoELayer:
         desc.workspace, desc.workspace_bytes = base, nbytes
         self.workspace_bytes = nbytes
         torch.cuda.synchronize(self.device)
-        if options:
-            o = cmoe_options()
-            o.force_path = -1
-            for key, val in options.items():
-                setattr(o, key, int(val))
-            self.handle = cmoe_create_ex(desc, o)
+        if opts is not None:
+            self.handle = cmoe_create_ex(desc, opts)
         else:
             self.handle = cmoe_create(desc)
         self.info = cmoe_get_info(self.handle)
@@ -340,9 +347,14 @@ class ClusteredMoELayer:
         T = x.shape[0]
         k = self.shape.k
         assert x.is_cuda and x.dtype == torch.float16 and x.is_contiguous() and x.shape[1] == self.shape.d
-        cid = torch.empty(T, dtype=torch.int32, device=x.device)
-        eid = torch.empty((T, k), dtype=torch.int32, device=x.device)
-        gates = torch.empty((T, k), dtype=torch.float32, device=x.device)
+        if self.g1 > 1:           # clusters_per_token: [T][g1], [T][g1][k], [T][g1][k]
+            cid = torch.empty((T, self.g1), dtype=torch.int32, device=x.device)
+            eid = torch.empty((T, self.g1, k), dtype=torch.int32, device=x.device)
+            gates = torch.empty((T, self.g1, k), dtype=torch.float32, device=x.device)
+        else:
+            cid = torch.empty(T, dtype=torch.int32, device=x.device)
+            eid = torch.empty((T, k), dtype=torch.int32, device=x.device)
+            gates = torch.empty((T, k), dtype=torch.float32, device=x.device)
         cmoe_route(self.handle, x.data_ptr(), T, cid.data_ptr(), eid.data_ptr(), gates.data_ptr(), self._stream())
         return cid, eid, gates
 

@@ -35,8 +35,11 @@ long long binom_ll(int n, int m) {
   return r;
 }
 
-int validate_dims(const cmoe_desc* desc, Dims* D) {
+int validate_dims(const cmoe_desc* desc, int g1, Dims* D) {
   if (!desc) return CMOE_ERR_INVALID_ARG;
+  if (g1 < 0 || g1 > 2) return CMOE_ERR_INVALID_ARG;
+  if (g1 < 1) g1 = 1;
+  if (g1 > desc->G) return CMOE_ERR_UNSUPPORTED_SHAPE;
   if (desc->d <= 0 || desc->d_ff <= 0 || desc->E <= 0 || desc->G <= 0 || desc->k <= 0 ||
       desc->r < 0 || desc->T_max <= 0)
     return CMOE_ERR_INVALID_ARG;
@@ -47,9 +50,10 @@ int validate_dims(const cmoe_desc* desc, Dims* D) {
   if (!(desc->r == 0 || desc->r == 4 || desc->r == 8 || desc->r == 16 || desc->r == 32))
     return CMOE_ERR_UNSUPPORTED_SHAPE;
   if (desc->quant_group != 32) return CMOE_ERR_UNSUPPORTED_SHAPE;
-  if (desc->T_max > (1 << 22)) return CMOE_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)desc->T_max * g1 > (1 << 22)) return CMOE_ERR_UNSUPPORTED_SHAPE;
   D->d = desc->d; D->d_ff = desc->d_ff; D->E = desc->E; D->G = desc->G; D->K = K;
-  D->r = desc->r; D->k = desc->k; D->T_max = desc->T_max;
+  // with g1 clusters per token everything below the entry points works on g1 virtual tokens per token
+  D->r = desc->r; D->k = desc->k; D->g1 = g1; D->T_user = desc->T_max; D->T_max = desc->T_max * g1;
   const long long combos = binom_ll(K, desc->k);
   if (combos <= 64) { D->nsub = (int)combos; D->sub_is_combo = 1; }
   else              { D->nsub = K;           D->sub_is_combo = 0; }
@@ -102,6 +106,10 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   s.row_slot = A.take<int>(P * k);
   s.row_gate = A.take<float>(P * k);
   s.x_perm = A.take<__half>(P * d);
+  if (D.g1 > 1) {
+    s.x_rep = A.take<__half>(T * d);
+    s.y_rep = A.take<__half>(T * d);
+  }
   s.t = A.take<float>(P * k * r + 4);
   s.abar = A.take<__half>(P * f);
   s.s = A.take<float>(P * k * r + 4);
@@ -140,7 +148,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 
 int check_call(cmoe_layer* L, const void* x, int32_t T) {
   if (!L) return CMOE_ERR_INVALID_ARG;
   if (T < 0) return CMOE_ERR_INVALID_ARG;
-  if (T > L->dims.T_max) return CMOE_ERR_T_EXCEEDS_MAX;
+  if (T > L->dims.T_user) return CMOE_ERR_T_EXCEEDS_MAX;
   if (T > 0 && (!x || !aligned16(x))) return CMOE_ERR_INVALID_ARG;
   return CMOE_OK;
 }
@@ -149,10 +157,12 @@ int check_call(cmoe_layer* L, const void* x, int32_t T) {
 
 extern "C" {
 
-int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) {
+int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) { return cmoe_workspace_bytes_ex(desc, nullptr, out_bytes); }
+
+int cmoe_workspace_bytes_ex(const cmoe_desc* desc, const cmoe_options* opt, size_t* out_bytes) {
   if (!out_bytes) return CMOE_ERR_INVALID_ARG;
   Dims D{};
-  int rc = validate_dims(desc, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, &D);
   if (rc) return rc;
   Arena A;
   plan(D, A, nullptr, nullptr);
@@ -166,7 +176,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   if (!out_layer) return CMOE_ERR_INVALID_ARG;
   *out_layer = nullptr;
   Dims D{};
-  int rc = validate_dims(desc, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, &D);
   if (rc) return rc;
   if (!desc->C || !desc->R || !desc->B1 || !desc->B2 || !desc->workspace) return CMOE_ERR_INVALID_ARG;
   if (D.r > 0 && (!desc->U1q || !desc->V1q || !desc->U2q || !desc->V2q || !desc->U1s ||
@@ -177,7 +187,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   for (const void* p : ptrs)
     if (!aligned16(p)) return CMOE_ERR_INVALID_ARG;
   size_t need = 0;
-  cmoe_workspace_bytes(desc, &need);
+  cmoe_workspace_bytes_ex(desc, opt, &need);
   if (desc->workspace_bytes < need) return CMOE_ERR_WORKSPACE_TOO_SMALL;
 
   cmoe_options o{};
@@ -185,7 +195,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   if (opt) o = *opt;
   if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
       o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks || o.row_gather < 0 || o.row_gather > 1 ||
-      o.reserved[0] != 0 || o.reserved[1] != 0) return CMOE_ERR_INVALID_ARG;
+      o.reserved[0] != 0) return CMOE_ERR_INVALID_ARG;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -325,6 +335,12 @@ int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int
   if (T == 0) return CMOE_OK;
   if (!cluster_id || !expert_ids || !gates) return CMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (L->dims.g1 > 1) {
+    // g1 virtual tokens per token: the outputs are [T][g1], [T][g1][k], [T][g1][k]
+    CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, st));
+    x = L->sc.x_rep;
+    T *= L->dims.g1;
+  }
   if (L->router_tc && T >= 1024)
     CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st));
   else
@@ -333,11 +349,25 @@ int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int
   return CMOE_OK;
 }
 
+static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream);
+
 int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream) {
   int rc = check_call(L, x, T);
   if (rc) return rc;
   if (T == 0) return CMOE_OK;
   if (!y || !aligned16(y)) return CMOE_ERR_INVALID_ARG;
+  if (L->dims.g1 <= 1) return forward_rows(L, x, T, y, cuda_stream);
+  // g1 clusters per token: every row g1 times, the layer on the virtual tokens, the g1 outputs of a token summed
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, st));
+  rc = forward_rows(L, L->sc.x_rep, T * L->dims.g1, L->sc.y_rep, cuda_stream);
+  if (rc) return rc;
+  CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, st));
+  return CMOE_OK;
+}
+
+// the layer on T rows of x as the kernels see them (virtual tokens when g1 > 1)
+static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Dims& D = L->dims;
   const Scratch& S = L->sc;
@@ -394,7 +424,7 @@ int cmoe_forward_host(cmoe_layer* L, const void* x_host, int32_t T, void* y_host
                       void* x_stage, void* y_stage, void* cuda_stream) {
   if (!L) return CMOE_ERR_INVALID_ARG;
   if (T < 0) return CMOE_ERR_INVALID_ARG;
-  if (T > L->dims.T_max) return CMOE_ERR_T_EXCEEDS_MAX;
+  if (T > L->dims.T_user) return CMOE_ERR_T_EXCEEDS_MAX;
   if (T == 0) return CMOE_OK;
   if (!x_host || !y_host || !x_stage || !y_stage || !aligned16(x_stage) || !aligned16(y_stage)) return CMOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -455,7 +485,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
-                               : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1));
+                               : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.g1 > 1 ? 2 : 0);
   out->memsets_forward = 0;
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;

@@ -26,7 +26,9 @@ struct Dims {
   int d, d_ff, E, G, K, r, k;
   int nsub;        // permutation sub-keys per cluster (expert combinations, or lowest expert)
   int nkey;        // G * nsub
-  int T_max;
+  int T_max;       // most tokens of a call as the kernels see them: g1 virtual tokens per caller token
+  int T_user;      // most tokens of a call as the caller counts them (T_max = g1 * T_user)
+  int g1;          // clusters per token (Sec. 3.3); 0 and 1 both mean one
   int T_pad_max;   // rows of the permuted buffers
   int row_align;   // a cluster's rows start at a multiple of this
   int sub_is_combo;
@@ -70,6 +72,8 @@ struct Scratch {
   int* row_slot;      // [T_pad][k]  expert slot ids (g*K+i), ascending
   float* row_gate;    // [T_pad][k]  gates in the same order (0 for padding rows)
   __half* x_perm;     // [T_pad][d]
+  __half* x_rep;      // [T_max][d]  g1 > 1: every token's row g1 times (one virtual token per kept cluster)
+  __half* y_rep;      // [T_max][d]  g1 > 1: the virtual tokens' outputs, summed per token at the end
   float* t;           // [T_pad][k][r]   x U1_e
   __half* abar;       // [T_pad][d_ff]   sum_j p_j GELU(h_j)
   float* s;           // [T_pad][k][r]   GELU(h_j) U2_e, accumulated with atomics
@@ -169,6 +173,10 @@ void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs);
 // x_src: not null when the t kernel gathers the rows of x itself (tc2_gathers_rows)
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 bool tc2_gathers_rows(const cmoe_layer* L);
+
+// multi_cluster.cu (g1 > 1): x_rep[g1 t + c] = x[t];  y[t] = sum_c y_rep[g1 t + c]
+cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, cudaStream_t st);
+cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, cudaStream_t st);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);

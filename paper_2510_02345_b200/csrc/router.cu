@@ -17,6 +17,7 @@
 #include "launch.cuh"
 #include "device_utils.cuh"
 #include "stage_factors.cuh"
+#include "cluster_pick.cuh"
 
 namespace cmoe {
 
@@ -41,7 +42,8 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& xv, const float4& 
 // renormalised over the kept experts); one thread per token, logits read from `lg`.
 __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, int g, int t,
                                                  const int* __restrict__ label, int* __restrict__ expert_ids,
-                                                 float* __restrict__ gates, int* __restrict__ slot_local) {
+                                                 float* __restrict__ gates, int* __restrict__ slot_local,
+                                                 float cluster_weight = 1.f) {
   unsigned taken = 0;
   float selv[kMaxKsel];
   int seli[kMaxKsel];
@@ -63,7 +65,7 @@ __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, 
   float sum = 0.f;
   for (int s = 0; s < k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
   for (int s = 0; s < k; ++s) {
-    if (gates) gates[(size_t)t * k + s] = ev[s] / sum;
+    if (gates) gates[(size_t)t * k + s] = cluster_weight == 1.f ? ev[s] / sum : cluster_weight * (ev[s] / sum);
     if (expert_ids) expert_ids[(size_t)t * k + s] = label[g * K + seli[s]];
     if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
   }
@@ -80,6 +82,7 @@ struct RouterArgs {
   int* slot_local;
   FactorStage fs;  // per-token kernel only: factor staging that rides in the blocks past the router's own (all words zero: none)
   int n_route_blocks, n_riders;
+  int g1;          // clusters per token: token index t is virtual token t % g1 of caller token t / g1 (x holds its row g1 times)
   int dc;          // columns of the cluster prototypes staged in shared memory at a time
   int crows;       // prototype rows staged at a time: min(G, 8)
 };
@@ -93,6 +96,9 @@ router_tile_kernel(const RouterArgs a) {
   __shared__ int s_cid[kTileTokens];
   __shared__ int s_order[kTileTokens];
   __shared__ float s_zbest[kTileTokens];
+  __shared__ float s_z2[kTileTokens];                      // two clusters per token: second-best logit, its cluster,
+  __shared__ int s_cid2[kTileTokens];                      // and the weight of the cluster the virtual token goes to
+  __shared__ float s_weight[kTileTokens];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int tok0 = blockIdx.x * kTileTokens;
@@ -143,11 +149,27 @@ router_tile_kernel(const RouterArgs a) {
         if (j < ng && lane == t) {
           const float zb = z + a.bc[g0 + j];
           const int slot = warp * kTokPerWarp + t;
-          if ((g0 + j) == 0 || zb > s_zbest[slot]) { s_zbest[slot] = zb; s_cid[slot] = g0 + j; }   // strict >: lowest index wins ties
+          if (a.g1 < 2) {
+            if ((g0 + j) == 0 || zb > s_zbest[slot]) { s_zbest[slot] = zb; s_cid[slot] = g0 + j; }   // strict >: lowest index wins ties
+          } else {
+            TwoBest b{s_zbest[slot], s_z2[slot], (g0 + j) == 0 ? -1 : s_cid[slot], (g0 + j) <= 1 ? -1 : s_cid2[slot]};
+            two_best_add(b, g0 + j, zb);
+            s_zbest[slot] = b.z1; s_z2[slot] = b.z2; s_cid[slot] = b.c1; s_cid2[slot] = b.c2;
+          }
         }
       }
     }
     __syncwarp();
+  }
+  __syncthreads();
+  if (a.g1 >= 2 && threadIdx.x < kTileTokens) {
+    // virtual token 2 t + c takes the token's c-th most probable cluster
+    const TwoBest b{s_zbest[threadIdx.x], s_z2[threadIdx.x], s_cid[threadIdx.x], s_cid2[threadIdx.x]};
+    int g;
+    float w;
+    two_best_pick(b, (tok0 + threadIdx.x) & 1, g, w);
+    s_cid[threadIdx.x] = g;
+    s_weight[threadIdx.x] = w;
   }
   __syncthreads();
 
@@ -227,7 +249,7 @@ router_tile_kernel(const RouterArgs a) {
   // ---- top-k and gates: one thread per token
   if (threadIdx.x < kTileTokens && tok0 + threadIdx.x < a.T)
     select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
-                     a.expert_ids, a.gates, a.slot_local);
+                     a.expert_ids, a.gates, a.slot_local, a.g1 >= 2 ? s_weight[threadIdx.x] : 1.f);
 }
 
 // One block per token; warp w computes the rows w, w + nwarp, ... of the router matrix, each over all of d
@@ -238,6 +260,7 @@ router_token_kernel(const RouterArgs a) {
   if ((int)blockIdx.x >= a.n_route_blocks) { stage_block(a.fs, blockIdx.x - a.n_route_blocks); return; }
   __shared__ float lg[kMaxG];           // cluster logits, then the expert logits (kMaxK <= kMaxG)
   __shared__ int s_g;
+  __shared__ float s_w;                 // weight of the chosen cluster (two clusters per token), else 1
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   const int t = blockIdx.x, d = a.d;
   const __half* xr = a.x + (size_t)t * d;
@@ -274,16 +297,25 @@ router_token_kernel(const RouterArgs a) {
     if (pass == 0) {
       if (threadIdx.x == 0) {
         int gs = 0;
-        float zb = lg[0];
-        for (int g = 1; g < a.G; ++g)
-          if (lg[g] > zb) { zb = lg[g]; gs = g; }          // strict >: lowest index wins ties
+        float w = 1.f;
+        if (a.g1 < 2) {
+          float zb = lg[0];
+          for (int g = 1; g < a.G; ++g)
+            if (lg[g] > zb) { zb = lg[g]; gs = g; }        // strict >: lowest index wins ties
+        } else {
+          TwoBest b;
+          two_best_init(b);
+          for (int g = 0; g < a.G; ++g) two_best_add(b, g, lg[g]);
+          two_best_pick(b, t & 1, gs, w);
+        }
         s_g = gs;
+        s_w = w;
         a.cluster_id[t] = gs;
       }
       __syncthreads();
     }
   }
-  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local);
+  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, s_w);
 }
 
 }  // namespace
@@ -297,7 +329,7 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
   // permutation's row-move kernel)
   if (fs && T < 1024) a.fs = *fs;
   a.n_riders = stage_blocks(a.fs, 256);          // one 32-bit word of packed codes per thread
-  a.x = x; a.T = T; a.d = D.d; a.G = D.G; a.K = D.K; a.k = D.k;
+  a.x = x; a.T = T; a.d = D.d; a.G = D.G; a.K = D.K; a.k = D.k; a.g1 = D.g1;
   a.Ct = W.Ct; a.Rt = W.Rt; a.bc = W.bc; a.be = W.be; a.label = W.label;
   a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;
   if (T < 1024) {

@@ -15,6 +15,7 @@
 #include "launch.cuh"
 #include "tc_ptx.cuh"
 #include "perm_keys.cuh"
+#include "cluster_pick.cuh"
 
 namespace cmoe {
 
@@ -40,6 +41,7 @@ struct RtcParams {
   int* status;
   KeyCount kc;     // key counting for the permutation (keys == nullptr: routing only)
   int stages;      // stages of the operand ring
+  int g1;          // clusters per token (token index = virtual token)
 };
 
 // fp32 router rows -> the two fp16 pieces, rows [hi_0 .. hi_{rp-1}, lo_0 .. lo_{rp-1}] x d (padding rows zero)
@@ -150,10 +152,19 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
       if (tok < p.T) {
         const int rp = p.rp, G = p.G, K = p.K;
         int gs = 0;
-        float zbest = 0.f;
-        for (int g = 0; g < G; ++g) {
-          const float z = fmaf(mine[rp + g], 1.f / 2048.f, mine[g]) + p.bc[g];
-          if (g == 0 || z > zbest) { zbest = z; gs = g; }          // strict >: lowest index wins ties
+        float cluster_weight = 1.f;
+        if (p.g1 < 2) {
+          float zbest = 0.f;
+          for (int g = 0; g < G; ++g) {
+            const float z = fmaf(mine[rp + g], 1.f / 2048.f, mine[g]) + p.bc[g];
+            if (g == 0 || z > zbest) { zbest = z; gs = g; }        // strict >: lowest index wins ties
+          }
+        } else {
+          // two clusters per token: this is virtual token tok % 2 of its token
+          TwoBest b;
+          two_best_init(b);
+          for (int g = 0; g < G; ++g) two_best_add(b, g, fmaf(mine[rp + g], 1.f / 2048.f, mine[g]) + p.bc[g]);
+          two_best_pick(b, tok & 1, gs, cluster_weight);
         }
         p.cluster_id[tok] = gs;
         // expert logits of the chosen cluster, in place over the cluster columns (no longer needed)
@@ -180,7 +191,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         float sum = 0.f;
         for (int s = 0; s < p.k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
         for (int s = 0; s < p.k; ++s) {
-          ev[s] = ev[s] / sum;
+          ev[s] = cluster_weight == 1.f ? ev[s] / sum : cluster_weight * (ev[s] / sum);
           if (p.gates) p.gates[(size_t)tok * p.k + s] = ev[s];
           if (p.expert_ids) p.expert_ids[(size_t)tok * p.k + s] = p.label[gs * K + seli[s]];
           if (p.slot_local) p.slot_local[(size_t)tok * p.k + s] = seli[s];
@@ -296,7 +307,7 @@ cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* c
   CUtensorMap mx;
   if (!make_map3(&mx, x, (uint64_t)T, D.d, RBM)) return cudaErrorInvalidValue;   // x is the caller's buffer: a map per call
   RtcParams p{};
-  p.T = T; p.d = D.d; p.G = D.G; p.K = D.K; p.k = D.k; p.E = D.E; p.rp = router_tc_rp(D);
+  p.T = T; p.d = D.d; p.G = D.G; p.K = D.K; p.k = D.k; p.E = D.E; p.rp = router_tc_rp(D); p.g1 = D.g1;
   p.bc = L->w.bc; p.be = L->w.be; p.label = L->w.label;
   p.cluster_id = cluster_id; p.expert_ids = expert_ids; p.gates = gates; p.slot_local = slot_local; p.status = L->sc.status;
   if (kc) p.kc = *kc;

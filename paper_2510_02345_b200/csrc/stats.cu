@@ -135,7 +135,7 @@ extern "C" int cmoe_selftest_wait_timeout(cmoe_layer* L, int64_t limit_cycles, v
 extern "C" int cmoe_expert_stats(cmoe_layer* L, const void* x, int32_t T, int32_t* loads, float* xbar,
                                  float* mu, float beta, float* cov, void* cuda_stream) {
   if (!L || T < 0 || !loads) return CMOE_ERR_INVALID_ARG;
-  if (T > L->dims.T_max) return CMOE_ERR_T_EXCEEDS_MAX;
+  if (T > L->dims.T_user) return CMOE_ERR_T_EXCEEDS_MAX;
   if (T > 0 && (!x || (reinterpret_cast<uintptr_t>(x) & 15))) return CMOE_ERR_INVALID_ARG;
   if (!(beta >= 0.f && beta <= 1.f)) return CMOE_ERR_INVALID_ARG;
   const Dims& D = L->dims;
@@ -150,6 +150,12 @@ extern "C" int cmoe_expert_stats(cmoe_layer* L, const void* x, int32_t T, int32_
     return CMOE_OK;
   }
   const __half* xh = static_cast<const __half*>(x);
+  if (D.g1 > 1) {
+    // g1 virtual tokens per token: an expert's load counts the tokens that reach it through either kept cluster
+    STAT_CUDA(launch_repeat_rows(D, xh, S.x_rep, T, st));
+    xh = S.x_rep;
+    T *= D.g1;
+  }
   if (L->router_tc && T >= 1024) STAT_CUDA(launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   else STAT_CUDA(launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   STAT_CUDA(launch_chained(loads_kernel, dim3((T + kStatThreads - 1) / kStatThreads), dim3(kStatThreads),
