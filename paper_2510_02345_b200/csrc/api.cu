@@ -35,7 +35,7 @@ long long binom_ll(int n, int m) {
   return r;
 }
 
-int validate_dims(const cmoe_desc* desc, int g1, Dims* D) {
+int validate_dims(const cmoe_desc* desc, int g1, bool allow_split, Dims* D) {
   if (!desc) return CMOE_ERR_INVALID_ARG;
   if (g1 < 0 || g1 > 2) return CMOE_ERR_INVALID_ARG;
   if (g1 < 1) g1 = 1;
@@ -54,9 +54,19 @@ int validate_dims(const cmoe_desc* desc, int g1, Dims* D) {
   D->d = desc->d; D->d_ff = desc->d_ff; D->E = desc->E; D->G = desc->G; D->K = K;
   // with g1 clusters per token everything below the entry points works on g1 virtual tokens per token
   D->r = desc->r; D->k = desc->k; D->g1 = g1; D->T_user = desc->T_max; D->T_max = desc->T_max * g1;
-  const long long combos = binom_ll(K, desc->k);
+  D->split = 0; D->rep = g1;
+  // K r beyond the pair path's expanded rank index: two expert halves per cluster where that makes the shape fit
+  if (allow_split && g1 == 1 && D->T_max > 128 && K % 2 == 0 && desc->k <= K / 2 && 2 * desc->G <= kMaxG &&
+      (long long)desc->T_max * 2 <= (1 << 22)) {
+    Dims V = *D;
+    V.K = K / 2; V.G = 2 * desc->G; V.T_max = 2 * desc->T_max;
+    if (!tc2_supported(*D) && tc2_supported(V)) {
+      D->split = 2; D->rep = 2; D->K = V.K; D->G = V.G; D->T_max = V.T_max;
+    }
+  }
+  const long long combos = binom_ll(D->K, desc->k);
   if (combos <= 64) { D->nsub = (int)combos; D->sub_is_combo = 1; }
-  else              { D->nsub = K;           D->sub_is_combo = 0; }
+  else              { D->nsub = D->K;        D->sub_is_combo = 0; }
   D->nkey = D->G * D->nsub;
   if (D->nkey > kMaxKeys) return CMOE_ERR_UNSUPPORTED_SHAPE;
   D->tc2 = (tc2_supported(*D) && D->T_max > 128) ? 1 : 0;
@@ -71,6 +81,7 @@ int validate_dims(const cmoe_desc* desc, int g1, Dims* D) {
 void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r, k = D.k;
   const size_t T = D.T_max, P = D.T_pad_max;
+  const size_t Gb = real_G(D);                       // bases and cluster prototypes: one per real cluster
   const size_t nblk = (T + kMinCountTile - 1) / kMinCountTile;
   Weights w{};
   Scratch s{};
@@ -80,8 +91,8 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   w.be = A.take<float>(E);
   w.label = A.take<int>(E);
   w.live = A.take<int>(E);
-  w.B1t = A.take<__half>(G * d * f);
-  w.B2t = A.take<__half>(G * d * f);
+  w.B1t = A.take<__half>(Gb * d * f);
+  w.B2t = A.take<__half>(Gb * d * f);
   w.U1q = A.take<uint8_t>(E * r * d / 2 + 16);
   w.V1q = A.take<uint8_t>(E * f * r / 2 + 16);
   w.U2q = A.take<uint8_t>(E * r * f / 2 + 16);
@@ -106,7 +117,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   s.row_slot = A.take<int>(P * k);
   s.row_gate = A.take<float>(P * k);
   s.x_perm = A.take<__half>(P * d);
-  if (D.g1 > 1) {
+  if (D.rep > 1) {
     s.x_rep = A.take<__half>(T * d);
     s.y_rep = A.take<__half>(T * d);
   }
@@ -162,7 +173,7 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) { return cmoe
 int cmoe_workspace_bytes_ex(const cmoe_desc* desc, const cmoe_options* opt, size_t* out_bytes) {
   if (!out_bytes) return CMOE_ERR_INVALID_ARG;
   Dims D{};
-  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || opt->force_path != kPathGeneric, &D);
   if (rc) return rc;
   Arena A;
   plan(D, A, nullptr, nullptr);
@@ -176,7 +187,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   if (!out_layer) return CMOE_ERR_INVALID_ARG;
   *out_layer = nullptr;
   Dims D{};
-  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || opt->force_path != kPathGeneric, &D);
   if (rc) return rc;
   if (!desc->C || !desc->R || !desc->B1 || !desc->B2 || !desc->workspace) return CMOE_ERR_INVALID_ARG;
   if (D.r > 0 && (!desc->U1q || !desc->V1q || !desc->U2q || !desc->V2q || !desc->U1s ||
@@ -224,7 +235,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
 
   cudaStream_t st = 0;
   const Weights& W = L->w;
-  const size_t d = D.d, f = D.d_ff, E = D.E, G = D.G, r = D.r;
+  const size_t d = D.d, f = D.d_ff, E = D.E, G = real_G(D), r = D.r;      // (router weights and bases: real clusters)
   auto fail = [&](cudaError_t) {
     cmoe_destroy(L);
     return CMOE_ERR_CUDA;
@@ -252,8 +263,8 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
     }
   }
   // router: C [d][G] -> Ct [G][d];  R [G][d][K] -> Rt [G][K][d]
-  if ((e = launch_transpose_f32(desc->C, const_cast<float*>(W.Ct), 1, D.d, D.G, st))) return fail(e);
-  if ((e = launch_transpose_f32(desc->R, const_cast<float*>(W.Rt), D.G, D.d, D.K, st))) return fail(e);
+  if ((e = launch_transpose_f32(desc->C, const_cast<float*>(W.Ct), 1, D.d, real_G(D), st))) return fail(e);
+  if ((e = launch_transpose_f32(desc->R, const_cast<float*>(W.Rt), real_G(D), D.d, real_K(D), st))) return fail(e);
   if (desc->b_c) e = cudaMemcpyAsync(const_cast<float*>(W.bc), desc->b_c, G * 4, cudaMemcpyDeviceToDevice, st);
   else           e = cudaMemsetAsync(const_cast<float*>(W.bc), 0, G * 4, st);
   if (e) return fail(e);
@@ -276,11 +287,11 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   const __half* B1src = reinterpret_cast<const __half*>(desc->B1);
   const __half* B2src = reinterpret_cast<const __half*>(desc->B2);
   if (streamed) {
-    if ((e = launch_stage_major_fp16(B1src, const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
-    if ((e = launch_stage_major_fp16(B2src, const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_stage_major_fp16(B1src, const_cast<__half*>(W.B1t), real_G(D), D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_stage_major_fp16(B2src, const_cast<__half*>(W.B2t), real_G(D), D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
   } else {
-    if ((e = launch_transpose_fp16(B1src, const_cast<__half*>(W.B1t), D.G, D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
-    if ((e = launch_transpose_fp16(B2src, const_cast<__half*>(W.B2t), D.G, D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_transpose_fp16(B1src, const_cast<__half*>(W.B1t), real_G(D), D.d, D.d_ff, st, o.base_dtype == 1))) return fail(e);
+    if ((e = launch_transpose_fp16(B2src, const_cast<__half*>(W.B2t), real_G(D), D.d_ff, D.d, st, o.base_dtype == 1))) return fail(e);
   }
   if (r > 0) {
     struct { const void* src; const void* dst; size_t bytes; } cp[] = {
@@ -337,14 +348,15 @@ int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   if (L->dims.g1 > 1) {
     // g1 virtual tokens per token: the outputs are [T][g1], [T][g1][k], [T][g1][k]
-    CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, st));
+    CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, L->dims.g1, st));
     x = L->sc.x_rep;
     T *= L->dims.g1;
   }
+  // (a layer that works on expert halves still reports the token's own routes)
   if (L->router_tc && T >= 1024)
-    CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st));
+    CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st, nullptr, true));
   else
-    CMOE_CUDA(L, launch_router(L->dims, L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
+    CMOE_CUDA(L, launch_router(plain_dims(L->dims), L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
                                gates, nullptr, st));
   return CMOE_OK;
 }
@@ -356,13 +368,15 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   if (rc) return rc;
   if (T == 0) return CMOE_OK;
   if (!y || !aligned16(y)) return CMOE_ERR_INVALID_ARG;
-  if (L->dims.g1 <= 1) return forward_rows(L, x, T, y, cuda_stream);
-  // g1 clusters per token: every row g1 times, the layer on the virtual tokens, the g1 outputs of a token summed
+  const int n = L->dims.rep;
+  if (n <= 1) return forward_rows(L, x, T, y, cuda_stream);
+  // virtual tokens (g1 clusters per token, or expert halves): every row n times, the layer on the virtual
+  // tokens, the n outputs of a token summed
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, st));
-  rc = forward_rows(L, L->sc.x_rep, T * L->dims.g1, L->sc.y_rep, cuda_stream);
+  CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, n, st));
+  rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream);
   if (rc) return rc;
-  CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, st));
+  CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, n, st));
   return CMOE_OK;
 }
 
@@ -485,7 +499,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
-                               : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.g1 > 1 ? 2 : 0);
+                               : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.rep > 1 ? 2 : 0);
   out->memsets_forward = 0;
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;

@@ -3,6 +3,8 @@
 // cluster's kept experts are scaled by the cluster's weight, Eq. 9's p_g renormalised over the two kept clusters.
 #pragma once
 
+#include "cmoe_internal.h"
+
 namespace cmoe {
 
 // Running best and second-best cluster logit; clusters are added in ascending index and ties keep the lower index.
@@ -20,6 +22,23 @@ __device__ __forceinline__ void two_best_pick(const TwoBest& b, int rank, int& g
   const float e2 = expf(b.z2 - b.z1);            // p_second / p_first <= 1
   if (rank == 0) { g = b.c1; w = 1.f / (1.f + e2); }
   else           { g = b.c2; w = e2 / (1.f + e2); }
+}
+
+// Expert halves (Dims::split): virtual token `half` (0 or 1) of a token keeps those of the token's k experts that
+// lie in that half of the cluster's K experts, renumbered inside the half, and fills its remaining slots with
+// other experts of the half (lowest index first) at gate zero.  sel / gate: in the token's k kept experts (local
+// index 0 .. K-1, gates summing to one), out this virtual token's k slots (local index 0 .. K/2-1).
+__device__ __forceinline__ void split_half(int K, int k, int half, int* sel, float* gate) {
+  const int Kh = K >> 1;
+  int si[kMaxKsel];
+  float gv[kMaxKsel];
+  unsigned used = 0;
+  int n = 0;
+  for (int s = 0; s < k; ++s)
+    if (sel[s] / Kh == half) { si[n] = sel[s] - half * Kh; gv[n] = gate[s]; used |= 1u << si[n]; ++n; }
+  for (int i = 0; n < k && i < Kh; ++i)
+    if (!((used >> i) & 1u)) { si[n] = i; gv[n] = 0.f; ++n; }
+  for (int s = 0; s < k; ++s) { sel[s] = si[s]; gate[s] = gv[s]; }
 }
 
 }  // namespace cmoe

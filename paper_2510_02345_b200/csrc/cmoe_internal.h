@@ -22,6 +22,12 @@ constexpr int kMinCountTile = 128; // token tile of the router kernel that count
 
 enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
 
+// Expert halves (split == 2): a cluster whose K r exceeds the 64 columns of the pair path's expanded rank index is
+// handled as two virtual clusters of K / 2 experts (virtual cluster 2 g + c = experts c K / 2 .. of cluster g: the
+// expert numbering e = g K + i does not change) that share the base of cluster g.  A token becomes two virtual
+// tokens, one per half, each with those of its kept experts that lie in the half and, in its remaining slots,
+// other experts of the half at gate zero; their outputs are summed.  G and K below are then the virtual counts
+// (2 G, K / 2): everything behind the router sees an ordinary layer; the router and the bases use real_G / real_K.
 struct Dims {
   int d, d_ff, E, G, K, r, k;
   int nsub;        // permutation sub-keys per cluster (expert combinations, or lowest expert)
@@ -29,6 +35,8 @@ struct Dims {
   int T_max;       // most tokens of a call as the kernels see them: g1 virtual tokens per caller token
   int T_user;      // most tokens of a call as the caller counts them (T_max = g1 * T_user)
   int g1;          // clusters per token (Sec. 3.3); 0 and 1 both mean one
+  int split;       // 2: the clusters are handled as two halves of K / 2 experts each (below); else 0
+  int rep;         // rows of the kernels' x per caller token: max(g1, split, 1)
   int T_pad_max;   // rows of the permuted buffers
   int row_align;   // a cluster's rows start at a multiple of this
   int sub_is_combo;
@@ -126,6 +134,8 @@ struct cmoe_layer {
 namespace cmoe {
 
 inline int round_up(int a, int b) { return (a + b - 1) / b * b; }
+inline int real_G(const Dims& D) { return D.split > 1 ? D.G / D.split : D.G; }
+inline int real_K(const Dims& D) { return D.split > 1 ? D.K * D.split : D.K; }
 inline int t_pad_bound(const Dims& D, int T) { return round_up(T, D.row_align) + D.G * D.row_align; }
 
 // ---- launchers (each returns the cudaError_t of its launches) ----------------------------------
@@ -143,7 +153,9 @@ bool router_tc_supported(const Dims& D);
 cudaError_t router_tc_init(cmoe_layer* L);
 // kc (or null): the kernel also writes every token's permutation key and the key counts of its 128-token tiles
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
-                             int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr);
+                             int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr, bool plain = false);
+// plain: the routes as the caller sees them even when the layer works on expert halves (Dims::split)
+inline Dims plain_dims(const Dims& D) { Dims R = D; R.G = real_G(D); R.K = real_K(D); R.split = 0; return R; }
 int router_tc_tile_tokens();
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
@@ -174,9 +186,9 @@ void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs);
 cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __half* y, cudaStream_t st, cudaEvent_t* marks);
 bool tc2_gathers_rows(const cmoe_layer* L);
 
-// multi_cluster.cu (g1 > 1): x_rep[g1 t + c] = x[t];  y[t] = sum_c y_rep[g1 t + c]
-cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, cudaStream_t st);
-cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, cudaStream_t st);
+// multi_cluster.cu (virtual tokens): x_rep[n t + c] = x[t];  y[t] = sum_c y_rep[n t + c]
+cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, int n, cudaStream_t st);
+cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, cudaStream_t st);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);

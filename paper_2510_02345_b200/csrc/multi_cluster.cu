@@ -1,7 +1,8 @@
-// Two clusters per token (Sec. 3.3, "Top-g1 groups"): the layer runs on g1 virtual tokens per token.  Before the
+// Virtual tokens.  Two clusters per token (Sec. 3.3, "Top-g1 groups"): the layer runs on g1 virtual tokens per token.  Before the
 // router every row of x is written g1 times (virtual token g1 t + c is token t on its way to its c-th most
 // probable cluster); after the un-permuting store the g1 output rows of a token are summed.  The gates already
-// carry the clusters' weights, so the sum is the mixture.
+// carry the clusters' weights, so the sum is the mixture.  Expert halves (Dims::split) use the same two kernels: a
+// token's two virtual tokens carry the experts of one half of its cluster each.
 #include "cmoe_internal.h"
 
 namespace cmoe {
@@ -40,17 +41,17 @@ int grid_for(long long n, int sm_count) {
 
 }  // namespace
 
-cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, cudaStream_t st) {
+cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, int n, cudaStream_t st) {
   const long long vec = D.d / 8;
   repeat_rows_kernel<<<grid_for((long long)T * vec, D.sm_count), 256, 0, st>>>(
-      reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(x_rep), vec, T, D.g1);
+      reinterpret_cast<const uint4*>(x), reinterpret_cast<uint4*>(x_rep), vec, T, n);
   return cudaGetLastError();
 }
 
-cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, cudaStream_t st) {
+cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, cudaStream_t st) {
   const long long pairs = D.d / 2;
   sum_rows_kernel<<<grid_for((long long)T * pairs, D.sm_count), 256, 0, st>>>(
-      reinterpret_cast<const __half2*>(y_rep), reinterpret_cast<__half2*>(y), pairs, T, D.g1);
+      reinterpret_cast<const __half2*>(y_rep), reinterpret_cast<__half2*>(y), pairs, T, n);
   return cudaGetLastError();
 }
 

@@ -43,7 +43,7 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& xv, const float4& 
 __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, int g, int t,
                                                  const int* __restrict__ label, int* __restrict__ expert_ids,
                                                  float* __restrict__ gates, int* __restrict__ slot_local,
-                                                 float cluster_weight = 1.f) {
+                                                 float cluster_weight = 1.f, int half = -1) {
   unsigned taken = 0;
   float selv[kMaxKsel];
   int seli[kMaxKsel];
@@ -64,6 +64,16 @@ __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, 
   float ev[kMaxKsel];
   float sum = 0.f;
   for (int s = 0; s < k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
+  if (half >= 0) {
+    // expert halves: this virtual token's share of the token's experts (internal routes only: no labels)
+    for (int s = 0; s < k; ++s) ev[s] = ev[s] / sum;
+    split_half(K, k, half, seli, ev);
+    for (int s = 0; s < k; ++s) {
+      if (gates) gates[(size_t)t * k + s] = ev[s];
+      if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
+    }
+    return;
+  }
   for (int s = 0; s < k; ++s) {
     if (gates) gates[(size_t)t * k + s] = cluster_weight == 1.f ? ev[s] / sum : cluster_weight * (ev[s] / sum);
     if (expert_ids) expert_ids[(size_t)t * k + s] = label[g * K + seli[s]];
@@ -82,6 +92,8 @@ struct RouterArgs {
   int* slot_local;
   FactorStage fs;  // per-token kernel only: factor staging that rides in the blocks past the router's own (all words zero: none)
   int n_route_blocks, n_riders;
+  int split;       // 2: expert halves; token index t is virtual token (half) t % 2 of caller token t / 2, and the
+                   // cluster id written is 2 g + half
   int g1;          // clusters per token: token index t is virtual token t % g1 of caller token t / g1 (x holds its row g1 times)
   int dc;          // columns of the cluster prototypes staged in shared memory at a time
   int crows;       // prototype rows staged at a time: min(G, 8)
@@ -182,7 +194,7 @@ router_tile_kernel(const RouterArgs a) {
       rank += (cu < c || (cu == c && u < me)) ? 1 : 0;
     }
     s_order[rank] = me;
-    if (tok0 + me < a.T) a.cluster_id[tok0 + me] = c;
+    if (tok0 + me < a.T) a.cluster_id[tok0 + me] = a.split > 1 ? 2 * c + ((tok0 + me) & 1) : c;
   }
   __syncthreads();
 
@@ -249,7 +261,8 @@ router_tile_kernel(const RouterArgs a) {
   // ---- top-k and gates: one thread per token
   if (threadIdx.x < kTileTokens && tok0 + threadIdx.x < a.T)
     select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
-                     a.expert_ids, a.gates, a.slot_local, a.g1 >= 2 ? s_weight[threadIdx.x] : 1.f);
+                     a.expert_ids, a.gates, a.slot_local, a.g1 >= 2 ? s_weight[threadIdx.x] : 1.f,
+                     a.split > 1 ? (int)((tok0 + threadIdx.x) & 1) : -1);
 }
 
 // One block per token; warp w computes the rows w, w + nwarp, ... of the router matrix, each over all of d
@@ -310,12 +323,12 @@ router_token_kernel(const RouterArgs a) {
         }
         s_g = gs;
         s_w = w;
-        a.cluster_id[t] = gs;
+        a.cluster_id[t] = a.split > 1 ? 2 * gs + (t & 1) : gs;
       }
       __syncthreads();
     }
   }
-  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, s_w);
+  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, s_w, a.split > 1 ? (t & 1) : -1);
 }
 
 }  // namespace
@@ -329,7 +342,7 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
   // permutation's row-move kernel)
   if (fs && T < 1024) a.fs = *fs;
   a.n_riders = stage_blocks(a.fs, 256);          // one 32-bit word of packed codes per thread
-  a.x = x; a.T = T; a.d = D.d; a.G = D.G; a.K = D.K; a.k = D.k; a.g1 = D.g1;
+  a.x = x; a.T = T; a.d = D.d; a.G = real_G(D); a.K = real_K(D); a.k = D.k; a.g1 = D.g1; a.split = D.split;
   a.Ct = W.Ct; a.Rt = W.Rt; a.bc = W.bc; a.be = W.be; a.label = W.label;
   a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;
   if (T < 1024) {
@@ -340,12 +353,12 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
     return cudaGetLastError();
   }
   // chunk of the prototypes staged at a time: at most 32 KB for a group of eight clusters
-  const int rows = D.G < kGroup ? D.G : kGroup;
+  const int rows = a.G < kGroup ? a.G : kGroup;
   int dc = 32768 / (4 * rows) / 256 * 256;
   if (dc > D.d) dc = D.d;
   a.dc = dc;
   a.crows = rows;
-  const size_t sh = sizeof(float) * ((size_t)rows * dc + (size_t)kTileTokens * D.K);      // at most 32 KB + 8 KB
+  const size_t sh = sizeof(float) * ((size_t)rows * dc + (size_t)kTileTokens * a.K);      // at most 32 KB + 8 KB
   static std::atomic<unsigned long long> smem_set{0};      // devices the kernel's shared-memory limit has been raised on
   if (cudaError_t e = ensure_dynamic_smem(router_tile_kernel, 64 * 1024, smem_set)) return e;
   launch_chained(router_tile_kernel, dim3((T + kTileTokens - 1) / kTileTokens), dim3(kTileWarps * 32), sh, st, 1,

@@ -152,18 +152,19 @@ extern "C" int cmoe_expert_stats(cmoe_layer* L, const void* x, int32_t T, int32_
   const __half* xh = static_cast<const __half*>(x);
   if (D.g1 > 1) {
     // g1 virtual tokens per token: an expert's load counts the tokens that reach it through either kept cluster
-    STAT_CUDA(launch_repeat_rows(D, xh, S.x_rep, T, st));
+    STAT_CUDA(launch_repeat_rows(D, xh, S.x_rep, T, D.g1, st));
     xh = S.x_rep;
     T *= D.g1;
   }
-  if (L->router_tc && T >= 1024) STAT_CUDA(launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
-  else STAT_CUDA(launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
+  // (the token's own routes, also when the layer works on expert halves)
+  if (L->router_tc && T >= 1024) STAT_CUDA(launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, nullptr, true));
+  else STAT_CUDA(launch_router(plain_dims(D), L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   STAT_CUDA(launch_chained(loads_kernel, dim3((T + kStatThreads - 1) / kStatThreads), dim3(kStatThreads),
-                           sizeof(int) * (size_t)D.E, st, 1, (int)T, D.K, D.k, D.E, (const int*)S.cluster_id,
+                           sizeof(int) * (size_t)D.E, st, 1, (int)T, real_K(D), D.k, D.E, (const int*)S.cluster_id,
                            (const int*)S.slot, (int*)loads));
   if (xbar || mu)
     STAT_CUDA(launch_chained(xbar_kernel, dim3(D.E, (D.d + kStatCols - 1) / kStatCols), dim3(kStatThreads), 0, st, 1,
-                             (int)T, D.d, D.K, D.k, xh, (const int*)S.cluster_id, (const int*)S.slot,
+                             (int)T, D.d, real_K(D), D.k, xh, (const int*)S.cluster_id, (const int*)S.slot,
                              (const int*)loads, xbar, mu, beta));
   if (cov) STAT_CUDA(launch_chained(cov_kernel, dim3(1), dim3(kStatThreads), 0, st, 1, D.E, (const int*)loads, cov));
 #undef STAT_CUDA

@@ -362,7 +362,9 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
         tile_of(w, pt, nt);
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
-        const int brow = g * p.N + nt * BN_UP + (int)rank * (BN_UP / 2);
+        const int ncol = nt * BN_UP + (int)rank * (BN_UP / 2);
+        const int brow = (g >> p.bshift) * p.N + ncol;        // base rows: of the cluster that owns the base
+        const int vrow = g * p.N + ncol;                      // staged factor rows: of this (virtual) cluster
         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
         if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
         const uint32_t a_dst = base + s * UP_STAGE_BYTES, b_dst = a_dst + UP_A_BYTES;
@@ -374,10 +376,10 @@ tc2_up_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_constant__ 
           // expanded-index stage: atom 0 = (A0, V1f) for P, atom 1 = (Ad, V1f) for Q
           if (leader) mbar_expect_tx(local(B_FULL + s), 2 * KSEL * (UP_A_ATOM + UP_B_ATOM));
           tma2_load_2d(a_dst, &tmA0, lead(B_FULL + s), 0, arow);
-          tma2_load_2d(b_dst, &tmV1, lead(B_FULL + s), 0, brow);
+          tma2_load_2d(b_dst, &tmV1, lead(B_FULL + s), 0, vrow);
           if (KSEL == 2) {
             tma2_load_2d(a_dst + UP_A_ATOM, &tmAd, lead(B_FULL + s), 0, arow);
-            tma2_load_2d(b_dst + UP_B_ATOM, &tmV1, lead(B_FULL + s), 0, brow);
+            tma2_load_2d(b_dst + UP_B_ATOM, &tmV1, lead(B_FULL + s), 0, vrow);
           }
         }
       }
@@ -675,6 +677,7 @@ struct Down2Params {
   __half* y;           // [T][N], original token order
   int* status;
   int KC, NT, N;
+  int bshift;          // the base of cluster g is that of g >> bshift (expert halves share their cluster's base)
   // Not null: the up kernel left the sums s = a_j U2_e in fp32 (its work units were parts of a row tile) and this
   // kernel turns them into its own operand As[row][block of e_j] = fp16(p_j s_j), row tile by row tile, in the
   // epilogue warps while they wait for the tile's main loop.
@@ -762,7 +765,9 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
         const int pt = w / NT, nt = w - pt * NT;
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
-        const int brow = g * p.N + nt * BN + (int)rank * (BN / 2);
+        const int ncol = nt * BN + (int)rank * (BN / 2);
+        const int brow = (g >> p.bshift) * p.N + ncol;        // base rows: of the cluster that owns the base
+        const int vrow = g * p.N + ncol;                      // staged factor rows: of this (virtual) cluster
         const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
         if (!mbar_wait_cluster(local(B_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
         const uint32_t a_dst = base + s * STAGE_BYTES, b_dst = a_dst + Cfg::A_BYTES;
@@ -775,7 +780,7 @@ tc2_down_kernel(const __grid_constant__ CUtensorMap tmA3, const __grid_constant_
           if (p.s && !mbar_wait(local(B_ASREADY), (uint32_t)ti & 1u, abort_flag)) { failed = true; break; }
           if (leader) mbar_expect_tx(local(B_FULL + s), 2 * (Cfg::A_ATOM + Cfg::B_ATOM));
           tma2_load_2d(a_dst, &tmAs, lead(B_FULL + s), 0, arow);
-          tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, brow);
+          tma2_load_2d(b_dst, &tmV2, lead(B_FULL + s), 0, vrow);
         }
       }
     }
@@ -1041,13 +1046,13 @@ cudaError_t tc2_init(cmoe_layer* L) {
   ts->log2r = D.r > 0 ? ilog2(D.r) : 0;
   ts->sm_count = D.sm_count;
   cudaError_t e;
-  const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G;
+  const uint64_t P = (uint64_t)D.T_pad_max, G = (uint64_t)D.G, Gb = (uint64_t)real_G(D);     // Gb: bases, one per real cluster
   bool ok = make_map(&ts->mX, S.x_perm, P, D.d, BM) &&
             make_map3(&ts->mX3, S.x_perm, P, D.d, BM) &&
-            make_map3(&ts->mB13, L->w.B1t, G * D.d_ff, D.d, BN_UP / 2) &&
-            make_map3(&ts->mB13w, L->w.B1t, G * D.d_ff, D.d, BN_WIDE / 2) &&
+            make_map3(&ts->mB13, L->w.B1t, Gb * D.d_ff, D.d, BN_UP / 2) &&
+            make_map3(&ts->mB13w, L->w.B1t, Gb * D.d_ff, D.d, BN_WIDE / 2) &&
             make_map3(&ts->mAbar3, S.abar, P, D.d_ff, BM) &&
-            make_map3(&ts->mB23, L->w.B2t, G * D.d, D.d_ff, ts->bn_down / 2);
+            make_map3(&ts->mB23, L->w.B2t, Gb * D.d, D.d_ff, ts->bn_down / 2);
   if (ok && D.r > 0) {
     ok = make_map(&ts->mA0, S.A0, P, KE, BM) && make_map(&ts->mAd, S.Ad, P, KE, BM) &&
          make_map(&ts->mAs, S.As, P, KE, BM) &&
@@ -1140,6 +1145,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __ha
   up.n_rows = S.n_rows; up.tile_cluster = S.tile_cluster; up.tile_mask = S.tile_mask; up.row_slot = S.row_slot;
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
   up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
+  up.bshift = D.split > 1 ? 1 : 0;
   const UpPlan plan = plan_up(ts, D, T);
   {
     up.NT = plan.NT;
@@ -1159,6 +1165,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __ha
   Down2Params dn{};
   dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask_dn; dn.row_token = S.row_token;
   dn.y = y; dn.status = S.status; dn.KC = D.d_ff / (BK * KA); dn.NT = D.d / ts.bn_down; dn.N = D.d;
+  dn.bshift = D.split > 1 ? 1 : 0;
   if (D.r > 0 && !plan.direct) {
     dn.s = S.s; dn.row_slot = S.row_slot; dn.row_gate = S.row_gate; dn.As = S.As; dn.K = D.K; dn.k = D.k; dn.r = D.r;
   }

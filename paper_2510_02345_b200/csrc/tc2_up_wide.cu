@@ -144,7 +144,9 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
         tile_of(w, pt, nt);
         const int g = p.tile_cluster[pt];
         const int arow = (2 * pt + (int)rank) * BM;
-        const int brow = g * p.N + nt * BN_WIDE + (int)rank * (BN_WIDE / 2);
+        const int ncol = nt * BN_WIDE + (int)rank * (BN_WIDE / 2);
+        const int brow = (g >> p.bshift) * p.N + ncol;        // base rows: of the cluster that owns the base
+        const int vrow = g * p.N + ncol;                      // staged factor rows: of this (virtual) cluster
         for (; c < spt; c += UW_PRODUCERS) {
           if (!mbar_wait_cluster(local(W_EMPTY + s), ph ^ 1u, abort_flag)) { failed = true; break; }
           const uint32_t a_dst = base + s * UW_STAGE_BYTES, b_dst = a_dst + UW_A_BYTES;
@@ -157,7 +159,7 @@ tc2_up_wide_kernel(const __grid_constant__ CUtensorMap tmX3, const __grid_consta
             if (leader) mbar_expect_tx(local(W_FULL + s), 2 * (KSEL * UW_A_ATOM + UW_B_ATOM));
             tma2_load_2d(a_dst, &tmA0, lead(W_FULL + s), 0, arow);
             if (KSEL == 2) tma2_load_2d(a_dst + UW_A_ATOM, &tmAd, lead(W_FULL + s), 0, arow);
-            tma2_load_2d(b_dst, &tmV1, lead(W_FULL + s), 0, brow);
+            tma2_load_2d(b_dst, &tmV1, lead(W_FULL + s), 0, vrow);
           }
           s += UW_PRODUCERS;
           if (s >= (uint32_t)STAGES) { s -= STAGES; ph ^= 1u; }

@@ -606,12 +606,46 @@ def test_headline_shape_variants(kw):
 
 
 def test_many_experts_beyond_the_pair_path():
-    """E = 128 in G = 16 clusters with r = 16 (K r = 128 > 64): the first tensor-core path with the rank-r terms in
-    its epilogue takes it; sampled rows."""
+    """E = 128 in G = 16 clusters with r = 16 (K r = 128 > 64, the expanded rank index of the pair path holds 64): the
+    clusters are handled as two halves of four experts on the pair path; sampled rows."""
     s = inputs.small_shape(T=4096, d=1024, d_ff=4096, E=128, G=16, r=16, k=2)
     L = inputs.make_layer(s, 8)
     got = full_check(L, L["x"], sample=512)
     assert got["module"].info.path == 1
+
+
+@pytest.mark.parametrize("T,kw", [
+    (700, dict(d=256, d_ff=256, E=16, G=2, r=16, k=2)),        # K = 8, r = 16: halves of four experts
+    (1500, dict(d=128, d_ff=512, E=8, G=2, r=32, k=2)),        # K = 4, r = 32: halves of two experts, both kept or one each
+    (1111, dict(d=256, d_ff=256, E=32, G=2, r=8, k=1)),        # K = 16, r = 8, one kept expert: one half has none
+    (129, dict(d=128, d_ff=256, E=24, G=3, r=16, k=2)),        # ragged, mostly padding rows
+    (2048, dict(d=256, d_ff=512, E=32, G=4, r=16, k=3)),       # k = 3 of K = 8: generic fallback of the pair path? (k <= 2 only)
+], ids=["K8r16", "K4r32", "K16r8k1", "ragged", "k3"])
+def test_expert_halves(T, kw):
+    """K r > 64: every cluster as two virtual clusters of K / 2 experts sharing its base, two virtual tokens per token
+    (its kept experts of that half, the other slots at gate zero), outputs summed.  Every row against the oracle."""
+    s = inputs.small_shape(T=T, **kw)
+    L = inputs.make_layer(s, 17)
+    got = full_check(L, L["x"])
+    if kw["k"] <= 2:
+        assert got["module"].info.path == 1
+        assert got["module"].info.T_pad_max >= 2 * T            # two virtual tokens per token
+
+
+def test_expert_halves_report_the_tokens_own_routes_and_loads():
+    """cmoe_route and cmoe_expert_stats of a layer that works on expert halves: the token's k experts among all K
+    of its cluster (full_check compares them with the oracle), every token counted k times."""
+    import torch
+    s = inputs.small_shape(T=900, d=128, d_ff=256, E=16, G=2, r=16, k=2)
+    L = inputs.make_layer(s, 18)
+    got = full_check(L, L["x"])
+    assert got["eid"].shape == (s.T, s.k) and got["eid"].max() >= s.E // 2
+    m = got["module"]
+    loads, _, _ = m.expert_stats(torch.from_numpy(L["x"]).cuda())
+    torch.cuda.synchronize()
+    want = np.bincount(ref.Layer(L).route(L["x"])["expert_slot"].reshape(-1), minlength=s.E)
+    assert int(loads.sum()) == s.k * s.T
+    assert np.abs(loads.cpu().numpy() - want).sum() <= 16          # near-tie tokens only
 
 
 # ---- zero residual blocks (Sec. 3.4: blocks pruned by the cosine gate) are found at create time and skipped ----
