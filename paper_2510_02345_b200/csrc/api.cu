@@ -121,6 +121,11 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
     s.x_rep = A.take<__half>(T * d);
     s.y_rep = A.take<__half>(T * d);
   }
+  if (D.split > 1) {
+    s.r_cluster = A.take<int>(D.T_user);
+    s.r_slot = A.take<int>((size_t)D.T_user * k);
+    s.r_gates = A.take<float>((size_t)D.T_user * k);
+  }
   s.t = A.take<float>(P * k * r + 4);
   s.abar = A.take<__half>(P * f);
   s.s = A.take<float>(P * k * r + 4);
@@ -354,14 +359,14 @@ int cmoe_route(cmoe_layer* L, const void* x, int32_t T, int32_t* cluster_id, int
   }
   // (a layer that works on expert halves still reports the token's own routes)
   if (L->router_tc && T >= 1024)
-    CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st, nullptr, true));
+    CMOE_CUDA(L, launch_router_tc(L, static_cast<const __half*>(x), T, cluster_id, expert_ids, gates, nullptr, st));
   else
     CMOE_CUDA(L, launch_router(plain_dims(L->dims), L->w, static_cast<const __half*>(x), T, cluster_id, expert_ids,
                                gates, nullptr, st));
   return CMOE_OK;
 }
 
-static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream);
+static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream, const void* x_tokens);
 
 int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream) {
   int rc = check_call(L, x, T);
@@ -369,19 +374,23 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   if (T == 0) return CMOE_OK;
   if (!y || !aligned16(y)) return CMOE_ERR_INVALID_ARG;
   const int n = L->dims.rep;
-  if (n <= 1) return forward_rows(L, x, T, y, cuda_stream);
+  if (n <= 1) return forward_rows(L, x, T, y, cuda_stream, nullptr);
   // virtual tokens (g1 clusters per token, or expert halves): every row n times, the layer on the virtual
   // tokens, the n outputs of a token summed
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, n, st));
-  rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream);
+  rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream, L->dims.split > 1 ? x : nullptr);
   if (rc) return rc;
-  CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, n, st));
+  // (expert halves: a half without any of the token's experts has no row)
+  CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, n,
+                               L->dims.split > 1 ? L->sc.cluster_id : nullptr, st));
   return CMOE_OK;
 }
 
-// the layer on T rows of x as the kernels see them (virtual tokens when g1 > 1)
-static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream) {
+// The layer on T rows of x as the kernels see them (virtual tokens when Dims::rep > 1).  x_tokens: not null for a
+// layer on expert halves: the caller's T / 2 tokens, which are routed once over the real clusters; their routes are
+// then split into those of the virtual tokens.
+static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream, const void* x_tokens) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const Dims& D = L->dims;
   const Scratch& S = L->sc;
@@ -399,13 +408,22 @@ static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* 
   KeyCount kc{};
   kc.keys = S.keys; kc.block_counts = S.block_counts; kc.nsub = D.nsub; kc.nkey = D.nkey; kc.sub_is_combo = D.sub_is_combo;
   int counted_tile = 0;
-  if (L->router_tc && T >= 1024) {
-    CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc));
-    counted_tile = router_tc_tile_tokens();
+  if (x_tokens) {
+    const __half* xt = static_cast<const __half*>(x_tokens);
+    const int Tt = T / D.split;
+    if (L->router_tc && Tt >= 1024) CMOE_CUDA(L, launch_router_tc(L, xt, Tt, S.r_cluster, nullptr, S.r_gates, S.r_slot, st));
+    else CMOE_CUDA(L, launch_router(plain_dims(D), L->w, xt, Tt, S.r_cluster, nullptr, S.r_gates, S.r_slot, st, &fs));
+    CMOE_CUDA(L, launch_split_routes(D, S, Tt, st));
+    if (Tt < 1024) fs = FactorStage{};  // staged beside the per-token router (else by the row-move kernel)
   } else {
-    CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &fs));
+    if (L->router_tc && T >= 1024) {
+      CMOE_CUDA(L, launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &kc));
+      counted_tile = router_tc_tile_tokens();
+    } else {
+      CMOE_CUDA(L, launch_router(D, L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, &fs));
+    }
+    if (T < 1024) fs = FactorStage{};   // staged beside the per-token router (else by the row-move kernel)
   }
-  if (T < 1024) fs = FactorStage{};     // staged beside the per-token router (else by the row-move kernel)
   CMOE_MARK();
   {
     // fp32 buffer that later kernels add into: the K ranges of y on the streaming path, else s

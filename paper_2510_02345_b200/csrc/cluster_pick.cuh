@@ -27,8 +27,9 @@ __device__ __forceinline__ void two_best_pick(const TwoBest& b, int rank, int& g
 // Expert halves (Dims::split): virtual token `half` (0 or 1) of a token keeps those of the token's k experts that
 // lie in that half of the cluster's K experts, renumbered inside the half, and fills its remaining slots with
 // other experts of the half (lowest index first) at gate zero.  sel / gate: in the token's k kept experts (local
-// index 0 .. K-1, gates summing to one), out this virtual token's k slots (local index 0 .. K/2-1).
-__device__ __forceinline__ void split_half(int K, int k, int half, int* sel, float* gate) {
+// index 0 .. K-1, gates summing to one), out this virtual token's k slots (local index 0 .. K/2-1).  Returns the
+// number of kept experts in the half (0: the virtual token contributes nothing).
+__device__ __forceinline__ int split_half(int K, int k, int half, int* sel, float* gate) {
   const int Kh = K >> 1;
   int si[kMaxKsel];
   float gv[kMaxKsel];
@@ -36,9 +37,11 @@ __device__ __forceinline__ void split_half(int K, int k, int half, int* sel, flo
   int n = 0;
   for (int s = 0; s < k; ++s)
     if (sel[s] / Kh == half) { si[n] = sel[s] - half * Kh; gv[n] = gate[s]; used |= 1u << si[n]; ++n; }
+  const int kept = n;
   for (int i = 0; n < k && i < Kh; ++i)
     if (!((used >> i) & 1u)) { si[n] = i; gv[n] = 0.f; ++n; }
   for (int s = 0; s < k; ++s) { sel[s] = si[s]; gate[s] = gv[s]; }
+  return kept;          // how many of the token's experts lie in this half
 }
 
 }  // namespace cmoe

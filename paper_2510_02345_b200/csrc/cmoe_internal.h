@@ -82,6 +82,9 @@ struct Scratch {
   __half* x_perm;     // [T_pad][d]
   __half* x_rep;      // [T_max][d]  g1 > 1: every token's row g1 times (one virtual token per kept cluster)
   __half* y_rep;      // [T_max][d]  g1 > 1: the virtual tokens' outputs, summed per token at the end
+  int* r_cluster;     // [T_user]     expert halves: the token's own routes, before they are split
+  int* r_slot;        // [T_user][k]
+  float* r_gates;     // [T_user][k]
   float* t;           // [T_pad][k][r]   x U1_e
   __half* abar;       // [T_pad][d_ff]   sum_j p_j GELU(h_j)
   float* s;           // [T_pad][k][r]   GELU(h_j) U2_e, accumulated with atomics
@@ -153,8 +156,8 @@ bool router_tc_supported(const Dims& D);
 cudaError_t router_tc_init(cmoe_layer* L);
 // kc (or null): the kernel also writes every token's permutation key and the key counts of its 128-token tiles
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
-                             int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr, bool plain = false);
-// plain: the routes as the caller sees them even when the layer works on expert halves (Dims::split)
+                             int* slot_local, cudaStream_t st, const KeyCount* kc = nullptr);
+// the routers work on the real clusters, also when the layer behind them works on expert halves (Dims::split)
 inline Dims plain_dims(const Dims& D) { Dims R = D; R.G = real_G(D); R.K = real_K(D); R.split = 0; return R; }
 int router_tc_tile_tokens();
 // permute.cu : histogram, scan, scatter (+ row gather), padding rows
@@ -188,7 +191,10 @@ bool tc2_gathers_rows(const cmoe_layer* L);
 
 // multi_cluster.cu (virtual tokens): x_rep[n t + c] = x[t];  y[t] = sum_c y_rep[n t + c]
 cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, int T, int n, cudaStream_t st);
-cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, cudaStream_t st);
+// cluster_id (or null): virtual tokens whose entry is negative have no row
+cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, const int* cluster_id, cudaStream_t st);
+// expert halves: the token's own routes in Scratch::r_* -> the virtual tokens' routes (cluster_id, slot, gates)
+cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st);
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);

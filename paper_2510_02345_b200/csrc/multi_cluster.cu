@@ -4,6 +4,7 @@
 // carry the clusters' weights, so the sum is the mixture.  Expert halves (Dims::split) use the same two kernels: a
 // token's two virtual tokens carry the experts of one half of its cluster each.
 #include "cmoe_internal.h"
+#include "cluster_pick.cuh"
 
 namespace cmoe {
 
@@ -20,17 +21,39 @@ repeat_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ x_rep, long 
 }
 
 __global__ void __launch_bounds__(256)
-sum_rows_kernel(const __half2* __restrict__ y_rep, __half2* __restrict__ y, long long pairs_per_row, long long T, int g1) {
+sum_rows_kernel(const __half2* __restrict__ y_rep, __half2* __restrict__ y, long long pairs_per_row, long long T, int g1,
+                const int* __restrict__ cluster_id) {
   const long long n = T * pairs_per_row;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
     const long long t = i / pairs_per_row, v = i - t * pairs_per_row;
     float2 acc = make_float2(0.f, 0.f);
     for (int c = 0; c < g1; ++c) {
+      if (cluster_id && cluster_id[t * g1 + c] < 0) continue;        // a virtual token that was dropped: no row
       const float2 f = __half22float2(y_rep[(t * g1 + c) * pairs_per_row + v]);
       acc.x += f.x;
       acc.y += f.y;
     }
     y[i] = __floats2half2_rn(acc.x, acc.y);
+  }
+}
+
+// Expert halves: the token's own routes (real cluster g, k experts among its K, gates) -> the routes of its two virtual
+// tokens.  A half without any of the token's experts gets cluster id -1: the permutation gives it no row.
+__global__ void __launch_bounds__(256)
+split_routes_kernel(int T, int K, int k, const int* __restrict__ r_cluster, const int* __restrict__ r_slot,
+                    const float* __restrict__ r_gates, int* __restrict__ cluster_id, int* __restrict__ slot,
+                    float* __restrict__ gates) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const int g = r_cluster[t];
+  for (int half = 0; half < 2; ++half) {
+    int sel[kMaxKsel];
+    float gv[kMaxKsel];
+    for (int s = 0; s < k; ++s) { sel[s] = r_slot[(size_t)t * k + s]; gv[s] = r_gates[(size_t)t * k + s]; }
+    const int kept = split_half(K, k, half, sel, gv);
+    const size_t vt = (size_t)2 * t + half;
+    cluster_id[vt] = kept > 0 ? 2 * g + half : -1;
+    for (int s = 0; s < k; ++s) { slot[vt * k + s] = sel[s]; gates[vt * k + s] = gv[s]; }
   }
 }
 
@@ -48,10 +71,16 @@ cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, in
   return cudaGetLastError();
 }
 
-cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, cudaStream_t st) {
+cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, const int* cluster_id, cudaStream_t st) {
   const long long pairs = D.d / 2;
   sum_rows_kernel<<<grid_for((long long)T * pairs, D.sm_count), 256, 0, st>>>(
-      reinterpret_cast<const __half2*>(y_rep), reinterpret_cast<__half2*>(y), pairs, T, n);
+      reinterpret_cast<const __half2*>(y_rep), reinterpret_cast<__half2*>(y), pairs, T, n, cluster_id);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st) {
+  split_routes_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, real_K(D), D.k, S.r_cluster, S.r_slot, S.r_gates, S.cluster_id,
+                                                       S.slot, S.gates);
   return cudaGetLastError();
 }
 

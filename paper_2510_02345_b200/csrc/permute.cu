@@ -38,9 +38,10 @@ hist_kernel(int T, int k, int nsub, int nkey, int sub_is_combo,
     int cs[kMaxKsel];
     float cg[kMaxKsel];
     int sub = canonical_slots(slot + (size_t)t * k, gates + (size_t)t * k, k, sub_is_combo, cs, cg);
-    int key = cluster_id[t] * nsub + sub;
+    const int g = cluster_id[t];
+    const int key = g >= 0 ? g * nsub + sub : -1;       // (a virtual token without a cluster gets no row)
     keys[t] = key;
-    atomicAdd(&sh_cnt[key], 1);
+    if (key >= 0) atomicAdd(&sh_cnt[key], 1);
   }
   __syncthreads();
   for (int i = threadIdx.x; i < nkey; i += blockDim.x)
@@ -237,8 +238,9 @@ scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int t = blockIdx.x * tile + threadIdx.x;              // a block takes the tokens one counting block took,
-  const bool live = (int)threadIdx.x < tile && t < T;         // a thread each (the block may have more threads: they help with the sums above)
-  const int key = live ? keys[t] : -1 - lane;     // dead lanes get unique keys: groups of one
+  const int my_key = ((int)threadIdx.x < tile && t < T) ? keys[t] : -1;       // a thread each (the block may have more threads: they help with the sums above)
+  const bool live = my_key >= 0;                  // (a virtual token without a cluster has key -1 and gets no row)
+  const int key = live ? my_key : -1 - lane;      // dead lanes get unique keys: groups of one
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
   const bool leader = rank_in_warp == 0;
@@ -332,8 +334,8 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
   if (t < T) {
     const int sub = canonical_slots(slot + (size_t)t * k, gates + (size_t)t * k, k, sub_is_combo, cs, cg);
     g = cluster_id[t];
-    key = g * nsub + sub;
-    atomicAdd(&cnt[key], 1);
+    key = g >= 0 ? g * nsub + sub : -1;                  // (a virtual token without a cluster gets no row)
+    if (key >= 0) atomicAdd(&cnt[key], 1);
   }
   keys[t] = key;
   __syncthreads();
@@ -357,7 +359,7 @@ permute_small_kernel(int T, int G, int K, int k, int nsub, int nkey, int sub_is_
     *n_rows = off;
   }
   __syncthreads();
-  if (t < T) {
+  if (t < T && key >= 0) {
     int rank = 0;
     for (int u = 0; u < t; ++u) rank += keys[u] == key ? 1 : 0;
     const int row = cnt[key] + rank;

@@ -43,7 +43,7 @@ __device__ __forceinline__ void fma8(float& acc, const uint4& xv, const float4& 
 __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, int g, int t,
                                                  const int* __restrict__ label, int* __restrict__ expert_ids,
                                                  float* __restrict__ gates, int* __restrict__ slot_local,
-                                                 float cluster_weight = 1.f, int half = -1) {
+                                                 float cluster_weight = 1.f) {
   unsigned taken = 0;
   float selv[kMaxKsel];
   int seli[kMaxKsel];
@@ -64,16 +64,6 @@ __device__ __forceinline__ void select_and_store(const float* lg, int K, int k, 
   float ev[kMaxKsel];
   float sum = 0.f;
   for (int s = 0; s < k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
-  if (half >= 0) {
-    // expert halves: this virtual token's share of the token's experts (internal routes only: no labels)
-    for (int s = 0; s < k; ++s) ev[s] = ev[s] / sum;
-    split_half(K, k, half, seli, ev);
-    for (int s = 0; s < k; ++s) {
-      if (gates) gates[(size_t)t * k + s] = ev[s];
-      if (slot_local) slot_local[(size_t)t * k + s] = seli[s];
-    }
-    return;
-  }
   for (int s = 0; s < k; ++s) {
     if (gates) gates[(size_t)t * k + s] = cluster_weight == 1.f ? ev[s] / sum : cluster_weight * (ev[s] / sum);
     if (expert_ids) expert_ids[(size_t)t * k + s] = label[g * K + seli[s]];
@@ -92,8 +82,6 @@ struct RouterArgs {
   int* slot_local;
   FactorStage fs;  // per-token kernel only: factor staging that rides in the blocks past the router's own (all words zero: none)
   int n_route_blocks, n_riders;
-  int split;       // 2: expert halves; token index t is virtual token (half) t % 2 of caller token t / 2, and the
-                   // cluster id written is 2 g + half
   int g1;          // clusters per token: token index t is virtual token t % g1 of caller token t / g1 (x holds its row g1 times)
   int dc;          // columns of the cluster prototypes staged in shared memory at a time
   int crows;       // prototype rows staged at a time: min(G, 8)
@@ -194,7 +182,7 @@ router_tile_kernel(const RouterArgs a) {
       rank += (cu < c || (cu == c && u < me)) ? 1 : 0;
     }
     s_order[rank] = me;
-    if (tok0 + me < a.T) a.cluster_id[tok0 + me] = a.split > 1 ? 2 * c + ((tok0 + me) & 1) : c;
+    if (tok0 + me < a.T) a.cluster_id[tok0 + me] = c;
   }
   __syncthreads();
 
@@ -261,8 +249,7 @@ router_tile_kernel(const RouterArgs a) {
   // ---- top-k and gates: one thread per token
   if (threadIdx.x < kTileTokens && tok0 + threadIdx.x < a.T)
     select_and_store(lg + (size_t)threadIdx.x * K, K, a.k, s_cid[threadIdx.x], tok0 + threadIdx.x, a.label,
-                     a.expert_ids, a.gates, a.slot_local, a.g1 >= 2 ? s_weight[threadIdx.x] : 1.f,
-                     a.split > 1 ? (int)((tok0 + threadIdx.x) & 1) : -1);
+                     a.expert_ids, a.gates, a.slot_local, a.g1 >= 2 ? s_weight[threadIdx.x] : 1.f);
 }
 
 // One block per token; warp w computes the rows w, w + nwarp, ... of the router matrix, each over all of d
@@ -323,12 +310,12 @@ router_token_kernel(const RouterArgs a) {
         }
         s_g = gs;
         s_w = w;
-        a.cluster_id[t] = a.split > 1 ? 2 * gs + (t & 1) : gs;
+        a.cluster_id[t] = gs;
       }
       __syncthreads();
     }
   }
-  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, s_w, a.split > 1 ? (t & 1) : -1);
+  if (threadIdx.x == 0) select_and_store(lg, a.K, a.k, s_g, t, a.label, a.expert_ids, a.gates, a.slot_local, s_w);
 }
 
 }  // namespace
@@ -342,7 +329,8 @@ cudaError_t launch_router(const Dims& D, const Weights& W, const __half* x, int 
   // permutation's row-move kernel)
   if (fs && T < 1024) a.fs = *fs;
   a.n_riders = stage_blocks(a.fs, 256);          // one 32-bit word of packed codes per thread
-  a.x = x; a.T = T; a.d = D.d; a.G = real_G(D); a.K = real_K(D); a.k = D.k; a.g1 = D.g1; a.split = D.split;
+  a.x = x; a.T = T; a.d = D.d; a.G = real_G(D); a.K = real_K(D); a.k = D.k; a.g1 = D.g1;
+  // (a layer on expert halves routes its tokens over the real clusters; the routes are split afterwards)
   a.Ct = W.Ct; a.Rt = W.Rt; a.bc = W.bc; a.be = W.be; a.label = W.label;
   a.cluster_id = cluster_id; a.expert_ids = expert_ids; a.gates = gates; a.slot_local = slot_local;
   if (T < 1024) {

@@ -42,7 +42,6 @@ struct RtcParams {
   KeyCount kc;     // key counting for the permutation (keys == nullptr: routing only)
   int stages;      // stages of the operand ring
   int g1;          // clusters per token (token index = virtual token)
-  int split;       // 2: expert halves (token index = virtual token; G, K are the real counts)
 };
 
 // fp32 router rows -> the two fp16 pieces, rows [hi_0 .. hi_{rp-1}, lo_0 .. lo_{rp-1}] x d (padding rows zero)
@@ -167,7 +166,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
           for (int g = 0; g < G; ++g) two_best_add(b, g, fmaf(mine[rp + g], 1.f / 2048.f, mine[g]) + p.bc[g]);
           two_best_pick(b, tok & 1, gs, cluster_weight);
         }
-        p.cluster_id[tok] = p.split > 1 ? 2 * gs + (tok & 1) : gs;
+        p.cluster_id[tok] = gs;
         // expert logits of the chosen cluster, in place over the cluster columns (no longer needed)
         const int e0 = G + gs * K;
         for (int i = 0; i < K; ++i) mine[i] = fmaf(mine[rp + e0 + i], 1.f / 2048.f, mine[e0 + i]) + p.be[gs * K + i];
@@ -192,11 +191,6 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         float sum = 0.f;
         for (int s = 0; s < p.k; ++s) { ev[s] = expf(selv[s] - lmax); sum += ev[s]; }
         for (int s = 0; s < p.k; ++s) ev[s] = cluster_weight == 1.f ? ev[s] / sum : cluster_weight * (ev[s] / sum);
-        int key_cluster = gs;
-        if (p.split > 1) {        // expert halves: this virtual token's share of the token's experts
-          split_half(K, p.k, tok & 1, seli, ev);
-          key_cluster = 2 * gs + (tok & 1);
-        }
         for (int s = 0; s < p.k; ++s) {
           if (p.gates) p.gates[(size_t)tok * p.k + s] = ev[s];
           if (p.expert_ids) p.expert_ids[(size_t)tok * p.k + s] = p.label[gs * K + seli[s]];
@@ -205,7 +199,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         if (p.kc.keys) {
           int cs[kMaxKsel];
           float cg[kMaxKsel];
-          key = key_cluster * p.kc.nsub + canonical_slots(seli, ev, p.k, p.kc.sub_is_combo, cs, cg);
+          key = gs * p.kc.nsub + canonical_slots(seli, ev, p.k, p.kc.sub_is_combo, cs, cg);
           p.kc.keys[tok] = key;
         }
       }
@@ -308,13 +302,12 @@ cudaError_t router_tc_init(cmoe_layer* L) {
 int router_tc_tile_tokens() { return RBM; }
 
 cudaError_t launch_router_tc(const cmoe_layer* L, const __half* x, int T, int* cluster_id, int* expert_ids, float* gates,
-                             int* slot_local, cudaStream_t st, const KeyCount* kc, bool plain) {
+                             int* slot_local, cudaStream_t st, const KeyCount* kc) {
   const Dims& D = L->dims;
   CUtensorMap mx;
   if (!make_map3(&mx, x, (uint64_t)T, D.d, RBM)) return cudaErrorInvalidValue;   // x is the caller's buffer: a map per call
   RtcParams p{};
   p.T = T; p.d = D.d; p.G = real_G(D); p.K = real_K(D); p.k = D.k; p.E = D.E; p.rp = router_tc_rp(D); p.g1 = D.g1;
-  p.split = plain ? 0 : D.split;
   p.bc = L->w.bc; p.be = L->w.be; p.label = L->w.label;
   p.cluster_id = cluster_id; p.expert_ids = expert_ids; p.gates = gates; p.slot_local = slot_local; p.status = L->sc.status;
   if (kc) p.kc = *kc;

@@ -157,7 +157,7 @@ extern "C" int cmoe_expert_stats(cmoe_layer* L, const void* x, int32_t T, int32_
     T *= D.g1;
   }
   // (the token's own routes, also when the layer works on expert halves)
-  if (L->router_tc && T >= 1024) STAT_CUDA(launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st, nullptr, true));
+  if (L->router_tc && T >= 1024) STAT_CUDA(launch_router_tc(L, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   else STAT_CUDA(launch_router(plain_dims(D), L->w, xh, T, S.cluster_id, nullptr, S.gates, S.slot, st));
   STAT_CUDA(launch_chained(loads_kernel, dim3((T + kStatThreads - 1) / kStatThreads), dim3(kStatThreads),
                            sizeof(int) * (size_t)D.E, st, 1, (int)T, real_K(D), D.k, D.E, (const int*)S.cluster_id,
