@@ -63,7 +63,8 @@ typedef struct cmoe_layer cmoe_layer; /* opaque, host object owned by the librar
  * 1 <= k <= min(K, 8), d % 32 == 0, d_ff % 32 == 0, r in {0, 4, 8, 16, 32}, quant_group == 32,
  * T_max >= 1.  With r == 0 the factor pointers are ignored (plain shared-base experts).
  * Speed, not results, depends on the shape: the fastest large-batch kernels need d and d_ff multiples of 128, k <= 2
- * and K*r <= 64 (or, with K even and k <= K/2, (K/2)*r <= 64: the clusters are then handled as two halves).
+ * and K*r <= 64 (or, for n = 2 or 4 with K a multiple of n, k <= K/n and n*G <= 64, (K/n)*r <= 64: the clusters are then
+ * handled as n parts of K/n experts sharing the cluster's base).
  * All weight pointers must be 16-byte aligned.
  */
 typedef struct {

@@ -55,13 +55,14 @@ int validate_dims(const cmoe_desc* desc, int g1, bool allow_split, Dims* D) {
   // with g1 clusters per token everything below the entry points works on g1 virtual tokens per token
   D->r = desc->r; D->k = desc->k; D->g1 = g1; D->T_user = desc->T_max; D->T_max = desc->T_max * g1;
   D->split = 0; D->rep = g1;
-  // K r beyond the pair path's expanded rank index: two expert halves per cluster where that makes the shape fit
-  if (allow_split && g1 == 1 && D->T_max > 128 && K % 2 == 0 && desc->k <= K / 2 && 2 * desc->G <= kMaxG &&
-      (long long)desc->T_max * 2 <= (1 << 22)) {
-    Dims V = *D;
-    V.K = K / 2; V.G = 2 * desc->G; V.T_max = 2 * desc->T_max;
-    if (!tc2_supported(*D) && tc2_supported(V)) {
-      D->split = 2; D->rep = 2; D->K = V.K; D->G = V.G; D->T_max = V.T_max;
+  // K r beyond the pair path's expanded rank index: every cluster as two halves, else four quarters, of its experts
+  // where that makes the shape fit
+  if (allow_split && g1 == 1 && D->T_max > 128 && !tc2_supported(*D)) {
+    for (int parts = 2; parts <= 4 && D->split == 0; parts *= 2) {
+      if (K % parts || desc->k > K / parts || parts * desc->G > kMaxG || (long long)desc->T_max * parts > (1 << 22)) continue;
+      Dims V = *D;
+      V.K = K / parts; V.G = parts * desc->G; V.T_max = parts * desc->T_max;
+      if (tc2_supported(V)) { D->split = parts; D->rep = parts; D->K = V.K; D->G = V.G; D->T_max = V.T_max; }
     }
   }
   const long long combos = binom_ll(D->K, desc->k);
@@ -381,14 +382,14 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, n, st));
   rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream, L->dims.split > 1 ? x : nullptr);
   if (rc) return rc;
-  // (expert halves: a half without any of the token's experts has no row)
+  // (expert parts: a part without any of the token's experts has no row)
   CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, n,
                                L->dims.split > 1 ? L->sc.cluster_id : nullptr, st));
   return CMOE_OK;
 }
 
 // The layer on T rows of x as the kernels see them (virtual tokens when Dims::rep > 1).  x_tokens: not null for a
-// layer on expert halves: the caller's T / 2 tokens, which are routed once over the real clusters; their routes are
+// layer on expert halves or quarters: the caller's T / split tokens, which are routed once over the real clusters; their routes are
 // then split into those of the virtual tokens.
 static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_stream, const void* x_tokens) {
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

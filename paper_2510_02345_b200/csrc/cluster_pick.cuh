@@ -24,24 +24,24 @@ __device__ __forceinline__ void two_best_pick(const TwoBest& b, int rank, int& g
   else           { g = b.c2; w = e2 / (1.f + e2); }
 }
 
-// Expert halves (Dims::split): virtual token `half` (0 or 1) of a token keeps those of the token's k experts that
-// lie in that half of the cluster's K experts, renumbered inside the half, and fills its remaining slots with
-// other experts of the half (lowest index first) at gate zero.  sel / gate: in the token's k kept experts (local
-// index 0 .. K-1, gates summing to one), out this virtual token's k slots (local index 0 .. K/2-1).  Returns the
-// number of kept experts in the half (0: the virtual token contributes nothing).
-__device__ __forceinline__ int split_half(int K, int k, int half, int* sel, float* gate) {
-  const int Kh = K >> 1;
+// Expert parts (Dims::split = 2 or 4): virtual token `part` (0 .. parts-1) of a token keeps those of the token's k
+// experts that lie in that part of the cluster's K experts (part c = experts c K / parts ..), renumbered inside the
+// part, and fills its remaining slots with other experts of the part (lowest index first) at gate zero.  sel / gate:
+// in the token's k kept experts (local index 0 .. K-1, gates summing to one), out this virtual token's k slots (local
+// index 0 .. K/parts-1).  Returns the number of kept experts in the part (0: the virtual token contributes nothing).
+__device__ __forceinline__ int split_part(int K, int parts, int k, int part, int* sel, float* gate) {
+  const int Kp = K / parts;
   int si[kMaxKsel];
   float gv[kMaxKsel];
   unsigned used = 0;
   int n = 0;
   for (int s = 0; s < k; ++s)
-    if (sel[s] / Kh == half) { si[n] = sel[s] - half * Kh; gv[n] = gate[s]; used |= 1u << si[n]; ++n; }
+    if (sel[s] / Kp == part) { si[n] = sel[s] - part * Kp; gv[n] = gate[s]; used |= 1u << si[n]; ++n; }
   const int kept = n;
-  for (int i = 0; n < k && i < Kh; ++i)
+  for (int i = 0; n < k && i < Kp; ++i)
     if (!((used >> i) & 1u)) { si[n] = i; gv[n] = 0.f; ++n; }
   for (int s = 0; s < k; ++s) { sel[s] = si[s]; gate[s] = gv[s]; }
-  return kept;          // how many of the token's experts lie in this half
+  return kept;          // how many of the token's experts lie in this part
 }
 
 }  // namespace cmoe

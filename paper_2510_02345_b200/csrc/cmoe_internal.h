@@ -22,12 +22,13 @@ constexpr int kMinCountTile = 128; // token tile of the router kernel that count
 
 enum Path { kPathGeneric = 0, kPathTensor = 1, kPathStream = 2 };
 
-// Expert halves (split == 2): a cluster whose K r exceeds the 64 columns of the pair path's expanded rank index is
-// handled as two virtual clusters of K / 2 experts (virtual cluster 2 g + c = experts c K / 2 .. of cluster g: the
-// expert numbering e = g K + i does not change) that share the base of cluster g.  A token becomes two virtual
-// tokens, one per half, each with those of its kept experts that lie in the half and, in its remaining slots,
-// other experts of the half at gate zero; their outputs are summed.  G and K below are then the virtual counts
-// (2 G, K / 2): everything behind the router sees an ordinary layer; the router and the bases use real_G / real_K.
+// Expert parts (split == 2 or 4): a cluster whose K r exceeds the 64 columns of the pair path's expanded rank index is
+// handled as `split` virtual clusters of K / split experts (virtual cluster split g + c = experts c K / split .. of
+// cluster g: the expert numbering e = g K + i does not change) that share the base of cluster g.  A token becomes
+// `split` virtual tokens, one per part, each with those of its kept experts that lie in the part and, in its remaining
+// slots, other experts of the part at gate zero; a part without any of the token's experts has no row; the outputs are
+// summed.  G and K below are then the virtual counts (split G, K / split): everything behind the router sees an
+// ordinary layer; the router and the bases use real_G / real_K.
 struct Dims {
   int d, d_ff, E, G, K, r, k;
   int nsub;        // permutation sub-keys per cluster (expert combinations, or lowest expert)
@@ -35,7 +36,7 @@ struct Dims {
   int T_max;       // most tokens of a call as the kernels see them: g1 virtual tokens per caller token
   int T_user;      // most tokens of a call as the caller counts them (T_max = g1 * T_user)
   int g1;          // clusters per token (Sec. 3.3); 0 and 1 both mean one
-  int split;       // 2: the clusters are handled as two halves of K / 2 experts each (below); else 0
+  int split;       // 2 or 4: the clusters are handled as that many parts of K / split experts each (above); else 0
   int rep;         // rows of the kernels' x per caller token: max(g1, split, 1)
   int T_pad_max;   // rows of the permuted buffers
   int row_align;   // a cluster's rows start at a multiple of this

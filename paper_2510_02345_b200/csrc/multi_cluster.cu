@@ -1,8 +1,8 @@
 // Virtual tokens.  Two clusters per token (Sec. 3.3, "Top-g1 groups"): the layer runs on g1 virtual tokens per token.  Before the
 // router every row of x is written g1 times (virtual token g1 t + c is token t on its way to its c-th most
 // probable cluster); after the un-permuting store the g1 output rows of a token are summed.  The gates already
-// carry the clusters' weights, so the sum is the mixture.  Expert halves (Dims::split) use the same two kernels: a
-// token's two virtual tokens carry the experts of one half of its cluster each.
+// carry the clusters' weights, so the sum is the mixture.  Expert parts (Dims::split = 2 or 4) use the same two kernels:
+// a token's virtual tokens carry the experts of one half, or one quarter, of its cluster each.
 #include "cmoe_internal.h"
 #include "cluster_pick.cuh"
 
@@ -37,22 +37,22 @@ sum_rows_kernel(const __half2* __restrict__ y_rep, __half2* __restrict__ y, long
   }
 }
 
-// Expert halves: the token's own routes (real cluster g, k experts among its K, gates) -> the routes of its two virtual
-// tokens.  A half without any of the token's experts gets cluster id -1: the permutation gives it no row.
+// Expert parts: the token's own routes (real cluster g, k experts among its K, gates) -> the routes of its `parts`
+// virtual tokens.  A part without any of the token's experts gets cluster id -1: the permutation gives it no row.
 __global__ void __launch_bounds__(256)
-split_routes_kernel(int T, int K, int k, const int* __restrict__ r_cluster, const int* __restrict__ r_slot,
+split_routes_kernel(int T, int K, int parts, int k, const int* __restrict__ r_cluster, const int* __restrict__ r_slot,
                     const float* __restrict__ r_gates, int* __restrict__ cluster_id, int* __restrict__ slot,
                     float* __restrict__ gates) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= T) return;
   const int g = r_cluster[t];
-  for (int half = 0; half < 2; ++half) {
+  for (int part = 0; part < parts; ++part) {
     int sel[kMaxKsel];
     float gv[kMaxKsel];
     for (int s = 0; s < k; ++s) { sel[s] = r_slot[(size_t)t * k + s]; gv[s] = r_gates[(size_t)t * k + s]; }
-    const int kept = split_half(K, k, half, sel, gv);
-    const size_t vt = (size_t)2 * t + half;
-    cluster_id[vt] = kept > 0 ? 2 * g + half : -1;
+    const int kept = split_part(K, parts, k, part, sel, gv);
+    const size_t vt = (size_t)parts * t + part;
+    cluster_id[vt] = kept > 0 ? parts * g + part : -1;
     for (int s = 0; s < k; ++s) { slot[vt * k + s] = sel[s]; gates[vt * k + s] = gv[s]; }
   }
 }
@@ -79,7 +79,7 @@ cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T
 }
 
 cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st) {
-  split_routes_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, real_K(D), D.k, S.r_cluster, S.r_slot, S.r_gates, S.cluster_id,
+  split_routes_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, real_K(D), D.split, D.k, S.r_cluster, S.r_slot, S.r_gates, S.cluster_id,
                                                        S.slot, S.gates);
   return cudaGetLastError();
 }

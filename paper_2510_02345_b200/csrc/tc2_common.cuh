@@ -62,7 +62,7 @@ struct Up2Params {
   int* status;
   int KC, NT, N, K, k, r, log2r;
   int unit;            // N tiles per work unit (divides NT)
-  int bshift;          // the base of cluster g is that of g >> bshift (expert halves share their cluster's base)
+  int bshift;          // the base of cluster g is that of g >> bshift (expert halves or quarters share their cluster's base)
   __half* As_direct;   // [rows][KE] or null.  Not null: a unit is a whole row tile (unit == NT), so S is complete at its
                        // end and the gated rows p_j s_j go straight into the down kernel's operand (zeroed by the caller)
 };

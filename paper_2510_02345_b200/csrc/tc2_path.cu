@@ -677,7 +677,7 @@ struct Down2Params {
   __half* y;           // [T][N], original token order
   int* status;
   int KC, NT, N;
-  int bshift;          // the base of cluster g is that of g >> bshift (expert halves share their cluster's base)
+  int bshift;          // the base of cluster g is that of g >> bshift (expert halves or quarters share their cluster's base)
   // Not null: the up kernel left the sums s = a_j U2_e in fp32 (its work units were parts of a row tile) and this
   // kernel turns them into its own operand As[row][block of e_j] = fp16(p_j s_j), row tile by row tile, in the
   // epilogue warps while they wait for the tile's main loop.
@@ -1145,7 +1145,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __ha
   up.n_rows = S.n_rows; up.tile_cluster = S.tile_cluster; up.tile_mask = S.tile_mask; up.row_slot = S.row_slot;
   up.row_gate = S.row_gate; up.row_token = S.row_token; up.s_out = S.s; up.abar = S.abar; up.status = S.status;
   up.KC = D.d / (BK * KA); up.NT = D.d_ff / BN_UP; up.N = D.d_ff; up.K = D.K; up.k = D.k; up.r = D.r; up.log2r = ts.log2r;
-  up.bshift = D.split > 1 ? 1 : 0;
+  up.bshift = D.split > 1 ? ilog2(D.split) : 0;
   const UpPlan plan = plan_up(ts, D, T);
   {
     up.NT = plan.NT;
@@ -1165,7 +1165,7 @@ cudaError_t launch_tc2_ffn(const cmoe_layer* L, const __half* x_src, int T, __ha
   Down2Params dn{};
   dn.n_rows = S.n_rows; dn.tile_cluster = S.tile_cluster; dn.tile_mask = S.tile_mask_dn; dn.row_token = S.row_token;
   dn.y = y; dn.status = S.status; dn.KC = D.d_ff / (BK * KA); dn.NT = D.d / ts.bn_down; dn.N = D.d;
-  dn.bshift = D.split > 1 ? 1 : 0;
+  dn.bshift = D.split > 1 ? ilog2(D.split) : 0;
   if (D.r > 0 && !plan.direct) {
     dn.s = S.s; dn.row_slot = S.row_slot; dn.row_gate = S.row_gate; dn.As = S.As; dn.K = D.K; dn.k = D.k; dn.r = D.r;
   }

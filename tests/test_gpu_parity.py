@@ -605,6 +605,15 @@ def test_headline_shape_variants(kw):
     assert got["module"].info.path == 1
 
 
+def test_decode_shaped_layer_on_a_large_batch():
+    """The decode-shaped layer (K = 8, r = 32: K r = 256) on a prefill-sized batch: quarters of two experts on the pair
+    path; sampled rows."""
+    s = inputs.small_shape(T=2048, d=4096, d_ff=14336, E=64, G=8, r=32, k=2)
+    L = inputs.make_layer(s, 9)
+    got = full_check(L, L["x"], sample=256)
+    assert got["module"].info.path == 1
+
+
 def test_many_experts_beyond_the_pair_path():
     """E = 128 in G = 16 clusters with r = 16 (K r = 128 > 64, the expanded rank index of the pair path holds 64): the
     clusters are handled as two halves of four experts on the pair path; sampled rows."""
@@ -620,10 +629,15 @@ def test_many_experts_beyond_the_pair_path():
     (1111, dict(d=256, d_ff=256, E=32, G=2, r=8, k=1)),        # K = 16, r = 8, one kept expert: one half has none
     (129, dict(d=128, d_ff=256, E=24, G=3, r=16, k=2)),        # ragged, mostly padding rows
     (2048, dict(d=256, d_ff=512, E=32, G=4, r=16, k=3)),       # k = 3 of K = 8: generic fallback of the pair path? (k <= 2 only)
-], ids=["K8r16", "K4r32", "K16r8k1", "ragged", "k3"])
+    (1200, dict(d=128, d_ff=256, E=16, G=2, r=32, k=2)),       # K = 8, r = 32: quarters of two experts
+    (900, dict(d=256, d_ff=512, E=32, G=2, r=16, k=2)),        # K = 16, r = 16: quarters of four experts
+    (1300, dict(d=128, d_ff=512, E=24, G=3, r=32, k=1)),       # K = 8, r = 32, one kept expert: three quarters have none
+    (131, dict(d=128, d_ff=256, E=16, G=2, r=32, k=2)),        # quarters, ragged, mostly padding rows
+], ids=["K8r16", "K4r32", "K16r8k1", "ragged", "k3", "K8r32", "K16r16", "K8r32k1", "quarters_ragged"])
 def test_expert_halves(T, kw):
-    """K r > 64: every cluster as two virtual clusters of K / 2 experts sharing its base, two virtual tokens per token
-    (its kept experts of that half, the other slots at gate zero), outputs summed.  Every row against the oracle."""
+    """K r > 64: every cluster as two (else four) virtual clusters of K / 2 (K / 4) experts sharing its base, as many
+    virtual tokens per token (its kept experts of that part, the other slots at gate zero; no row for a part without
+    any), outputs summed.  Every row against the oracle."""
     s = inputs.small_shape(T=T, **kw)
     L = inputs.make_layer(s, 17)
     got = full_check(L, L["x"])
