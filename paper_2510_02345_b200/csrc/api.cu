@@ -515,7 +515,8 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   *out = cmoe_info{};
   out->path = L->path;
   out->launches_route = 1;
-  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0) +
+  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0,
+                                              L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L)) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.rep > 1 ? 2 : 0);

@@ -168,7 +168,7 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                            size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile);
 // kernels of the permutation: 2 for batches of at most 256 tokens, 4 below 1024 tokens, else 3 (the router counts the
 // keys) or 2 (and the scatter kernel sums the small count table itself; see launch_permute)
-int permute_launches(const Dims& D, int T, int counted_tile);
+int permute_launches(const Dims& D, int T, int counted_tile, bool gathered);
 // generic_path.cu : CUDA-core path for any supported shape
 // `marks` (or null): three events recorded before the residual-t, up and down stages
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,

@@ -11,7 +11,8 @@
 //   scatter  each token's row = key offset + earlier blocks' count + its rank inside the block;
 //            writes the row tables
 //   move     copies every token's activations to its row with 16-byte vectors (a block per row;
-//            padding rows get zeros) and clears the buffer the later stages accumulate into
+//            padding rows get zeros) and clears the buffer the later stages accumulate into; when the scatter blocks
+//            do the sums themselves they also move the rows of their own token tile and this kernel is not launched
 //
 // The result is deterministic: rows of one key keep the token order.
 #include "cmoe_internal.h"
@@ -137,6 +138,17 @@ struct ScanInline {
   int *seg_off, *seg_cnt, *n_rows, *tile_cluster;
 };
 
+// The row move done by the scatter blocks themselves (MoveInline.on; only with ScanInline): a block copies the rows
+// of its own token tile, which are contiguous in x, to their places in x_perm, zeroes its share of the clusters'
+// padding rows and of the accumulation buffer; blocks nblk.. stage the INT4 factors.  One launch less, and the rows'
+// places never travel through memory.
+struct MoveInline {
+  int on;
+  uint4* zero_ptr;
+  size_t zero_n;
+  FactorStage fs;
+};
+
 __global__ void __launch_bounds__(512)      // at least `tile` threads: the token tile of the kernel that counted the keys
 scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
                const __half* __restrict__ x, const int* __restrict__ cluster_id,
@@ -144,13 +156,15 @@ scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
                const int* __restrict__ keys, const int* __restrict__ block_base,
                const int* __restrict__ key_off,
                int* __restrict__ row_token, int* __restrict__ row_slot, float* __restrict__ row_gate,
-               __half* __restrict__ x_perm, const ScanInline si) {
+               __half* __restrict__ x_perm, const ScanInline si, const MoveInline mv) {
   pdl_wait();
+  if (mv.on && (int)blockIdx.x >= si.nblk) { stage_block(mv.fs, blockIdx.x - si.nblk); return; }
   extern __shared__ int sh_next[];   // next free row of each key for this block
+  __shared__ int sh_seg[kMaxG + 1];
+  __shared__ int sh_segcnt[kMaxG];
+  __shared__ int sh_row[512];        // fused move: the row of each token of this block's tile (-1: none)
   if (si.counts) {
     int* sh_tot = sh_next + nkey;    // [nkey] tokens of each key in the whole batch
-    __shared__ int sh_seg[kMaxG + 1];
-    __shared__ int sh_segcnt[kMaxG];
     // Column sums of the count table, read along its rows: lanes over the keys (four columns of 32 keys per pass),
     // warps over the counting blocks; a key's total and the part of the blocks before this one.
     for (int key = threadIdx.x; key < nkey; key += blockDim.x) { sh_tot[key] = 0; sh_next[key] = 0; }
@@ -267,6 +281,44 @@ scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
         row_gate[(size_t)row * k + j] = cg[j];
       }
   }
+  if (!mv.on) return;
+  // ---- the row move, by the block that placed the rows
+  if ((int)threadIdx.x < tile) sh_row[threadIdx.x] = row;
+  __syncthreads();
+  const int vec_per_row = d / 8, nthr = (int)blockDim.x;
+  {
+    // this tile's tokens are consecutive rows of x: vector i of the tile is vector i % vec_per_row of token i / vec_per_row
+    const int t0 = blockIdx.x * tile, nt = min(tile, T - t0);
+    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t0 * d);
+    const int nvec = nt * vec_per_row;
+    for (int i0 = threadIdx.x; i0 < nvec; i0 += 8 * nthr) {
+      uint4 val[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * nthr;
+        if (i < nvec) val[u] = src[i];
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = i0 + u * nthr;
+        if (i < nvec) {
+          const int tt = i / vec_per_row, r = sh_row[tt];
+          if (r >= 0) reinterpret_cast<uint4*>(x_perm + (size_t)r * d)[i - tt * vec_per_row] = val[u];
+        }
+      }
+    }
+  }
+  // padding rows of every cluster: block b takes every nblk-th of them
+  for (int g = 0; g < si.G; ++g) {
+    const int first = sh_seg[g] + sh_segcnt[g], last = sh_seg[g + 1];
+    for (int prow = first + (int)blockIdx.x; prow < last; prow += si.nblk) {
+      uint4* dstp = reinterpret_cast<uint4*>(x_perm + (size_t)prow * d);
+      for (int v = threadIdx.x; v < vec_per_row; v += nthr) dstp[v] = make_uint4(0, 0, 0, 0);
+    }
+  }
+  // the accumulation buffer of the later stages starts at zero
+  for (size_t i = (size_t)blockIdx.x * nthr + threadIdx.x; i < mv.zero_n; i += (size_t)si.nblk * nthr)
+    mv.zero_ptr[i] = make_uint4(0, 0, 0, 0);
 }
 
 // x_perm[row] = x[row_token[row]], zeros for padding rows; a block per row, 16 bytes per thread
@@ -398,10 +450,10 @@ bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk 
 
 }  // namespace
 
-int permute_launches(const Dims& D, int T, int counted_tile) {
+int permute_launches(const Dims& D, int T, int counted_tile, bool gathered) {
   if (T <= kSmallT) return 2;
   if (counted_tile <= 0) return 4;
-  return inline_scan_ok(D, (T + counted_tile - 1) / counted_tile, counted_tile) ? 2 : 3;
+  return inline_scan_ok(D, (T + counted_tile - 1) / counted_tile, counted_tile) ? (gathered ? 2 : 1) : 3;
 }
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
@@ -440,11 +492,17 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                                     S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
                                     S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
   }
-  launch_chained(scatter_kernel, dim3(nblk), dim3(inline_scan ? 512 : tile), sh * (inline_scan ? 2 : 1), st, 1,
+  // with the inline sums the scatter blocks also move their tile's rows (unless a later kernel gathers them)
+  MoveInline mv{};
+  const bool fused_move = inline_scan && x != nullptr && tile <= 512;
+  if (fused_move) { mv.on = 1; mv.zero_ptr = static_cast<uint4*>(zero_ptr); mv.zero_n = zero_bytes / 16; mv.fs = fs; }
+  launch_chained(scatter_kernel, dim3(nblk + (fused_move ? stage_blocks(fs, 512) : 0)), dim3(inline_scan ? 512 : tile),
+                 sh * (inline_scan ? 2 : 1), st, 1,
       T, tile, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
                                                S.cluster_id, S.slot, S.gates, S.keys, S.block_base,
                                                S.key_off, S.row_token, S.row_slot, S.row_gate,
-                                               S.x_perm, si);
+                                               S.x_perm, si, mv);
+  if (fused_move) return cudaGetLastError();
   const int move_max = (D.sm_count > 0 ? D.sm_count : 148) * 32;      // resident blocks of 128 threads
   const int move_grid = rows_bound < move_max ? rows_bound : move_max;
   launch_chained(move_rows_kernel, dim3(move_grid + stage_blocks(fs, 128)), dim3(128), 0, st, 1,
