@@ -103,6 +103,8 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
 /* cmoe_create with kernel-selection switches for A/B measurements and tests (NULL options = cmoe_create).
  * Results stay within the same tolerances whatever is chosen; only speed changes.
  *   force_path   -1 automatic (default); 0 keeps the generic CUDA-core path for every shape
+ *                 3 automatic, but clusters are never handled as halves or quarters: shapes with K*r > 64 then
+ *                 take the tensor-core path that evaluates the rank-r terms in its epilogue
  *   router_fp32   1 keeps batches of 1024 tokens and more on the fp32 CUDA-core router instead of the
  *                 tensor-core router (which splits the fp32 router matrices into two fp16 pieces; logit error
  *                 about 1e-6)

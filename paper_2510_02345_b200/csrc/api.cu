@@ -179,7 +179,7 @@ int cmoe_workspace_bytes(const cmoe_desc* desc, size_t* out_bytes) { return cmoe
 int cmoe_workspace_bytes_ex(const cmoe_desc* desc, const cmoe_options* opt, size_t* out_bytes) {
   if (!out_bytes) return CMOE_ERR_INVALID_ARG;
   Dims D{};
-  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || opt->force_path != kPathGeneric, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || (opt->force_path != kPathGeneric && opt->force_path != 3), &D);
   if (rc) return rc;
   Arena A;
   plan(D, A, nullptr, nullptr);
@@ -193,7 +193,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   if (!out_layer) return CMOE_ERR_INVALID_ARG;
   *out_layer = nullptr;
   Dims D{};
-  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || opt->force_path != kPathGeneric, &D);
+  int rc = validate_dims(desc, opt ? opt->clusters_per_token : 1, !opt || (opt->force_path != kPathGeneric && opt->force_path != 3), &D);
   if (rc) return rc;
   if (!desc->C || !desc->R || !desc->B1 || !desc->B2 || !desc->workspace) return CMOE_ERR_INVALID_ARG;
   if (D.r > 0 && (!desc->U1q || !desc->V1q || !desc->U2q || !desc->V2q || !desc->U1s ||
@@ -210,7 +210,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   cmoe_options o{};
   o.force_path = -1;
   if (opt) o = *opt;
-  if (o.force_path < -1 || o.force_path > 0 || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
+  if (o.force_path < -1 || (o.force_path > 0 && o.force_path != 3) || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
       o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks || o.row_gather < 0 || o.row_gather > 1 ||
       o.reserved[0] != 0) return CMOE_ERR_INVALID_ARG;
   {

@@ -234,8 +234,12 @@ def test_tensor_path_ragged(T):
 def test_tensor_path_variants(kw):
     s = inputs.small_shape(T=700, **kw)
     L = inputs.make_layer(s, 13)
-    got = full_check(L, L["x"])
+    # K r > 64: kept on the path with the rank-r terms in its epilogue (clusters not split into parts)
+    whole = s.E // s.G * s.r > 64
+    got = full_check(L, L["x"], options=dict(force_path=3) if whole else None)
     assert got["module"].info.path == 1
+    if whole:
+        assert got["module"].info.T_pad_max < 2 * 700
 
 
 def test_tensor_path_empty_cluster():
@@ -410,8 +414,11 @@ _RESID_CASES = [
     ("generic_r4_k2", dict(T=200, d=96, d_ff=224, E=8, G=2, r=4, k=2), None),
     ("generic_r32_k3", dict(T=200, d=96, d_ff=224, E=16, G=2, r=32, k=3), None),
     # first tensor-core path: K * r > 64, rank-r terms in the epilogue
-    ("tc1_K8_r32", dict(T=700, d=384, d_ff=256, E=16, G=2, r=32, k=2), None),
-    ("tc1_K8_r16_k1", dict(T=700, d=256, d_ff=384, E=16, G=2, r=16, k=1), None),
+    ("tc1_K8_r32", dict(T=700, d=384, d_ff=256, E=16, G=2, r=32, k=2), dict(force_path=3)),
+    ("tc1_K8_r16_k1", dict(T=700, d=256, d_ff=384, E=16, G=2, r=16, k=1), dict(force_path=3)),
+    # the same shapes as halves / quarters of the clusters on the pair path
+    ("parts_K8_r32", dict(T=700, d=384, d_ff=256, E=16, G=2, r=32, k=2), None),
+    ("parts_K8_r16_k1", dict(T=700, d=256, d_ff=384, E=16, G=2, r=16, k=1), None),
     # pair path, 256-column up tiles: several units per row tile, whole-row units (direct rows), both k
     ("pair_wide_units", dict(T=1500, d=256, d_ff=1024, E=8, G=2, r=16, k=2), None),
     ("pair_wide_direct_r4", dict(T=1500, d=128, d_ff=256, E=8, G=2, r=4, k=2), None),
@@ -448,9 +455,10 @@ def test_residual_dominated_layers(name, kw, options, mode):
 @pytest.mark.parametrize("kw", [
     dict(d=96, d_ff=224, E=8, G=2, r=4, k=2),          # generic path
     dict(d=384, d_ff=256, E=16, G=2, r=32, k=2),       # first tensor-core path
+    dict(d=256, d_ff=256, E=16, G=2, r=16, k=2),       # pair path, clusters as halves (virtual tokens)
     dict(d=128, d_ff=256, E=8, G=2, r=16, k=2),        # pair path, wide tiles
     dict(d=256, d_ff=384, E=8, G=2, r=8, k=2),         # pair path, narrow tiles
-], ids=["generic", "tc1", "pair_wide", "pair_narrow"])
+], ids=["generic", "tc1", "pair_halves", "pair_wide", "pair_narrow"])
 @pytest.mark.parametrize("T", [1, 127, 129, 257, 1500])
 def test_nothing_is_written_outside_the_arena_or_y(kw, T):
     import torch
@@ -458,7 +466,8 @@ def test_nothing_is_written_outside_the_arena_or_y(kw, T):
     s = inputs.small_shape(T=1500, **kw)
     L = inputs.make_layer(s, 71)
     # arena pre-filled with 0xFF (NaN as fp16 / fp32, -1 as int32): nothing may rely on zeroed scratch
-    m = ClusteredMoELayer(L, T_max=1500, guard_bytes=1 << 16, fill_byte=0xFF)
+    whole = s.E // s.G * s.r > 64          # first tensor-core path: the clusters are not split into parts
+    m = ClusteredMoELayer(L, T_max=1500, guard_bytes=1 << 16, fill_byte=0xFF, options=dict(force_path=3) if whole else None)
     x_np = inputs.make_tokens(s, T, seed=T)
     band = 4096
     buf = torch.full((T * s.d + 2 * band,), float("nan"), dtype=torch.float16, device="cuda")
