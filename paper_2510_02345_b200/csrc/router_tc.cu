@@ -31,7 +31,7 @@ constexpr int R_MAX_STAGES = 4;    // stages of the operand ring: as many as sha
 
 struct RtcParams {
   int T, d, G, K, k, E;
-  int rp;                        // G + E rounded up to 8: the hi pieces are columns 0..rp-1, the lo pieces rp..2rp-1
+  int rp;                        // G + E rounded up to 8 (to 16 beyond 128): the hi pieces are columns 0..rp-1, the lo pieces rp..2rp-1
   const float *bc, *be;
   const int* label;
   int* cluster_id;
@@ -69,6 +69,10 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* sm = smem_raw + (base - raw);
   const int N = 2 * p.rp;
+  // A router wider than one MMA (N > 256) is issued piece by piece: two MMAs of N / 2 columns per step, the pieces'
+  // operand rows loaded by a TMA box each (a box has at most 256 rows) and lying one behind the other in the stage
+  const int pieces = N > 256 ? 2 : 1, Np = N / pieces;
+  const uint32_t tcols = N > 256 ? 512u : 256u;
   const uint32_t a_atom = RBM * RBK * 2, b_atom = (uint32_t)N * RBK * 2;
   const uint32_t a_bytes = RKA * a_atom, b_bytes = RKA * b_atom, st_bytes = a_bytes + b_bytes;   // b_atom is a multiple of 1024
   const int R_STAGES = p.stages;
@@ -92,7 +96,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   if (warp == 1) {
     __syncwarp();
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(tmem_holder)), "r"(256u) : "memory");
+                 ::"r"(smem_u32(tmem_holder)), "r"(tcols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -109,12 +113,14 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         const uint32_t a_dst = base + s * st_bytes, b_dst = a_dst + a_bytes;
         mbar_expect_tx(full0 + 8 * s, st_bytes);
         tma_load_3d(a_dst, &tmX, full0 + 8 * s, 0, tile * RBM, c * RKA);    // rows past T read as zeros
-        tma_load_3d(b_dst, &tmW, full0 + 8 * s, 0, 0, c * RKA);
+        for (int h = 0; h < pieces; ++h)
+          tma_load_3d(b_dst + h * (b_bytes / pieces), &tmW, full0 + 8 * s, 0, h * Np, c * RKA);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = idesc_f16(RBM, N);
+      const uint32_t idesc = idesc_f16(RBM, Np);
+      const uint32_t bp_atom = b_atom / pieces;          // one K atom of one piece
       for (int c = 0; c < KC; ++c) {
         const uint32_t s = c % R_STAGES, ph = (c / R_STAGES) & 1u;
         if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) { failed = true; break; }
@@ -125,8 +131,9 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
         for (int a = 0; a < RKA; ++a)
 #pragma unroll
           for (int ks = 0; ks < RBK / 16; ++ks)
-            umma_f16(tmem_base, adesc + a * (a_atom >> 4) + 2 * ks, bdesc + a * (b_atom >> 4) + 2 * ks, idesc,
-                     (c | a | ks) != 0 ? 1u : 0u);
+            for (int h = 0; h < pieces; ++h)
+              umma_f16(tmem_base + h * Np, adesc + a * (a_atom >> 4) + 2 * ks,
+                       bdesc + ((h * RKA + a) * bp_atom >> 4) + 2 * ks, idesc, (c | a | ks) != 0 ? 1u : 0u);
         umma_commit(empty0 + 8 * s);
       }
       if (!failed) umma_commit(tfull);
@@ -222,7 +229,7 @@ router_tc_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant_
   }
   tc_fence_after();
   if (warp == 1)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tcols) : "memory");
   if (p.kc.keys) {
     // keys of this tile counted in shared memory: the permutation's histogram, for free
     for (int i = threadIdx.x; i < p.kc.nkey; i += blockDim.x) cnt[i] = 0;
@@ -279,11 +286,14 @@ int rtc_stages(int N) {
 
 }  // namespace
 
-int router_tc_rp(const Dims& D) { return (real_G(D) + D.E + 7) / 8 * 8; }
+int router_tc_rp(const Dims& D) {
+  const int n = real_G(D) + D.E;
+  return n <= 128 ? (n + 7) / 8 * 8 : (n + 15) / 16 * 16;      // (beyond 128 every piece is an MMA of its own: N a multiple of 16)
+}
 
 bool router_tc_supported(const Dims& D) {
   const int N = 2 * router_tc_rp(D);
-  return D.d % (RBK * RKA) == 0 && N <= 256 && D.T_max >= 1024 && rtc_stages(N) > 0;
+  return D.d % (RBK * RKA) == 0 && N <= 512 && D.T_max >= 1024 && rtc_stages(N) > 0;
 }
 
 cudaError_t router_tc_init(cmoe_layer* L) {
@@ -293,7 +303,7 @@ cudaError_t router_tc_init(cmoe_layer* L) {
   router_split_kernel<<<(unsigned)((n + 255) / 256), 256>>>(L->w.Ct, L->w.Rt, real_G(D), D.E, rp, D.d, L->sc.Wsplit);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (!make_map3(&L->router_map_w, L->sc.Wsplit, (uint64_t)2 * rp, D.d, (uint32_t)(2 * rp))) return cudaErrorInvalidValue;
+  if (!make_map3(&L->router_map_w, L->sc.Wsplit, (uint64_t)2 * rp, D.d, (uint32_t)(2 * rp > 256 ? rp : 2 * rp))) return cudaErrorInvalidValue;
   e = cudaFuncSetAttribute(router_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rtc_smem(2 * rp, rtc_stages(2 * rp)));
   if (e != cudaSuccess) return e;
   return cudaDeviceSynchronize();

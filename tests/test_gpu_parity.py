@@ -180,7 +180,9 @@ def test_router_tile_kernel_shapes(kw):
     dict(T=1100, d=128, d_ff=64, E=36, G=12, r=0, k=2),     # 48 router rows -> 96 MMA columns
     dict(T=1500, d=256, d_ff=64, E=10, G=2, r=0, k=3),      # K = 5
     dict(T=1027, d=1024, d_ff=32, E=8, G=8, r=0, k=1),      # ragged last tile of 128 tokens
-], ids=["G12", "K5", "ragged"])
+    dict(T=1300, d=256, d_ff=64, E=128, G=16, r=0, k=2),    # 144 router rows: two MMAs of 144 columns per step
+    dict(T=1100, d=384, d_ff=64, E=144, G=16, r=0, k=3),    # 160 router rows, K = 9: the widest router the ring has room for
+], ids=["G12", "K5", "ragged", "rows144", "rows160"])
 def test_router_tensor_core_shapes(kw):
     """Large batches are routed on the tensor cores from split fp16 router matrices: same routes as the
     oracle outside the near-tie band, gates to 1e-5."""
