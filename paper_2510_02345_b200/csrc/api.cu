@@ -119,7 +119,7 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   s.row_gate = A.take<float>(P * k);
   s.x_perm = A.take<__half>(P * d);
   if (D.rep > 1) {
-    s.x_rep = A.take<__half>(T * d);
+    if (D.g1 > 1) s.x_rep = A.take<__half>(T * d);       // (expert parts read the token's own row)
     s.y_rep = A.take<__half>(T * d);
   }
   if (D.split > 1) {
@@ -379,8 +379,13 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   // virtual tokens (g1 clusters per token, or expert halves): every row n times, the layer on the virtual
   // tokens, the n outputs of a token summed
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, n, st));
-  rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream, L->dims.split > 1 ? x : nullptr);
+  if (L->dims.split > 1) {
+    // expert parts: the virtual tokens of a token share its row of x (the row move reads row t / n)
+    rc = forward_rows(L, x, T * n, L->sc.y_rep, cuda_stream, x);
+  } else {
+    CMOE_CUDA(L, launch_repeat_rows(L->dims, static_cast<const __half*>(x), L->sc.x_rep, T, n, st));
+    rc = forward_rows(L, L->sc.x_rep, T * n, L->sc.y_rep, cuda_stream, nullptr);
+  }
   if (rc) return rc;
   // (expert parts: a part without any of the token's experts has no row)
   CMOE_CUDA(L, launch_sum_rows(L->dims, L->sc.y_rep, static_cast<__half*>(y), T, n,
@@ -414,7 +419,9 @@ static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* 
     const int Tt = T / D.split;
     if (L->router_tc && Tt >= 1024) CMOE_CUDA(L, launch_router_tc(L, xt, Tt, S.r_cluster, nullptr, S.r_gates, S.r_slot, st));
     else CMOE_CUDA(L, launch_router(plain_dims(D), L->w, xt, Tt, S.r_cluster, nullptr, S.r_gates, S.r_slot, st, &fs));
-    CMOE_CUDA(L, launch_split_routes(D, S, Tt, st));
+    // (the splitting kernel writes the virtual tokens' permutation keys and counts them per block)
+    CMOE_CUDA(L, launch_split_routes(D, S, Tt, st, &kc));
+    counted_tile = split_routes_tile();
     if (Tt < 1024) fs = FactorStage{};  // staged beside the per-token router (else by the row-move kernel)
   } else {
     if (L->router_tc && T >= 1024) {
@@ -435,7 +442,7 @@ static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* 
     LowrankTok lr{};                      // nothing rides along unless the streaming path has residual factors
     if (L->path == kPathStream) stream_lowrank_rider(L, xh, T, &lr);
     const bool gather = L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L);
-    CMOE_CUDA(L, launch_permute(D, S, gather ? nullptr : xh, T, st, zp, zb, fs, lr, counted_tile));
+    CMOE_CUDA(L, launch_permute(D, S, gather ? nullptr : xh, T, st, zp, zb, fs, lr, counted_tile, x_tokens ? D.split : 1));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, tc2_gathers_rows(L) ? xh : nullptr, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
@@ -515,7 +522,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   *out = cmoe_info{};
   out->path = L->path;
   out->launches_route = 1;
-  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0,
+  out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, L->dims.split > 1 ? split_routes_tile() : (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0,
                                               L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L)) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)

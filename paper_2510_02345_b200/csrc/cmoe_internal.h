@@ -165,7 +165,7 @@ int router_tc_tile_tokens();
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
 // counted_tile > 0: the router kernel has already written the keys and the key counts of its tiles of that many tokens
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile);
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div = 1);
 // kernels of the permutation: 2 for batches of at most 256 tokens, 4 below 1024 tokens, else 3 (the router counts the
 // keys) or 2 (and the scatter kernel sums the small count table itself; see launch_permute)
 int permute_launches(const Dims& D, int T, int counted_tile, bool gathered);
@@ -195,7 +195,11 @@ cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, in
 // cluster_id (or null): virtual tokens whose entry is negative have no row
 cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, const int* cluster_id, cudaStream_t st);
 // expert halves: the token's own routes in Scratch::r_* -> the virtual tokens' routes (cluster_id, slot, gates)
-cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st);
+struct KeyCount;
+// routes of the T tokens -> routes of their virtual tokens; with kc the kernel also writes the virtual tokens' permutation
+// keys and counts them per block of split_routes_tile() virtual tokens
+cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st, const KeyCount* kc);
+int split_routes_tile();
 // stream_path.cu : small batches, bound by streaming the bases from HBM
 bool stream_supported(const Dims& D);
 cudaError_t stream_init(cmoe_layer* L);

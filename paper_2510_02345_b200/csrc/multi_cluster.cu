@@ -5,6 +5,7 @@
 // a token's virtual tokens carry the experts of one half, or one quarter, of its cluster each.
 #include "cmoe_internal.h"
 #include "cluster_pick.cuh"
+#include "perm_keys.cuh"
 
 namespace cmoe {
 
@@ -38,22 +39,42 @@ sum_rows_kernel(const __half2* __restrict__ y_rep, __half2* __restrict__ y, long
 }
 
 // Expert parts: the token's own routes (real cluster g, k experts among its K, gates) -> the routes of its `parts`
-// virtual tokens.  A part without any of the token's experts gets cluster id -1: the permutation gives it no row.
-__global__ void __launch_bounds__(256)
+// virtual tokens, a thread per virtual token.  A part without any of the token's experts gets cluster id -1: the
+// permutation gives it no row.  With kc.keys the kernel also writes every virtual token's permutation key and counts
+// the keys of its block's kSplitTile virtual tokens, so that the permutation starts from a finished histogram.
+constexpr int kSplitTile = 256;
+
+__global__ void __launch_bounds__(kSplitTile)
 split_routes_kernel(int T, int K, int parts, int k, const int* __restrict__ r_cluster, const int* __restrict__ r_slot,
                     const float* __restrict__ r_gates, int* __restrict__ cluster_id, int* __restrict__ slot,
-                    float* __restrict__ gates) {
-  const int t = blockIdx.x * blockDim.x + threadIdx.x;
-  if (t >= T) return;
-  const int g = r_cluster[t];
-  for (int part = 0; part < parts; ++part) {
+                    float* __restrict__ gates, const KeyCount kc) {
+  __shared__ int cnt[kMaxKeys];
+  if (kc.keys) {
+    for (int i = threadIdx.x; i < kc.nkey; i += blockDim.x) cnt[i] = 0;
+    __syncthreads();
+  }
+  const long long vt = (long long)blockIdx.x * kSplitTile + threadIdx.x;
+  const int t = (int)(vt / parts), part = (int)(vt - (long long)t * parts);
+  if (t < T) {
+    const int g = r_cluster[t];
     int sel[kMaxKsel];
     float gv[kMaxKsel];
     for (int s = 0; s < k; ++s) { sel[s] = r_slot[(size_t)t * k + s]; gv[s] = r_gates[(size_t)t * k + s]; }
     const int kept = split_part(K, parts, k, part, sel, gv);
-    const size_t vt = (size_t)parts * t + part;
-    cluster_id[vt] = kept > 0 ? parts * g + part : -1;
+    const int vg = kept > 0 ? parts * g + part : -1;
+    cluster_id[vt] = vg;
     for (int s = 0; s < k; ++s) { slot[vt * k + s] = sel[s]; gates[vt * k + s] = gv[s]; }
+    if (kc.keys) {
+      int cs[kMaxKsel];
+      float cg[kMaxKsel];
+      const int key = vg >= 0 ? vg * kc.nsub + canonical_slots(sel, gv, k, kc.sub_is_combo, cs, cg) : -1;
+      kc.keys[vt] = key;
+      if (key >= 0) atomicAdd(&cnt[key], 1);
+    }
+  }
+  if (kc.keys) {
+    __syncthreads();
+    for (int i = threadIdx.x; i < kc.nkey; i += blockDim.x) kc.block_counts[(size_t)blockIdx.x * kc.nkey + i] = cnt[i];
   }
 }
 
@@ -78,9 +99,12 @@ cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T
   return cudaGetLastError();
 }
 
-cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st) {
-  split_routes_kernel<<<(T + 255) / 256, 256, 0, st>>>(T, real_K(D), D.split, D.k, S.r_cluster, S.r_slot, S.r_gates, S.cluster_id,
-                                                       S.slot, S.gates);
+int split_routes_tile() { return kSplitTile; }
+
+cudaError_t launch_split_routes(const Dims& D, const Scratch& S, int T, cudaStream_t st, const KeyCount* kc) {
+  const long long vts = (long long)T * D.split;
+  split_routes_kernel<<<(unsigned)((vts + kSplitTile - 1) / kSplitTile), kSplitTile, 0, st>>>(
+      T, real_K(D), D.split, D.k, S.r_cluster, S.r_slot, S.r_gates, S.cluster_id, S.slot, S.gates, kc ? *kc : KeyCount{});
   return cudaGetLastError();
 }
 

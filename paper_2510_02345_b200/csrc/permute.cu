@@ -144,6 +144,7 @@ struct ScanInline {
 // places never travel through memory.
 struct MoveInline {
   int on;
+  int rep;             // rows of x are shared by `rep` consecutive (virtual) tokens: token t reads row t / rep
   uint4* zero_ptr;
   size_t zero_n;
   FactorStage fs;
@@ -287,16 +288,20 @@ scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
   __syncthreads();
   const int vec_per_row = d / 8, nthr = (int)blockDim.x;
   {
-    // this tile's tokens are consecutive rows of x: vector i of the tile is vector i % vec_per_row of token i / vec_per_row
+    // this tile's tokens are consecutive rows of x (every row mv.rep times when the tokens are virtual ones): vector i
+    // of the tile is vector i % vec_per_row of token i / vec_per_row
     const int t0 = blockIdx.x * tile, nt = min(tile, T - t0);
-    const uint4* src = reinterpret_cast<const uint4*>(x + (size_t)t0 * d);
-    const int nvec = nt * vec_per_row;
+    const uint4* src = reinterpret_cast<const uint4*>(x);
+    const int nvec = nt * vec_per_row, rdiv = mv.rep;
     for (int i0 = threadIdx.x; i0 < nvec; i0 += 8 * nthr) {
       uint4 val[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int i = i0 + u * nthr;
-        if (i < nvec) val[u] = src[i];
+        if (i < nvec) {
+          const int tt = i / vec_per_row;
+          val[u] = src[(size_t)((t0 + tt) / rdiv) * vec_per_row + (i - tt * vec_per_row)];
+        }
       }
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
@@ -325,7 +330,7 @@ scatter_kernel(int T, int tile, int d, int K, int k, int nkey, int sub_is_combo,
 __global__ void __launch_bounds__(128)
 move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ row_token,
                  const __half* __restrict__ x, __half* __restrict__ x_perm, uint4* __restrict__ zero_ptr, size_t zero_n,
-                 int n_move, const FactorStage fs) {
+                 int n_move, const FactorStage fs, int rdiv) {
   pdl_wait();
   // blocks n_move.. decode the layer's INT4 factors for the tensor-core residual products (weights only; a few MB
   // more for a kernel that is bound by memory bandwidth anyway)
@@ -345,7 +350,7 @@ move_rows_kernel(int d, const int* __restrict__ n_rows, const int* __restrict__ 
       uint4 val[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
-        val[i] = tok[i] >= 0 ? reinterpret_cast<const uint4*>(x + (size_t)tok[i] * d)[v] : make_uint4(0, 0, 0, 0);
+        val[i] = tok[i] >= 0 ? reinterpret_cast<const uint4*>(x + (size_t)(tok[i] / rdiv) * d)[v] : make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         if (tok[i] != -2) reinterpret_cast<uint4*>(x_perm + (size_t)(row0 + i * n_move) * d)[v] = val[i];
@@ -453,11 +458,14 @@ bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk 
 int permute_launches(const Dims& D, int T, int counted_tile, bool gathered) {
   if (T <= kSmallT) return 2;
   if (counted_tile <= 0) return 4;
-  return inline_scan_ok(D, (T + counted_tile - 1) / counted_tile, counted_tile) ? (gathered ? 2 : 1) : 3;
+  const int nblk = (T + counted_tile - 1) / counted_tile, sms = D.sm_count > 0 ? D.sm_count : 148;
+  const bool fused = !gathered && counted_tile <= 512 && (long long)T * D.d * 2 / (nblk < sms ? nblk : sms) <= 600 * 1024;
+  return inline_scan_ok(D, nblk, counted_tile) ? (fused ? 1 : 2) : 3;
 }
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile) {
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div) {
+  if (x_div < 1) x_div = 1;
 
   const int rows_bound = t_pad_bound(D, T);
   if (T <= kSmallT) {
@@ -467,7 +475,7 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
         T, D.G, D.K, D.k, D.nsub, D.nkey, D.sub_is_combo, D.row_align, D.T_pad_max / D.row_align, S.cluster_id, S.slot,
         S.gates, S.seg_off, S.seg_cnt, S.n_rows, S.tile_cluster, S.row_token, S.row_slot, S.row_gate, lr);
     launch_chained(move_rows_kernel, dim3(rows_bound), dim3(128), 0, st, 1,
-      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, rows_bound, FactorStage{});
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, rows_bound, FactorStage{}, x_div);
     return cudaGetLastError();
   }
   // counting blocks: the router's token tiles when it counted the keys itself (counted_tile tokens each), else
@@ -494,8 +502,11 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
   }
   // with the inline sums the scatter blocks also move their tile's rows (unless a later kernel gathers them)
   MoveInline mv{};
-  const bool fused_move = inline_scan && x != nullptr && tile <= 512;
-  if (fused_move) { mv.on = 1; mv.zero_ptr = static_cast<uint4*>(zero_ptr); mv.zero_n = zero_bytes / 16; mv.fs = fs; }
+  // (not when that would leave each of too few blocks with megabytes to move: the row-move kernel then does better)
+  const int sms = D.sm_count > 0 ? D.sm_count : 148;
+  const bool fused_move = inline_scan && x != nullptr && tile <= 512 &&
+                          (long long)T * D.d * 2 / (nblk < sms ? nblk : sms) <= 600 * 1024;
+  if (fused_move) { mv.on = 1; mv.rep = x_div; mv.zero_ptr = static_cast<uint4*>(zero_ptr); mv.zero_n = zero_bytes / 16; mv.fs = fs; }
   launch_chained(scatter_kernel, dim3(nblk + (fused_move ? stage_blocks(fs, 512) : 0)), dim3(inline_scan ? 512 : tile),
                  sh * (inline_scan ? 2 : 1), st, 1,
       T, tile, D.d, D.K, D.k, D.nkey, D.sub_is_combo, x,
@@ -506,7 +517,7 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
   const int move_max = (D.sm_count > 0 ? D.sm_count : 148) * 32;      // resident blocks of 128 threads
   const int move_grid = rows_bound < move_max ? rows_bound : move_max;
   launch_chained(move_rows_kernel, dim3(move_grid + stage_blocks(fs, 128)), dim3(128), 0, st, 1,
-      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, move_grid, fs);
+      D.d, S.n_rows, S.row_token, x, S.x_perm, static_cast<uint4*>(zero_ptr), zero_bytes / 16, move_grid, fs, x_div);
   return cudaGetLastError();
 }
 

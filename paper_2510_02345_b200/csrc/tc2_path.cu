@@ -1096,7 +1096,7 @@ void tc2_factor_stage(const cmoe_layer* L, FactorStage* fs) {
 }
 
 // (option) the t kernel reads x by row_token and writes x_perm itself: the permutation then moves no rows
-bool tc2_gathers_rows(const cmoe_layer* L) { return L->dims.r > 0 && L->opt.row_gather == 1; }
+bool tc2_gathers_rows(const cmoe_layer* L) { return L->dims.r > 0 && L->opt.row_gather == 1 && L->dims.split <= 1; }
 
 int tc2_launch_count(const cmoe_layer* L) {
   const Dims& D = L->dims;
