@@ -115,6 +115,9 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *                 the kernel that projects the tokens onto U1 reads them from x by TMA row gather (four rows of 128
  *                 bytes per instruction) and writes the permuted copy as it goes: one pass over x less, but slower
  *                 as measured (the gathers are issued at a fraction of the rate of tiled loads)
+ *   move_in_scatter  0 (default): large batches are permuted by a kernel that places the tokens and a kernel that
+ *                 moves their rows; 1: the placing blocks move the rows of their own token tile themselves (one
+ *                 launch less; measured equal on one B200 of the pool and 3-7 us slower on another, so off)
  * and one switch that changes what the descriptor means:
  *   base_dtype    0: desc.B1 / desc.B2 hold fp16 bits (the paper's storage format, Sec. 3.4); 1: they hold bfloat16
  *                 bits.  The tensor cores take both operands of a product in one 16-bit type and the activations
@@ -132,7 +135,7 @@ int cmoe_create(const cmoe_desc* desc, cmoe_layer** out_layer);
  *                 on two virtual tokens per token (2 T rows through router, permutation and expert FFNs, then one
  *                 sum per token), so a call costs about what one of 2 T tokens costs, and the workspace must be sized
  *                 with cmoe_workspace_bytes_ex.
- * Other values: CMOE_ERR_INVALID_ARG.  reserved must be zero. */
+ * Other values: CMOE_ERR_INVALID_ARG.  */
 typedef struct {
   int32_t force_path;
   int32_t router_fp32;
@@ -141,7 +144,7 @@ typedef struct {
   int32_t host_chunks;
   int32_t row_gather;
   int32_t clusters_per_token;
-  int32_t reserved[1];
+  int32_t move_in_scatter;
 } cmoe_options;
 int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* options, cmoe_layer** out_layer);
 /* cmoe_workspace_bytes for a handle that cmoe_create_ex will make with these options (NULL = cmoe_workspace_bytes):

@@ -42,7 +42,7 @@ class cmoe_desc(C.Structure):
 
 class cmoe_options(C.Structure):
     _fields_ = [("force_path", C.c_int32), ("router_fp32", C.c_int32), ("up_tile", C.c_int32), ("base_dtype", C.c_int32),
-                ("host_chunks", C.c_int32), ("row_gather", C.c_int32), ("clusters_per_token", C.c_int32), ("reserved", C.c_int32 * 1)]
+                ("host_chunks", C.c_int32), ("row_gather", C.c_int32), ("clusters_per_token", C.c_int32), ("move_in_scatter", C.c_int32)]
 
 
 class cmoe_compress_desc(C.Structure):

@@ -212,7 +212,7 @@ int cmoe_create_ex(const cmoe_desc* desc, const cmoe_options* opt, cmoe_layer** 
   if (opt) o = *opt;
   if (o.force_path < -1 || (o.force_path > 0 && o.force_path != 3) || (o.up_tile != 0 && o.up_tile != 128 && o.up_tile != 256) ||
       o.base_dtype < 0 || o.base_dtype > 1 || o.host_chunks < 0 || o.host_chunks > kMaxHostChunks || o.row_gather < 0 || o.row_gather > 1 ||
-      o.reserved[0] != 0) return CMOE_ERR_INVALID_ARG;
+      o.move_in_scatter < 0 || o.move_in_scatter > 1) return CMOE_ERR_INVALID_ARG;
   {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&D.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
@@ -442,7 +442,7 @@ static int forward_rows(cmoe_layer* L, const void* x, int32_t T, void* y, void* 
     LowrankTok lr{};                      // nothing rides along unless the streaming path has residual factors
     if (L->path == kPathStream) stream_lowrank_rider(L, xh, T, &lr);
     const bool gather = L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L);
-    CMOE_CUDA(L, launch_permute(D, S, gather ? nullptr : xh, T, st, zp, zb, fs, lr, counted_tile, x_tokens ? D.split : 1));
+    CMOE_CUDA(L, launch_permute(D, S, gather ? nullptr : xh, T, st, zp, zb, fs, lr, counted_tile, x_tokens ? D.split : 1, L->opt.move_in_scatter == 1));
   }
   if (L->path == kPathTensor && L->tc_variant == 2)
     CMOE_CUDA(L, launch_tc2_ffn(L, tc2_gathers_rows(L) ? xh : nullptr, T, static_cast<__half*>(y), st, L->profiling ? L->events + stage : nullptr));
@@ -523,7 +523,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
   out->path = L->path;
   out->launches_route = 1;
   out->launches_forward = 1 + permute_launches(L->dims, L->dims.T_max, L->dims.split > 1 ? split_routes_tile() : (L->dims.T_max >= 1024 && L->router_tc) ? router_tc_tile_tokens() : 0,
-                                              L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L)) +
+                                              (L->path == kPathTensor && L->tc_variant == 2 && tc2_gathers_rows(L)) || L->opt.move_in_scatter != 1) +
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.rep > 1 ? 2 : 0);

@@ -165,10 +165,11 @@ int router_tc_tile_tokens();
 // also clears zero_bytes (a multiple of 16) at zero_ptr: the buffer the later stages accumulate into
 // counted_tile > 0: the router kernel has already written the keys and the key counts of its tiles of that many tokens
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div = 1);
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div = 1,
+                           bool move_in_scatter = false);
 // kernels of the permutation: 2 for batches of at most 256 tokens, 4 below 1024 tokens, else 3 (the router counts the
 // keys) or 2 (and the scatter kernel sums the small count table itself; see launch_permute)
-int permute_launches(const Dims& D, int T, int counted_tile, bool gathered);
+int permute_launches(const Dims& D, int T, int counted_tile, bool separate_move);
 // generic_path.cu : CUDA-core path for any supported shape
 // `marks` (or null): three events recorded before the residual-t, up and down stages
 cudaError_t launch_generic_ffn(const Dims& D, const Weights& W, const Scratch& S, int T, __half* y,

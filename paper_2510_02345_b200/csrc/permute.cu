@@ -455,16 +455,17 @@ bool inline_scan_ok(const Dims& D, int nblk, int tile) { return (long long)nblk 
 
 }  // namespace
 
-int permute_launches(const Dims& D, int T, int counted_tile, bool gathered) {
+int permute_launches(const Dims& D, int T, int counted_tile, bool separate_move) {
   if (T <= kSmallT) return 2;
   if (counted_tile <= 0) return 4;
   const int nblk = (T + counted_tile - 1) / counted_tile, sms = D.sm_count > 0 ? D.sm_count : 148;
-  const bool fused = !gathered && counted_tile <= 512 && (long long)T * D.d * 2 / (nblk < sms ? nblk : sms) <= 600 * 1024;
+  const bool fused = !separate_move && counted_tile <= 512 && (long long)T * D.d * 2 / (nblk < sms ? nblk : sms) <= 600 * 1024;
   return inline_scan_ok(D, nblk, counted_tile) ? (fused ? 1 : 2) : 3;
 }
 
 cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int T, cudaStream_t st, void* zero_ptr,
-                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div) {
+                           size_t zero_bytes, const FactorStage& fs, const LowrankTok& lr, int counted_tile, int x_div,
+                           bool move_in_scatter) {
   if (x_div < 1) x_div = 1;
 
   const int rows_bound = t_pad_bound(D, T);
@@ -500,11 +501,11 @@ cudaError_t launch_permute(const Dims& D, const Scratch& S, const __half* x, int
                                     S.block_counts, S.block_base, S.key_cnt, S.key_off, S.seg_off,
                                     S.seg_cnt, S.n_rows, S.tile_cluster, D.K, D.k, S.row_token, S.row_slot, S.row_gate);
   }
-  // with the inline sums the scatter blocks also move their tile's rows (unless a later kernel gathers them)
+  // on request (cmoe_options.move_in_scatter) the scatter blocks that do the sums also move their tile's rows
   MoveInline mv{};
   // (not when that would leave each of too few blocks with megabytes to move: the row-move kernel then does better)
   const int sms = D.sm_count > 0 ? D.sm_count : 148;
-  const bool fused_move = inline_scan && x != nullptr && tile <= 512 &&
+  const bool fused_move = move_in_scatter && inline_scan && x != nullptr && tile <= 512 &&
                           (long long)T * D.d * 2 / (nblk < sms ? nblk : sms) <= 600 * 1024;
   if (fused_move) { mv.on = 1; mv.rep = x_div; mv.zero_ptr = static_cast<uint4*>(zero_ptr); mv.zero_n = zero_bytes / 16; mv.fs = fs; }
   launch_chained(scatter_kernel, dim3(nblk + (fused_move ? stage_blocks(fs, 512) : 0)), dim3(inline_scan ? 512 : tile),

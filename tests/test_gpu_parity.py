@@ -625,6 +625,25 @@ def test_decode_shaped_layer_on_a_large_batch():
     assert got["module"].info.path == 1
 
 
+@pytest.mark.parametrize("T,kw", [
+    (1027, dict(d=128, d_ff=256, E=8, G=2, r=16, k=2)),        # ragged last router tile
+    (4096, dict(d=768, d_ff=3072, E=16, G=4, r=16, k=2)),      # the bert shape
+    (3000, dict(d=256, d_ff=512, E=12, G=3, r=8, k=1)),        # one kept expert; an empty cluster (bias below)
+    (2500, dict(d=256, d_ff=256, E=16, G=2, r=16, k=2)),       # expert halves: virtual tokens share their token's row
+], ids=["ragged", "bert", "empty_cluster", "halves"])
+def test_rows_moved_by_the_scatter_blocks(T, kw):
+    """cmoe_options.move_in_scatter: the blocks that place the tokens of a router tile also move their rows (one
+    launch less).  Every row against the oracle."""
+    s = inputs.small_shape(T=T, **kw)
+    L = inputs.make_layer(s, 23)
+    if s.G == 3:
+        L["b_c"] = np.array([0.0, -50.0, 0.0], np.float32)
+    plain = run_gpu(L, L["x"])["module"].info.launches_forward
+    got = full_check(L, L["x"], options=dict(move_in_scatter=1))
+    assert got["module"].info.path == 1
+    assert got["module"].info.launches_forward == plain - 1
+
+
 def test_many_experts_beyond_the_pair_path():
     """E = 128 in G = 16 clusters with r = 16 (K r = 128 > 64, the expanded rank index of the pair path holds 64): the
     clusters are handled as two halves of four experts on the pair path; sampled rows."""
