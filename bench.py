@@ -66,7 +66,7 @@ def stage_work(s, T, stage, active_clusters, active_experts):
 # profiles/.  The figure is reported only while
 # the kernel sources still have the hash they had at the capture; otherwise "traffic" is null.
 NCU_TRAFFIC = {
-    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 124.950528e6 + 112.657920e6,
+    "gpt2m": {"kernel": "tc2_up_wide_kernel<true,2>", "bytes": 121.410560e6 + 113.126912e6,
               "sha1": {"tc2_up_wide.cu": "4af5ed7641eb5387e18a572ad07b739a68937757",
                        "tc2_common.cuh": "f6446e474cd1a42f4e9a7cc20120ebd7f01b50b3",
                        "tc_ptx.cuh": "5939df29cafb85df0df022be40abbaa547d366c8"}},
