@@ -81,3 +81,38 @@ def test_null_handles(lib):
     assert lib.cmoe_destroy(None) == -1
     assert lib.cmoe_status(None, None) == -1
     assert binding.strerror(0) == "ok" and "workspace" in binding.strerror(-3)
+
+
+def _bytes_ex(lib, d, **opt):
+    o = binding.cmoe_options()
+    o.force_path = -1
+    for k, v in opt.items():
+        setattr(o, k, v)
+    out = C.c_size_t()
+    rc = lib.cmoe_workspace_bytes_ex(C.byref(d), C.byref(o), C.byref(out))
+    return rc, out.value
+
+
+def test_clusters_handled_as_parts_need_a_larger_arena(lib):
+    """K r > 64 on a large batch: the clusters are handled as halves (K r <= 128) or quarters (K r <= 256) with as
+    many virtual tokens per token, which shows in the arena the host query asks for; force_path = 3 keeps the
+    clusters whole.  Shapes the split does not apply to ask for the same arena either way."""
+    shape = dict(d=256, d_ff=512, G=2, k=2, T_max=2048)
+    rows = []
+    for E, r in ((8, 16), (16, 16), (16, 32)):          # K r = 64 (whole), 128 (halves), 256 (quarters)
+        rc, whole = _bytes_ex(lib, desc(E=E, r=r, **shape), force_path=3)
+        assert rc == 0
+        rc, auto = _bytes_ex(lib, desc(E=E, r=r, **shape))
+        assert rc == 0
+        rows.append(auto / whole)
+    assert rows[0] == 1.0
+    # (the pair path also keeps staged fp16 factors and 256-row segments, so the factors are above 2 and 4)
+    assert 1.5 < rows[1] < 4.0 and 1.3 * rows[1] < rows[2] < 8.0, rows
+    # k = 3 of K = 8: neither halves (k <= 4 but (K/2) r = 128 > 64 at r = 32) nor quarters (k > 2) apply
+    rc, a = _bytes_ex(lib, desc(E=16, r=32, d=256, d_ff=512, G=2, k=3, T_max=2048))
+    rc2, b = _bytes_ex(lib, desc(E=16, r=32, d=256, d_ff=512, G=2, k=3, T_max=2048), force_path=3)
+    assert rc == 0 and rc2 == 0 and a == b
+    # small batches never split (the weight-streaming path takes them)
+    rc, a = _bytes_ex(lib, desc(E=16, r=32, d=256, d_ff=512, G=2, k=2, T_max=128))
+    rc2, b = _bytes_ex(lib, desc(E=16, r=32, d=256, d_ff=512, G=2, k=2, T_max=128), force_path=3)
+    assert a == b
