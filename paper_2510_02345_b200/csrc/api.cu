@@ -54,15 +54,22 @@ int validate_dims(const cmoe_desc* desc, int g1, bool allow_split, Dims* D) {
   D->d = desc->d; D->d_ff = desc->d_ff; D->E = desc->E; D->G = desc->G; D->K = K;
   // with g1 clusters per token everything below the entry points works on g1 virtual tokens per token
   D->r = desc->r; D->k = desc->k; D->g1 = g1; D->T_user = desc->T_max; D->T_max = desc->T_max * g1;
-  D->split = 0; D->rep = g1;
+  D->split = 0; D->rep = g1; D->seq = 0;
   // K r beyond the pair path's expanded rank index: every cluster as two halves, else four quarters, of its experts
   // where that makes the shape fit
   if (allow_split && g1 == 1 && D->T_max > 128 && !tc2_supported(*D)) {
-    for (int parts = 2; parts <= 4 && D->split == 0; parts *= 2) {
+    for (int parts = 2; parts <= 4 && D->split == 0 && D->seq == 0; parts *= 2) {
       if (K % parts || desc->k > K / parts || parts * desc->G > kMaxG || (long long)desc->T_max * parts > (1 << 22)) continue;
       Dims V = *D;
       V.K = K / parts; V.G = parts * desc->G; V.T_max = parts * desc->T_max;
-      if (tc2_supported(V)) { D->split = parts; D->rep = parts; D->K = V.K; D->G = V.G; D->T_max = V.T_max; }
+      if (!tc2_supported(V)) continue;
+      // Up to kSeqTokens tokens the weight-streaming path, taken in pieces of 128 tokens, is the faster one: every
+      // piece reads the weights once, where the parts read each base `parts` times on mostly empty 256-row tiles
+      // (decode-shaped layer, 129 tokens: 1371 us as quarters, about 750 us as two pieces)
+      Dims W = *D;
+      W.T_max = 128;
+      if (desc->T_max <= kSeqTokens && stream_supported(W)) { D->seq = 128; D->T_max = 128; continue; }
+      D->split = parts; D->rep = parts; D->K = V.K; D->G = V.G; D->T_max = V.T_max;
     }
   }
   const long long combos = binom_ll(D->K, desc->k);
@@ -102,9 +109,10 @@ void plan(const Dims& D, Arena& A, Weights* W, Scratch* S) {
   w.V1s = A.take<__half>(E * f * r / 32 + 8);
   w.U2s = A.take<__half>(E * r * f / 32 + 8);
   w.V2s = A.take<__half>(E * d * r / 32 + 8);
-  s.cluster_id = A.take<int>(T);
-  s.slot = A.take<int>(T * k);
-  s.gates = A.take<float>(T * k);
+  const size_t Tr = D.seq > 0 ? (size_t)D.T_user : T;      // (cmoe_expert_stats routes a whole call at once)
+  s.cluster_id = A.take<int>(Tr);
+  s.slot = A.take<int>(Tr * k);
+  s.gates = A.take<float>(Tr * k);
   s.keys = A.take<int>(T);
   s.block_counts = A.take<int>(nblk * D.nkey);
   s.block_base = A.take<int>(nblk * D.nkey);
@@ -375,6 +383,16 @@ int cmoe_forward(cmoe_layer* L, const void* x, int32_t T, void* y, void* cuda_st
   if (T == 0) return CMOE_OK;
   if (!y || !aligned16(y)) return CMOE_ERR_INVALID_ARG;
   const int n = L->dims.rep;
+  if (L->dims.seq > 0 && T > L->dims.seq) {
+    // consecutive pieces of at most seq tokens, one after the other on the caller's stream
+    const size_t row = sizeof(__half) * (size_t)L->dims.d;
+    for (int t0 = 0; t0 < T; t0 += L->dims.seq) {
+      const int tc = T - t0 < L->dims.seq ? T - t0 : L->dims.seq;
+      rc = forward_rows(L, static_cast<const char*>(x) + row * t0, tc, static_cast<char*>(y) + row * t0, cuda_stream, nullptr);
+      if (rc) return rc;
+    }
+    return CMOE_OK;
+  }
   if (n <= 1) return forward_rows(L, x, T, y, cuda_stream, nullptr);
   // virtual tokens (g1 clusters per token, or expert halves): every row n times, the layer on the virtual
   // tokens, the n outputs of a token summed
@@ -527,6 +545,7 @@ int cmoe_get_info(const cmoe_layer* L, cmoe_info* out) {
                           (L->path == kPathTensor && L->tc_variant == 2
                                ? tc2_launch_count(L)
                                : L->path == kPathStream ? stream_launch_count(L->dims) : (L->dims.r > 0 ? kGenericFfnLaunches : kGenericFfnLaunches - 1)) + (L->dims.rep > 1 ? 2 : 0);
+  if (L->dims.seq > 0) out->launches_forward *= (L->dims.T_user + L->dims.seq - 1) / L->dims.seq;    // (a call of T_max tokens)
   out->memsets_forward = 0;
   out->n_stages = L->n_stages;
   out->row_align = L->dims.row_align;

@@ -17,6 +17,7 @@ constexpr int kMaxK = 32;          // experts per cluster (one lane each in the 
 constexpr int kMaxKsel = 8;        // k
 constexpr int kMaxKeys = 4096;     // permutation keys (cluster x expert combination)
 constexpr int kMaxHostChunks = 8; // most chunks cmoe_forward_host cuts a batch into
+constexpr int kSeqTokens = 384;    // largest T_max that is served in pieces of 128 tokens on the weight-streaming path (Dims::seq)
 constexpr int kPermBlock = 256;    // tokens per block in the permutation kernels (when they count the keys themselves)
 constexpr int kMinCountTile = 128; // token tile of the router kernel that counts keys (router_tc.cu)
 
@@ -38,6 +39,9 @@ struct Dims {
   int g1;          // clusters per token (Sec. 3.3); 0 and 1 both mean one
   int split;       // 2 or 4: the clusters are handled as that many parts of K / split experts each (above); else 0
   int rep;         // rows of the kernels' x per caller token: max(g1, split, 1)
+  int seq;         // > 0: a call's tokens go through the layer in consecutive pieces of at most `seq` tokens (= T_max):
+                   // few tokens on a layer whose clusters would have to be split (below) stream the weights once per
+                   // piece instead of computing two to four base products per token
   int T_pad_max;   // rows of the permuted buffers
   int row_align;   // a cluster's rows start at a multiple of this
   int sub_is_combo;

@@ -35,10 +35,10 @@ def run_gpu(L, x_np, T_max=None, options=None):
     return out
 
 
-def full_check(L, x_np, sample=None, seed=0, label=None, options=None):
+def full_check(L, x_np, sample=None, seed=0, label=None, options=None, T_max=None):
     s = L["shape"]
     o = ref.Layer(L)
-    got = run_gpu(L, x_np, options=options)
+    got = run_gpu(L, x_np, T_max=T_max, options=options)
     T = x_np.shape[0]
     idx = None
     if sample is not None and sample < T:
@@ -616,6 +616,31 @@ def test_headline_shape_variants(kw):
     assert got["module"].info.path == 1
 
 
+@pytest.mark.parametrize("T,T_max", [(129, 129), (300, 384), (384, 384), (128, 384), (50, 200)])
+def test_wide_clusters_on_few_tokens_stream_in_pieces(T, T_max):
+    """K r > 64 with 128 < T_max <= 384: the call's tokens go through the weight-streaming kernels in consecutive pieces of
+    128 tokens (splitting the clusters would compute up to four base products per token on mostly empty tiles).  Every
+    row against the oracle; routes and expert loads of the whole call."""
+    import torch
+    s = inputs.small_shape(T=T, d=256, d_ff=512, E=16, G=2, r=32, k=2)
+    L = inputs.make_layer(s, 27)
+    got = full_check(L, L["x"], T_max=T_max)
+    m = got["module"]
+    assert m.info.path == 2 and m.info.T_pad_max < 2 * 128 + 64
+    loads, _, _ = m.expert_stats(torch.from_numpy(L["x"]).cuda())
+    torch.cuda.synchronize()
+    want = np.bincount(ref.Layer(L).route(L["x"])["expert_slot"].reshape(-1), minlength=s.E)
+    assert int(loads.sum()) == s.k * T and np.abs(loads.cpu().numpy() - want).sum() <= 8
+
+
+def test_wide_clusters_beyond_the_streamed_pieces():
+    """The same layer with T_max = 385 is past the limit of the pieces: clusters as quarters on the pair path."""
+    s = inputs.small_shape(T=385, d=256, d_ff=512, E=16, G=2, r=32, k=2)
+    L = inputs.make_layer(s, 27)
+    got = full_check(L, L["x"])
+    assert got["module"].info.path == 1 and got["module"].info.T_pad_max >= 4 * 385
+
+
 def test_decode_shaped_layer_on_a_large_batch():
     """The decode-shaped layer (K = 8, r = 32: K r = 256) on a prefill-sized batch: quarters of two experts on the pair
     path; sampled rows."""
@@ -671,9 +696,11 @@ def test_expert_halves(T, kw):
     s = inputs.small_shape(T=T, **kw)
     L = inputs.make_layer(s, 17)
     got = full_check(L, L["x"])
-    if kw["k"] <= 2:
+    if kw["k"] <= 2 and T > 384:
         assert got["module"].info.path == 1
         assert got["module"].info.T_pad_max >= 2 * T            # two virtual tokens per token
+    elif kw["k"] <= 2:
+        assert got["module"].info.path == 2                     # few tokens: pieces of 128 on the streaming path
 
 
 def test_expert_halves_report_the_tokens_own_routes_and_loads():
