@@ -155,6 +155,9 @@ VARIANTS = {
     "gpt2m_G16_K4": dict(E=64, G=16), "gpt2m_K8_r8": dict(E=64, r=8), "gpt2m_E128_G16": dict(E=128, G=16),
     "gpt2m_bf16_bases": dict(),
     "decode_layer_T4096": dict(T=4096, d=4096, d_ff=14336, E=64, G=8, r=32),   # K r = 256: quarters of two experts
+    "decode_layer_T129": dict(T=129, d=4096, d_ff=14336, E=64, G=8, r=32),     # few tokens: two pieces on the streaming path
+    "decode_layer_T256": dict(T=256, d=4096, d_ff=14336, E=64, G=8, r=32),
+    "decode_layer_T512": dict(T=512, d=4096, d_ff=14336, E=64, G=8, r=32),     # past the pieces: quarters on mostly empty tiles
     "gpt2m_two_clusters": dict(T=8192),      # Sec. 3.3 "Top-g1 groups", g1 = 2: 8192 tokens, two clusters each
 }
 VARIANT_OPTIONS = {"gpt2m_two_clusters": dict(clusters_per_token=2)}
