@@ -21,20 +21,30 @@ repeat_rows_kernel(const uint4* __restrict__ x, uint4* __restrict__ x_rep, long 
   }
 }
 
+// y[t] = sum of the token's n output rows (fp32 sums, one rounding), eight columns per thread
 __global__ void __launch_bounds__(256)
-sum_rows_kernel(const __half2* __restrict__ y_rep, __half2* __restrict__ y, long long pairs_per_row, long long T, int g1,
+sum_rows_kernel(const uint4* __restrict__ y_rep, uint4* __restrict__ y, long long vec_per_row, long long T, int g1,
                 const int* __restrict__ cluster_id) {
-  const long long n = T * pairs_per_row;
+  const long long n = T * vec_per_row;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-    const long long t = i / pairs_per_row, v = i - t * pairs_per_row;
-    float2 acc = make_float2(0.f, 0.f);
+    const long long t = i / vec_per_row, v = i - t * vec_per_row;
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
     for (int c = 0; c < g1; ++c) {
       if (cluster_id && cluster_id[t * g1 + c] < 0) continue;        // a virtual token that was dropped: no row
-      const float2 f = __half22float2(y_rep[(t * g1 + c) * pairs_per_row + v]);
-      acc.x += f.x;
-      acc.y += f.y;
+      const uint4 q = y_rep[(t * g1 + c) * vec_per_row + v];
+      const __half2* h = reinterpret_cast<const __half2*>(&q);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const float2 f = __half22float2(h[u]);
+        acc[2 * u] += f.x;
+        acc[2 * u + 1] += f.y;
+      }
     }
-    y[i] = __floats2half2_rn(acc.x, acc.y);
+    uint4 o;
+    __half2* oh = reinterpret_cast<__half2*>(&o);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) oh[u] = __floats2half2_rn(acc[2 * u], acc[2 * u + 1]);
+    y[i] = o;
   }
 }
 
@@ -93,9 +103,9 @@ cudaError_t launch_repeat_rows(const Dims& D, const __half* x, __half* x_rep, in
 }
 
 cudaError_t launch_sum_rows(const Dims& D, const __half* y_rep, __half* y, int T, int n, const int* cluster_id, cudaStream_t st) {
-  const long long pairs = D.d / 2;
-  sum_rows_kernel<<<grid_for((long long)T * pairs, D.sm_count), 256, 0, st>>>(
-      reinterpret_cast<const __half2*>(y_rep), reinterpret_cast<__half2*>(y), pairs, T, n, cluster_id);
+  const long long vec = D.d / 8;
+  sum_rows_kernel<<<grid_for((long long)T * vec, D.sm_count), 256, 0, st>>>(
+      reinterpret_cast<const uint4*>(y_rep), reinterpret_cast<uint4*>(y), vec, T, n, cluster_id);
   return cudaGetLastError();
 }
 
