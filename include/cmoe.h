@@ -64,8 +64,9 @@ typedef struct cmoe_layer cmoe_layer; /* opaque, host object owned by the librar
  * T_max >= 1.  With r == 0 the factor pointers are ignored (plain shared-base experts).
  * Speed, not results, depends on the shape: the fastest large-batch kernels need d and d_ff multiples of 128, k <= 2
  * and K*r <= 64 (or, for n = 2 or 4 with K a multiple of n, k <= K/n and n*G <= 64, (K/n)*r <= 64: the clusters are then
- * handled as n parts of K/n experts sharing the cluster's base; with T_max <= 384 such a layer instead runs a call's
- * tokens in consecutive pieces of 128 on the kernels for small batches, which read the weights once per piece).
+ * handled as n parts of K/n experts sharing the cluster's base; with T_max <= 384 and enough weights for it to pay
+ * such a layer instead runs a call's tokens in consecutive pieces of 128 on the kernels for small batches, which read
+ * the weights once per piece).
  * All weight pointers must be 16-byte aligned.
  */
 typedef struct {

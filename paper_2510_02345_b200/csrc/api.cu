@@ -3,6 +3,8 @@
 #include <cstdlib>
 #include <new>
 
+#include <cmath>
+
 #include "cmoe_internal.h"
 #include "stage_factors.cuh"
 #include "lowrank.cuh"
@@ -35,6 +37,26 @@ long long binom_ll(int n, int m) {
   return r;
 }
 
+// Few tokens on a layer whose clusters would be handled as `parts` parts: pieces of 128 tokens on the streaming
+// kernels, or the parts on the pair kernels?  Estimates in us, fitted to measurements on a B200 (four layers from
+// 134 MB to 1.9 GB of bases, 129 to 384 tokens; the constants do not depend on the device so that the host query and
+// cmoe_create always agree):
+//   a piece     80 + bytes of the bases / 6.0 TB/s      (one pass over the weights and the launch chain)
+//   the parts   60 + rounds of 256 x 256 pair tiles on 74 CTA pairs: parts * G row tiles (one per virtual cluster at
+//               these sizes), 8.6 us * d / 1024 per up tile, 6.7 us * d_ff / 1024 per down tile (half for 128 columns)
+// Pieces are taken when they come out at least 15 % ahead.
+bool pieces_win(const cmoe_desc& desc, int parts) {
+  const double d = desc.d, f = desc.d_ff, G = desc.G;
+  const double piece = 80.0 + 2.0 * G * d * f * 2.0 / 6.0e6;
+  const double n_pieces = (desc.T_max + 127) / 128;
+  const double row_tiles = (double)parts * G, pairs = 74.0;
+  const double up_rounds = std::ceil(row_tiles * std::ceil(f / 256.0) / pairs);
+  const bool dn_wide = desc.d % 256 == 0;
+  const double dn_rounds = std::ceil(row_tiles * std::ceil(d / (dn_wide ? 256.0 : 128.0)) / pairs);
+  const double split = 60.0 + up_rounds * 8.6 * d / 1024.0 + dn_rounds * (dn_wide ? 6.7 : 3.35) * f / 1024.0;
+  return n_pieces * piece < 0.85 * split;
+}
+
 int validate_dims(const cmoe_desc* desc, int g1, bool allow_split, Dims* D) {
   if (!desc) return CMOE_ERR_INVALID_ARG;
   if (g1 < 0 || g1 > 2) return CMOE_ERR_INVALID_ARG;
@@ -63,12 +85,12 @@ int validate_dims(const cmoe_desc* desc, int g1, bool allow_split, Dims* D) {
       Dims V = *D;
       V.K = K / parts; V.G = parts * desc->G; V.T_max = parts * desc->T_max;
       if (!tc2_supported(V)) continue;
-      // Up to kSeqTokens tokens the weight-streaming path, taken in pieces of 128 tokens, is the faster one: every
-      // piece reads the weights once, where the parts read each base `parts` times on mostly empty 256-row tiles
-      // (decode-shaped layer, 129 tokens: 1371 us as quarters, about 750 us as two pieces)
+      // Few tokens (at most kSeqTokens): the weight-streaming path, taken in pieces of 128 tokens, reads the weights
+      // once per piece, where the parts run parts * G row tiles that are mostly padding.  Which is faster depends
+      // on the layer's size; pieces_win() compares two fitted estimates.
       Dims W = *D;
       W.T_max = 128;
-      if (desc->T_max <= kSeqTokens && stream_supported(W)) { D->seq = 128; D->T_max = 128; continue; }
+      if (desc->T_max <= kSeqTokens && stream_supported(W) && pieces_win(*desc, parts)) { D->seq = 128; D->T_max = 128; continue; }
       D->split = parts; D->rep = parts; D->K = V.K; D->G = V.G; D->T_max = V.T_max;
     }
   }

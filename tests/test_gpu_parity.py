@@ -616,29 +616,51 @@ def test_headline_shape_variants(kw):
     assert got["module"].info.path == 1
 
 
-@pytest.mark.parametrize("T,T_max", [(129, 129), (300, 384), (384, 384), (128, 384), (50, 200)])
+_wide_layer = {}
+
+
+def _wide_clusters_layer():
+    """d = 2048, d_ff = 8192, K = 8, r = 32 (K r = 256; 537 MB of bases): large enough for the pieces to win."""
+    if not _wide_layer:
+        s = inputs.small_shape(T=256, d=2048, d_ff=8192, E=64, G=8, r=32, k=2)
+        _wide_layer["L"] = inputs.make_layer(s, 27)
+    return _wide_layer["L"]
+
+
+@pytest.mark.parametrize("T,T_max", [(129, 129), (200, 256), (256, 256), (128, 256), (50, 200)])
 def test_wide_clusters_on_few_tokens_stream_in_pieces(T, T_max):
-    """K r > 64 with 128 < T_max <= 384: the call's tokens go through the weight-streaming kernels in consecutive pieces of
-    128 tokens (splitting the clusters would compute up to four base products per token on mostly empty tiles).  Every
-    row against the oracle; routes and expert loads of the whole call."""
+    """K r > 64 with 128 < T_max <= 384 on a layer with enough weights: the call's tokens go through the weight-streaming
+    kernels in consecutive pieces of 128 tokens (splitting the clusters would run 4 G row tiles that are mostly padding).
+    Every row against the oracle; routes and expert loads of the whole call."""
     import torch
-    s = inputs.small_shape(T=T, d=256, d_ff=512, E=16, G=2, r=32, k=2)
-    L = inputs.make_layer(s, 27)
-    got = full_check(L, L["x"], T_max=T_max)
+    L = _wide_clusters_layer()
+    s = L["shape"]
+    x = L["x"][:T]
+    got = full_check(L, x, T_max=T_max)
     m = got["module"]
-    assert m.info.path == 2 and m.info.T_pad_max < 2 * 128 + 64
-    loads, _, _ = m.expert_stats(torch.from_numpy(L["x"]).cuda())
+    assert m.info.path == 2 and m.info.T_pad_max < 2 * 128 + 8 * 16
+    loads, _, _ = m.expert_stats(torch.from_numpy(x).cuda())
     torch.cuda.synchronize()
-    want = np.bincount(ref.Layer(L).route(L["x"])["expert_slot"].reshape(-1), minlength=s.E)
+    want = np.bincount(ref.Layer(L).route(x)["expert_slot"].reshape(-1), minlength=s.E)
     assert int(loads.sum()) == s.k * T and np.abs(loads.cpu().numpy() - want).sum() <= 8
 
 
-def test_wide_clusters_beyond_the_streamed_pieces():
-    """The same layer with T_max = 385 is past the limit of the pieces: clusters as quarters on the pair path."""
-    s = inputs.small_shape(T=385, d=256, d_ff=512, E=16, G=2, r=32, k=2)
-    L = inputs.make_layer(s, 27)
-    got = full_check(L, L["x"])
-    assert got["module"].info.path == 1 and got["module"].info.T_pad_max >= 4 * 385
+@pytest.mark.parametrize("T,kw", [
+    (385, dict(d=2048, d_ff=8192, E=64, G=8, r=32, k=2)),     # past the limit of the pieces
+    (300, dict(d=256, d_ff=512, E=16, G=2, r=32, k=2)),       # a small layer: the quarters are estimated faster
+], ids=["T385", "small_layer"])
+def test_wide_clusters_beyond_the_streamed_pieces(T, kw):
+    """Where the pieces would not pay (more than 384 tokens, or a layer with few weights) the clusters run as
+    quarters on the pair path; sampled rows."""
+    if kw["d"] == 2048:
+        L = dict(_wide_clusters_layer())
+        s = inputs.small_shape(T=T, **kw)
+        L["shape"] = s
+        L["x"] = inputs.make_tokens(s, T, seed=5)
+    else:
+        L = inputs.make_layer(inputs.small_shape(T=T, **kw), 27)
+    got = full_check(L, L["x"], sample=128)
+    assert got["module"].info.path == 1 and got["module"].info.T_pad_max >= 4 * T
 
 
 def test_decode_shaped_layer_on_a_large_batch():
@@ -696,11 +718,9 @@ def test_expert_halves(T, kw):
     s = inputs.small_shape(T=T, **kw)
     L = inputs.make_layer(s, 17)
     got = full_check(L, L["x"])
-    if kw["k"] <= 2 and T > 384:
+    if kw["k"] <= 2:
         assert got["module"].info.path == 1
         assert got["module"].info.T_pad_max >= 2 * T            # two virtual tokens per token
-    elif kw["k"] <= 2:
-        assert got["module"].info.path == 2                     # few tokens: pieces of 128 on the streaming path
 
 
 def test_expert_halves_report_the_tokens_own_routes_and_loads():
